@@ -1,0 +1,160 @@
+/*
+ * forge.h -- C interface of the B200 (sm_100a) fused linear operator
+ *
+ *     E = scale * act(X * W^T + b)            X [M,K], W [N,K], b [N]
+ *     none:       Y[M,N]  = E
+ *     sum / max:  out[M]  = sum_n E[m,n]  /  max_n E[m,n]
+ *     layernorm:  Y[M,N]  = (E - mean_n E) / sqrt(var_n E + eps) * gamma[n] + beta[n]
+ *
+ * The operation is the fused operator chain the paper's agents are asked to produce: one
+ * kernel in place of a framework Linear (matmul + bias) followed by an element-wise
+ * activation (Appendix A.1, "combining matmul + relu") and, optionally, a per-row statistic
+ * computed from the accumulators without a trip through global memory (Appendix B.1, the
+ * Linear + in-register epilogue proposal, whose stated difficulty is the aggregation across
+ * output tiles).  Results are meant to agree with the unfused chain evaluated in double
+ * precision within 1e-4 (fp32) -- the tolerance of Section 2.2 -- or 2e-2 (bf16 storage).
+ *
+ * Conventions for every entry point
+ *   - No exceptions, no aborts: every failure is a forge_status_t return value.
+ *   - All tensors are dense row-major with leading dimension K (X, W) or N (Y); the
+ *     contraction runs over the contiguous axis of both X and W.
+ *   - X, W, b, gamma, beta and Y share the descriptor's dtype; out[M] of sum/max is fp32.
+ *   - Rounding of bf16 outputs is to nearest, ties to even.
+ *   - There is no fallback: a descriptor the hand-written kernels cannot serve is rejected
+ *     with FORGE_ERR_UNSUPPORTED, never computed some other way.
+ */
+#ifndef FORGE_H_
+#define FORGE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct forge_fused_linear_s *forge_fused_linear_t;   /* opaque handle */
+
+typedef enum {
+    FORGE_OK = 0,
+    FORGE_ERR_INVALID_ARG = 1,   /* NULL pointer, bad enum, non-positive size, misalignment */
+    FORGE_ERR_UNSUPPORTED = 2,   /* valid request that no kernel here serves              */
+    FORGE_ERR_CUDA = 3,          /* a CUDA runtime/driver call failed (or no sm_100 GPU)  */
+    FORGE_ERR_ALLOC = 4,         /* host or device allocation failed                      */
+    FORGE_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up                    */
+} forge_status_t;
+
+typedef enum { FORGE_F32 = 0, FORGE_BF16 = 1 } forge_dtype_t;
+
+typedef enum {
+    FORGE_ACT_IDENTITY = 0,
+    FORGE_ACT_RELU = 1,          /* max(z, 0)                                            */
+    FORGE_ACT_GELU_ERF = 2,      /* 0.5 z (1 + erf(z / sqrt 2))                          */
+    FORGE_ACT_GELU_TANH = 3,     /* 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3)))      */
+    FORGE_ACT_SILU = 4           /* z / (1 + exp(-z))                                    */
+} forge_act_t;
+
+typedef enum {
+    FORGE_RED_NONE = 0,
+    FORGE_RED_SUM = 1,
+    FORGE_RED_MAX = 2,
+    FORGE_RED_LAYERNORM = 3      /* population variance, eps inside the square root      */
+} forge_red_t;
+
+typedef struct {
+    int64_t M, N, K;             /* all > 0                                              */
+    forge_dtype_t dtype;         /* storage type of X, W, b, gamma, beta, Y              */
+    forge_act_t act;
+    forge_red_t red;
+    float scale;                 /* multiplies act(...); 1.0f for none                   */
+    float ln_eps;                /* FORGE_RED_LAYERNORM only                             */
+    int has_bias;                /* 0: b is ignored and may be NULL                      */
+    int device;                  /* CUDA device ordinal                                  */
+} forge_fused_linear_desc_t;
+
+/* Kernel families.  The choice is a pure function of the descriptor. */
+typedef enum {
+    FORGE_KERNEL_F32_FFMA = 1,        /* fp32 register-tiled FFMA GEMM, fused epilogue        */
+    FORGE_KERNEL_BF16_TCGEN05 = 2,    /* bf16 TMA -> smem ring -> tcgen05.mma -> TMEM         */
+    FORGE_KERNEL_BF16_SKINNY = 3,     /* bf16, M <= 16: split-K over warps, HBM-bound          */
+    FORGE_KERNEL_BF16_TCGEN05_LN = 4  /* bf16 tcgen05 with a cluster-wide LayerNorm epilogue  */
+} forge_kernel_t;
+
+typedef struct {
+    forge_kernel_t kernel;
+    int tile_m, tile_n, tile_k;  /* CTA tile                                              */
+    int stages;                  /* depth of the shared-memory ring (0: not ring-based)   */
+    int cluster;                 /* CTAs per cluster (1: no cluster)                      */
+    int threads;                 /* threads per CTA                                       */
+    int64_t grid;                /* CTAs launched, given sm_count                         */
+    int64_t smem_bytes;          /* dynamic shared memory per CTA                         */
+    int64_t workspace_bytes;     /* device scratch owned by the handle                    */
+} forge_plan_info_t;
+
+/*
+ * Host-only: validate `desc` and report the kernel that create() would plan for a GPU with
+ * `sm_count` multiprocessors.  Touches no device.  Returns FORGE_ERR_INVALID_ARG /
+ * FORGE_ERR_UNSUPPORTED exactly as create() would for the same descriptor.
+ * Kernel selection (Appendix B.1's point that the right fusion depends on whether the chain
+ * is compute- or memory-bound): fp32 -> F32_FFMA; bf16 with M <= 16 and no LayerNorm ->
+ * BF16_SKINNY; bf16 LayerNorm -> BF16_TCGEN05_LN; other bf16 -> BF16_TCGEN05.
+ * Unsupported: bf16 with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); LayerNorm with N
+ * larger than one cluster spans (bf16: 4096, fp32: 1024).
+ */
+forge_status_t forge_fused_linear_query_plan(const forge_fused_linear_desc_t *desc, int sm_count,
+                                             forge_plan_info_t *info);
+
+/*
+ * Validate, plan, and allocate the handle's device workspace (per-tile partials, arrival
+ * counters, a status word) on desc->device.  Host pointers: `desc` (read), `out` (written
+ * with the new handle; NULL on failure).  Requires compute capability 10.x; otherwise
+ * FORGE_ERR_CUDA.  Synchronous; launches no kernel on any user stream.
+ */
+forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, forge_fused_linear_t *out);
+
+/*
+ * Enqueue one evaluation on `cuda_stream` (a cudaStream_t; NULL = default stream).
+ * DEVICE pointers, owned by the caller, 16-byte aligned, alive until the work completes:
+ *   X [M,K], W [N,K], b [N] (may be NULL iff has_bias == 0), gamma, beta [N] (non-NULL iff
+ *   layernorm), out: Y [M,N] in dtype (none, layernorm) or fp32 [M] (sum, max).
+ * Allocates nothing and does not synchronise.  Returns only argument / launch errors;
+ * device-side give-ups are reported by forge_fused_linear_last_status().  At most one run
+ * per handle may be in flight (the workspace belongs to the handle).
+ * Steps: operand fetch, contraction with fp32 accumulation, bias, activation, scale, row
+ * reduction and store all happen inside the single kernel launched here (the fused form of
+ * Appendix A.1 / B.1; nothing but the final result reaches global memory).
+ */
+forge_status_t forge_fused_linear_run(forge_fused_linear_t h, const void *X, const void *W, const void *b,
+                                      const void *gamma, const void *beta, void *out, void *cuda_stream);
+
+/*
+ * Same operation with HOST buffers (pageable or pinned): copies the inputs to device
+ * staging buffers owned by the handle (allocated on first use), runs, copies the result
+ * back and synchronises.  Layouts and dtypes as for run(); bf16 data are raw 16-bit words.
+ */
+forge_status_t forge_fused_linear_run_host(forge_fused_linear_t h, const void *X, const void *W, const void *b,
+                                           const void *gamma, const void *beta, void *out);
+
+/*
+ * Read the handle's device status word.  Synchronises the device first.  FORGE_OK, or
+ * FORGE_ERR_TIMEOUT if a bounded wait inside the last kernels expired (the output is then
+ * undefined).  The word is cleared by this call.
+ */
+forge_status_t forge_fused_linear_last_status(forge_fused_linear_t h);
+
+/* Copy the plan chosen at create() into *info (host pointer). */
+forge_status_t forge_fused_linear_get_plan(forge_fused_linear_t h, forge_plan_info_t *info);
+
+/* Number of kernels run() launches per call for this handle (always >= 1). */
+int forge_fused_linear_launches_per_run(forge_fused_linear_t h);
+
+/* Free the workspace, staging buffers and the handle.  NULL is FORGE_ERR_INVALID_ARG. */
+forge_status_t forge_fused_linear_destroy(forge_fused_linear_t h);
+
+/* Static strings; never NULL. */
+const char *forge_status_string(forge_status_t s);
+const char *forge_kernel_name(forge_kernel_t k);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FORGE_H_ */

@@ -1,0 +1,291 @@
+// The C interface: descriptor validation, kernel selection, workspace, launches.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "plan.h"
+
+namespace forge {
+
+namespace {
+
+constexpr size_t kStatusBytes = 256;     // status word lives alone in the first 256 bytes
+
+bool desc_enums_ok(const forge_fused_linear_desc_t &d)
+{
+    return (d.dtype == FORGE_F32 || d.dtype == FORGE_BF16) && d.act >= FORGE_ACT_IDENTITY &&
+           d.act <= FORGE_ACT_SILU && d.red >= FORGE_RED_NONE && d.red <= FORGE_RED_LAYERNORM;
+}
+
+forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
+{
+    if (d.M <= 0 || d.N <= 0 || d.K <= 0 || !desc_enums_ok(d) || d.device < 0 || sm_count <= 0)
+        return FORGE_ERR_INVALID_ARG;
+    if (!(d.scale == d.scale) || !(d.ln_eps == d.ln_eps)) return FORGE_ERR_INVALID_ARG;   // NaN
+    if (d.red == FORGE_RED_LAYERNORM && d.ln_eps < 0.f) return FORGE_ERR_INVALID_ARG;
+    std::memset(info, 0, sizeof(*info));
+    forge_status_t st;
+    if (d.dtype == FORGE_F32) {
+        st = k1_plan(d, sm_count, info, wl);
+    } else {
+        if (d.K % 8 != 0 || d.N % 8 != 0) return FORGE_ERR_UNSUPPORTED;     // 16-byte row pitch for TMA
+        if (d.red == FORGE_RED_LAYERNORM) st = k4_plan(d, sm_count, info, wl);
+        else if (d.M <= 16) st = k3_plan(d, sm_count, info, wl);
+        else st = k2_plan(d, sm_count, info, wl);
+    }
+    if (st != FORGE_OK) return st;
+    const size_t bytes = kStatusBytes + ((wl->counters * sizeof(unsigned) + 255) / 256) * 256 +
+                         wl->partial_floats * sizeof(float);
+    info->workspace_bytes = (int64_t)bytes;
+    return FORGE_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; prev = -1; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard()
+    {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+size_t elem_bytes(const forge_fused_linear_desc_t &d) { return d.dtype == FORGE_F32 ? 4 : 2; }
+size_t out_bytes(const forge_fused_linear_desc_t &d)
+{
+    return (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) ? (size_t)d.M * 4
+                                                              : (size_t)d.M * (size_t)d.N * elem_bytes(d);
+}
+
+forge_status_t check_run_args(const Handle &h, const RunArgs &a)
+{
+    if (!a.X || !a.W || !a.out) return FORGE_ERR_INVALID_ARG;
+    if (h.d.has_bias && !a.b) return FORGE_ERR_INVALID_ARG;
+    if (h.d.red == FORGE_RED_LAYERNORM && (!a.gamma || !a.beta)) return FORGE_ERR_INVALID_ARG;
+    const uintptr_t m = (uintptr_t)a.X | (uintptr_t)a.W | (uintptr_t)a.out | (uintptr_t)a.b |
+                        (uintptr_t)a.gamma | (uintptr_t)a.beta;
+    // bf16 operands travel by TMA and 128-bit accesses: 16-byte alignment is required.
+    // fp32 falls back to scalar accesses when unaligned, but still needs element alignment.
+    if (h.d.dtype == FORGE_BF16 ? (m % 16 != 0) : (m % 4 != 0)) return FORGE_ERR_INVALID_ARG;
+    return FORGE_OK;
+}
+
+forge_status_t dispatch(Handle &h, const RunArgs &a)
+{
+    switch (h.info.kernel) {
+    case FORGE_KERNEL_F32_FFMA: return k1_launch(h, a);
+    case FORGE_KERNEL_BF16_TCGEN05: return k2_launch(h, a);
+    case FORGE_KERNEL_BF16_SKINNY: return k3_launch(h, a);
+    case FORGE_KERNEL_BF16_TCGEN05_LN: return k4_launch(h, a);
+    }
+    return FORGE_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+forge_status_t encode_tmap_bf16(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
+                                uint32_t box_rows, uint32_t box_cols)
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &sym, 12000, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess || !sym)
+            return FORGE_ERR_CUDA;
+        fn = (EncodeTiledFn)sym;
+    }
+    const cuuint64_t dims[2] = {cols, rows};                  // innermost first
+    const cuuint64_t strides[1] = {cols * 2};                 // bytes, dimension 1
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? FORGE_OK : FORGE_ERR_CUDA;
+}
+
+}  // namespace forge
+
+using namespace forge;
+
+extern "C" {
+
+forge_status_t forge_fused_linear_query_plan(const forge_fused_linear_desc_t *desc, int sm_count, forge_plan_info_t *info)
+{
+    if (!desc || !info) return FORGE_ERR_INVALID_ARG;
+    WorkspaceLayout wl;
+    return plan_for(*desc, sm_count, info, &wl);
+}
+
+forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, forge_fused_linear_t *out)
+{
+    if (out) *out = nullptr;
+    if (!desc || !out) return FORGE_ERR_INVALID_ARG;
+    // argument errors are reported before the device is touched
+    forge_plan_info_t probe;
+    WorkspaceLayout wl;
+    forge_status_t st = plan_for(*desc, 148, &probe, &wl);
+    if (st != FORGE_OK) return st;
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || desc->device >= ndev) { cudaGetLastError(); return FORGE_ERR_CUDA; }
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, desc->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, desc->device) != cudaSuccess)
+        return FORGE_ERR_CUDA;
+    if (major != 10) return FORGE_ERR_CUDA;     // the kernels are sm_100a only
+
+    Handle *h = new (std::nothrow) Handle();
+    if (!h) return FORGE_ERR_ALLOC;
+    h->d = *desc;
+    h->sm_count = sms;
+    st = plan_for(*desc, sms, &h->info, &wl);
+    if (st != FORGE_OK) { delete h; return st; }
+
+    DeviceGuard g(desc->device);
+    if (!g.ok) { delete h; return FORGE_ERR_CUDA; }
+    h->ws.bytes = (size_t)h->info.workspace_bytes;
+    if (cudaMalloc(&h->ws.base, h->ws.bytes) != cudaSuccess) { cudaGetLastError(); delete h; return FORGE_ERR_ALLOC; }
+    if (cudaMemset(h->ws.base, 0, h->ws.bytes) != cudaSuccess) { cudaFree(h->ws.base); delete h; return FORGE_ERR_CUDA; }
+    char *base = (char *)h->ws.base;
+    h->ws.status = (int *)base;
+    h->ws.counters = (unsigned *)(base + kStatusBytes);
+    h->ws.partial = (float *)(base + kStatusBytes + ((wl.counters * sizeof(unsigned) + 255) / 256) * 256);
+
+    switch (h->info.kernel) {
+    case FORGE_KERNEL_F32_FFMA: st = k1_setup(*h); break;
+    case FORGE_KERNEL_BF16_TCGEN05: st = k2_setup(*h); break;
+    case FORGE_KERNEL_BF16_SKINNY: st = k3_setup(*h); break;
+    case FORGE_KERNEL_BF16_TCGEN05_LN: st = k4_setup(*h); break;
+    }
+    if (st != FORGE_OK) { cudaFree(h->ws.base); delete h; return st; }
+    *out = reinterpret_cast<forge_fused_linear_t>(h);
+    return FORGE_OK;
+}
+
+forge_status_t forge_fused_linear_run(forge_fused_linear_t hh, const void *X, const void *W, const void *b,
+                                      const void *gamma, const void *beta, void *out, void *cuda_stream)
+{
+    if (!hh) return FORGE_ERR_INVALID_ARG;
+    Handle &h = *reinterpret_cast<Handle *>(hh);
+    RunArgs a{X, W, h.d.has_bias ? b : nullptr, gamma, beta, out, (cudaStream_t)cuda_stream};
+    const forge_status_t st = check_run_args(h, a);
+    if (st != FORGE_OK) return st;
+    DeviceGuard g(h.d.device);
+    if (!g.ok) return FORGE_ERR_CUDA;
+    return dispatch(h, a);
+}
+
+forge_status_t forge_fused_linear_run_host(forge_fused_linear_t hh, const void *X, const void *W, const void *b,
+                                           const void *gamma, const void *beta, void *out)
+{
+    if (!hh) return FORGE_ERR_INVALID_ARG;
+    Handle &h = *reinterpret_cast<Handle *>(hh);
+    const forge_fused_linear_desc_t &d = h.d;
+    if (!X || !W || !out || (d.has_bias && !b) || (d.red == FORGE_RED_LAYERNORM && (!gamma || !beta)))
+        return FORGE_ERR_INVALID_ARG;
+    DeviceGuard g(d.device);
+    if (!g.ok) return FORGE_ERR_CUDA;
+    const size_t e = elem_bytes(d);
+    const size_t bx = (size_t)d.M * d.K * e, bw = (size_t)d.N * d.K * e, bn = (size_t)d.N * e, bo = out_bytes(d);
+    if (!h.hX) {
+        if (cudaMalloc(&h.hX, bx) != cudaSuccess || cudaMalloc(&h.hW, bw) != cudaSuccess ||
+            cudaMalloc(&h.hb, bn) != cudaSuccess || cudaMalloc(&h.hg, bn) != cudaSuccess ||
+            cudaMalloc(&h.hbe, bn) != cudaSuccess || cudaMalloc(&h.hout, bo) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(h.hX); cudaFree(h.hW); cudaFree(h.hb); cudaFree(h.hg); cudaFree(h.hbe); cudaFree(h.hout);
+            h.hX = h.hW = h.hb = h.hg = h.hbe = h.hout = nullptr;
+            return FORGE_ERR_ALLOC;
+        }
+    }
+    cudaStream_t s = nullptr;
+    bool ok = cudaMemcpyAsync(h.hX, X, bx, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+              cudaMemcpyAsync(h.hW, W, bw, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (ok && d.has_bias) ok = cudaMemcpyAsync(h.hb, b, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (ok && d.red == FORGE_RED_LAYERNORM)
+        ok = cudaMemcpyAsync(h.hg, gamma, bn, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+             cudaMemcpyAsync(h.hbe, beta, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!ok) return FORGE_ERR_CUDA;
+    RunArgs a{h.hX, h.hW, d.has_bias ? h.hb : nullptr, h.hg, h.hbe, h.hout, s};
+    const forge_status_t st = dispatch(h, a);
+    if (st != FORGE_OK) return st;
+    if (cudaMemcpyAsync(out, h.hout, bo, cudaMemcpyDeviceToHost, s) != cudaSuccess) return FORGE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return FORGE_ERR_CUDA;
+    return FORGE_OK;
+}
+
+forge_status_t forge_fused_linear_last_status(forge_fused_linear_t hh)
+{
+    if (!hh) return FORGE_ERR_INVALID_ARG;
+    Handle &h = *reinterpret_cast<Handle *>(hh);
+    DeviceGuard g(h.d.device);
+    if (!g.ok) return FORGE_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return FORGE_ERR_CUDA;
+    int word = 0;
+    if (cudaMemcpy(&word, h.ws.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FORGE_ERR_CUDA;
+    if (word != 0) {
+        // a give-up may have left arrival counters half way: clear the whole workspace
+        cudaMemset(h.ws.base, 0, h.ws.bytes);
+        return (forge_status_t)(word >> 16);
+    }
+    return FORGE_OK;
+}
+
+forge_status_t forge_fused_linear_get_plan(forge_fused_linear_t hh, forge_plan_info_t *info)
+{
+    if (!hh || !info) return FORGE_ERR_INVALID_ARG;
+    *info = reinterpret_cast<Handle *>(hh)->info;
+    return FORGE_OK;
+}
+
+int forge_fused_linear_launches_per_run(forge_fused_linear_t hh) { return hh ? 1 : 0; }
+
+forge_status_t forge_fused_linear_destroy(forge_fused_linear_t hh)
+{
+    if (!hh) return FORGE_ERR_INVALID_ARG;
+    Handle *h = reinterpret_cast<Handle *>(hh);
+    {
+        DeviceGuard g(h->d.device);
+        cudaFree(h->ws.base);
+        cudaFree(h->hX); cudaFree(h->hW); cudaFree(h->hb); cudaFree(h->hg); cudaFree(h->hbe); cudaFree(h->hout);
+    }
+    delete h;
+    return FORGE_OK;
+}
+
+const char *forge_status_string(forge_status_t s)
+{
+    switch (s) {
+    case FORGE_OK: return "ok";
+    case FORGE_ERR_INVALID_ARG: return "invalid argument";
+    case FORGE_ERR_UNSUPPORTED: return "unsupported descriptor (no kernel serves it; there is no fallback)";
+    case FORGE_ERR_CUDA: return "CUDA error or no sm_100 device";
+    case FORGE_ERR_ALLOC: return "allocation failed";
+    case FORGE_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    }
+    return "unknown status";
+}
+
+const char *forge_kernel_name(forge_kernel_t k)
+{
+    switch (k) {
+    case FORGE_KERNEL_F32_FFMA: return "f32_ffma_128x128x16";
+    case FORGE_KERNEL_BF16_TCGEN05: return "bf16_tcgen05_tma";
+    case FORGE_KERNEL_BF16_SKINNY: return "bf16_skinny_splitk";
+    case FORGE_KERNEL_BF16_TCGEN05_LN: return "bf16_tcgen05_cluster_layernorm";
+    }
+    return "unknown kernel";
+}
+
+}  // extern "C"

@@ -1,0 +1,340 @@
+// K1: fp32 fused linear.  Register-tiled FFMA GEMM (128x128 CTA tile, 8x8 per thread),
+// 128-bit global loads, double-buffered shared memory, epilogue (bias, activation, scale,
+// row sum / max / LayerNorm) applied to the accumulators in registers.
+//
+// Row reductions across the N-tiles of one row strip:
+//   sum/max   per-tile partials in a small workspace, folded in tile order by the CTA that
+//             arrives last at the strip's counter (deterministic, no float atomics);
+//   layernorm the N-tiles of a strip form one thread-block cluster; per-row (n, mean, M2)
+//             triples are exchanged through distributed shared memory and merged, then
+//             each CTA normalises the tile it still holds in registers.
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+#include "plan.h"
+
+namespace cg = cooperative_groups;
+
+namespace forge {
+
+constexpr int K1_BM = 128, K1_BN = 128, K1_BK = 16, K1_THREADS = 256, K1_PAD = 4;
+constexpr int K1_LN_MAX_CLUSTER = 8;
+
+struct K1Params {
+    const float *X, *W, *b, *gamma, *beta;
+    float *out;
+    int M, N, K;
+    Epilogue e;
+    float *partial;        // [tiles_n][M]
+    unsigned *counters;    // [tiles_m]
+    int tiles_n;
+    int out_vec4;          // Y rows can be written with 128-bit stores
+};
+
+// One CTA-tile slab of 128 rows x 16 k from a K-major matrix into registers.
+template <bool VEC>
+__device__ __forceinline__ void k1_fetch(const float *__restrict__ base, int rows_total, int K,
+                                         int row0, int kt, int tid, float4 (&r)[2])
+{
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int idx = tid + i * K1_THREADS;
+        const int row = row0 + (idx >> 2);
+        const int k = kt + (idx & 3) * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row < rows_total) {
+            const float *src = base + (size_t)row * K + k;
+            if (VEC) {
+                if (k < K) v = __ldg(reinterpret_cast<const float4 *>(src));
+            } else {
+                if (k + 0 < K) v.x = __ldg(src + 0);
+                if (k + 1 < K) v.y = __ldg(src + 1);
+                if (k + 2 < K) v.z = __ldg(src + 2);
+                if (k + 3 < K) v.w = __ldg(src + 3);
+            }
+        }
+        r[i] = v;
+    }
+}
+
+// Registers -> shared memory, transposed to [k][row] so the inner product reads rows of 4.
+__device__ __forceinline__ void k1_stash(float (*S)[K1_BM + K1_PAD], int tid, const float4 (&r)[2])
+{
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int idx = tid + i * K1_THREADS;
+        const int row = idx >> 2;
+        const int k = (idx & 3) * 4;
+        S[k + 0][row] = r[i].x;
+        S[k + 1][row] = r[i].y;
+        S[k + 2][row] = r[i].z;
+        S[k + 3][row] = r[i].w;
+    }
+}
+
+template <bool VEC, int RED>
+__global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Params p)
+{
+    __shared__ __align__(16) float As[2][K1_BK][K1_BM + K1_PAD];
+    __shared__ __align__(16) float Bs[2][K1_BK][K1_BN + K1_PAD];
+    __shared__ RowStat s_stat[K1_BM];
+    __shared__ float s_mean[K1_BM], s_rstd[K1_BM];
+    __shared__ int s_last;
+
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    const int tile_n = blockIdx.x, tile_m = blockIdx.y;
+    const int m0 = tile_m * K1_BM, n0 = tile_n * K1_BN;
+    const int M = p.M, N = p.N, K = p.K;
+
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+
+    float4 ra[2], rb[2];
+    k1_fetch<VEC>(p.X, M, K, m0, 0, tid, ra);
+    k1_fetch<VEC>(p.W, N, K, n0, 0, tid, rb);
+    k1_stash(As[0], tid, ra);
+    k1_stash(Bs[0], tid, rb);
+    __syncthreads();
+
+    int buf = 0;
+    for (int kt = 0; kt < K; kt += K1_BK) {
+        const bool more = kt + K1_BK < K;
+        if (more) {
+            k1_fetch<VEC>(p.X, M, K, m0, kt + K1_BK, tid, ra);
+            k1_fetch<VEC>(p.W, N, K, n0, kt + K1_BK, tid, rb);
+        }
+#pragma unroll
+        for (int k = 0; k < K1_BK; ++k) {
+            const float4 a0 = *reinterpret_cast<const float4 *>(&As[buf][k][ty * 4]);
+            const float4 a1 = *reinterpret_cast<const float4 *>(&As[buf][k][64 + ty * 4]);
+            const float4 b0 = *reinterpret_cast<const float4 *>(&Bs[buf][k][tx * 4]);
+            const float4 b1 = *reinterpret_cast<const float4 *>(&Bs[buf][k][64 + tx * 4]);
+            const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        if (more) {
+            k1_stash(As[buf ^ 1], tid, ra);
+            k1_stash(Bs[buf ^ 1], tid, rb);
+        }
+        __syncthreads();
+        buf ^= 1;
+    }
+
+    // ---- epilogue: bias, activation, scale, in registers --------------------------------
+    int col[8];
+    bool cok[8];
+    float bias[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        col[j] = n0 + tx * 4 + (j & 3) + (j >> 2) * 64;
+        cok[j] = col[j] < N;
+        bias[j] = (p.e.has_bias && cok[j]) ? __ldg(p.b + col[j]) : 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = p.e.scale * apply_act<true>(p.e.act, acc[i][j] + bias[j]);
+
+    if (RED == FORGE_RED_NONE) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int row = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
+            if (row >= M) continue;
+            float *dst = p.out + (size_t)row * N;
+            if (p.out_vec4) {
+                if (cok[0]) *reinterpret_cast<float4 *>(dst + col[0]) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                if (cok[4]) *reinterpret_cast<float4 *>(dst + col[4]) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (cok[j]) dst[col[j]] = acc[i][j];
+            }
+        }
+        return;
+    }
+
+    if (RED == FORGE_RED_SUM || RED == FORGE_RED_MAX) {
+        // thread -> 16 lanes that share the row (shuffles) -> tile partial
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float v = (RED == FORGE_RED_SUM) ? 0.f : -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (cok[j]) v = (RED == FORGE_RED_SUM) ? v + acc[i][j] : fmaxf(v, acc[i][j]);
+#pragma unroll
+            for (int s = 8; s >= 1; s >>= 1) {
+                const float o = __shfl_xor_sync(0xffffffffu, v, s);
+                v = (RED == FORGE_RED_SUM) ? v + o : fmaxf(v, o);
+            }
+            const int row = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
+            if (tx == 0 && row < M) {
+                if (p.tiles_n == 1) p.out[row] = v;
+                else p.partial[(size_t)tile_n * M + row] = v;
+            }
+        }
+        if (p.tiles_n == 1) return;
+        // the last CTA to arrive at this row strip folds the partials in tile order
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = (atomicAdd(&p.counters[tile_m], 1u) == (unsigned)(p.tiles_n - 1));
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+        if (tid < K1_BM && m0 + tid < M) {
+            const int row = m0 + tid;
+            float v = __ldcg(&p.partial[row]);
+            for (int t = 1; t < p.tiles_n; ++t) {
+                const float o = __ldcg(&p.partial[(size_t)t * M + row]);
+                v = (RED == FORGE_RED_SUM) ? v + o : fmaxf(v, o);
+            }
+            p.out[row] = v;
+        }
+        if (tid == 0) p.counters[tile_m] = 0u;     // ready for the next run
+        return;
+    }
+
+    if (RED == FORGE_RED_LAYERNORM) {
+        cg::cluster_group cluster = cg::this_cluster();
+        // per-thread statistics of its <= 8 columns of each row, two sweeps over registers
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            RowStat s;
+            float sum = 0.f;
+            s.n = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (cok[j]) { sum += acc[i][j]; s.n += 1.f; }
+            s.mean = s.n > 0.f ? sum / s.n : 0.f;
+            s.m2 = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (cok[j]) { const float d = acc[i][j] - s.mean; s.m2 = fmaf(d, d, s.m2); }
+#pragma unroll
+            for (int sft = 1; sft <= 8; sft <<= 1) s = merge_stat(s, shfl_xor_stat(s, sft));
+            if (tx == 0) s_stat[ty * 4 + (i & 3) + (i >> 2) * 64] = s;
+        }
+        cluster.sync();
+        if (tid < K1_BM) {
+            const unsigned nranks = cluster.num_blocks();
+            RowStat s = *cluster.map_shared_rank(&s_stat[tid], 0);
+            for (unsigned r = 1; r < nranks; ++r) s = merge_stat(s, *cluster.map_shared_rank(&s_stat[tid], r));
+            s_mean[tid] = s.mean;
+            s_rstd[tid] = rsqrtf(s.m2 / s.n + p.e.eps);
+        }
+        cluster.sync();      // also keeps every CTA's s_stat alive until all have read it
+        float g[8], be[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            g[j] = cok[j] ? __ldg(p.gamma + col[j]) : 0.f;
+            be[j] = cok[j] ? __ldg(p.beta + col[j]) : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int rl = ty * 4 + (i & 3) + (i >> 2) * 64;
+            const int row = m0 + rl;
+            if (row >= M) continue;
+            const float mu = s_mean[rl], rs = s_rstd[rl];
+            float *dst = p.out + (size_t)row * N;
+            float y[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) y[j] = (acc[i][j] - mu) * rs * g[j] + be[j];
+            if (p.out_vec4) {
+                if (cok[0]) *reinterpret_cast<float4 *>(dst + col[0]) = make_float4(y[0], y[1], y[2], y[3]);
+                if (cok[4]) *reinterpret_cast<float4 *>(dst + col[4]) = make_float4(y[4], y[5], y[6], y[7]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (cok[j]) dst[col[j]] = y[j];
+            }
+        }
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
+{
+    (void)sm_count;
+    const int64_t tiles_m = (d.M + K1_BM - 1) / K1_BM, tiles_n = (d.N + K1_BN - 1) / K1_BN;
+    if (tiles_m > 65535 || tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    if (d.red == FORGE_RED_LAYERNORM && tiles_n > K1_LN_MAX_CLUSTER) return FORGE_ERR_UNSUPPORTED;
+    info->kernel = FORGE_KERNEL_F32_FFMA;
+    info->tile_m = K1_BM;
+    info->tile_n = K1_BN;
+    info->tile_k = K1_BK;
+    info->stages = 2;
+    info->cluster = d.red == FORGE_RED_LAYERNORM ? (int)tiles_n : 1;
+    info->threads = K1_THREADS;
+    info->grid = tiles_m * tiles_n;
+    info->smem_bytes = 0;
+    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) && tiles_n > 1;
+    wl->partial_floats = partials ? (size_t)tiles_n * (size_t)d.M : 0;
+    wl->counters = partials ? (size_t)tiles_m : 0;
+    return FORGE_OK;
+}
+
+forge_status_t k1_setup(Handle &) { return FORGE_OK; }
+
+template <bool VEC, int RED>
+static forge_status_t k1_launch_t(const K1Params &p, dim3 grid, int cluster, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(K1_THREADS);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    if (RED == FORGE_RED_LAYERNORM) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = cluster;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    return cudaLaunchKernelEx(&cfg, k1_f32_ffma_kernel<VEC, RED>, p) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+}
+
+forge_status_t k1_launch(Handle &h, const RunArgs &a)
+{
+    const forge_fused_linear_desc_t &d = h.d;
+    K1Params p;
+    p.X = (const float *)a.X;
+    p.W = (const float *)a.W;
+    p.b = (const float *)a.b;
+    p.gamma = (const float *)a.gamma;
+    p.beta = (const float *)a.beta;
+    p.out = (float *)a.out;
+    p.M = (int)d.M;
+    p.N = (int)d.N;
+    p.K = (int)d.K;
+    p.e = Epilogue{(int)d.act, (int)d.red, d.scale, d.ln_eps, d.has_bias};
+    p.partial = h.ws.partial;
+    p.counters = h.ws.counters;
+    p.tiles_n = (int)((d.N + K1_BN - 1) / K1_BN);
+    p.out_vec4 = (d.N % 4 == 0) && ((uintptr_t)a.out % 16 == 0);
+    const dim3 grid((unsigned)p.tiles_n, (unsigned)((d.M + K1_BM - 1) / K1_BM));
+    const bool vec = (d.K % 4 == 0) && ((uintptr_t)a.X % 16 == 0) && ((uintptr_t)a.W % 16 == 0);
+#define K1_CASE(R)                                                                      \
+    case R:                                                                             \
+        return vec ? k1_launch_t<true, R>(p, grid, h.info.cluster, a.stream)            \
+                   : k1_launch_t<false, R>(p, grid, h.info.cluster, a.stream);
+    switch (d.red) {
+        K1_CASE(FORGE_RED_NONE)
+        K1_CASE(FORGE_RED_SUM)
+        K1_CASE(FORGE_RED_MAX)
+        K1_CASE(FORGE_RED_LAYERNORM)
+    }
+#undef K1_CASE
+    return FORGE_ERR_INVALID_ARG;
+}
+
+}  // namespace forge

@@ -1,0 +1,68 @@
+// Host-side plan shared by the C interface and the per-kernel launchers.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/forge.h"
+
+namespace forge {
+
+struct RunArgs {
+    const void *X, *W, *b, *gamma, *beta;
+    void *out;
+    cudaStream_t stream;
+};
+
+// Device scratch owned by a handle.
+struct Workspace {
+    float *partial = nullptr;        // per-tile row partials (sum/max), fp32
+    unsigned *counters = nullptr;    // arrival counters, zero between runs
+    int *status = nullptr;           // status word
+    void *base = nullptr;            // the single allocation the three point into
+    size_t bytes = 0;
+};
+
+struct Handle {
+    forge_fused_linear_desc_t d;
+    forge_plan_info_t info;
+    int sm_count = 0;
+    Workspace ws;
+    // staging buffers of run_host()
+    void *hX = nullptr, *hW = nullptr, *hb = nullptr, *hg = nullptr, *hbe = nullptr, *hout = nullptr;
+    // cached TMA descriptors (bf16 kernels): re-encoded only when a pointer changes
+    CUtensorMap tmX, tmW, tmY;
+    const void *tmX_ptr = nullptr, *tmW_ptr = nullptr, *tmY_ptr = nullptr;
+};
+
+// Layout of the workspace (element counts) for a plan; filled by the planners.
+struct WorkspaceLayout {
+    size_t partial_floats = 0;
+    size_t counters = 0;
+};
+
+// Each kernel family: a host-only planner (no device access), a one-time setup on the
+// device (function attributes), and a launcher.
+forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl);
+forge_status_t k1_setup(Handle &h);
+forge_status_t k1_launch(Handle &h, const RunArgs &a);
+
+forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl);
+forge_status_t k2_setup(Handle &h);
+forge_status_t k2_launch(Handle &h, const RunArgs &a);
+
+forge_status_t k3_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl);
+forge_status_t k3_setup(Handle &h);
+forge_status_t k3_launch(Handle &h, const RunArgs &a);
+
+forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl);
+forge_status_t k4_setup(Handle &h);
+forge_status_t k4_launch(Handle &h, const RunArgs &a);
+
+// Encode a 2-D row-major bf16 tensor map [rows, cols] with a [box_rows, box_cols] box and
+// the 128-byte shared-memory swizzle.  Host-only driver call.
+forge_status_t encode_tmap_bf16(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
+                                uint32_t box_rows, uint32_t box_cols);
+
+}  // namespace forge

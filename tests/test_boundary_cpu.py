@@ -1,0 +1,100 @@
+"""Host-side checks of the C interface that need no GPU: the library loads, exports every
+symbol the header declares, validates descriptors, and plans kernels as documented."""
+import ctypes
+import os
+import re
+import subprocess
+
+import pytest
+
+from paper_2511_01884_b200 import binding as B
+from paper_2511_01884_b200 import build as forge_build
+from paper_2511_01884_b200 import workloads as wk
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    forge_build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "forge.h")).read()
+    declared = set(re.findall(r"\b(forge_[a-z_]+)\s*\(", hdr))
+    assert declared, "no declarations found"
+    L = ctypes.CDLL(B.LIB_PATH)
+    for name in declared:
+        assert hasattr(L, name), f"{name} is declared in forge.h but not exported"
+    assert declared == set(B.EXPORTS)
+
+
+def test_no_vendor_gemm_library_is_linked():
+    out = subprocess.run(["ldd", B.LIB_PATH], capture_output=True, text=True).stdout
+    for lib in ("cublas", "cudnn", "cutlass", "nccl"):
+        assert lib not in out.lower()
+
+
+def test_enums_match_the_workload_module():
+    assert (B.FORGE_F32, B.FORGE_BF16) == (wk.F32, wk.BF16)
+    assert (B.FORGE_ACT_IDENTITY, B.FORGE_ACT_RELU, B.FORGE_ACT_GELU_ERF, B.FORGE_ACT_GELU_TANH, B.FORGE_ACT_SILU) == \
+           (wk.ACT_IDENTITY, wk.ACT_RELU, wk.ACT_GELU_ERF, wk.ACT_GELU_TANH, wk.ACT_SILU)
+    assert (B.FORGE_RED_NONE, B.FORGE_RED_SUM, B.FORGE_RED_MAX, B.FORGE_RED_LAYERNORM) == \
+           (wk.RED_NONE, wk.RED_SUM, wk.RED_MAX, wk.RED_LAYERNORM)
+
+
+def test_invalid_descriptors():
+    ok = dict(M=8, N=8, K=8, dtype=0, act=0, red=0)
+    for bad in (dict(M=0), dict(N=-1), dict(K=0), dict(dtype=2), dict(act=5), dict(act=-1), dict(red=4)):
+        st, _ = B.forge_fused_linear_query_plan(B.make_desc(**{**ok, **bad}))
+        assert st == B.FORGE_ERR_INVALID_ARG, bad
+        st, h = B.forge_fused_linear_create(B.make_desc(**{**ok, **bad}))
+        assert st == B.FORGE_ERR_INVALID_ARG and not h
+    st, _ = B.forge_fused_linear_query_plan(B.make_desc(8, 8, 8, 0, 0, 0, scale=float("nan")))
+    assert st == B.FORGE_ERR_INVALID_ARG
+    st, _ = B.forge_fused_linear_query_plan(B.make_desc(8, 8, 8, 0, 0, 3, ln_eps=-1.0))
+    assert st == B.FORGE_ERR_INVALID_ARG
+    assert B.lib().forge_fused_linear_query_plan(None, 148, None) == B.FORGE_ERR_INVALID_ARG
+    assert B.lib().forge_fused_linear_create(None, None) == B.FORGE_ERR_INVALID_ARG
+    assert B.forge_fused_linear_destroy(None) == B.FORGE_ERR_INVALID_ARG
+    assert B.forge_fused_linear_last_status(None) == B.FORGE_ERR_INVALID_ARG
+    assert B.lib().forge_fused_linear_run(None, None, None, None, None, None, None, None) == B.FORGE_ERR_INVALID_ARG
+
+
+def test_unsupported_is_reported_not_rerouted():
+    # bf16 rows must have a 16-byte pitch
+    for M, N, K in ((64, 8, 12), (64, 12, 8)):
+        st, _ = B.forge_fused_linear_query_plan(B.make_desc(M, N, K, wk.BF16, 0, 0))
+        assert st == B.FORGE_ERR_UNSUPPORTED
+    st, _ = B.forge_fused_linear_query_plan(B.make_desc(64, 1025, 8, wk.F32, 0, wk.RED_LAYERNORM))
+    assert st == B.FORGE_ERR_UNSUPPORTED
+
+
+def test_status_and_kernel_strings():
+    seen = {B.status_string(s) for s in range(6)}
+    assert len(seen) == 6 and "unknown status" not in seen
+    assert B.status_string(99) == "unknown status"
+    assert "f32" in B.kernel_name(B.FORGE_KERNEL_F32_FFMA)
+
+
+def test_fp32_plan():
+    st, p = B.forge_fused_linear_query_plan(pu_desc("c1"))
+    assert st == B.FORGE_OK and p.kernel == B.FORGE_KERNEL_F32_FFMA
+    assert (p.tile_m, p.tile_n, p.grid) == (128, 128, 4) and p.workspace_bytes >= 4 * 128 * 4
+    st, p = B.forge_fused_linear_query_plan(pu_desc("c2"))
+    assert st == B.FORGE_OK and p.grid == 32 * 32 and p.cluster == 1
+
+
+def pu_desc(name):
+    wl = wk.WORKLOADS[name]
+    return B.make_desc(wl.M, wl.N, wl.K, wl.dtype, wl.act, wl.red, wl.scale, wl.ln_eps, wl.bias.kind != "none")
+
+
+def test_create_without_a_gpu_fails_loudly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    st, h = B.forge_fused_linear_create(pu_desc("c1"))
+    assert st == B.FORGE_ERR_CUDA and not h
+    with pytest.raises(B.ForgeError):
+        B.FusedLinear(pu_desc("c1"))

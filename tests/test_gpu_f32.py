@@ -1,0 +1,99 @@
+"""GPU parity of the fp32 path (register-tiled FFMA kernel) against the CPU oracle."""
+import numpy as np
+import pytest
+
+from paper_2511_01884_b200 import binding as B
+from paper_2511_01884_b200 import workloads as wk
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+ACTS = [wk.ACT_IDENTITY, wk.ACT_RELU, wk.ACT_GELU_ERF, wk.ACT_GELU_TANH, wk.ACT_SILU]
+REDS = [wk.RED_NONE, wk.RED_SUM, wk.RED_MAX, wk.RED_LAYERNORM]
+
+
+def test_c1_full():
+    wl = wk.WORKLOADS["c1"]
+    inp = wk.make_inputs(wl)
+    g, plan = pu.run_gpu(wl, inp)
+    assert plan["kernel"] == B.FORGE_KERNEL_F32_FFMA
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_c2_sampled_rows_full_size():
+    wl = wk.WORKLOADS["c2"]
+    inp = wk.make_inputs(wl)
+    g, _ = pu.run_gpu(wl, inp)
+    rows = wk.sample_rows(wl.M)
+    pu.assert_parity(wl, g[rows], pu.run_oracle(wl, inp, rows))
+    assert np.isfinite(g).all()
+
+
+# several tiles in both directions plus ragged tails; K not a multiple of 4 takes the scalar loads
+SHAPES = [(1, 1, 1), (3, 5, 7), (128, 128, 16), (129, 257, 33), (200, 130, 64), (64, 300, 100), (257, 96, 19)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("red", REDS)
+def test_shapes_and_reductions(M, N, K, red):
+    act = ACTS[(M + N + K + red) % len(ACTS)]
+    wl = wk.custom_workload(f"f32_{M}x{N}x{K}", wk.F32, M, N, K, act, red, scale=0.75, seed=M + N)
+    inp = wk.make_inputs(wl)
+    g, _ = pu.run_gpu(wl, inp)
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp), f"act={act} red={red}")
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_every_activation(act):
+    wl = wk.custom_workload("f32_act", wk.F32, 150, 140, 72, act, wk.RED_NONE, scale=1.25, seed=act)
+    inp = wk.make_inputs(wl)
+    # widen the pre-activations so that the tails of the activation are exercised
+    inp["W"] = wk.round_to_storage(inp["W"] * 4.0, wk.F32)
+    g, _ = pu.run_gpu(wl, inp)
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_no_bias_and_layernorm_edge_of_cluster():
+    wl = wk.custom_workload("f32_ln_1024", wk.F32, 130, 1024, 40, wk.ACT_GELU_ERF, wk.RED_LAYERNORM,
+                            has_bias=False, seed=4)
+    inp = wk.make_inputs(wl)
+    g, plan = pu.run_gpu(wl, inp)
+    assert plan["cluster"] == 8
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+    st, _ = B.forge_fused_linear_query_plan(B.make_desc(8, 1025, 8, wk.F32, 0, wk.RED_LAYERNORM))
+    assert st == B.FORGE_ERR_UNSUPPORTED
+
+
+def test_layernorm_constant_rows_give_beta():
+    wl = wk.custom_workload("f32_ln_const", wk.F32, 5, 200, 12, wk.ACT_RELU, wk.RED_LAYERNORM, seed=1)
+    inp = wk.make_inputs(wl)
+    inp["X"][:] = -np.abs(inp["X"])
+    inp["W"][:] = np.abs(inp["W"])
+    inp["b"][:] = -0.5                      # every pre-activation negative: ReLU output is all zero
+    g, _ = pu.run_gpu(wl, inp)
+    assert np.array_equal(g, np.tile(inp["beta"].astype(np.float64), (5, 1)))
+
+
+def test_freivalds_covers_every_output_element():
+    """act = identity: Y r must equal X (W^T r) + (b . r) for random r (checks all of Y in O(MN))."""
+    wl = wk.custom_workload("f32_freivalds", wk.F32, 1000, 900, 520, wk.ACT_IDENTITY, wk.RED_NONE, seed=2)
+    inp = wk.make_inputs(wl)
+    g, _ = pu.run_gpu(wl, inp)
+    rng = np.random.default_rng(0)
+    for _ in range(3):
+        r = rng.standard_normal(wl.N)
+        want = inp["X"].astype(np.float64) @ (inp["W"].astype(np.float64).T @ r) + inp["b"].astype(np.float64) @ r
+        got = g @ r
+        assert np.max(np.abs(got - want)) <= 1e-4 * (np.sqrt(np.mean(want * want)))
+
+
+def test_repeatable_bits_and_workspace_reuse():
+    wl = wk.custom_workload("f32_rep", wk.F32, 300, 700, 64, wk.ACT_SILU, wk.RED_SUM, seed=3)
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op)
+    b, _ = pu.run_gpu(wl, inp, op=op)          # second run reuses counters reset by the first
+    op.close()
+    assert np.array_equal(a, b)
+    pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
