@@ -65,6 +65,26 @@ __device__ __forceinline__ float apply_act(int act, float z)
     }
 }
 
+// v[i] = scale * act(v[i]) for a register array; the activation is selected once, outside
+// the element loop.
+template <bool ACCURATE, int ACT, int N>
+__device__ __forceinline__ void apply_act_fixed(float (&v)[N], float scale)
+{
+#pragma unroll
+    for (int i = 0; i < N; ++i) v[i] = scale * apply_act<ACCURATE>(ACT, v[i]);
+}
+template <bool ACCURATE, int N>
+__device__ __forceinline__ void apply_act_array(int act, float (&v)[N], float scale)
+{
+    switch (act) {
+    case FORGE_ACT_RELU: apply_act_fixed<ACCURATE, FORGE_ACT_RELU>(v, scale); break;
+    case FORGE_ACT_GELU_ERF: apply_act_fixed<ACCURATE, FORGE_ACT_GELU_ERF>(v, scale); break;
+    case FORGE_ACT_GELU_TANH: apply_act_fixed<ACCURATE, FORGE_ACT_GELU_TANH>(v, scale); break;
+    case FORGE_ACT_SILU: apply_act_fixed<ACCURATE, FORGE_ACT_SILU>(v, scale); break;
+    default: apply_act_fixed<ACCURATE, FORGE_ACT_IDENTITY>(v, scale); break;
+    }
+}
+
 // ---- row statistics (count, mean, sum of squared deviations) -------------------------
 // Merging rule of Chan, Golub & LeVeque for partitioned samples; the single-pass form of
 // the variance that lets LayerNorm statistics be combined across threads, warps and CTAs

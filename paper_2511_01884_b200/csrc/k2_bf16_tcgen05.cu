@@ -1,0 +1,286 @@
+// K2: bf16 fused linear on the 5th-generation tensor cores.
+//
+// Persistent, warp-specialised CTA (one per SM):
+//   warp 0      TMA producer: X and W tiles (128x64 and 256x64 bf16, 128-byte swizzle) into a
+//               4-stage shared-memory ring, completion counted in bytes on "full" mbarriers;
+//   warp 1      MMA issuer: one elected thread issues tcgen05.mma (128x256x16, fp32 accumulate
+//               in TMEM); tcgen05.commit releases ring stages and publishes finished tiles;
+//   warps 2..5  epilogue: tcgen05.ld of the accumulator (thread <-> output row), bias,
+//               activation, scale, then either bf16 stores of Y or the row sum / max.
+// TMEM holds two 128x256 fp32 accumulators, so the epilogue of tile i overlaps the MMAs of
+// tile i+1.  No load is multicast; every wait is bounded (see ptx::mbar_wait).
+#include "common.cuh"
+#include "plan.h"
+#include "sm100_ptx.cuh"
+
+namespace forge {
+
+constexpr int K2_BM = 128, K2_BN = 256, K2_BK = 64, K2_STAGES = 4;
+constexpr int K2_THREADS = 192;
+constexpr int K2_EPI_THREADS = 128;
+constexpr uint32_t K2_A_BYTES = K2_BM * K2_BK * 2;
+constexpr uint32_t K2_B_BYTES = K2_BN * K2_BK * 2;
+constexpr uint32_t K2_STAGE_BYTES = K2_A_BYTES + K2_B_BYTES;
+constexpr uint32_t K2_TMEM_COLS = 512;
+constexpr int K2_GROUP_M = 16;      // row tiles per rasterisation group (keeps a wave's operands in L2)
+
+struct K2Smem {
+    uint64_t full[K2_STAGES];
+    uint64_t empty[K2_STAGES];
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint32_t tmem_base;
+    int last_flag;
+    int abort_flag;
+    float bias[2][K2_BN];
+};
+constexpr size_t K2_SMEM_BYTES = 1024 + (size_t)K2_STAGES * K2_STAGE_BYTES + sizeof(K2Smem);
+
+struct K2Params {
+    const __nv_bfloat16 *b;
+    void *out;
+    int M, N, K;
+    Epilogue e;
+    float *partial;       // [tiles_n][M]
+    unsigned *counters;   // [tiles_m]
+    int *status;
+    int tiles_m, tiles_n, num_kb;
+};
+
+__device__ __forceinline__ void k2_tile_coords(int t, int tiles_m, int tiles_n, int &tm, int &tn)
+{
+    const int group_size = K2_GROUP_M * tiles_n;
+    const int g = t / group_size, r = t - g * group_size;
+    const int gm = min(K2_GROUP_M, tiles_m - g * K2_GROUP_M);
+    tm = g * K2_GROUP_M + r % gm;
+    tn = r / gm;
+}
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(K2_EPI_THREADS) : "memory"); }
+
+__global__ void __launch_bounds__(K2_THREADS, 1)
+k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const K2Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    K2Smem &s = *reinterpret_cast<K2Smem *>(tiles + (size_t)K2_STAGES * K2_STAGE_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = p.tiles_m * p.tiles_n;
+    bool ok = true;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < K2_STAGES; ++i) { ptx::mbar_init(&s.full[i], 1); ptx::mbar_init(&s.empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&s.acc_full[i], 1); ptx::mbar_init(&s.acc_empty[i], 4); }
+        s.abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmX);
+        ptx::prefetch_tmap(&tmW);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(&s.tmem_base, K2_TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = s.tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (ptx::elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                int tm, tn;
+                k2_tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
+                    uint8_t *a = tiles + (size_t)stage * K2_STAGE_BYTES;
+                    ptx::mbar_expect_tx(&s.full[stage], K2_STAGE_BYTES);
+                    ptx::tma_load_2d(a, &tmX, &s.full[stage], kb * K2_BK, tm * K2_BM);
+                    ptx::tma_load_2d(a + K2_A_BYTES, &tmW, &s.full[stage], kb * K2_BK, tn * K2_BN);
+                    if (++stage == K2_STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (ptx::elect_one()) {
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(K2_BM, K2_BN);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                if (!ptx::mbar_wait(&s.acc_empty[acc], acc_phase ^ 1, p.status, SITE_ACC_EMPTY)) { ok = false; break; }
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * K2_BN;
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    if (!ptx::mbar_wait(&s.full[stage], phase, p.status, SITE_TMA_FULL)) { ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint8_t *a = tiles + (size_t)stage * K2_STAGE_BYTES;
+                    const uint64_t adesc = ptx::smem_desc_k_sw128(a);
+                    const uint64_t bdesc = ptx::smem_desc_k_sw128(a + K2_A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < K2_BK / 16; ++k)      // 16 bf16 = 32 bytes = 2 descriptor units
+                        ptx::umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                    ptx::umma_commit(&s.empty[stage]);
+                    if (++stage == K2_STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                ptx::umma_commit(&s.acc_full[acc]);
+                if ((acc ^= 1) == 0) acc_phase ^= 1;
+            }
+        }
+    } else {
+        // ---------------- epilogue ----------------
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int et = threadIdx.x - 64;              // 0..127
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+            int tm, tn;
+            k2_tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
+            const int m0 = tm * K2_BM, n0 = tn * K2_BN;
+            // bias of this tile -> shared memory (fp32), two values per thread
+            for (int j = et; j < K2_BN; j += K2_EPI_THREADS)
+                s.bias[acc][j] = (p.e.has_bias && n0 + j < p.N) ? __bfloat162float(p.b[n0 + j]) : 0.f;
+            // the give-up decision must be taken by all 128 epilogue threads together
+            if (!ptx::mbar_wait(&s.acc_full[acc], acc_phase, p.status, SITE_ACC_FULL)) s.abort_flag = 1;
+            epi_bar_sync();
+            if (*(volatile int *)&s.abort_flag) { ok = false; break; }
+            ptx::tc_fence_after();
+
+            const int row = m0 + q * 32 + lane;
+            const uint32_t taddr = tmem_base + (uint32_t)acc * K2_BN + ((uint32_t)(q * 32) << 16);
+            float red = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY;
+#pragma unroll 1
+            for (int c = 0; c < K2_BN / 32; ++c) {
+                const int col0 = n0 + c * 32;
+                if (col0 >= p.N) break;
+                uint32_t r[32];
+                ptx::tmem_ld_32x32(taddr + c * 32, r);
+                ptx::tmem_ld_wait();
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + s.bias[acc][c * 32 + j];
+                apply_act_array<false>(p.e.act, v, p.e.scale);
+                if (reduce) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (col0 + j < p.N) red = p.e.red == FORGE_RED_SUM ? red + v[j] : fmaxf(red, v[j]);
+                } else if (row < p.M) {
+                    __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)row * p.N + col0;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if (col0 + i * 8 < p.N) {
+                            uint4 w;
+                            w.x = ptx::pack_bf16x2(v[i * 8 + 0], v[i * 8 + 1]);
+                            w.y = ptx::pack_bf16x2(v[i * 8 + 2], v[i * 8 + 3]);
+                            w.z = ptx::pack_bf16x2(v[i * 8 + 4], v[i * 8 + 5]);
+                            w.w = ptx::pack_bf16x2(v[i * 8 + 6], v[i * 8 + 7]);
+                            *reinterpret_cast<uint4 *>(dst + i * 8) = w;
+                        }
+                    }
+                }
+            }
+            // accumulator drained: hand the TMEM buffer back to the MMA warp
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&s.acc_empty[acc]);
+
+            if (reduce) {
+                float *out = reinterpret_cast<float *>(p.out);
+                if (p.tiles_n == 1) {
+                    if (row < p.M) out[row] = red;
+                } else {
+                    if (row < p.M) p.partial[(size_t)tn * p.M + row] = red;
+                    __threadfence();
+                    epi_bar_sync();
+                    if (et == 0) s.last_flag = (atomicAdd(&p.counters[tm], 1u) == (unsigned)(p.tiles_n - 1));
+                    epi_bar_sync();
+                    if (s.last_flag) {
+                        __threadfence();
+                        if (row < p.M) {
+                            float v = __ldcg(&p.partial[row]);
+                            for (int i = 1; i < p.tiles_n; ++i) {
+                                const float o = __ldcg(&p.partial[(size_t)i * p.M + row]);
+                                v = p.e.red == FORGE_RED_SUM ? v + o : fmaxf(v, o);
+                            }
+                            out[row] = v;
+                        }
+                        if (et == 0) p.counters[tm] = 0u;
+                    }
+                }
+            }
+            if ((acc ^= 1) == 0) acc_phase ^= 1;
+        }
+    }
+
+    // ---------------- teardown ----------------
+    if (!ok) __nanosleep(200000);      // give-up path: let copies and MMAs already in flight land
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, K2_TMEM_COLS);
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
+{
+    if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    const int64_t tiles_m = (d.M + K2_BM - 1) / K2_BM, tiles_n = (d.N + K2_BN - 1) / K2_BN;
+    if (tiles_m * tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    info->kernel = FORGE_KERNEL_BF16_TCGEN05;
+    info->tile_m = K2_BM;
+    info->tile_n = K2_BN;
+    info->tile_k = K2_BK;
+    info->stages = K2_STAGES;
+    info->cluster = 1;
+    info->threads = K2_THREADS;
+    info->grid = tiles_m * tiles_n < sm_count ? tiles_m * tiles_n : sm_count;
+    info->smem_bytes = (int64_t)K2_SMEM_BYTES;
+    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) && tiles_n > 1;
+    wl->partial_floats = partials ? (size_t)tiles_n * (size_t)d.M : 0;
+    wl->counters = partials ? (size_t)tiles_m : 0;
+    return FORGE_OK;
+}
+
+forge_status_t k2_setup(Handle &)
+{
+    return cudaFuncSetAttribute(k2_bf16_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES) == cudaSuccess
+               ? FORGE_OK : FORGE_ERR_CUDA;
+}
+
+forge_status_t k2_launch(Handle &h, const RunArgs &a)
+{
+    const forge_fused_linear_desc_t &d = h.d;
+    forge_status_t st;
+    if (h.tmX_ptr != a.X) {
+        if ((st = encode_tmap_bf16(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, K2_BM, K2_BK)) != FORGE_OK) return st;
+        h.tmX_ptr = a.X;
+    }
+    if (h.tmW_ptr != a.W) {
+        if ((st = encode_tmap_bf16(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, K2_BN, K2_BK)) != FORGE_OK) return st;
+        h.tmW_ptr = a.W;
+    }
+    K2Params p;
+    p.b = (const __nv_bfloat16 *)a.b;
+    p.out = a.out;
+    p.M = (int)d.M;
+    p.N = (int)d.N;
+    p.K = (int)d.K;
+    p.e = Epilogue{(int)d.act, (int)d.red, d.scale, d.ln_eps, d.has_bias};
+    p.partial = h.ws.partial;
+    p.counters = h.ws.counters;
+    p.status = h.ws.status;
+    p.tiles_m = (int)((d.M + K2_BM - 1) / K2_BM);
+    p.tiles_n = (int)((d.N + K2_BN - 1) / K2_BN);
+    p.num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
+    k2_bf16_tcgen05_kernel<<<(unsigned)h.info.grid, K2_THREADS, K2_SMEM_BYTES, a.stream>>>(h.tmX, h.tmW, p);
+    return cudaGetLastError() == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+}
+
+}  // namespace forge

@@ -1,0 +1,99 @@
+"""GPU parity of the bf16 tcgen05 path (TMA -> shared-memory ring -> tcgen05.mma -> TMEM ->
+fused epilogue) against the CPU oracle."""
+import numpy as np
+import pytest
+
+from paper_2511_01884_b200 import binding as B
+from paper_2511_01884_b200 import workloads as wk
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+ACTS = [wk.ACT_IDENTITY, wk.ACT_RELU, wk.ACT_GELU_ERF, wk.ACT_GELU_TANH, wk.ACT_SILU]
+
+
+def _case(M, N, K, act, red, seed=0, scale=1.0, has_bias=True):
+    return wk.custom_workload(f"bf16_{M}x{N}x{K}", wk.BF16, M, N, K, act, red, scale=scale, seed=seed,
+                              has_bias=has_bias)
+
+
+def test_one_tile_one_k_block_identity_weight():
+    """W = I (N = K = 64 padded into one 256-wide tile): Y must reproduce bf16(X) exactly --
+    any mistake in the shared-memory / instruction descriptors or the swizzle shows here."""
+    wl = _case(128, 64, 64, wk.ACT_IDENTITY, wk.RED_NONE, has_bias=False)
+    inp = wk.make_inputs(wl)
+    inp["W"] = np.eye(64, dtype=np.float32)
+    g, plan = pu.run_gpu(wl, inp)
+    assert plan["kernel"] == B.FORGE_KERNEL_BF16_TCGEN05
+    assert np.array_equal(g, inp["X"].astype(np.float64))
+
+
+def test_k_steps_inside_and_across_swizzle_atoms():
+    for K in (16, 32, 64, 128, 136, 512):
+        wl = _case(128, 256, K, wk.ACT_IDENTITY, wk.RED_NONE, seed=K)
+        inp = wk.make_inputs(wl)
+        g, _ = pu.run_gpu(wl, inp)
+        pu.assert_parity(wl, g, pu.run_oracle(wl, inp), f"K={K}")
+
+
+SHAPES = [(17, 8, 8), (128, 256, 64), (129, 264, 72), (300, 520, 200), (1000, 776, 328), (2048, 1024, 512)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("red", [wk.RED_NONE, wk.RED_SUM, wk.RED_MAX])
+def test_shapes_and_reductions(M, N, K, red):
+    act = ACTS[(M + N + K + red) % len(ACTS)]
+    wl = _case(M, N, K, act, red, seed=M + K, scale=0.75)
+    inp = wk.make_inputs(wl)
+    g, _ = pu.run_gpu(wl, inp)
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp), f"act={act} red={red}")
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_every_activation(act):
+    wl = _case(256, 512, 128, act, wk.RED_NONE, seed=act, scale=1.25)
+    inp = wk.make_inputs(wl)
+    inp["W"] = wk.round_to_storage(inp["W"] * 4.0, wk.BF16)
+    g, _ = pu.run_gpu(wl, inp)
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_more_tiles_than_sms_and_both_accumulator_buffers():
+    wl = _case(128 * 20, 256 * 9, 192, wk.ACT_SILU, wk.RED_NONE, seed=5)      # 180 tiles on 148 CTAs
+    inp = wk.make_inputs(wl)
+    g, plan = pu.run_gpu(wl, inp)
+    assert plan["grid"] <= 148
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_freivalds_covers_every_output_element():
+    wl = _case(1536, 1280, 640, wk.ACT_IDENTITY, wk.RED_NONE, seed=2)
+    inp = wk.make_inputs(wl)
+    g, _ = pu.run_gpu(wl, inp)
+    rng = np.random.default_rng(0)
+    r = rng.standard_normal(wl.N)
+    want = inp["X"].astype(np.float64) @ (inp["W"].astype(np.float64).T @ r) + inp["b"].astype(np.float64) @ r
+    # bf16 rounding of each output (2^-9 relative) averages out over N terms
+    assert np.max(np.abs(g @ r - want)) <= 2e-2 * np.sqrt(np.mean(want * want))
+
+
+def test_repeatable_bits_and_workspace_reuse():
+    wl = _case(700, 1304, 256, wk.ACT_GELU_TANH, wk.RED_MAX, seed=3)
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op)
+    b, _ = pu.run_gpu(wl, inp, op=op)
+    op.close()
+    assert np.array_equal(a, b)
+    pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
+
+
+def test_c3_sampled_rows_full_size():
+    wl = wk.WORKLOADS["c3"]
+    inp = wk.make_inputs(wl)
+    g, plan = pu.run_gpu(wl, inp)
+    assert plan["kernel"] == B.FORGE_KERNEL_BF16_TCGEN05
+    assert np.isfinite(g).all()
+    rows = wk.sample_rows(wl.M)
+    pu.assert_parity(wl, g[rows], pu.run_oracle(wl, inp, rows))
