@@ -237,6 +237,7 @@ forge_status_t forge_fused_linear_last_status(forge_fused_linear_t hh)
     if (word != 0) {
         // a give-up may have left arrival counters half way: clear the whole workspace
         cudaMemset(h.ws.base, 0, h.ws.bytes);
+        h.run_gen = 0;
         return (forge_status_t)(word >> 16);
     }
     return FORGE_OK;
@@ -283,7 +284,7 @@ const char *forge_kernel_name(forge_kernel_t k)
     case FORGE_KERNEL_F32_FFMA: return "f32_ffma_128x128x16";
     case FORGE_KERNEL_BF16_TCGEN05: return "bf16_tcgen05_tma";
     case FORGE_KERNEL_BF16_SKINNY: return "bf16_skinny_splitk";
-    case FORGE_KERNEL_BF16_TCGEN05_LN: return "bf16_tcgen05_cluster_layernorm";
+    case FORGE_KERNEL_BF16_TCGEN05_LN: return "bf16_tcgen05_tma_layernorm";
     }
     return "unknown kernel";
 }

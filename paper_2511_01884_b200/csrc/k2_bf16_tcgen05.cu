@@ -9,6 +9,17 @@
 //               activation, scale, then either bf16 stores of Y or the row sum / max.
 // TMEM holds two 128x256 fp32 accumulators, so the epilogue of tile i overlaps the MMAs of
 // tile i+1.  No load is multicast; every wait is bounded (see ptx::mbar_wait).
+//
+// K4 (LayerNorm over N) is the same kernel with a different tile order and epilogue: the
+// N-tiles of one 128-row strip are consecutive tiles, hence run on different SMs at about
+// the same time.  Each epilogue makes one sweep over its accumulator (bias, activation,
+// scale, per-row (n, mean, M2) of its 256 columns, activated values written back to TMEM),
+// publishes the row triples to a small workspace, waits -- bounded -- until the strip's
+// other tiles have published theirs, merges the triples in tile order (Chan et al.), and
+// makes a second sweep over TMEM to normalise and store.  Only the 16-byte triples travel
+// through global memory; the un-normalised tile never leaves the SM.  The wait is hidden
+// behind the MMAs of the next tile (other TMEM buffer).  CTAs wait on one another, so the
+// launch is cooperative and a strip may not have more tiles than there are CTAs.
 #include "common.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
@@ -33,6 +44,8 @@ struct K2Smem {
     int last_flag;
     int abort_flag;
     float bias[2][K2_BN];
+    float gamma[2][K2_BN];
+    float beta[2][K2_BN];
 };
 constexpr size_t K2_SMEM_BYTES = 1024 + (size_t)K2_STAGES * K2_STAGE_BYTES + sizeof(K2Smem);
 
@@ -41,14 +54,22 @@ struct K2Params {
     void *out;
     int M, N, K;
     Epilogue e;
-    float *partial;       // [tiles_n][M]
+    const __nv_bfloat16 *gamma, *beta;
+    float *partial;       // sum/max: [tiles_n][M] floats; layernorm: [tiles_n][M] float4 triples
     unsigned *counters;   // [tiles_m]
     int *status;
     int tiles_m, tiles_n, num_kb;
+    unsigned ln_target;   // layernorm: counter value at which a strip is complete in this run
 };
 
+template <bool LN>
 __device__ __forceinline__ void k2_tile_coords(int t, int tiles_m, int tiles_n, int &tm, int &tn)
 {
+    if (LN) {            // a strip's N-tiles are neighbours in the schedule
+        tm = t / tiles_n;
+        tn = t - tm * tiles_n;
+        return;
+    }
     const int group_size = K2_GROUP_M * tiles_n;
     const int g = t / group_size, r = t - g * group_size;
     const int gm = min(K2_GROUP_M, tiles_m - g * K2_GROUP_M);
@@ -58,6 +79,14 @@ __device__ __forceinline__ void k2_tile_coords(int t, int tiles_m, int tiles_n, 
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(K2_EPI_THREADS) : "memory"); }
 
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+template <bool LN>
 __global__ void __launch_bounds__(K2_THREADS, 1)
 k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const K2Params p)
 {
@@ -93,7 +122,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             uint32_t phase = 0;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 int tm, tn;
-                k2_tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
+                k2_tile_coords<LN>(t, p.tiles_m, p.tiles_n, tm, tn);
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
                     uint8_t *a = tiles + (size_t)stage * K2_STAGE_BYTES;
@@ -140,11 +169,18 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             int tm, tn;
-            k2_tile_coords(t, p.tiles_m, p.tiles_n, tm, tn);
+            k2_tile_coords<LN>(t, p.tiles_m, p.tiles_n, tm, tn);
             const int m0 = tm * K2_BM, n0 = tn * K2_BN;
             // bias of this tile -> shared memory (fp32), two values per thread
             for (int j = et; j < K2_BN; j += K2_EPI_THREADS)
                 s.bias[acc][j] = (p.e.has_bias && n0 + j < p.N) ? __bfloat162float(p.b[n0 + j]) : 0.f;
+            if (LN) {
+                for (int j = et; j < K2_BN; j += K2_EPI_THREADS) {
+                    const bool in = n0 + j < p.N;
+                    s.gamma[acc][j] = in ? __bfloat162float(p.gamma[n0 + j]) : 0.f;
+                    s.beta[acc][j] = in ? __bfloat162float(p.beta[n0 + j]) : 0.f;
+                }
+            }
             // the give-up decision must be taken by all 128 epilogue threads together
             if (!ptx::mbar_wait(&s.acc_full[acc], acc_phase, p.status, SITE_ACC_FULL)) s.abort_flag = 1;
             epi_bar_sync();
@@ -153,6 +189,108 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 
             const int row = m0 + q * 32 + lane;
             const uint32_t taddr = tmem_base + (uint32_t)acc * K2_BN + ((uint32_t)(q * 32) << 16);
+
+            if (LN) {
+                // ---- sweep 1: activated values back to TMEM, row statistics of this tile ----
+                RowStat rs{0.f, 0.f, 0.f};
+#pragma unroll 1
+                for (int c = 0; c < K2_BN / 32; ++c) {
+                    const int col0 = n0 + c * 32;
+                    if (col0 >= p.N) break;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(taddr + c * 32, r);
+                    ptx::tmem_ld_wait();
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + s.bias[acc][c * 32 + j];
+                    apply_act_array<false>(p.e.act, v, p.e.scale);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(v[j]);
+                    ptx::tmem_st_32x32(taddr + c * 32, r);
+                    const int nv = min(32, p.N - col0);
+                    float sum = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) sum += j < nv ? v[j] : 0.f;
+                    RowStat cs;
+                    cs.n = (float)nv;
+                    cs.mean = sum / cs.n;
+                    cs.m2 = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float dlt = j < nv ? v[j] - cs.mean : 0.f;
+                        cs.m2 = fmaf(dlt, dlt, cs.m2);
+                    }
+                    rs = merge_stat(rs, cs);
+                }
+                ptx::tmem_st_wait();
+                float4 *stats = reinterpret_cast<float4 *>(p.partial);
+                if (row < p.M) stats[(size_t)tn * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
+                // ---- publish, then wait (bounded) for the other tiles of this strip ----
+                __threadfence();
+                epi_bar_sync();
+                if (et == 0) {
+                    atomicAdd(&p.counters[tm], 1u);
+                    uint64_t t0 = 0;
+                    for (uint32_t it = 1; (int)(ld_acquire_u32(&p.counters[tm]) - p.ln_target) < 0; ++it) {
+                        if ((it & 0xff) == 0) {
+                            if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
+                            const uint64_t now = ptx::globaltimer_ns();
+                            if (t0 == 0) t0 = now;
+                            else if (now - t0 > ptx::kWaitBudgetNs) {
+                                report_timeout(p.status, SITE_ARRIVAL);
+                                s.abort_flag = 1;
+                                break;
+                            }
+                        }
+                    }
+                }
+                epi_bar_sync();
+                if (*(volatile int *)&s.abort_flag) { ok = false; break; }
+                __threadfence();
+                if (row < p.M) {
+                    const float4 f = __ldcg(&stats[row]);
+                    rs = RowStat{f.x, f.y, f.z};
+                    for (int i = 1; i < p.tiles_n; ++i) {
+                        const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
+                        rs = merge_stat(rs, RowStat{o.x, o.y, o.z});
+                    }
+                }
+                const float mean = rs.mean, rstd = rsqrtf(rs.m2 / rs.n + p.e.eps);
+                // ---- sweep 2: normalise out of TMEM and store ----
+#pragma unroll 1
+                for (int c = 0; c < K2_BN / 32; ++c) {
+                    const int col0 = n0 + c * 32;
+                    if (col0 >= p.N) break;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(taddr + c * 32, r);
+                    ptx::tmem_ld_wait();
+                    if (row < p.M) {
+                        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)row * p.N + col0;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            if (col0 + i * 8 < p.N) {
+                                float y[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    const int cc = c * 32 + i * 8 + j;
+                                    y[j] = fmaf((__uint_as_float(r[i * 8 + j]) - mean) * rstd, s.gamma[acc][cc], s.beta[acc][cc]);
+                                }
+                                uint4 w;
+                                w.x = ptx::pack_bf16x2(y[0], y[1]);
+                                w.y = ptx::pack_bf16x2(y[2], y[3]);
+                                w.z = ptx::pack_bf16x2(y[4], y[5]);
+                                w.w = ptx::pack_bf16x2(y[6], y[7]);
+                                *reinterpret_cast<uint4 *>(dst + i * 8) = w;
+                            }
+                        }
+                    }
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&s.acc_empty[acc]);
+                if ((acc ^= 1) == 0) acc_phase ^= 1;
+                continue;
+            }
             float red = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY;
 #pragma unroll 1
             for (int c = 0; c < K2_BN / 32; ++c) {
@@ -250,11 +388,36 @@ forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
 
 forge_status_t k2_setup(Handle &)
 {
-    return cudaFuncSetAttribute(k2_bf16_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES) == cudaSuccess
+    return cudaFuncSetAttribute(k2_bf16_tcgen05_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES) == cudaSuccess
                ? FORGE_OK : FORGE_ERR_CUDA;
 }
 
-forge_status_t k2_launch(Handle &h, const RunArgs &a)
+forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
+{
+    const forge_status_t st = k2_plan(d, sm_count, info, wl);
+    if (st != FORGE_OK) return st;
+    const int64_t tiles_m = (d.M + K2_BM - 1) / K2_BM, tiles_n = (d.N + K2_BN - 1) / K2_BN;
+    // the tiles of a strip wait for one another: they must all be resident at once
+    if (tiles_n > sm_count) return FORGE_ERR_UNSUPPORTED;
+    info->kernel = FORGE_KERNEL_BF16_TCGEN05_LN;
+    wl->partial_floats = 4 * (size_t)tiles_n * (size_t)d.M;
+    wl->counters = (size_t)tiles_m;
+    return FORGE_OK;
+}
+
+forge_status_t k4_setup(Handle &h)
+{
+    if (cudaFuncSetAttribute(k2_bf16_tcgen05_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES) != cudaSuccess)
+        return FORGE_ERR_CUDA;
+    int coop = 0, per_sm = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h.d.device) != cudaSuccess || !coop) return FORGE_ERR_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2_bf16_tcgen05_kernel<true>, K2_THREADS, K2_SMEM_BYTES) != cudaSuccess ||
+        (int64_t)per_sm * h.sm_count < h.info.grid)
+        return FORGE_ERR_CUDA;
+    return FORGE_OK;
+}
+
+static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
 {
     const forge_fused_linear_desc_t &d = h.d;
     forge_status_t st;
@@ -268,6 +431,8 @@ forge_status_t k2_launch(Handle &h, const RunArgs &a)
     }
     K2Params p;
     p.b = (const __nv_bfloat16 *)a.b;
+    p.gamma = (const __nv_bfloat16 *)a.gamma;
+    p.beta = (const __nv_bfloat16 *)a.beta;
     p.out = a.out;
     p.M = (int)d.M;
     p.N = (int)d.N;
@@ -279,8 +444,20 @@ forge_status_t k2_launch(Handle &h, const RunArgs &a)
     p.tiles_m = (int)((d.M + K2_BM - 1) / K2_BM);
     p.tiles_n = (int)((d.N + K2_BN - 1) / K2_BN);
     p.num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
-    k2_bf16_tcgen05_kernel<<<(unsigned)h.info.grid, K2_THREADS, K2_SMEM_BYTES, a.stream>>>(h.tmX, h.tmW, p);
-    return cudaGetLastError() == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+    p.ln_target = 0;
+    if (!ln) {
+        k2_bf16_tcgen05_kernel<false><<<(unsigned)h.info.grid, K2_THREADS, K2_SMEM_BYTES, a.stream>>>(h.tmX, h.tmW, p);
+        return cudaGetLastError() == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+    }
+    // Strip counters only ever grow: run r completes a strip at r * tiles_n arrivals.
+    h.run_gen += 1;
+    p.ln_target = h.run_gen * (unsigned)p.tiles_n;
+    void *args[] = {(void *)&h.tmX, (void *)&h.tmW, (void *)&p};
+    return cudaLaunchCooperativeKernel((const void *)k2_bf16_tcgen05_kernel<true>, dim3((unsigned)h.info.grid), dim3(K2_THREADS),
+                                       args, K2_SMEM_BYTES, a.stream) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
 }
+
+forge_status_t k2_launch(Handle &h, const RunArgs &a) { return k24_launch(h, a, false); }
+forge_status_t k4_launch(Handle &h, const RunArgs &a) { return k24_launch(h, a, true); }
 
 }  // namespace forge

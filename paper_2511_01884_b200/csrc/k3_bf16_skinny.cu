@@ -1,0 +1,330 @@
+// K3: bf16 fused linear for M <= 16 (HBM-bound: the weight matrix is read once and that is
+// the whole cost).
+//
+// Each CTA owns a contiguous range of 8-column groups of the output (8 rows of W per group)
+// sized so that all CTAs stream the same number of bytes.  A producer warp streams W (and
+// the matching slice of X, which stays L2-resident) through a 10-stage TMA ring; 8 consumer
+// warps feed the tiles to mma.sync.m16n8k16 straight from shared memory (ldmatrix on the
+// 128-byte-swizzled layout).  The warps split the work 2 (halves of the strip's columns) x
+// 4 (K: ring stages are dealt round-robin), so the partial accumulators of the 4 K-slices
+// are summed -- before bias and activation, which are nonlinear -- through shared memory in
+// a fixed order.  Row sum / max: two shuffles inside the 4-lane groups that share a row,
+// then per-CTA partials folded by the CTA that arrives last.
+//
+// Every thread of the CTA stays resident until the common exit barrier, so that no copy can
+// still be in flight towards the shared memory of a CTA that has left.
+#include "common.cuh"
+#include "plan.h"
+#include "sm100_ptx.cuh"
+
+namespace forge {
+
+constexpr int K3_BK = 64;                       // k per stage: one 128-byte swizzle row
+constexpr int K3_MAX_GROUPS = 16;               // 8-column groups per strip (128 rows of W)
+constexpr int K3_STAGES = 10;
+constexpr int K3_KSPLIT = 4, K3_NSPLIT = 2;
+constexpr int K3_CONSUMER_WARPS = K3_KSPLIT * K3_NSPLIT;
+constexpr int K3_CONSUMERS = K3_CONSUMER_WARPS * 32;
+constexpr int K3_THREADS = K3_CONSUMERS + 32;
+constexpr uint32_t K3_W_BYTES = K3_MAX_GROUPS * 8 * K3_BK * 2;     // 16 KiB (full strip)
+constexpr uint32_t K3_X_BYTES = 16 * K3_BK * 2;                    // 2 KiB
+constexpr uint32_t K3_STAGE_BYTES = K3_W_BYTES + K3_X_BYTES;
+constexpr int K3_GH = K3_MAX_GROUPS / K3_NSPLIT;                   // groups per column half
+
+struct K3Smem {
+    uint64_t full[K3_STAGES];
+    uint64_t empty[K3_STAGES];
+    float4 red[K3_KSPLIT][K3_MAX_GROUPS][32];    // partial accumulators of the K-slices
+    float rowred[K3_MAX_GROUPS][16];
+    int last_flag;
+    int abort_flag;
+};
+constexpr size_t K3_SMEM_BYTES = 1024 + (size_t)K3_STAGES * K3_STAGE_BYTES + sizeof(K3Smem);
+
+struct K3Params {
+    const __nv_bfloat16 *b;
+    void *out;
+    int M, N, K;
+    Epilogue e;
+    float *partial;       // [grid][16]
+    unsigned *counters;   // [1]
+    int *status;
+    int num_kb;
+    int groups;           // N / 8
+    int box_groups;       // groups per strip = rows of the W box / 8
+};
+
+// Debug build (-DFORGE_DEBUG_BOUNDS): indices are range-checked; a bad one is recorded in the
+// status word as (0x7f << 16 | site) and the access is skipped.
+#ifdef FORGE_DEBUG_BOUNDS
+#define K3_INRANGE(cond, site) ((cond) ? true : (atomicCAS(p.status, 0, (0x7f << 16) | (site)), false))
+#else
+#define K3_INRANGE(cond, site) true
+#endif
+
+__device__ __forceinline__ void k3_consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(K3_CONSUMERS) : "memory"); }
+
+__global__ void __launch_bounds__(K3_THREADS, 1)
+k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const K3Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    K3Smem &s = *reinterpret_cast<K3Smem *>(ring + (size_t)K3_STAGES * K3_STAGE_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // this CTA's share of the column groups, and its strips
+    const int g_lo = (int)((long long)p.groups * blockIdx.x / gridDim.x);
+    const int g_hi = (int)((long long)p.groups * (blockIdx.x + 1) / gridDim.x);
+    const int strips = (g_hi - g_lo + p.box_groups - 1) / p.box_groups;
+    const uint32_t stage_tx = (uint32_t)p.box_groups * 8 * K3_BK * 2 + K3_X_BYTES;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < K3_STAGES; ++i) { ptx::mbar_init(&s.full[i], 1); ptx::mbar_init(&s.empty[i], K3_NSPLIT); }
+        s.abort_flag = 0;
+        s.last_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmX);
+        ptx::prefetch_tmap(&tmW);
+    }
+    __syncthreads();
+
+    if (warp == K3_CONSUMER_WARPS) {
+        // ---------------- TMA producer ----------------
+        if (ptx::elect_one()) {
+            int slot = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int st = 0; st < strips && ok; ++st) {
+                const int row0 = (g_lo + st * p.box_groups) * 8;
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    if (!ptx::mbar_wait(&s.empty[slot], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
+                    if (!K3_INRANGE(row0 >= 0 && row0 < p.N && kb * K3_BK < p.K, 1)) { ok = false; break; }
+                    uint8_t *dst = ring + (size_t)slot * K3_STAGE_BYTES;
+                    ptx::mbar_expect_tx(&s.full[slot], stage_tx);
+                    ptx::tma_load_2d(dst, &tmW, &s.full[slot], kb * K3_BK, row0);
+                    ptx::tma_load_2d(dst + K3_W_BYTES, &tmX, &s.full[slot], kb * K3_BK, 0);
+                    if (++slot == K3_STAGES) { slot = 0; phase ^= 1; }
+                }
+            }
+            if (!ok) s.abort_flag = 1;
+        }
+    } else {
+        // ---------------- consumers ----------------
+        const int nh = warp & 1;            // which half of the strip's groups
+        const int ks = warp >> 1;           // which K-slice (ring stages with index % 4 == ks)
+        const int t = threadIdx.x;          // 0..255
+        const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX;
+        bool ok = true;
+        float running = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY;     // threads 0..15: row t
+
+        // ldmatrix lane addressing on the 128-byte-swizzled tiles (16-byte chunk c of row r
+        // sits at r*128 + ((c ^ (r & 7)) << 4)).
+        const int lm = lane >> 3, lr = lane & 7;
+        const int a_row = (lm & 1) * 8 + lr, a_chunk = lm >> 1;     // X: (r0-7,k0-7) (r8-15,k0-7) (r0-7,k8-15) (r8-15,k8-15)
+        const int b_row = (lm >> 1) * 8 + lr, b_chunk = lm & 1;     // W: (g,k0-7) (g,k8-15) (g+1,k0-7) (g+1,k8-15)
+
+        // ring position of the next stage this warp consumes: sequence index, slot and phase
+        int seq = ks, slot = ks;
+        uint32_t phase = 0;
+        int seq_end = 0;                    // first sequence index past the current strip
+
+        for (int st = 0; st < strips; ++st) {
+            seq_end += p.num_kb;
+            const int gbase = g_lo + st * p.box_groups;
+            const int ng = min(p.box_groups, p.groups - gbase);      // groups present in this strip's box
+            float acc[K3_GH][4];
+#pragma unroll
+            for (int g = 0; g < K3_GH; ++g) acc[g][0] = acc[g][1] = acc[g][2] = acc[g][3] = 0.f;
+
+            for (; seq < seq_end; seq += K3_KSPLIT) {
+                if (ok && !ptx::mbar_wait(&s.full[slot], phase, p.status, SITE_TMA_FULL)) ok = false;
+                if (ok) {
+                    const uint32_t wbase = ptx::smem_u32(ring + (size_t)slot * K3_STAGE_BYTES);
+                    const uint32_t xbase = wbase + K3_W_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < K3_BK / 16; ++kk) {
+                        uint32_t a[4];
+                        ptx::ldmatrix_x4(a, xbase + a_row * 128 + (((2 * kk + a_chunk) ^ (a_row & 7)) << 4));
+#pragma unroll
+                        for (int gp = 0; gp < K3_GH / 2; ++gp) {
+                            const int g0 = nh * K3_GH + gp * 2;
+                            if (g0 < ng) {
+                                uint32_t b[4];
+                                const int r = g0 * 8 + b_row;
+                                ptx::ldmatrix_x4(b, wbase + r * 128 + (((2 * kk + b_chunk) ^ (r & 7)) << 4));
+                                ptx::mma_m16n8k16_bf16(acc[gp * 2], a, b[0], b[1]);
+                                ptx::mma_m16n8k16_bf16(acc[gp * 2 + 1], a, b[2], b[3]);
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&s.empty[slot]);
+                }
+                slot += K3_KSPLIT;
+                if (slot >= K3_STAGES) { slot -= K3_STAGES; phase ^= 1; }
+            }
+
+            // ---- sum the K-slices (fixed order), then the epilogue on the full pre-activations
+#pragma unroll
+            for (int g = 0; g < K3_GH; ++g)
+                s.red[ks][nh * K3_GH + g][lane] = make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]);
+            k3_consumer_sync();
+
+#pragma unroll
+            for (int j = 0; j < K3_MAX_GROUPS * 32 / K3_CONSUMERS; ++j) {
+                const int g = warp + j * K3_CONSUMER_WARPS;        // fragment lane == this thread's lane
+                float4 z = s.red[0][g][lane];
+#pragma unroll
+                for (int k = 1; k < K3_KSPLIT; ++k) {
+                    const float4 o = s.red[k][g][lane];
+                    z.x += o.x; z.y += o.y; z.z += o.z; z.w += o.w;
+                }
+                const int col = (gbase + g) * 8 + (lane & 3) * 2;
+                const bool live = g < ng && gbase + g < g_hi && col + 1 < p.N;   // in the box, in this CTA's share
+                float b0 = 0.f, b1 = 0.f;
+                if (live && p.e.has_bias) {
+                    const __nv_bfloat162 bb = *reinterpret_cast<const __nv_bfloat162 *>(p.b + col);
+                    b0 = __low2float(bb);
+                    b1 = __high2float(bb);
+                }
+                float v[4] = {z.x + b0, z.y + b1, z.z + b0, z.w + b1};
+                apply_act_array<false>(p.e.act, v, p.e.scale);
+                const int r0 = lane >> 2, r1 = r0 + 8;
+                if (reduce) {
+                    float m0, m1;
+                    if (p.e.red == FORGE_RED_SUM) {
+                        m0 = live ? v[0] + v[1] : 0.f;
+                        m1 = live ? v[2] + v[3] : 0.f;
+                        m0 += __shfl_xor_sync(0xffffffffu, m0, 1);
+                        m1 += __shfl_xor_sync(0xffffffffu, m1, 1);
+                        m0 += __shfl_xor_sync(0xffffffffu, m0, 2);
+                        m1 += __shfl_xor_sync(0xffffffffu, m1, 2);
+                    } else {
+                        m0 = live ? fmaxf(v[0], v[1]) : -INFINITY;
+                        m1 = live ? fmaxf(v[2], v[3]) : -INFINITY;
+                        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
+                        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
+                        m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+                        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+                    }
+                    if ((lane & 3) == 0) {
+                        s.rowred[g][r0] = m0;
+                        s.rowred[g][r1] = m1;
+                    }
+                } else if (live) {
+                    __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(p.out);
+                    if (r0 < p.M) *reinterpret_cast<uint32_t *>(Y + (size_t)r0 * p.N + col) = ptx::pack_bf16x2(v[0], v[1]);
+                    if (r1 < p.M) *reinterpret_cast<uint32_t *>(Y + (size_t)r1 * p.N + col) = ptx::pack_bf16x2(v[2], v[3]);
+                }
+            }
+            k3_consumer_sync();
+            if (reduce && t < 16) {
+                for (int g = 0; g < K3_MAX_GROUPS; ++g) {
+                    const float o = s.rowred[g][t];
+                    running = p.e.red == FORGE_RED_SUM ? running + o : fmaxf(running, o);
+                }
+            }
+        }
+        if (!ok) s.abort_flag = 1;
+
+        // ---- fold the CTAs' partials: the last CTA to arrive does it, in CTA order ----
+        if (reduce) {
+            float *out = reinterpret_cast<float *>(p.out);
+            if (gridDim.x == 1) {
+                if (t < p.M) out[t] = running;
+            } else {
+                if (t < 16) p.partial[(size_t)blockIdx.x * 16 + t] = running;
+                __threadfence();
+                k3_consumer_sync();
+                if (t == 0) s.last_flag = (atomicAdd(&p.counters[0], 1u) == gridDim.x - 1);
+                k3_consumer_sync();
+                if (s.last_flag) {
+                    __threadfence();
+                    if (t < p.M) {
+                        float v = __ldcg(&p.partial[t]);
+                        for (unsigned c = 1; c < gridDim.x; ++c) {
+                            const float o = __ldcg(&p.partial[(size_t)c * 16 + t]);
+                            v = p.e.red == FORGE_RED_SUM ? v + o : fmaxf(v, o);
+                        }
+                        out[t] = v;
+                    }
+                    if (t == 0) p.counters[0] = 0u;
+                }
+            }
+        }
+    }
+
+    // ---------------- common exit ----------------
+    __syncthreads();
+    // give-up path only: copies already issued may still be landing in this CTA's shared memory
+    if (*(volatile int *)&s.abort_flag) __nanosleep(500000);
+}
+
+// ---- host side ---------------------------------------------------------------------------
+static int k3_grid(const forge_fused_linear_desc_t &d, int sm_count)
+{
+    const int64_t groups = d.N / 8;
+    return (int)(groups < sm_count ? groups : sm_count);
+}
+static int k3_box_groups(const forge_fused_linear_desc_t &d, int grid)
+{
+    const int64_t groups = d.N / 8;
+    const int64_t per_cta = (groups + grid - 1) / grid;
+    return (int)(per_cta < K3_MAX_GROUPS ? per_cta : K3_MAX_GROUPS);
+}
+
+forge_status_t k3_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
+{
+    if (d.M > 16 || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    const int grid = k3_grid(d, sm_count);
+    info->kernel = FORGE_KERNEL_BF16_SKINNY;
+    info->tile_m = 16;
+    info->tile_n = k3_box_groups(d, grid) * 8;
+    info->tile_k = K3_BK;
+    info->stages = K3_STAGES;
+    info->cluster = 1;
+    info->threads = K3_THREADS;
+    info->grid = grid;
+    info->smem_bytes = (int64_t)K3_SMEM_BYTES;
+    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) && grid > 1;
+    wl->partial_floats = partials ? (size_t)grid * 16 : 0;
+    wl->counters = partials ? 1 : 0;
+    return FORGE_OK;
+}
+
+forge_status_t k3_setup(Handle &)
+{
+    return cudaFuncSetAttribute(k3_bf16_skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K3_SMEM_BYTES) == cudaSuccess
+               ? FORGE_OK : FORGE_ERR_CUDA;
+}
+
+forge_status_t k3_launch(Handle &h, const RunArgs &a)
+{
+    const forge_fused_linear_desc_t &d = h.d;
+    forge_status_t st;
+    if (h.tmX_ptr != a.X) {
+        if ((st = encode_tmap_bf16(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, 16, K3_BK)) != FORGE_OK) return st;
+        h.tmX_ptr = a.X;
+    }
+    if (h.tmW_ptr != a.W) {
+        if ((st = encode_tmap_bf16(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, (uint32_t)h.info.tile_n, K3_BK)) != FORGE_OK) return st;
+        h.tmW_ptr = a.W;
+    }
+    K3Params p;
+    p.b = (const __nv_bfloat16 *)a.b;
+    p.out = a.out;
+    p.M = (int)d.M;
+    p.N = (int)d.N;
+    p.K = (int)d.K;
+    p.e = Epilogue{(int)d.act, (int)d.red, d.scale, d.ln_eps, d.has_bias};
+    p.partial = h.ws.partial;
+    p.counters = h.ws.counters;
+    p.status = h.ws.status;
+    p.num_kb = (int)((d.K + K3_BK - 1) / K3_BK);
+    p.groups = (int)(d.N / 8);
+    p.box_groups = h.info.tile_n / 8;
+    k3_bf16_skinny_kernel<<<(unsigned)h.info.grid, K3_THREADS, K3_SMEM_BYTES, a.stream>>>(h.tmX, h.tmW, p);
+    return cudaGetLastError() == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+}
+
+}  // namespace forge

@@ -28,6 +28,7 @@ struct Handle {
     forge_fused_linear_desc_t d;
     forge_plan_info_t info;
     int sm_count = 0;
+    unsigned run_gen = 0;            // runs launched since the workspace was last cleared
     Workspace ws;
     // staging buffers of run_host()
     void *hX = nullptr, *hW = nullptr, *hb = nullptr, *hg = nullptr, *hbe = nullptr, *hout = nullptr;

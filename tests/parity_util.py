@@ -31,8 +31,9 @@ def desc_of(wl: wk.Workload, M=None, device=0):
                        wl.bias.kind != "none", device)
 
 
-def run_gpu(wl: wk.Workload, inp, check_status=True, op=None):
-    """One call through the C interface; returns (float64 numpy result, plan dict)."""
+def run_gpu(wl: wk.Workload, inp, check_status=True, op=None, repeats=1):
+    """``repeats`` calls through the C interface (no synchronisation between them); returns
+    (float64 numpy result of the last one, plan dict)."""
     import torch
     dev = {k: to_device(v, wl.dtype) for k, v in inp.items()}
     M = inp["X"].shape[0]
@@ -44,7 +45,8 @@ def run_gpu(wl: wk.Workload, inp, check_status=True, op=None):
     else:
         out = torch.full((M, wl.N), float("nan"), dtype=torch.float32 if wl.dtype == wk.F32 else torch.bfloat16,
                          device="cuda")
-    op(dev["X"], dev["W"], dev["b"], dev["gamma"], dev["beta"], out)
+    for _ in range(repeats):
+        op(dev["X"], dev["W"], dev["b"], dev["gamma"], dev["beta"], out)
     torch.cuda.synchronize()
     if check_status:
         op.check()

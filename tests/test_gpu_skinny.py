@@ -1,0 +1,72 @@
+"""GPU parity of the skinny-M bf16 path (M <= 16: split-K over warps, mma.sync from a TMA
+ring, warp-shuffle row reductions) against the CPU oracle."""
+import numpy as np
+import pytest
+
+from paper_2511_01884_b200 import binding as B
+from paper_2511_01884_b200 import workloads as wk
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+ACTS = [wk.ACT_IDENTITY, wk.ACT_RELU, wk.ACT_GELU_ERF, wk.ACT_GELU_TANH, wk.ACT_SILU]
+
+
+def _case(M, N, K, act, red, seed=0, scale=1.0, has_bias=True):
+    return wk.custom_workload(f"skinny_{M}x{N}x{K}", wk.BF16, M, N, K, act, red, scale=scale, seed=seed,
+                              has_bias=has_bias)
+
+
+def test_identity_weight_reproduces_x():
+    wl = _case(16, 64, 64, wk.ACT_IDENTITY, wk.RED_NONE, has_bias=False)
+    inp = wk.make_inputs(wl)
+    inp["W"] = np.eye(64, dtype=np.float32)
+    g, plan = pu.run_gpu(wl, inp)
+    assert plan["kernel"] == B.FORGE_KERNEL_BF16_SKINNY
+    assert np.array_equal(g, inp["X"].astype(np.float64))
+
+
+# N/8 below, at and far above the SM count (1, several and many strips per CTA); K with a
+# ragged last block and fewer blocks than K-slices; M below 16
+SHAPES = [(16, 8, 8), (1, 64, 16), (5, 1184, 72), (16, 1192, 200), (16, 4096, 1024), (7, 20000, 264),
+          (16, 148 * 8 * 17, 128), (16, 148 * 8 * 40 + 8, 64)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("red", [wk.RED_NONE, wk.RED_SUM, wk.RED_MAX])
+def test_shapes_and_reductions(M, N, K, red):
+    act = ACTS[(M + N + K + red) % len(ACTS)]
+    wl = _case(M, N, K, act, red, seed=N + K, scale=0.75)
+    inp = wk.make_inputs(wl)
+    g, _ = pu.run_gpu(wl, inp)
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp), f"act={act} red={red}")
+
+
+def test_all_negative_rows_keep_their_maximum():
+    wl = _case(16, 2048, 128, wk.ACT_IDENTITY, wk.RED_MAX, has_bias=False, seed=8)
+    inp = wk.make_inputs(wl)
+    inp["X"] = -np.abs(inp["X"])
+    inp["W"] = np.abs(inp["W"])
+    g, _ = pu.run_gpu(wl, inp)
+    assert (g < 0).all()
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_repeatable_bits_and_back_to_back_runs():
+    wl = _case(16, 8192, 512, wk.ACT_SILU, wk.RED_SUM, seed=3)
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op)
+    b, _ = pu.run_gpu(wl, inp, op=op, repeats=4)      # four launches with no synchronisation between them
+    op.close()
+    assert np.array_equal(a, b)
+    pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
+
+
+def test_c4_full():
+    wl = wk.WORKLOADS["c4"]
+    inp = wk.make_inputs(wl)
+    g, plan = pu.run_gpu(wl, inp)
+    assert plan["kernel"] == B.FORGE_KERNEL_BF16_SKINNY
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
