@@ -141,6 +141,14 @@ forge_status_t forge_fused_linear_run_host(forge_fused_linear_t h, const void *X
  */
 forge_status_t forge_fused_linear_last_status(forge_fused_linear_t h);
 
+/*
+ * Diagnostics of the give-up that the most recent last_status() call reported (host pointer
+ * to 4 ints): [0] which wait (1 operand tile arrival, 2 ring stage release, 3 accumulator
+ * ready, 4 accumulator release, 5 arrival of the other tiles of a row strip), [1] a
+ * kernel-specific detail word, [2] CTA index, [3] thread index.  All zero if none.
+ */
+forge_status_t forge_fused_linear_last_wait_detail(forge_fused_linear_t h, int detail[4]);
+
 /* Copy the plan chosen at create() into *info (host pointer). */
 forge_status_t forge_fused_linear_get_plan(forge_fused_linear_t h, forge_plan_info_t *info);
 

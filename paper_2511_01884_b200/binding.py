@@ -19,8 +19,8 @@ FORGE_KERNEL_F32_FFMA, FORGE_KERNEL_BF16_TCGEN05, FORGE_KERNEL_BF16_SKINNY, FORG
 EXPORTS = [
     "forge_fused_linear_query_plan", "forge_fused_linear_create", "forge_fused_linear_run",
     "forge_fused_linear_run_host", "forge_fused_linear_last_status", "forge_fused_linear_get_plan",
-    "forge_fused_linear_launches_per_run", "forge_fused_linear_destroy", "forge_status_string",
-    "forge_kernel_name",
+    "forge_fused_linear_launches_per_run", "forge_fused_linear_destroy", "forge_fused_linear_last_wait_detail",
+    "forge_status_string", "forge_kernel_name",
 ]
 
 
@@ -67,11 +67,12 @@ def lib() -> ctypes.CDLL:
         L.forge_fused_linear_get_plan.argtypes = [vp, ctypes.POINTER(PlanInfo)]
         L.forge_fused_linear_launches_per_run.argtypes = [vp]
         L.forge_fused_linear_destroy.argtypes = [vp]
+        L.forge_fused_linear_last_wait_detail.argtypes = [vp, ctypes.POINTER(ctypes.c_int * 4)]
         L.forge_status_string.argtypes = [i]
         L.forge_status_string.restype = ctypes.c_char_p
         L.forge_kernel_name.argtypes = [i]
         L.forge_kernel_name.restype = ctypes.c_char_p
-        for n in EXPORTS[:8]:
+        for n in EXPORTS[:9]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -127,6 +128,15 @@ def forge_fused_linear_last_status(h) -> int:
     return lib().forge_fused_linear_last_status(h)
 
 
+def forge_fused_linear_last_wait_detail(h):
+    """[wait site, detail word, CTA, thread] of the give-up the last last_status() call saw."""
+    d = (ctypes.c_int * 4)()
+    st = lib().forge_fused_linear_last_wait_detail(h, ctypes.byref(d))
+    if st != FORGE_OK:
+        raise ForgeError(st, "last_wait_detail")
+    return list(d)
+
+
 def forge_fused_linear_get_plan(h) -> PlanInfo:
     info = PlanInfo()
     st = lib().forge_fused_linear_get_plan(h, ctypes.byref(info))
@@ -169,7 +179,7 @@ class FusedLinear:
     def check(self):
         st = forge_fused_linear_last_status(self.h)
         if st != FORGE_OK:
-            raise ForgeError(st, "forge_fused_linear_last_status")
+            raise ForgeError(st, f"forge_fused_linear_last_status (wait detail {forge_fused_linear_last_wait_detail(self.h)})")
 
     def close(self):
         if self.h:

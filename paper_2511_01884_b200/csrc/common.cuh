@@ -25,9 +25,15 @@ enum WaitSite : int {
     SITE_ARRIVAL = 5, SITE_STORE = 6, SITE_CLUSTER = 7
 };
 
-__device__ __forceinline__ void report_timeout(int *status, int site)
+// Words 1..3 of the status area describe the first give-up: a caller-chosen detail word, the
+// CTA index and the thread index.
+__device__ __forceinline__ void report_timeout(int *status, int site, int detail = 0)
 {
-    atomicCAS(status, 0, (int(FORGE_ERR_TIMEOUT) << 16) | site);
+    if (atomicCAS(status, 0, (int(FORGE_ERR_TIMEOUT) << 16) | site) == 0) {
+        status[1] = detail;
+        status[2] = (int)blockIdx.x;
+        status[3] = (int)threadIdx.x;
+    }
 }
 
 // ---- activations -------------------------------------------------------------------

@@ -232,14 +232,25 @@ forge_status_t forge_fused_linear_last_status(forge_fused_linear_t hh)
     DeviceGuard g(h.d.device);
     if (!g.ok) return FORGE_ERR_CUDA;
     if (cudaDeviceSynchronize() != cudaSuccess) return FORGE_ERR_CUDA;
-    int word = 0;
-    if (cudaMemcpy(&word, h.ws.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return FORGE_ERR_CUDA;
+    if (cudaMemcpy(h.last_detail, h.ws.status, sizeof(h.last_detail), cudaMemcpyDeviceToHost) != cudaSuccess) return FORGE_ERR_CUDA;
+    const int word = h.last_detail[0];
     if (word != 0) {
         // a give-up may have left arrival counters half way: clear the whole workspace
         cudaMemset(h.ws.base, 0, h.ws.bytes);
         h.run_gen = 0;
         return (forge_status_t)(word >> 16);
     }
+    return FORGE_OK;
+}
+
+forge_status_t forge_fused_linear_last_wait_detail(forge_fused_linear_t hh, int detail[4])
+{
+    if (!hh || !detail) return FORGE_ERR_INVALID_ARG;
+    const Handle &h = *reinterpret_cast<Handle *>(hh);
+    detail[0] = h.last_detail[0] & 0xffff;
+    detail[1] = h.last_detail[1];
+    detail[2] = h.last_detail[2];
+    detail[3] = h.last_detail[3];
     return FORGE_OK;
 }
 

@@ -5,8 +5,8 @@
 // sized so that all CTAs stream the same number of bytes.  A producer warp streams W (and
 // the matching slice of X, which stays L2-resident) through a 10-stage TMA ring; 8 consumer
 // warps feed the tiles to mma.sync.m16n8k16 straight from shared memory (ldmatrix on the
-// 128-byte-swizzled layout).  The warps split the work 2 (halves of the strip's columns) x
-// 4 (K: ring stages are dealt round-robin), so the partial accumulators of the 4 K-slices
+// 128-byte-swizzled layout).  The warps split the work 4 (quarters of the strip's columns) x
+// 2 (K: ring stages are dealt round-robin), so the partial accumulators of the 2 K-slices
 // are summed -- before bias and activation, which are nonlinear -- through shared memory in
 // a fixed order.  Row sum / max: two shuffles inside the 4-lane groups that share a row,
 // then per-CTA partials folded by the CTA that arrives last.
@@ -22,7 +22,12 @@ namespace forge {
 constexpr int K3_BK = 64;                       // k per stage: one 128-byte swizzle row
 constexpr int K3_MAX_GROUPS = 16;               // 8-column groups per strip (128 rows of W)
 constexpr int K3_STAGES = 10;
-constexpr int K3_KSPLIT = 4, K3_NSPLIT = 2;
+constexpr int K3_KSPLIT = 2, K3_NSPLIT = 4;
+// A ring slot must be consumed by the same warps on every pass.  The phase-parity wait only
+// tells "one phase further" from "not yet"; a warp that never consumed pass n of a slot has
+// nothing that orders its wait for pass n+1 after the completion of pass n, and would read a
+// spurious success while pass n is still in flight.
+static_assert(K3_STAGES % K3_KSPLIT == 0, "each ring slot belongs to one K-slice");
 constexpr int K3_CONSUMER_WARPS = K3_KSPLIT * K3_NSPLIT;
 constexpr int K3_CONSUMERS = K3_CONSUMER_WARPS * 32;
 constexpr int K3_THREADS = K3_CONSUMERS + 32;
@@ -97,7 +102,7 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             for (int st = 0; st < strips && ok; ++st) {
                 const int row0 = (g_lo + st * p.box_groups) * 8;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
-                    if (!ptx::mbar_wait(&s.empty[slot], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
+                    if (!ptx::mbar_wait(&s.empty[slot], phase ^ 1, p.status, SITE_STAGE_EMPTY, (slot << 16) | (kb & 0xffff))) { ok = false; break; }
                     if (!K3_INRANGE(row0 >= 0 && row0 < p.N && kb * K3_BK < p.K, 1)) { ok = false; break; }
                     uint8_t *dst = ring + (size_t)slot * K3_STAGE_BYTES;
                     ptx::mbar_expect_tx(&s.full[slot], stage_tx);
@@ -110,8 +115,8 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         }
     } else {
         // ---------------- consumers ----------------
-        const int nh = warp & 1;            // which half of the strip's groups
-        const int ks = warp >> 1;           // which K-slice (ring stages with index % 4 == ks)
+        const int nh = warp % K3_NSPLIT;    // which part of the strip's groups
+        const int ks = warp / K3_NSPLIT;    // which K-slice (ring stages with index % K3_KSPLIT == ks)
         const int t = threadIdx.x;          // 0..255
         const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX;
         bool ok = true;
@@ -137,7 +142,7 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             for (int g = 0; g < K3_GH; ++g) acc[g][0] = acc[g][1] = acc[g][2] = acc[g][3] = 0.f;
 
             for (; seq < seq_end; seq += K3_KSPLIT) {
-                if (ok && !ptx::mbar_wait(&s.full[slot], phase, p.status, SITE_TMA_FULL)) ok = false;
+                if (ok && !ptx::mbar_wait(&s.full[slot], phase, p.status, SITE_TMA_FULL, (slot << 16) | (seq & 0xffff))) ok = false;
                 if (ok) {
                     const uint32_t wbase = ptx::smem_u32(ring + (size_t)slot * K3_STAGE_BYTES);
                     const uint32_t xbase = wbase + K3_W_BYTES;

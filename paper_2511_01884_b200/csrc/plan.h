@@ -28,6 +28,7 @@ struct Handle {
     forge_fused_linear_desc_t d;
     forge_plan_info_t info;
     int sm_count = 0;
+    int last_detail[4] = {0, 0, 0, 0};   // status area as read by the last last_status() call
     unsigned run_gen = 0;            // runs launched since the workspace was last cleared
     Workspace ws;
     // staging buffers of run_host()

@@ -29,8 +29,9 @@ def test_identity_weight_reproduces_x():
 
 # N/8 below, at and far above the SM count (1, several and many strips per CTA); K with a
 # ragged last block and fewer blocks than K-slices; M below 16
+# ... and K long enough for many passes over the shared-memory ring
 SHAPES = [(16, 8, 8), (1, 64, 16), (5, 1184, 72), (16, 1192, 200), (16, 4096, 1024), (7, 20000, 264),
-          (16, 148 * 8 * 17, 128), (16, 148 * 8 * 40 + 8, 64)]
+          (16, 148 * 8 * 17, 128), (16, 148 * 8 * 40 + 8, 64), (16, 2368, 4096), (3, 1184 * 13, 2048)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
