@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the fused linear operator on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl reference]
+
+One "step" is one pass of the whole hot path (operand fetch, contraction, bias, activation,
+scale, row reduction, store: a single kernel launch) over one batch of seeded synthetic
+input.  The headline workload is C3 (bf16, M=N=K=8192, SiLU); at N=1 the line also carries
+short measurements of the other four workloads under "workloads".  With N>1 (launched by
+torch.distributed.run, one rank per GPU) every rank runs the workload on its own block of
+rows of a global X (rows are independent: no collective on the data path) and the value is
+the aggregate over ranks of work / max-over-ranks time.
+
+Timing: CUDA events on the stream the kernels are launched on, after >= 3 warm-up steps,
+barrier + synchronize on both sides.  L2: the operands of C2..C5 exceed the 126 MB L2; C1
+fits and is timed with an L2 flush (a 256 MiB write) before every call.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2511_01884_b200 import workloads as wk  # noqa: E402
+
+HEADLINE = "c3"
+NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel
+# from the ncu captures summarised under profiles/, keyed by workload, with the sha256 of the
+# kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
+NCU_TRAFFIC = {
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+def kernel_source_hash(kernel: int) -> str:
+    name = {1: "k1_f32_ffma.cu", 2: "k2_bf16_tcgen05.cu", 3: "k3_bf16_skinny.cu", 4: "k2_bf16_tcgen05.cu"}[kernel]
+    with open(os.path.join(ROOT, "paper_2511_01884_b200", "csrc", name), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+# ---- clocks during the timed region (NVML; nvidia-smi as a fallback) -------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h) if hasattr(
+                    nv, "nvmlDeviceGetCurrentClocksEventReasons") else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if self._nv is None or not self.samples:
+            return self._smi_once()
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples), "how": "nvml during the timed region"}
+
+    def _smi_once(self):
+        import subprocess
+        try:
+            out = subprocess.run(["nvidia-smi", f"--id={self.index}", "--query-gpu=clocks.sm,clocks.max.sm",
+                                  "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=10).stdout
+            a, b = [float(t) for t in out.strip().split(",")]
+            return {"sm_mhz": a, "sm_max_mhz": b, "reasons": [], "samples": 1, "how": "nvidia-smi after the timed region"}
+        except Exception:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "how": "unavailable"}
+
+
+# ---- device-side measurement ---------------------------------------------------------------------
+def device_tensors(wl, inp, torch):
+    def dev(a):
+        if a is None:
+            return None
+        t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
+        return (t.to(torch.bfloat16) if wl.dtype == wk.BF16 else t).cuda()
+    d = {k: dev(v) for k, v in inp.items()}
+    M = inp["X"].shape[0]
+    if wl.red in (wk.RED_SUM, wk.RED_MAX):
+        d["out"] = torch.empty((M,), dtype=torch.float32, device="cuda")
+    else:
+        d["out"] = torch.empty((M, wl.N), dtype=torch.bfloat16 if wl.dtype == wk.BF16 else torch.float32, device="cuda")
+    return d
+
+
+def make_op(wl, M, device):
+    from paper_2511_01884_b200 import binding as B
+    return B.FusedLinear(B.make_desc(M, wl.N, wl.K, wl.dtype, wl.act, wl.red, wl.scale, wl.ln_eps,
+                                     wl.bias.kind != "none", device))
+
+
+def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
+    """Average device milliseconds per step over exactly `steps` steps (CUDA events on the
+    launching stream).  With flush_buf every step is bracketed by its own events and L2 is
+    overwritten before it."""
+    for _ in range(warmup):
+        op(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
+    torch.cuda.synchronize()
+    op.check()
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    if flush_buf is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            op(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+    else:
+        tot = 0.0
+        for _ in range(steps):
+            flush_buf.fill_(1.0)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            op(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
+            e1.record()
+            torch.cuda.synchronize()
+            tot += e0.elapsed_time(e1)
+        ms = tot / steps
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    op.check()
+    return ms
+
+
+def roofline_of(wl, ms, peaks, kernel, sm_max_mhz, sm_count):
+    """Roofline of the (single) kernel of a step: achieved = algorithmic work / measured time."""
+    src = peaks["_source"]
+    if wl.name == "c4":
+        ach = wl.algorithmic_bytes / ms / 1e6
+        peak, unit, bound = peaks["hbm_gbs"], "GB/s", "hbm"
+        note = f"{wl.algorithmic_bytes} algorithmic bytes per launch; peak = copy bandwidth, of {src}"
+    elif wl.dtype == wk.BF16:
+        ach = wl.flops / ms / 1e9
+        peak, unit, bound = peaks["bf16_tflops"], "TFLOP/s", "tensor"
+        note = f"2MNK = {wl.flops} flops per launch; peak = cuBLAS bf16 burst, of {src}"
+    else:
+        ach = wl.flops / ms / 1e9
+        peak = sm_count * 128 * 2 * (sm_max_mhz or 1965.0) * 1e6 / 1e12
+        unit, bound = "TFLOP/s", "alu"
+        note = "fp32 FFMA peak = SMs x 128 lanes x 2 flop x max SM clock (derived, not measured)"
+    key = NCU_TRAFFIC.get(wl.name)
+    traffic = key["bytes"] if key and key["sha"] == kernel_source_hash(kernel) else None
+    return {"bound": bound, "achieved": round(ach, 2), "peak": round(peak, 2), "unit": unit,
+            "frac": round(ach / peak, 4), "traffic": traffic, "note": note}
+
+
+def unit_value(wl, ms, n_units=1):
+    if wl.name == "c4":
+        return n_units * wl.algorithmic_bytes / ms / 1e6, "GB/s"
+    return n_units * wl.flops / ms / 1e9, "TFLOP/s"
+
+
+# ---- CPU oracle leg -------------------------------------------------------------------------------
+def oracle_sample(wl, inp, target_s=12.0, max_rows=None):
+    """Time the oracle, as it stands, on a bounded sample of rows of the workload."""
+    import oracle
+    M = inp["X"].shape[0]
+    rows_all = wk.sample_rows(M)
+    probe = rows_all[: min(len(rows_all), 4)]
+    t = time.perf_counter()
+    oracle.fused_linear(inp["X"], inp["W"], inp["b"], inp["gamma"], inp["beta"], act=wl.act, scale=wl.scale,
+                        red=wl.red, eps=wl.ln_eps, rows=probe)
+    per_row = (time.perf_counter() - t) / len(probe)
+    n = int(max(len(probe), min(M, target_s / max(per_row, 1e-9))))
+    if max_rows:
+        n = min(n, max_rows)
+    rows = np.arange(n, dtype=np.int64) * (M // n) if n < M else np.arange(M, dtype=np.int64)
+    t = time.perf_counter()
+    oracle.fused_linear(inp["X"], inp["W"], inp["b"], inp["gamma"], inp["beta"], act=wl.act, scale=wl.scale,
+                        red=wl.red, eps=wl.ln_eps, rows=rows)
+    dt = time.perf_counter() - t
+    flops = 2.0 * len(rows) * wl.N * wl.K
+    if wl.name == "c4":
+        value, unit = (len(rows) / M) * wl.algorithmic_bytes / dt / 1e9, "GB/s"
+    else:
+        value, unit = flops / dt / 1e12, "TFLOP/s"
+    return {"value": value, "unit": unit, "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"{len(rows)} of {M} rows of {wl.name} (all N, all K), fp64 loops, {dt:.2f} s",
+            "seconds": dt, "rows": len(rows)}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, same metric and workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    wl = wk.WORKLOADS[args.workload]
+    inp = wk.make_inputs(wl)
+    per_step_target = max(1.0, min(10.0, 60.0 / max(1, args.steps + args.warmup)))
+    first = oracle_sample(wl, inp, target_s=per_step_target)
+    rows = first["rows"]
+    import oracle
+    sel = np.arange(rows, dtype=np.int64) * (wl.M // rows)
+    times = []
+    for i in range(args.warmup + args.steps):
+        t = time.perf_counter()
+        oracle.fused_linear(inp["X"], inp["W"], inp["b"], inp["gamma"], inp["beta"], act=wl.act, scale=wl.scale,
+                            red=wl.red, eps=wl.ln_eps, rows=sel)
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t)
+    ms = 1e3 * sum(times) / len(times)
+    if wl.name == "c4":
+        value, unit = (rows / wl.M) * wl.algorithmic_bytes / ms / 1e6, "GB/s"
+    else:
+        value, unit = 2.0 * rows * wl.N * wl.K / ms / 1e9, "TFLOP/s"
+    line = {"impl": "reference", "metric": f"fused-op {unit} ({wl.name})", "value": value, "unit": unit,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_of(wl, args.gpus, extra={"step": f"{rows} sampled rows of the workload per step"}),
+            "cpu_baseline": {"value": value, "unit": unit, "cores": first["cores"], "kind": "oracle",
+                             "sample": f"{rows} of {wl.M} rows of {wl.name} per step, fp64 loops"},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def config_of(wl, n_gpus, extra=None):
+    names = {wk.ACT_IDENTITY: "identity", wk.ACT_RELU: "relu", wk.ACT_GELU_ERF: "gelu_erf",
+             wk.ACT_GELU_TANH: "gelu_tanh", wk.ACT_SILU: "silu"}
+    reds = {wk.RED_NONE: "none", wk.RED_SUM: "row_sum", wk.RED_MAX: "row_max", wk.RED_LAYERNORM: "layernorm"}
+    c = {"workload": f"{wl.name}: {wl.note}", "M_per_gpu": wl.M, "N": wl.N, "K": wl.K,
+         "dtype": "bf16" if wl.dtype == wk.BF16 else "f32", "act": names[wl.act], "scale": wl.scale,
+         "reduction": reds[wl.red], "seed": wl.seed, "parallelism": f"rows sharded over {n_gpus} gpu(s), no collective",
+         "l2": "operands larger than L2 (126 MB): no flush" if wl.algorithmic_bytes > 130e6 else "L2 flushed before every call"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=HEADLINE, choices=sorted(wk.WORKLOADS))
+    ap.add_argument("--impl", default="forge", choices=["forge", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the short runs of the other workloads")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (sm_100a); there is no CPU fallback")
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    n_gpus = world
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    peaks = load_peaks()
+    props = torch.cuda.get_device_properties(local)
+    wl = wk.WORKLOADS[args.workload]
+
+    # this rank's block of rows of the global [world * M, K] input; W, b, gamma, beta replicated
+    inp = wk.make_inputs(wl, M=wl.M, row_offset=rank * wl.M)
+    d = device_tensors(wl, inp, torch)
+    op = make_op(wl, wl.M, local)
+    flush = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device="cuda") if wl.algorithmic_bytes < 130e6 else None
+
+    with ClockSampler(local) as cs:
+        ms = time_steps(op, d, args.steps, args.warmup, torch, flush_buf=flush, barrier=barrier)
+    clocks = cs.summary()
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    value, unit = unit_value(wl, ms_max, n_units=world)
+    launches = args.steps * 1
+
+    # ---- end to end: pinned host buffers in, result out, through the host entry point ----
+    e2e_steps = max(1, min(args.steps, 10))
+    host = {}
+    for k in ("X", "W", "b", "gamma", "beta"):
+        host[k] = None if d[k] is None else d[k].cpu().pin_memory()
+    host_out = torch.empty_like(d["out"], device="cpu").pin_memory()
+    h2d = sum(v.numel() * v.element_size() for v in host.values() if v is not None)
+    d2h = host_out.numel() * host_out.element_size()
+    op.run_host(host["X"], host["W"], host["b"], host["gamma"], host["beta"], host_out)   # warm-up, allocates staging
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        op.run_host(host["X"], host["W"], host["b"], host["gamma"], host["beta"], host_out)
+    torch.cuda.synchronize()
+    e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_val, _ = unit_value(wl, float(t.item()), n_units=world)
+    same = bool(torch.equal(host_out.cuda(), d["out"]))
+    op.check()
+
+    line = {"metric": f"fused-op {unit} ({wl.name})", "value": round(value, 2), "unit": unit, "n_gpus": n_gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_max, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == wk.BF16 else "f32",
+            "data": "synthetic", "config": config_of(wl, n_gpus, {"kernel": op.plan.as_dict()}),
+            "clocks": clocks,
+            "e2e": {"value": round(e2e_val, 3), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps, "ms_per_step": round(float(t.item()), 3),
+                    "matches_device_run": same, "how": "forge_fused_linear_run_host, pinned host buffers, wall clock"},
+            "gpu_launches": launches,
+            "roofline": roofline_of(wl, ms, peaks, op.plan.kernel, clocks.get("sm_max_mhz"), props.multi_processor_count),
+            "nominal_frac": round((value / world) / (NOMINAL["hbm_gbs"] if wl.name == "c4" else NOMINAL["bf16_tflops"]), 4)
+            if wl.dtype == wk.BF16 else None}
+    op.close()
+    del d, host
+
+    if rank == 0 and world == 1:
+        line["cpu_baseline"] = {k: v for k, v in oracle_sample(wl, inp).items() if k not in ("seconds", "rows")}
+        if not args.no_extras:
+            line["workloads"] = {}
+            for name in sorted(wk.WORKLOADS):
+                if name == wl.name:
+                    continue
+                w2 = wk.WORKLOADS[name]
+                torch.cuda.empty_cache()
+                i2 = wk.make_inputs(w2)
+                d2 = device_tensors(w2, i2, torch)
+                op2 = make_op(w2, w2.M, local)
+                fl = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device="cuda") if w2.algorithmic_bytes < 130e6 else None
+                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50}[name]
+                ms2 = time_steps(op2, d2, steps2, 3, torch, flush_buf=fl)
+                v2, u2 = unit_value(w2, ms2)
+                launches += steps2
+                line["workloads"][name] = {"us_per_call": round(ms2 * 1e3, 2), "value": round(v2, 2), "unit": u2,
+                                           "steps": steps2, "l2": "flushed before every call" if fl is not None else "operands larger than L2",
+                                           "kernel": op2.plan.as_dict()["kernel"],
+                                           "roofline": roofline_of(w2, ms2, peaks, op2.plan.kernel, clocks.get("sm_max_mhz"),
+                                                                   props.multi_processor_count)}
+                op2.close()
+                del d2, i2, fl
+            line["gpu_launches_all_workloads"] = launches
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
