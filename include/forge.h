@@ -40,7 +40,9 @@ typedef enum {
     FORGE_ERR_UNSUPPORTED = 2,   /* valid request that no kernel here serves              */
     FORGE_ERR_CUDA = 3,          /* a CUDA runtime/driver call failed (or no sm_100 GPU)  */
     FORGE_ERR_ALLOC = 4,         /* host or device allocation failed                      */
-    FORGE_ERR_TIMEOUT = 5        /* a bounded device-side wait gave up                    */
+    FORGE_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up                    */
+    FORGE_ERR_SCRATCH_LIMIT = 6  /* problem needs more scratch than the fixed buffer of   */
+                                 /* forge_fused_linear_f32_reduce_static() holds          */
 } forge_status_t;
 
 typedef enum { FORGE_F32 = 0, FORGE_BF16 = 1 } forge_dtype_t;
@@ -154,6 +156,43 @@ forge_status_t forge_fused_linear_get_plan(forge_fused_linear_t h, forge_plan_in
 
 /* Number of kernels run() launches per call for this handle (always >= 1). */
 int forge_fused_linear_launches_per_run(forge_fused_linear_t h);
+
+/*
+ * Row sum / row max of the fp32 fused linear without a handle and without any allocation.
+ * (The paper has no counterpart to this entry point: it exists for the benefit of callers,
+ * not of the method.)
+ *
+ * Who needs it: code that may not call cudaMalloc when it wants the result -- a plugin
+ * running inside someone else's memory pool or under a fixed memory budget, a real-time or
+ * latency-critical loop where an allocation (which can synchronise the whole device) is not
+ * acceptable, a process that has handed all device memory to its own allocator and cannot
+ * get more from the driver.  create() cannot serve them: it allocates the workspace in which
+ * the N-tiles of a row strip leave their partial sums / maxima and count their arrivals.
+ *
+ * Here that workspace is a fixed array of FORGE_STATIC_SCRATCH_BYTES inside the library
+ * image; every GPU that loads the library carries it until the process ends.  The call
+ * needs, for ceil(M/128) row strips and ceil(N/128) column tiles,
+ *     roundup(4 * ceil(M/128), 256) + (ceil(N/128) > 1 ? 4 * M * ceil(N/128) : 0)  bytes;
+ * a problem that needs more is refused with FORGE_ERR_SCRATCH_LIMIT (nothing is launched).
+ *
+ * Computes out[m] = sum_n or max_n of scale * act(X W^T + b), fp32, on the CURRENT device.
+ * DEVICE pointers, 4-byte aligned (16-byte alignment of X and W with K % 4 == 0 enables the
+ * 128-bit loads): X [M,K], W [N,K], b [N] or NULL for no bias, out [M] fp32.  `red` must be
+ * FORGE_RED_SUM or FORGE_RED_MAX.  Asynchronous on `cuda_stream`; calls neither cudaMalloc
+ * nor cudaFree nor any allocating library routine.
+ *
+ * The first call on each device looks up the device address of the array (a runtime query);
+ * make that first call outside any stream capture.  All calls in the process share the one
+ * array per device, and it keeps the previous call's contents: this function zeroes the
+ * arrival counters on the stream before the kernel, but two calls whose kernels overlap on
+ * the GPU (different streams, no dependency) race on it and give wrong results -- keep
+ * calls on one device ordered.  Results are identical to the handle-based path.
+ */
+#define FORGE_STATIC_SCRATCH_BYTES (1u << 20)
+forge_status_t forge_fused_linear_f32_reduce_static(int64_t M, int64_t N, int64_t K, forge_act_t act,
+                                                    forge_red_t red, float scale, const void *X,
+                                                    const void *W, const void *b, void *out,
+                                                    void *cuda_stream);
 
 /* Free the workspace, staging buffers and the handle.  NULL is FORGE_ERR_INVALID_ARG. */
 forge_status_t forge_fused_linear_destroy(forge_fused_linear_t h);

@@ -10,7 +10,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libforge.so")
 
 # enums of forge.h
-FORGE_OK, FORGE_ERR_INVALID_ARG, FORGE_ERR_UNSUPPORTED, FORGE_ERR_CUDA, FORGE_ERR_ALLOC, FORGE_ERR_TIMEOUT = range(6)
+(FORGE_OK, FORGE_ERR_INVALID_ARG, FORGE_ERR_UNSUPPORTED, FORGE_ERR_CUDA, FORGE_ERR_ALLOC, FORGE_ERR_TIMEOUT,
+ FORGE_ERR_SCRATCH_LIMIT) = range(7)
+FORGE_STATIC_SCRATCH_BYTES = 1 << 20
 FORGE_F32, FORGE_BF16 = 0, 1
 FORGE_ACT_IDENTITY, FORGE_ACT_RELU, FORGE_ACT_GELU_ERF, FORGE_ACT_GELU_TANH, FORGE_ACT_SILU = range(5)
 FORGE_RED_NONE, FORGE_RED_SUM, FORGE_RED_MAX, FORGE_RED_LAYERNORM = range(4)
@@ -20,7 +22,7 @@ EXPORTS = [
     "forge_fused_linear_query_plan", "forge_fused_linear_create", "forge_fused_linear_run",
     "forge_fused_linear_run_host", "forge_fused_linear_last_status", "forge_fused_linear_get_plan",
     "forge_fused_linear_launches_per_run", "forge_fused_linear_destroy", "forge_fused_linear_last_wait_detail",
-    "forge_status_string", "forge_kernel_name",
+    "forge_fused_linear_f32_reduce_static", "forge_status_string", "forge_kernel_name",
 ]
 
 
@@ -72,7 +74,9 @@ def lib() -> ctypes.CDLL:
         L.forge_status_string.restype = ctypes.c_char_p
         L.forge_kernel_name.argtypes = [i]
         L.forge_kernel_name.restype = ctypes.c_char_p
-        for n in EXPORTS[:9]:
+        L.forge_fused_linear_f32_reduce_static.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, i, i,
+                                                           ctypes.c_float, vp, vp, vp, vp, vp]
+        for n in EXPORTS[:10]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -147,6 +151,16 @@ def forge_fused_linear_get_plan(h) -> PlanInfo:
 
 def forge_fused_linear_launches_per_run(h) -> int:
     return lib().forge_fused_linear_launches_per_run(h)
+
+
+def forge_fused_linear_f32_reduce_static(M, N, K, act, red, scale, X, W, b, out, stream=None) -> int:
+    """fp32 row sum / max on the current device using the library's fixed scratch array: no
+    handle, no allocation (see forge.h for who needs this and for the size limit)."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    return lib().forge_fused_linear_f32_reduce_static(int(M), int(N), int(K), int(act), int(red), float(scale),
+                                                      _ptr(X), _ptr(W), _ptr(b), _ptr(out), stream)
 
 
 def forge_fused_linear_destroy(h) -> int:

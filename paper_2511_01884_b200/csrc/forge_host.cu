@@ -285,6 +285,7 @@ const char *forge_status_string(forge_status_t s)
     case FORGE_ERR_CUDA: return "CUDA error or no sm_100 device";
     case FORGE_ERR_ALLOC: return "allocation failed";
     case FORGE_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case FORGE_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the fixed no-allocation buffer holds";
     }
     return "unknown status";
 }

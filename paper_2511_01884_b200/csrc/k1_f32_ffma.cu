@@ -10,6 +10,8 @@
 //             each CTA normalises the tile it still holds in registers.
 #include <cooperative_groups.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "plan.h"
 
@@ -337,4 +339,83 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
     return FORGE_ERR_INVALID_ARG;
 }
 
+// ---- row sum / max without any allocation ---------------------------------------------------
+// Scratch of forge_fused_linear_f32_reduce_static(): one fixed array per GPU that loads this
+// library, held until the process exits.  Layout: arrival counters (one per 128-row strip,
+// padded to 256 bytes), then the per-tile row partials [tiles_n][M].
+constexpr size_t K1_STATIC_SCRATCH_BYTES = FORGE_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char k1_static_scratch[K1_STATIC_SCRATCH_BYTES];
+
+constexpr int K1_MAX_DEVICES = 64;
+static void *k1_static_scratch_addr[K1_MAX_DEVICES];      // device address of the array, per device
+static std::mutex k1_static_mutex;
+
+// `k1_static_scratch` names a host-side shadow here; the address the kernel needs comes from
+// the runtime, once per device, with that device current.
+static forge_status_t k1_static_scratch_on_current_device(void **addr)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= K1_MAX_DEVICES) return FORGE_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(k1_static_mutex);
+    if (!k1_static_scratch_addr[dev]) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || major != 10)
+            return FORGE_ERR_CUDA;
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, k1_static_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return FORGE_ERR_CUDA;
+        }
+        k1_static_scratch_addr[dev] = ptr;
+    }
+    *addr = k1_static_scratch_addr[dev];
+    return FORGE_OK;
+}
+
 }  // namespace forge
+
+extern "C" forge_status_t forge_fused_linear_f32_reduce_static(int64_t M, int64_t N, int64_t K, forge_act_t act,
+                                                               forge_red_t red, float scale, const void *X,
+                                                               const void *W, const void *b, void *out,
+                                                               void *cuda_stream)
+{
+    using namespace forge;
+    if (M <= 0 || N <= 0 || K <= 0 || !X || !W || !out) return FORGE_ERR_INVALID_ARG;
+    if (act < FORGE_ACT_IDENTITY || act > FORGE_ACT_SILU || !(scale == scale)) return FORGE_ERR_INVALID_ARG;
+    if (red != FORGE_RED_SUM && red != FORGE_RED_MAX) return FORGE_ERR_INVALID_ARG;
+    if (((uintptr_t)X | (uintptr_t)W | (uintptr_t)b | (uintptr_t)out) % 4 != 0) return FORGE_ERR_INVALID_ARG;
+    if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return FORGE_ERR_SCRATCH_LIMIT;
+    const int64_t tiles_m = (M + K1_BM - 1) / K1_BM, tiles_n = (N + K1_BN - 1) / K1_BN;
+    if (tiles_m > 65535) return FORGE_ERR_SCRATCH_LIMIT;
+    const size_t counter_bytes = (((size_t)tiles_m * sizeof(unsigned) + 255) / 256) * 256;
+    const size_t partial_bytes = tiles_n > 1 ? (size_t)tiles_n * (size_t)M * sizeof(float) : 0;
+    if (counter_bytes + partial_bytes > K1_STATIC_SCRATCH_BYTES) return FORGE_ERR_SCRATCH_LIMIT;
+
+    void *scratch = nullptr;
+    const forge_status_t st = k1_static_scratch_on_current_device(&scratch);
+    if (st != FORGE_OK) return st;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // the array keeps whatever the previous call left: the arrival counters must start at zero
+    if (cudaMemsetAsync(scratch, 0, counter_bytes, stream) != cudaSuccess) return FORGE_ERR_CUDA;
+
+    K1Params p;
+    p.X = (const float *)X;
+    p.W = (const float *)W;
+    p.b = (const float *)b;
+    p.gamma = nullptr;
+    p.beta = nullptr;
+    p.out = (float *)out;
+    p.M = (int)M;
+    p.N = (int)N;
+    p.K = (int)K;
+    p.e = Epilogue{(int)act, (int)red, scale, 0.f, b != nullptr};
+    p.counters = (unsigned *)scratch;
+    p.partial = (float *)((unsigned char *)scratch + counter_bytes);
+    p.tiles_n = (int)tiles_n;
+    p.out_vec4 = 0;
+    const dim3 grid((unsigned)tiles_n, (unsigned)tiles_m);
+    const bool vec = (K % 4 == 0) && ((uintptr_t)X % 16 == 0) && ((uintptr_t)W % 16 == 0);
+    if (red == FORGE_RED_SUM)
+        return vec ? k1_launch_t<true, FORGE_RED_SUM>(p, grid, 1, stream) : k1_launch_t<false, FORGE_RED_SUM>(p, grid, 1, stream);
+    return vec ? k1_launch_t<true, FORGE_RED_MAX>(p, grid, 1, stream) : k1_launch_t<false, FORGE_RED_MAX>(p, grid, 1, stream);
+}

@@ -21,7 +21,7 @@ def _built():
 
 def test_library_exports_every_declared_symbol():
     hdr = open(os.path.join(ROOT, "include", "forge.h")).read()
-    declared = set(re.findall(r"\b(forge_[a-z_]+)\s*\(", hdr))
+    declared = set(re.findall(r"\b(forge_[a-z0-9_]+)\s*\(", hdr))
     assert declared, "no declarations found"
     L = ctypes.CDLL(B.LIB_PATH)
     for name in declared:
@@ -71,8 +71,8 @@ def test_unsupported_is_reported_not_rerouted():
 
 
 def test_status_and_kernel_strings():
-    seen = {B.status_string(s) for s in range(6)}
-    assert len(seen) == 6 and "unknown status" not in seen
+    seen = {B.status_string(s) for s in range(7)}
+    assert len(seen) == 7 and "unknown status" not in seen
     assert B.status_string(99) == "unknown status"
     assert "f32" in B.kernel_name(B.FORGE_KERNEL_F32_FFMA)
 
