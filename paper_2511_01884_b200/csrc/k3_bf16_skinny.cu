@@ -99,9 +99,14 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             int slot = 0;
             uint32_t phase = 0;
             bool ok = true;
+            const int kb_rot = (int)((long long)p.num_kb * blockIdx.x / gridDim.x);
             for (int st = 0; st < strips && ok; ++st) {
                 const int row0 = (g_lo + st * p.box_groups) * 8;
-                for (int kb = 0; kb < p.num_kb; ++kb) {
+                for (int i = 0; i < p.num_kb; ++i) {
+                    // CTAs start at different k: if all of them walked K in lock step, the requests in
+                    // flight would share their low address bits and pile onto a few DRAM channels
+                    int kb = i + kb_rot;
+                    if (kb >= p.num_kb) kb -= p.num_kb;
                     if (!ptx::mbar_wait(&s.empty[slot], phase ^ 1, p.status, SITE_STAGE_EMPTY, (slot << 16) | (kb & 0xffff))) { ok = false; break; }
                     if (!K3_INRANGE(row0 >= 0 && row0 < p.N && kb * K3_BK < p.K, 1)) { ok = false; break; }
                     uint8_t *dst = ring + (size_t)slot * K3_STAGE_BYTES;
@@ -244,14 +249,24 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                 if (t == 0) s.last_flag = (atomicAdd(&p.counters[0], 1u) == gridDim.x - 1);
                 k3_consumer_sync();
                 if (s.last_flag) {
+                    // 16 threads per row: thread (row, j) folds CTAs j, j+16, ... in order, then
+                    // the 16 chunk results of a row are folded in order (fixed tree: repeatable)
                     __threadfence();
+                    const int row = t & 15, chunk = t >> 4;
+                    float v = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY;
+                    for (unsigned c = chunk; c < gridDim.x; c += 16) {
+                        const float o = __ldcg(&p.partial[(size_t)c * 16 + row]);
+                        v = p.e.red == FORGE_RED_SUM ? v + o : fmaxf(v, o);
+                    }
+                    s.rowred[chunk][row] = v;
+                    k3_consumer_sync();
                     if (t < p.M) {
-                        float v = __ldcg(&p.partial[t]);
-                        for (unsigned c = 1; c < gridDim.x; ++c) {
-                            const float o = __ldcg(&p.partial[(size_t)c * 16 + t]);
-                            v = p.e.red == FORGE_RED_SUM ? v + o : fmaxf(v, o);
+                        float r = s.rowred[0][t];
+                        for (int j = 1; j < 16; ++j) {
+                            const float o = s.rowred[j][t];
+                            r = p.e.red == FORGE_RED_SUM ? r + o : fmaxf(r, o);
                         }
-                        out[t] = v;
+                        out[t] = r;
                     }
                     if (t == 0) p.counters[0] = 0u;
                 }
