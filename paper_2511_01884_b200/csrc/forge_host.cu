@@ -109,9 +109,18 @@ forge_status_t encode_tmap_bf16(CUtensorMap *tm, const void *ptr, uint64_t rows,
     const cuuint64_t strides[1] = {cols * 2};                 // bytes, dimension 1
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
+    // FORGE_TMA_L2_PROMOTION = 0 | 64 | 128 | 256 overrides the L2 fetch granularity (tuning aid)
+    static int promo = -1;
+    if (promo < 0) {
+        const char *e = std::getenv("FORGE_TMA_L2_PROMOTION");
+        promo = e ? std::atoi(e) : 256;
+    }
+    const CUtensorMapL2promotion l2 = promo == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
+                                      : promo == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
+                                      : promo == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B
+                                                     : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
     const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, l2, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? FORGE_OK : FORGE_ERR_CUDA;
 }
 

@@ -3,7 +3,8 @@
 //
 // Each CTA owns a contiguous range of 8-column groups of the output (8 rows of W per group)
 // sized so that all CTAs stream the same number of bytes.  A producer warp streams W (and
-// the matching slice of X, which stays L2-resident) through a 10-stage TMA ring; 8 consumer
+// the matching slice of X, which stays L2-resident) through a 6-stage TMA ring (a stage is
+// 128 k of every row of the strip: two boxes, so 256 contiguous bytes per row); 8 consumer
 // warps feed the tiles to mma.sync.m16n8k16 straight from shared memory (ldmatrix on the
 // 128-byte-swizzled layout).  The warps split the work 4 (quarters of the strip's columns) x
 // 2 (K: ring stages are dealt round-robin), so the partial accumulators of the 2 K-slices
@@ -19,9 +20,11 @@
 
 namespace forge {
 
-constexpr int K3_BK = 64;                       // k per stage: one 128-byte swizzle row
-constexpr int K3_MAX_GROUPS = 16;               // 8-column groups per strip (128 rows of W)
-constexpr int K3_STAGES = 10;
+constexpr int K3_BK = 64;                       // k per TMA box: one 128-byte swizzle row
+constexpr int K3_KB = 2;                        // boxes per stage: 256 contiguous bytes of every W row at a time
+constexpr int K3_MAX_GROUPS = 14;               // 8-column groups per strip (112 rows of W)
+constexpr int K3_PAD_GROUPS = 16;               // group count the warp layout and the scratch arrays are sized for
+constexpr int K3_STAGES = 6;
 constexpr int K3_KSPLIT = 2, K3_NSPLIT = 4;
 // A ring slot must be consumed by the same warps on every pass.  The phase-parity wait only
 // tells "one phase further" from "not yet"; a warp that never consumed pass n of a slot has
@@ -31,16 +34,18 @@ static_assert(K3_STAGES % K3_KSPLIT == 0, "each ring slot belongs to one K-slice
 constexpr int K3_CONSUMER_WARPS = K3_KSPLIT * K3_NSPLIT;
 constexpr int K3_CONSUMERS = K3_CONSUMER_WARPS * 32;
 constexpr int K3_THREADS = K3_CONSUMERS + 32;
-constexpr uint32_t K3_W_BYTES = K3_MAX_GROUPS * 8 * K3_BK * 2;     // 16 KiB (full strip)
-constexpr uint32_t K3_X_BYTES = 16 * K3_BK * 2;                    // 2 KiB
-constexpr uint32_t K3_STAGE_BYTES = K3_W_BYTES + K3_X_BYTES;
-constexpr int K3_GH = K3_MAX_GROUPS / K3_NSPLIT;                   // groups per column half
+constexpr uint32_t K3_WBOX_BYTES = K3_MAX_GROUPS * 8 * K3_BK * 2;  // 14 KiB: one W box of a full strip
+constexpr uint32_t K3_XBOX_BYTES = 16 * K3_BK * 2;                 // 2 KiB: one X box
+constexpr uint32_t K3_W_BYTES = K3_KB * K3_WBOX_BYTES;
+constexpr uint32_t K3_X_BYTES = K3_KB * K3_XBOX_BYTES;
+constexpr uint32_t K3_STAGE_BYTES = K3_W_BYTES + K3_X_BYTES;       // 32 KiB
+constexpr int K3_GH = K3_PAD_GROUPS / K3_NSPLIT;                   // groups per warp column part
 
 struct K3Smem {
     uint64_t full[K3_STAGES];
     uint64_t empty[K3_STAGES];
-    float4 red[K3_KSPLIT][K3_MAX_GROUPS][32];    // partial accumulators of the K-slices
-    float rowred[K3_MAX_GROUPS][16];
+    float4 red[K3_KSPLIT][K3_PAD_GROUPS][32];    // partial accumulators of the K-slices
+    float rowred[K3_PAD_GROUPS][16];
     int last_flag;
     int abort_flag;
 };
@@ -81,7 +86,8 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const int g_lo = (int)((long long)p.groups * blockIdx.x / gridDim.x);
     const int g_hi = (int)((long long)p.groups * (blockIdx.x + 1) / gridDim.x);
     const int strips = (g_hi - g_lo + p.box_groups - 1) / p.box_groups;
-    const uint32_t stage_tx = (uint32_t)p.box_groups * 8 * K3_BK * 2 + K3_X_BYTES;
+    const uint32_t wbox_bytes = (uint32_t)p.box_groups * 8 * K3_BK * 2;       // multiple of 1024
+    const uint32_t stage_tx = K3_KB * wbox_bytes + K3_X_BYTES;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < K3_STAGES; ++i) { ptx::mbar_init(&s.full[i], 1); ptx::mbar_init(&s.empty[i], K3_NSPLIT); }
@@ -108,11 +114,15 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                     int kb = i + kb_rot;
                     if (kb >= p.num_kb) kb -= p.num_kb;
                     if (!ptx::mbar_wait(&s.empty[slot], phase ^ 1, p.status, SITE_STAGE_EMPTY, (slot << 16) | (kb & 0xffff))) { ok = false; break; }
-                    if (!K3_INRANGE(row0 >= 0 && row0 < p.N && kb * K3_BK < p.K, 1)) { ok = false; break; }
+                    if (!K3_INRANGE(row0 >= 0 && row0 < p.N && kb * K3_KB * K3_BK < p.K, 1)) { ok = false; break; }
                     uint8_t *dst = ring + (size_t)slot * K3_STAGE_BYTES;
                     ptx::mbar_expect_tx(&s.full[slot], stage_tx);
-                    ptx::tma_load_2d(dst, &tmW, &s.full[slot], kb * K3_BK, row0);
-                    ptx::tma_load_2d(dst + K3_W_BYTES, &tmX, &s.full[slot], kb * K3_BK, 0);
+                    // a box that starts at or past K (ragged last stage) is all zero fill
+#pragma unroll
+                    for (int j = 0; j < K3_KB; ++j) {
+                        ptx::tma_load_2d(dst + j * wbox_bytes, &tmW, &s.full[slot], (kb * K3_KB + j) * K3_BK, row0);
+                        ptx::tma_load_2d(dst + K3_W_BYTES + j * K3_XBOX_BYTES, &tmX, &s.full[slot], (kb * K3_KB + j) * K3_BK, 0);
+                    }
                     if (++slot == K3_STAGES) { slot = 0; phase ^= 1; }
                 }
             }
@@ -152,16 +162,17 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                     const uint32_t wbase = ptx::smem_u32(ring + (size_t)slot * K3_STAGE_BYTES);
                     const uint32_t xbase = wbase + K3_W_BYTES;
 #pragma unroll
-                    for (int kk = 0; kk < K3_BK / 16; ++kk) {
+                    for (int kq = 0; kq < K3_KB * K3_BK / 16; ++kq) {
+                        const int j = kq / (K3_BK / 16), kk = kq % (K3_BK / 16);     // box, 16-wide step inside it
                         uint32_t a[4];
-                        ptx::ldmatrix_x4(a, xbase + a_row * 128 + (((2 * kk + a_chunk) ^ (a_row & 7)) << 4));
+                        ptx::ldmatrix_x4(a, xbase + j * K3_XBOX_BYTES + a_row * 128 + (((2 * kk + a_chunk) ^ (a_row & 7)) << 4));
 #pragma unroll
                         for (int gp = 0; gp < K3_GH / 2; ++gp) {
                             const int g0 = nh * K3_GH + gp * 2;
                             if (g0 < ng) {
                                 uint32_t b[4];
                                 const int r = g0 * 8 + b_row;
-                                ptx::ldmatrix_x4(b, wbase + r * 128 + (((2 * kk + b_chunk) ^ (r & 7)) << 4));
+                                ptx::ldmatrix_x4(b, wbase + j * wbox_bytes + r * 128 + (((2 * kk + b_chunk) ^ (r & 7)) << 4));
                                 ptx::mma_m16n8k16_bf16(acc[gp * 2], a, b[0], b[1]);
                                 ptx::mma_m16n8k16_bf16(acc[gp * 2 + 1], a, b[2], b[3]);
                             }
@@ -181,7 +192,7 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             k3_consumer_sync();
 
 #pragma unroll
-            for (int j = 0; j < K3_MAX_GROUPS * 32 / K3_CONSUMERS; ++j) {
+            for (int j = 0; j < K3_PAD_GROUPS * 32 / K3_CONSUMERS; ++j) {
                 const int g = warp + j * K3_CONSUMER_WARPS;        // fragment lane == this thread's lane
                 float4 z = s.red[0][g][lane];
 #pragma unroll
@@ -229,7 +240,7 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
             }
             k3_consumer_sync();
             if (reduce && t < 16) {
-                for (int g = 0; g < K3_MAX_GROUPS; ++g) {
+                for (int g = 0; g < K3_PAD_GROUPS; ++g) {
                     const float o = s.rowred[g][t];
                     running = p.e.red == FORGE_RED_SUM ? running + o : fmaxf(running, o);
                 }
@@ -300,7 +311,7 @@ forge_status_t k3_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     info->kernel = FORGE_KERNEL_BF16_SKINNY;
     info->tile_m = 16;
     info->tile_n = k3_box_groups(d, grid) * 8;
-    info->tile_k = K3_BK;
+    info->tile_k = K3_KB * K3_BK;
     info->stages = K3_STAGES;
     info->cluster = 1;
     info->threads = K3_THREADS;
@@ -340,7 +351,7 @@ forge_status_t k3_launch(Handle &h, const RunArgs &a)
     p.partial = h.ws.partial;
     p.counters = h.ws.counters;
     p.status = h.ws.status;
-    p.num_kb = (int)((d.K + K3_BK - 1) / K3_BK);
+    p.num_kb = (int)((d.K + K3_KB * K3_BK - 1) / (K3_KB * K3_BK));
     p.groups = (int)(d.N / 8);
     p.box_groups = h.info.tile_n / 8;
     k3_bf16_skinny_kernel<<<(unsigned)h.info.grid, K3_THREADS, K3_SMEM_BYTES, a.stream>>>(h.tmX, h.tmW, p);
