@@ -97,7 +97,12 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         ptx::prefetch_tmap(&tmX);
         ptx::prefetch_tmap(&tmW);
     }
+    // This kernel is short (tens of microseconds), so the gap between two launches matters: let
+    // the next launch set itself up on each SM as soon as this CTA leaves it, and touch global
+    // memory only once everything earlier in the stream has completed.
+    ptx::pdl_launch_dependents();
     __syncthreads();
+    ptx::pdl_wait();
 
     if (warp == K3_CONSUMER_WARPS) {
         // ---------------- TMA producer ----------------
@@ -354,8 +359,17 @@ forge_status_t k3_launch(Handle &h, const RunArgs &a)
     p.num_kb = (int)((d.K + K3_KB * K3_BK - 1) / (K3_KB * K3_BK));
     p.groups = (int)(d.N / 8);
     p.box_groups = h.info.tile_n / 8;
-    k3_bf16_skinny_kernel<<<(unsigned)h.info.grid, K3_THREADS, K3_SMEM_BYTES, a.stream>>>(h.tmX, h.tmW, p);
-    return cudaGetLastError() == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)h.info.grid);
+    cfg.blockDim = dim3(K3_THREADS);
+    cfg.dynamicSmemBytes = K3_SMEM_BYTES;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k3_bf16_skinny_kernel, h.tmX, h.tmW, p) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
 }
 
 }  // namespace forge

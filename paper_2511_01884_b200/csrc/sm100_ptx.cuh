@@ -34,6 +34,14 @@ __device__ __forceinline__ bool elect_one()
     return pred != 0;
 }
 
+// ---- programmatic dependent launch --------------------------------------------------------
+// launch_dependents: the next kernel in the stream (if it was launched with programmatic
+// stream serialisation) may start placing CTAs as soon as every CTA of this grid has issued
+// this or exited.  wait: block until the previous grid has completed and its memory is visible;
+// nothing that depends on earlier work in the stream may be touched before it.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- mbarrier ----------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
 {
