@@ -388,6 +388,7 @@ def main():
                     continue
                 w2 = wk.WORKLOADS[name]
                 torch.cuda.empty_cache()
+                time.sleep(2.0)      # each workload is measured from the same (burst) power state, not in the wake of the previous one
                 i2 = wk.make_inputs(w2)
                 d2 = device_tensors(w2, i2, torch)
                 op2 = make_op(w2, w2.M, local)

@@ -5,8 +5,9 @@
 //               4-stage shared-memory ring, completion counted in bytes on "full" mbarriers;
 //   warp 1      MMA issuer: one elected thread issues tcgen05.mma (128x256x16, fp32 accumulate
 //               in TMEM); tcgen05.commit releases ring stages and publishes finished tiles;
-//   warps 2..5  epilogue: tcgen05.ld of the accumulator (thread <-> output row), bias,
-//               activation, scale, then either bf16 stores of Y or the row sum / max.
+//   warps 2..9  epilogue, two groups of four warps, each owning one 128-column half of every
+//               tile: tcgen05.ld of the accumulator (thread <-> output row), bias, activation,
+//               scale, then either bf16 stores of Y or the row sum / max.
 // TMEM holds two 128x256 fp32 accumulators, so the epilogue of tile i overlaps the MMAs of
 // tile i+1.  No load is multicast; every wait is bounded (see ptx::mbar_wait).
 //
@@ -27,7 +28,7 @@
 namespace forge {
 
 constexpr int K2_BM = 128, K2_BN = 256, K2_BK = 64, K2_STAGES = 4;
-constexpr int K2_THREADS = 192;
+constexpr int K2_THREADS = 320;              // TMA warp, MMA warp, 2 x 4 epilogue warps
 constexpr int K2_EPI_THREADS = 128;
 constexpr uint32_t K2_A_BYTES = K2_BM * K2_BK * 2;
 constexpr uint32_t K2_B_BYTES = K2_BN * K2_BK * 2;
@@ -41,7 +42,7 @@ struct K2Smem {
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint32_t tmem_base;
-    int last_flag;
+    int last_flag[2];
     int abort_flag;
     float bias[2][K2_BN];
     float gamma[2][K2_BN];
@@ -55,7 +56,7 @@ struct K2Params {
     int M, N, K;
     Epilogue e;
     const __nv_bfloat16 *gamma, *beta;
-    float *partial;       // sum/max: [tiles_n][M] floats; layernorm: [tiles_n][M] float4 triples
+    float *partial;       // per half tile: sum/max [2*tiles_n][M] floats; layernorm [2*tiles_n][M] float4 triples
     unsigned *counters;   // [tiles_m]
     int *status;
     int tiles_m, tiles_n, num_kb;
@@ -77,7 +78,8 @@ __device__ __forceinline__ void k2_tile_coords(int t, int tiles_m, int tiles_n, 
     tn = r / gm;
 }
 
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(K2_EPI_THREADS) : "memory"); }
+// named barrier of epilogue group g (ids 1 and 2; 0 is __syncthreads)
+__device__ __forceinline__ void epi_bar_sync(int g) { asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(K2_EPI_THREADS) : "memory"); }
 
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
 {
@@ -100,7 +102,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < K2_STAGES; ++i) { ptx::mbar_init(&s.full[i], 1); ptx::mbar_init(&s.empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&s.acc_full[i], 1); ptx::mbar_init(&s.acc_empty[i], 4); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&s.acc_full[i], 1); ptx::mbar_init(&s.acc_empty[i], 8); }
         s.abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmX);
@@ -162,39 +164,45 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         }
     } else {
         // ---------------- epilogue ----------------
+        // Two independent groups of four warps; group h owns columns [128h, 128h+128) of every
+        // tile ("part" 2*tn + h of the row strip) and has its own named barrier.
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
-        const int et = threadIdx.x - 64;              // 0..127
+        const int h = (warp - 2) >> 2;                // column half
+        const int et = (threadIdx.x - 64) & (K2_EPI_THREADS - 1);     // 0..127 inside the group
+        constexpr int HALF = K2_BN / 2, CHUNKS = HALF / 32;
+        const int parts = 2 * p.tiles_n;
         int acc = 0;
         uint32_t acc_phase = 0;
         const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             int tm, tn;
             k2_tile_coords<LN>(t, p.tiles_m, p.tiles_n, tm, tn);
-            const int m0 = tm * K2_BM, n0 = tn * K2_BN;
-            // bias of this tile -> shared memory (fp32), two values per thread
-            for (int j = et; j < K2_BN; j += K2_EPI_THREADS)
-                s.bias[acc][j] = (p.e.has_bias && n0 + j < p.N) ? __bfloat162float(p.b[n0 + j]) : 0.f;
-            if (LN) {
-                for (int j = et; j < K2_BN; j += K2_EPI_THREADS) {
-                    const bool in = n0 + j < p.N;
-                    s.gamma[acc][j] = in ? __bfloat162float(p.gamma[n0 + j]) : 0.f;
-                    s.beta[acc][j] = in ? __bfloat162float(p.beta[n0 + j]) : 0.f;
+            const int m0 = tm * K2_BM, n0 = tn * K2_BN + h * HALF;
+            const int part = 2 * tn + h;
+            float *sb = s.bias[acc] + h * HALF, *sg = s.gamma[acc] + h * HALF, *sbe = s.beta[acc] + h * HALF;
+            // bias (and gamma, beta) of this half tile -> shared memory as fp32, one value per thread
+            {
+                const bool in = n0 + et < p.N;
+                sb[et] = (p.e.has_bias && in) ? __bfloat162float(p.b[n0 + et]) : 0.f;
+                if (LN) {
+                    sg[et] = in ? __bfloat162float(p.gamma[n0 + et]) : 0.f;
+                    sbe[et] = in ? __bfloat162float(p.beta[n0 + et]) : 0.f;
                 }
             }
-            // the give-up decision must be taken by all 128 epilogue threads together
+            // the give-up decision must be taken by all threads of the group together
             if (!ptx::mbar_wait(&s.acc_full[acc], acc_phase, p.status, SITE_ACC_FULL)) s.abort_flag = 1;
-            epi_bar_sync();
+            epi_bar_sync(h);
             if (*(volatile int *)&s.abort_flag) { ok = false; break; }
             ptx::tc_fence_after();
 
             const int row = m0 + q * 32 + lane;
-            const uint32_t taddr = tmem_base + (uint32_t)acc * K2_BN + ((uint32_t)(q * 32) << 16);
+            const uint32_t taddr = tmem_base + (uint32_t)(acc * K2_BN + h * HALF) + ((uint32_t)(q * 32) << 16);
 
             if (LN) {
-                // ---- sweep 1: activated values back to TMEM, row statistics of this tile ----
+                // ---- sweep 1: activated values back to TMEM, row statistics of this half tile ----
                 RowStat rs{0.f, 0.f, 0.f};
 #pragma unroll 1
-                for (int c = 0; c < K2_BN / 32; ++c) {
+                for (int c = 0; c < CHUNKS; ++c) {
                     const int col0 = n0 + c * 32;
                     if (col0 >= p.N) break;
                     uint32_t r[32];
@@ -202,32 +210,42 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                     ptx::tmem_ld_wait();
                     float v[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + s.bias[acc][c * 32 + j];
+                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
                     apply_act_array<false>(p.e.act, v, p.e.scale);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(v[j]);
                     ptx::tmem_st_32x32(taddr + c * 32, r);
                     const int nv = min(32, p.N - col0);
-                    float sum = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) sum += j < nv ? v[j] : 0.f;
                     RowStat cs;
                     cs.n = (float)nv;
-                    cs.mean = sum / cs.n;
-                    cs.m2 = 0.f;
+                    if (nv == 32) {
+                        float sum = 0.f;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float dlt = j < nv ? v[j] - cs.mean : 0.f;
-                        cs.m2 = fmaf(dlt, dlt, cs.m2);
+                        for (int j = 0; j < 32; ++j) sum += v[j];
+                        cs.mean = sum * (1.0f / 32.0f);
+                        cs.m2 = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) { const float dlt = v[j] - cs.mean; cs.m2 = fmaf(dlt, dlt, cs.m2); }
+                    } else {
+                        float sum = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) sum += j < nv ? v[j] : 0.f;
+                        cs.mean = sum / cs.n;
+                        cs.m2 = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float dlt = j < nv ? v[j] - cs.mean : 0.f;
+                            cs.m2 = fmaf(dlt, dlt, cs.m2);
+                        }
                     }
                     rs = merge_stat(rs, cs);
                 }
                 ptx::tmem_st_wait();
                 float4 *stats = reinterpret_cast<float4 *>(p.partial);
-                if (row < p.M) stats[(size_t)tn * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
-                // ---- publish, then wait (bounded) for the other tiles of this strip ----
+                if (row < p.M) stats[(size_t)part * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
+                // ---- publish, then wait (bounded) for the other parts of this strip ----
                 __threadfence();
-                epi_bar_sync();
+                epi_bar_sync(h);
                 if (et == 0) {
                     atomicAdd(&p.counters[tm], 1u);
                     uint64_t t0 = 0;
@@ -237,28 +255,28 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                             const uint64_t now = ptx::globaltimer_ns();
                             if (t0 == 0) t0 = now;
                             else if (now - t0 > ptx::kWaitBudgetNs) {
-                                report_timeout(p.status, SITE_ARRIVAL);
+                                report_timeout(p.status, SITE_ARRIVAL, tm);
                                 s.abort_flag = 1;
                                 break;
                             }
                         }
                     }
                 }
-                epi_bar_sync();
+                epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
                 __threadfence();
                 if (row < p.M) {
                     const float4 f = __ldcg(&stats[row]);
                     rs = RowStat{f.x, f.y, f.z};
-                    for (int i = 1; i < p.tiles_n; ++i) {
+                    for (int i = 1; i < parts; ++i) {
                         const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
                         rs = merge_stat(rs, RowStat{o.x, o.y, o.z});
                     }
                 }
-                const float mean = rs.mean, rstd = rsqrtf(rs.m2 / rs.n + p.e.eps);
+                const float rstd = rsqrtf(rs.m2 / rs.n + p.e.eps), shift = -rs.mean * rstd;
                 // ---- sweep 2: normalise out of TMEM and store ----
 #pragma unroll 1
-                for (int c = 0; c < K2_BN / 32; ++c) {
+                for (int c = 0; c < CHUNKS; ++c) {
                     const int col0 = n0 + c * 32;
                     if (col0 >= p.N) break;
                     uint32_t r[32];
@@ -273,7 +291,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) {
                                     const int cc = c * 32 + i * 8 + j;
-                                    y[j] = fmaf((__uint_as_float(r[i * 8 + j]) - mean) * rstd, s.gamma[acc][cc], s.beta[acc][cc]);
+                                    y[j] = fmaf(fmaf(__uint_as_float(r[i * 8 + j]), rstd, shift), sg[cc], sbe[cc]);
                                 }
                                 uint4 w;
                                 w.x = ptx::pack_bf16x2(y[0], y[1]);
@@ -291,9 +309,10 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 if ((acc ^= 1) == 0) acc_phase ^= 1;
                 continue;
             }
+
             float red = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY;
 #pragma unroll 1
-            for (int c = 0; c < K2_BN / 32; ++c) {
+            for (int c = 0; c < CHUNKS; ++c) {
                 const int col0 = n0 + c * 32;
                 if (col0 >= p.N) break;
                 uint32_t r[32];
@@ -301,7 +320,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 ptx::tmem_ld_wait();
                 float v[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + s.bias[acc][c * 32 + j];
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
                 apply_act_array<false>(p.e.act, v, p.e.scale);
                 if (reduce) {
 #pragma unroll
@@ -328,27 +347,24 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             if (lane == 0) ptx::mbar_arrive(&s.acc_empty[acc]);
 
             if (reduce) {
+                // per-part row partials; the group that arrives last at the strip folds them in order
                 float *out = reinterpret_cast<float *>(p.out);
-                if (p.tiles_n == 1) {
-                    if (row < p.M) out[row] = red;
-                } else {
-                    if (row < p.M) p.partial[(size_t)tn * p.M + row] = red;
+                if (row < p.M) p.partial[(size_t)part * p.M + row] = red;
+                __threadfence();
+                epi_bar_sync(h);
+                if (et == 0) s.last_flag[h] = (atomicAdd(&p.counters[tm], 1u) == (unsigned)(parts - 1));
+                epi_bar_sync(h);
+                if (s.last_flag[h]) {
                     __threadfence();
-                    epi_bar_sync();
-                    if (et == 0) s.last_flag = (atomicAdd(&p.counters[tm], 1u) == (unsigned)(p.tiles_n - 1));
-                    epi_bar_sync();
-                    if (s.last_flag) {
-                        __threadfence();
-                        if (row < p.M) {
-                            float v = __ldcg(&p.partial[row]);
-                            for (int i = 1; i < p.tiles_n; ++i) {
-                                const float o = __ldcg(&p.partial[(size_t)i * p.M + row]);
-                                v = p.e.red == FORGE_RED_SUM ? v + o : fmaxf(v, o);
-                            }
-                            out[row] = v;
+                    if (row < p.M) {
+                        float v = __ldcg(&p.partial[row]);
+                        for (int i = 1; i < parts; ++i) {
+                            const float o = __ldcg(&p.partial[(size_t)i * p.M + row]);
+                            v = p.e.red == FORGE_RED_SUM ? v + o : fmaxf(v, o);
                         }
-                        if (et == 0) p.counters[tm] = 0u;
+                        out[row] = v;
                     }
+                    if (et == 0) p.counters[tm] = 0u;
                 }
             }
             if ((acc ^= 1) == 0) acc_phase ^= 1;
@@ -380,8 +396,8 @@ forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     info->threads = K2_THREADS;
     info->grid = tiles_m * tiles_n < sm_count ? tiles_m * tiles_n : sm_count;
     info->smem_bytes = (int64_t)K2_SMEM_BYTES;
-    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) && tiles_n > 1;
-    wl->partial_floats = partials ? (size_t)tiles_n * (size_t)d.M : 0;
+    const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX;      // one partial per row and half tile
+    wl->partial_floats = partials ? 2 * (size_t)tiles_n * (size_t)d.M : 0;
     wl->counters = partials ? (size_t)tiles_m : 0;
     return FORGE_OK;
 }
@@ -400,7 +416,7 @@ forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     // the tiles of a strip wait for one another: they must all be resident at once
     if (tiles_n > sm_count) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_BF16_TCGEN05_LN;
-    wl->partial_floats = 4 * (size_t)tiles_n * (size_t)d.M;
+    wl->partial_floats = 4 * 2 * (size_t)tiles_n * (size_t)d.M;          // one float4 per row and half tile
     wl->counters = (size_t)tiles_m;
     return FORGE_OK;
 }
@@ -449,9 +465,9 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
         k2_bf16_tcgen05_kernel<false><<<(unsigned)h.info.grid, K2_THREADS, K2_SMEM_BYTES, a.stream>>>(h.tmX, h.tmW, p);
         return cudaGetLastError() == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
     }
-    // Strip counters only ever grow: run r completes a strip at r * tiles_n arrivals.
+    // Strip counters only ever grow: run r completes a strip at r * 2 * tiles_n arrivals (half tiles).
     h.run_gen += 1;
-    p.ln_target = h.run_gen * (unsigned)p.tiles_n;
+    p.ln_target = h.run_gen * 2u * (unsigned)p.tiles_n;
     void *args[] = {(void *)&h.tmX, (void *)&h.tmW, (void *)&p};
     return cudaLaunchCooperativeKernel((const void *)k2_bf16_tcgen05_kernel<true>, dim3((unsigned)h.info.grid), dim3(K2_THREADS),
                                        args, K2_SMEM_BYTES, a.stream) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
