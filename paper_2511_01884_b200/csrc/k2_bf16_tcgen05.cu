@@ -21,24 +21,35 @@
 // through global memory; the un-normalised tile never leaves the SM.  The wait is hidden
 // behind the MMAs of the next tile (other TMEM buffer).  CTAs wait on one another, so the
 // launch is cooperative and a strip may not have more tiles than there are CTAs.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
 
 namespace forge {
 
-constexpr int K2_BM = 128, K2_BN = 256, K2_BK = 64, K2_STAGES = 4;
+constexpr int K2_BM = 128, K2_BN = 256, K2_BK = 64;
+constexpr int K2_MAX_STAGES = 6;
 constexpr int K2_THREADS = 320;              // TMA warp, MMA warp, 2 x 4 epilogue warps
 constexpr int K2_EPI_THREADS = 128;
 constexpr uint32_t K2_A_BYTES = K2_BM * K2_BK * 2;
-constexpr uint32_t K2_B_BYTES = K2_BN * K2_BK * 2;
-constexpr uint32_t K2_STAGE_BYTES = K2_A_BYTES + K2_B_BYTES;
 constexpr uint32_t K2_TMEM_COLS = 512;
+// Shared-memory ring.  One CTA per tile: a stage holds the 128-row X tile and the 256-row W tile
+// (48 KiB, 4 stages).  CTA pair (cta_group::2, 256x256 tile per pair): each CTA holds its own
+// 128 rows of X and its 128-row half of the W tile (32 KiB, 6 stages); the tensor cores of both
+// SMs read each half once.
+template <bool PAIR> struct K2Ring {
+    static constexpr uint32_t B_BYTES = (PAIR ? K2_BN / 2 : K2_BN) * K2_BK * 2;
+    static constexpr uint32_t STAGE_BYTES = K2_A_BYTES + B_BYTES;
+    static constexpr int STAGES = PAIR ? 6 : 4;
+    static constexpr uint32_t BYTES = STAGES * STAGE_BYTES;      // 192 KiB either way
+};
 constexpr int K2_GROUP_M = 16;      // row tiles per rasterisation group (keeps a wave's operands in L2)
 
 struct K2Smem {
-    uint64_t full[K2_STAGES];
-    uint64_t empty[K2_STAGES];
+    uint64_t full[K2_MAX_STAGES];
+    uint64_t empty[K2_MAX_STAGES];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint32_t tmem_base;
@@ -48,7 +59,8 @@ struct K2Smem {
     float gamma[2][K2_BN];
     float beta[2][K2_BN];
 };
-constexpr size_t K2_SMEM_BYTES = 1024 + (size_t)K2_STAGES * K2_STAGE_BYTES + sizeof(K2Smem);
+constexpr size_t K2_SMEM_BYTES = 1024 + (size_t)K2Ring<false>::BYTES + sizeof(K2Smem);
+static_assert(K2Ring<false>::BYTES == K2Ring<true>::BYTES, "both ring layouts use the same shared memory");
 
 struct K2Params {
     const __nv_bfloat16 *b;
@@ -59,7 +71,7 @@ struct K2Params {
     float *partial;       // per half tile: sum/max [2*tiles_n][M] floats; layernorm [2*tiles_n][M] float4 triples
     unsigned *counters;   // [tiles_m]
     int *status;
-    int tiles_m, tiles_n, num_kb;
+    int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     unsigned ln_target;   // layernorm: counter value at which a strip is complete in this run
 };
 
@@ -88,32 +100,53 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
     return v;
 }
 
-template <bool LN>
+// PAIR: the kernel runs as clusters of two CTAs on one TPC.  A pair owns a 256x256 output tile:
+// CTA `rank` loads rows [128 rank, 128 rank + 128) of the X tile and of the W tile; the leader
+// (rank 0) issues tcgen05.mma.cta_group::2, which accumulates 128 rows x 256 columns in the TMEM
+// of each CTA; each CTA runs the epilogue of its own 128 rows.  Barriers: both CTAs' loads are
+// credited to the leader's "full" barrier, tcgen05.commit signals the "empty" and "accumulator
+// full" barriers of both CTAs, the epilogues of both CTAs arrive on the leader's "accumulator
+// empty" barrier.
+template <bool LN, bool PAIR>
 __global__ void __launch_bounds__(K2_THREADS, 1)
 k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const K2Params p)
 {
+    using Ring = K2Ring<PAIR>;
+    constexpr int STAGES = Ring::STAGES;
+    constexpr uint32_t STAGE_BYTES = Ring::STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    K2Smem &s = *reinterpret_cast<K2Smem *>(tiles + (size_t)K2_STAGES * K2_STAGE_BYTES);
+    K2Smem &s = *reinterpret_cast<K2Smem *>(tiles + (size_t)Ring::BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int total_tiles = p.tiles_m * p.tiles_n;
+    const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;        // position in the pair; 0 leads
+    // work units: tiles (one CTA each) or 256-row pair tiles (one cluster each)
+    const int unit_rows = PAIR ? (p.tiles_m + 1) / 2 : p.tiles_m;
+    const int total_tiles = unit_rows * p.tiles_n;
+    const int first_unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int unit_stride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     bool ok = true;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < K2_STAGES; ++i) { ptx::mbar_init(&s.full[i], 1); ptx::mbar_init(&s.empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&s.acc_full[i], 1); ptx::mbar_init(&s.acc_empty[i], 8); }
+        for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&s.full[i], 1); ptx::mbar_init(&s.empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&s.acc_full[i], 1); ptx::mbar_init(&s.acc_empty[i], PAIR ? 16 : 8); }
         s.abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmX);
         ptx::prefetch_tmap(&tmW);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(&s.tmem_base, K2_TMEM_COLS);
-        ptx::tmem_relinquish();
+        if (PAIR) {
+            ptx::tmem_alloc_pair(&s.tmem_base, K2_TMEM_COLS);
+            ptx::tmem_relinquish_pair();
+        } else {
+            ptx::tmem_alloc(&s.tmem_base, K2_TMEM_COLS);
+            ptx::tmem_relinquish();
+        }
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (PAIR) ptx::cluster_sync_all();       // the peer's barriers exist before anything signals them
     ptx::tc_fence_after();
     const uint32_t tmem_base = s.tmem_base;
 
@@ -122,43 +155,57 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         if (ptx::elect_one()) {
             int stage = 0;
             uint32_t phase = 0;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int t = first_unit; t < total_tiles && ok; t += unit_stride) {
                 int tm, tn;
-                k2_tile_coords<LN>(t, p.tiles_m, p.tiles_n, tm, tn);
+                k2_tile_coords<LN>(t, unit_rows, p.tiles_n, tm, tn);
+                if (PAIR) tm = 2 * tm + (int)rank;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
-                    uint8_t *a = tiles + (size_t)stage * K2_STAGE_BYTES;
-                    ptx::mbar_expect_tx(&s.full[stage], K2_STAGE_BYTES);
-                    ptx::tma_load_2d(a, &tmX, &s.full[stage], kb * K2_BK, tm * K2_BM);
-                    ptx::tma_load_2d(a + K2_A_BYTES, &tmW, &s.full[stage], kb * K2_BK, tn * K2_BN);
-                    if (++stage == K2_STAGES) { stage = 0; phase ^= 1; }
+                    uint8_t *a = tiles + (size_t)stage * STAGE_BYTES;
+                    if (PAIR) {
+                        // the leader's barrier counts the bytes of both CTAs (rows past M or N are zero fill
+                        // and count in full)
+                        if (rank == 0) ptx::mbar_expect_tx(&s.full[stage], 2 * STAGE_BYTES);
+                        const uint32_t bar = ptx::mapa_u32(ptx::smem_u32(&s.full[stage]), 0);
+                        ptx::tma_load_2d_pair(a, &tmX, bar, kb * K2_BK, tm * K2_BM);
+                        ptx::tma_load_2d_pair(a + K2_A_BYTES, &tmW, bar, kb * K2_BK, tn * K2_BN + (int)rank * (K2_BN / 2));
+                    } else {
+                        ptx::mbar_expect_tx(&s.full[stage], STAGE_BYTES);
+                        ptx::tma_load_2d(a, &tmX, &s.full[stage], kb * K2_BK, tm * K2_BM);
+                        ptx::tma_load_2d(a + K2_A_BYTES, &tmW, &s.full[stage], kb * K2_BK, tn * K2_BN);
+                    }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (ptx::elect_one()) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(K2_BM, K2_BN);
+        if ((!PAIR || rank == 0) && ptx::elect_one()) {
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(PAIR ? 2 * K2_BM : K2_BM, K2_BN);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int t = first_unit; t < total_tiles && ok; t += unit_stride) {
                 if (!ptx::mbar_wait(&s.acc_empty[acc], acc_phase ^ 1, p.status, SITE_ACC_EMPTY)) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * K2_BN;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (!ptx::mbar_wait(&s.full[stage], phase, p.status, SITE_TMA_FULL)) { ok = false; break; }
                     ptx::tc_fence_after();
-                    const uint8_t *a = tiles + (size_t)stage * K2_STAGE_BYTES;
+                    const uint8_t *a = tiles + (size_t)stage * STAGE_BYTES;
                     const uint64_t adesc = ptx::smem_desc_k_sw128(a);
                     const uint64_t bdesc = ptx::smem_desc_k_sw128(a + K2_A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < K2_BK / 16; ++k)      // 16 bf16 = 32 bytes = 2 descriptor units
-                        ptx::umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
-                    ptx::umma_commit(&s.empty[stage]);
-                    if (++stage == K2_STAGES) { stage = 0; phase ^= 1; }
+                    for (int k = 0; k < K2_BK / 16; ++k) {     // 16 bf16 = 32 bytes = 2 descriptor units
+                        if (PAIR) ptx::umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                        else ptx::umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                    }
+                    if (PAIR) ptx::umma_commit_pair(&s.empty[stage], 3);
+                    else ptx::umma_commit(&s.empty[stage]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
-                ptx::umma_commit(&s.acc_full[acc]);
+                if (PAIR) ptx::umma_commit_pair(&s.acc_full[acc], 3);
+                else ptx::umma_commit(&s.acc_full[acc]);
                 if ((acc ^= 1) == 0) acc_phase ^= 1;
             }
         }
@@ -174,9 +221,12 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         int acc = 0;
         uint32_t acc_phase = 0;
         const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+        const uint32_t acc_empty_addr[2] = {ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[0]), 0),
+                                            ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[1]), 0)};   // the leader's (PAIR)
+        for (int t = first_unit; t < total_tiles; t += unit_stride) {
             int tm, tn;
-            k2_tile_coords<LN>(t, p.tiles_m, p.tiles_n, tm, tn);
+            k2_tile_coords<LN>(t, unit_rows, p.tiles_n, tm, tn);
+            if (PAIR) tm = 2 * tm + (int)rank;
             const int m0 = tm * K2_BM, n0 = tn * K2_BN + h * HALF;
             const int part = 2 * tn + h;
             float *sb = s.bias[acc] + h * HALF, *sg = s.gamma[acc] + h * HALF, *sbe = s.beta[acc] + h * HALF;
@@ -197,6 +247,14 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 
             const int row = m0 + q * 32 + lane;
             const uint32_t taddr = tmem_base + (uint32_t)(acc * K2_BN + h * HALF) + ((uint32_t)(q * 32) << 16);
+            if (PAIR && m0 >= p.M) {
+                // second half of the last pair tile lies past M: nothing to publish, free the accumulator
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
+                if ((acc ^= 1) == 0) acc_phase ^= 1;
+                continue;
+            }
 
             if (LN) {
                 // ---- sweep 1: activated values back to TMEM, row statistics of this half tile ----
@@ -305,7 +363,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&s.acc_empty[acc]);
+                if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
                 if ((acc ^= 1) == 0) acc_phase ^= 1;
                 continue;
             }
@@ -344,7 +402,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             // accumulator drained: hand the TMEM buffer back to the MMA warp
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&s.acc_empty[acc]);
+            if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
 
             if (reduce) {
                 // per-part row partials; the group that arrives last at the strip folds them in order
@@ -375,26 +433,46 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
     if (!ok) __nanosleep(200000);      // give-up path: let copies and MMAs already in flight land
     ptx::tc_fence_before();
     __syncthreads();
+    if (PAIR) ptx::cluster_sync_all();     // the peer no longer reads this CTA's shared memory or signals its barriers
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, K2_TMEM_COLS);
+        if (PAIR) ptx::tmem_dealloc_pair(tmem_base, K2_TMEM_COLS);
+        else ptx::tmem_dealloc(tmem_base, K2_TMEM_COLS);
     }
 }
 
 // ---- host side ---------------------------------------------------------------------------
+// CTA pairs need at least two 128-row strips and two SMs.  FORGE_K2_PAIR=0 forces one CTA per
+// tile (tuning aid).
+static bool k2_use_pair(const forge_fused_linear_desc_t &d, int sm_count)
+{
+    static int env = -1;
+    if (env < 0) {
+        const char *e = std::getenv("FORGE_K2_PAIR");
+        env = e ? (std::atoi(e) != 0) : 1;
+    }
+    return env && d.M > K2_BM && sm_count >= 2;
+}
+
 forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
     if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
     const int64_t tiles_m = (d.M + K2_BM - 1) / K2_BM, tiles_n = (d.N + K2_BN - 1) / K2_BN;
     if (tiles_m * tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    const bool pair = k2_use_pair(d, sm_count);
     info->kernel = FORGE_KERNEL_BF16_TCGEN05;
-    info->tile_m = K2_BM;
+    info->tile_m = pair ? 2 * K2_BM : K2_BM;
     info->tile_n = K2_BN;
     info->tile_k = K2_BK;
-    info->stages = K2_STAGES;
-    info->cluster = 1;
+    info->stages = pair ? K2Ring<true>::STAGES : K2Ring<false>::STAGES;
+    info->cluster = pair ? 2 : 1;
     info->threads = K2_THREADS;
-    info->grid = tiles_m * tiles_n < sm_count ? tiles_m * tiles_n : sm_count;
+    if (pair) {
+        const int64_t units = ((tiles_m + 1) / 2) * tiles_n, clusters = sm_count / 2;
+        info->grid = 2 * (units < clusters ? units : clusters);
+    } else {
+        info->grid = tiles_m * tiles_n < sm_count ? tiles_m * tiles_n : sm_count;
+    }
     info->smem_bytes = (int64_t)K2_SMEM_BYTES;
     const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX;      // one partial per row and half tile
     wl->partial_floats = partials ? 2 * (size_t)tiles_n * (size_t)d.M : 0;
@@ -402,11 +480,14 @@ forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     return FORGE_OK;
 }
 
-forge_status_t k2_setup(Handle &)
+template <bool LN, bool PAIR>
+static forge_status_t k2_prepare()
 {
-    return cudaFuncSetAttribute(k2_bf16_tcgen05_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES) == cudaSuccess
-               ? FORGE_OK : FORGE_ERR_CUDA;
+    return cudaFuncSetAttribute(k2_bf16_tcgen05_kernel<LN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)K2_SMEM_BYTES) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
 }
+
+forge_status_t k2_setup(Handle &h) { return h.info.cluster == 2 ? k2_prepare<false, true>() : k2_prepare<false, false>(); }
 
 forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
@@ -414,7 +495,7 @@ forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     if (st != FORGE_OK) return st;
     const int64_t tiles_m = (d.M + K2_BM - 1) / K2_BM, tiles_n = (d.N + K2_BN - 1) / K2_BN;
     // the tiles of a strip wait for one another: they must all be resident at once
-    if (tiles_n > sm_count) return FORGE_ERR_UNSUPPORTED;
+    if (tiles_n > sm_count / info->cluster) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_BF16_TCGEN05_LN;
     wl->partial_floats = 4 * 2 * (size_t)tiles_n * (size_t)d.M;          // one float4 per row and half tile
     wl->counters = (size_t)tiles_m;
@@ -423,26 +504,54 @@ forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
 
 forge_status_t k4_setup(Handle &h)
 {
-    if (cudaFuncSetAttribute(k2_bf16_tcgen05_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K2_SMEM_BYTES) != cudaSuccess)
-        return FORGE_ERR_CUDA;
+    const bool pair = h.info.cluster == 2;
+    if ((pair ? k2_prepare<true, true>() : k2_prepare<true, false>()) != FORGE_OK) return FORGE_ERR_CUDA;
     int coop = 0, per_sm = 0;
     if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h.d.device) != cudaSuccess || !coop) return FORGE_ERR_CUDA;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2_bf16_tcgen05_kernel<true>, K2_THREADS, K2_SMEM_BYTES) != cudaSuccess ||
-        (int64_t)per_sm * h.sm_count < h.info.grid)
-        return FORGE_ERR_CUDA;
+    const cudaError_t e = pair ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2_bf16_tcgen05_kernel<true, true>, K2_THREADS, K2_SMEM_BYTES)
+                               : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2_bf16_tcgen05_kernel<true, false>, K2_THREADS, K2_SMEM_BYTES);
+    if (e != cudaSuccess || (int64_t)per_sm * h.sm_count < h.info.grid) return FORGE_ERR_CUDA;
     return FORGE_OK;
+}
+
+template <bool LN, bool PAIR>
+static forge_status_t k2_launch_t(const Handle &h, const K2Params &p, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)h.info.grid);
+    cfg.blockDim = dim3(K2_THREADS);
+    cfg.dynamicSmemBytes = K2_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (PAIR) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = 2;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (LN) {           // CTAs wait on one another: all of them must be resident
+        attr[n].id = cudaLaunchAttributeCooperative;
+        attr[n].val.cooperative = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, k2_bf16_tcgen05_kernel<LN, PAIR>, h.tmX, h.tmW, p) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
 }
 
 static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
 {
     const forge_fused_linear_desc_t &d = h.d;
+    const bool pair = h.info.cluster == 2;
     forge_status_t st;
     if (h.tmX_ptr != a.X) {
         if ((st = encode_tmap_bf16(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, K2_BM, K2_BK)) != FORGE_OK) return st;
         h.tmX_ptr = a.X;
     }
     if (h.tmW_ptr != a.W) {
-        if ((st = encode_tmap_bf16(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, K2_BN, K2_BK)) != FORGE_OK) return st;
+        if ((st = encode_tmap_bf16(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, pair ? K2_BN / 2 : K2_BN, K2_BK)) != FORGE_OK) return st;
         h.tmW_ptr = a.W;
     }
     K2Params p;
@@ -461,16 +570,11 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     p.tiles_n = (int)((d.N + K2_BN - 1) / K2_BN);
     p.num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
     p.ln_target = 0;
-    if (!ln) {
-        k2_bf16_tcgen05_kernel<false><<<(unsigned)h.info.grid, K2_THREADS, K2_SMEM_BYTES, a.stream>>>(h.tmX, h.tmW, p);
-        return cudaGetLastError() == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
-    }
+    if (!ln) return pair ? k2_launch_t<false, true>(h, p, a.stream) : k2_launch_t<false, false>(h, p, a.stream);
     // Strip counters only ever grow: run r completes a strip at r * 2 * tiles_n arrivals (half tiles).
     h.run_gen += 1;
     p.ln_target = h.run_gen * 2u * (unsigned)p.tiles_n;
-    void *args[] = {(void *)&h.tmX, (void *)&h.tmW, (void *)&p};
-    return cudaLaunchCooperativeKernel((const void *)k2_bf16_tcgen05_kernel<true>, dim3((unsigned)h.info.grid), dim3(K2_THREADS),
-                                       args, K2_SMEM_BYTES, a.stream) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+    return pair ? k2_launch_t<true, true>(h, p, a.stream) : k2_launch_t<true, false>(h, p, a.stream);
 }
 
 forge_status_t k2_launch(Handle &h, const RunArgs &a) { return k24_launch(h, a, false); }
