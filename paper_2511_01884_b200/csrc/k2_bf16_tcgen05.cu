@@ -323,15 +323,26 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
                 __threadfence();
+                // Combine the strip's parts in part order, all at once (same result on every CTA):
+                // mean = sum n_i mean_i / sum n_i,  M2 = sum (M2_i + n_i (mean_i - mean)^2).
+                float rstd = 0.f, shift = 0.f;
                 if (row < p.M) {
-                    const float4 f = __ldcg(&stats[row]);
-                    rs = RowStat{f.x, f.y, f.z};
-                    for (int i = 1; i < parts; ++i) {
+                    float cnt = 0.f, wsum = 0.f;
+                    for (int i = 0; i < parts; ++i) {
                         const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
-                        rs = merge_stat(rs, RowStat{o.x, o.y, o.z});
+                        cnt += o.x;
+                        wsum = fmaf(o.x, o.y, wsum);
                     }
+                    const float mean = wsum / cnt;
+                    float m2 = 0.f;
+                    for (int i = 0; i < parts; ++i) {
+                        const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
+                        const float dm = o.y - mean;
+                        m2 += fmaf(o.x * dm, dm, o.z);
+                    }
+                    rstd = rsqrtf(m2 / cnt + p.e.eps);
+                    shift = -mean * rstd;
                 }
-                const float rstd = rsqrtf(rs.m2 / rs.n + p.e.eps), shift = -rs.mean * rstd;
                 // ---- sweep 2: normalise out of TMEM and store ----
 #pragma unroll 1
                 for (int c = 0; c < CHUNKS; ++c) {
