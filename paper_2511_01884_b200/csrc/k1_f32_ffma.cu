@@ -65,13 +65,32 @@ __device__ __forceinline__ void k1_stash(float (*S)[K1_BM + K1_PAD], int tid, co
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int idx = tid + i * K1_THREADS;
-        const int row = idx >> 2;
         const int k = (idx & 3) * 4;
+        // rows of the k-groups 8..15 are stored with bit 3 of the row index flipped: the four
+        // k-groups a warp writes at once then fall into four different bank octets
+        const int row = (idx >> 2) ^ (((k >> 3) & 1) << 3);
         S[k + 0][row] = r[i].x;
         S[k + 1][row] = r[i].y;
         S[k + 2][row] = r[i].z;
         S[k + 3][row] = r[i].w;
     }
+}
+
+// Two fp32 fused multiply-adds per instruction (sm_100 packed-pair FMA): the inner product is
+// bound by instruction issue, not by the FMA pipe, when it is written with scalar FFMA.
+__device__ __forceinline__ void ffma2(unsigned long long &d, unsigned long long a, unsigned long long b)
+{
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
+}
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
 
 template <bool VEC, int RED>
@@ -89,11 +108,11 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
     const int m0 = tile_m * K1_BM, n0 = tile_n * K1_BN;
     const int M = p.M, N = p.N, K = p.K;
 
-    float acc[8][8];
+    unsigned long long acc2[8][4];       // acc2[i][j] = accumulators (i, 2j) and (i, 2j+1)
 #pragma unroll
     for (int i = 0; i < 8; ++i)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+        for (int j = 0; j < 4; ++j) acc2[i][j] = 0ull;
 
     float4 ra[2], rb[2];
     k1_fetch<VEC>(p.X, M, K, m0, 0, tid, ra);
@@ -111,16 +130,19 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         }
 #pragma unroll
         for (int k = 0; k < K1_BK; ++k) {
-            const float4 a0 = *reinterpret_cast<const float4 *>(&As[buf][k][ty * 4]);
-            const float4 a1 = *reinterpret_cast<const float4 *>(&As[buf][k][64 + ty * 4]);
-            const float4 b0 = *reinterpret_cast<const float4 *>(&Bs[buf][k][tx * 4]);
-            const float4 b1 = *reinterpret_cast<const float4 *>(&Bs[buf][k][64 + tx * 4]);
+            const int flip = ((k >> 3) & 1) << 3;          // see k1_stash
+            const float4 a0 = *reinterpret_cast<const float4 *>(&As[buf][k][(ty * 4) ^ flip]);
+            const float4 a1 = *reinterpret_cast<const float4 *>(&As[buf][k][64 + ((ty * 4) ^ flip)]);
+            const ulonglong2 b0 = *reinterpret_cast<const ulonglong2 *>(&Bs[buf][k][(tx * 4) ^ flip]);
+            const ulonglong2 b1 = *reinterpret_cast<const ulonglong2 *>(&Bs[buf][k][64 + ((tx * 4) ^ flip)]);
             const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-            const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+            const unsigned long long b[4] = {b0.x, b0.y, b1.x, b1.y};      // column pairs as they lie in memory
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+            for (int i = 0; i < 8; ++i) {
+                const unsigned long long ai = pack2(a[i], a[i]);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+                for (int j = 0; j < 4; ++j) ffma2(acc2[i][j], ai, b[j]);
+            }
         }
         if (more) {
             k1_stash(As[buf ^ 1], tid, ra);
@@ -129,6 +151,12 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         __syncthreads();
         buf ^= 1;
     }
+
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) unpack2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
 
     // ---- epilogue: bias, activation, scale, in registers --------------------------------
     int col[8];
