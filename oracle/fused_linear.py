@@ -40,7 +40,7 @@ def _load():
         fp = ctypes.POINTER(ctypes.c_float)
         lib.forge_oracle_fused_linear.restype = ctypes.c_int
         lib.forge_oracle_fused_linear.argtypes = [
-            ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, fp, fp, fp, fp, fp,
+            ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, fp, fp, fp, fp, fp, fp,
             ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_double,
             ctypes.POINTER(ctypes.c_int64), ctypes.c_int64, ctypes.POINTER(ctypes.c_double)]
         lib.forge_oracle_act.restype = ctypes.c_double
@@ -68,8 +68,9 @@ def act(kind: int, z: float) -> float:
 def fused_linear(X: np.ndarray, W: np.ndarray, b: Optional[np.ndarray] = None,
                  gamma: Optional[np.ndarray] = None, beta: Optional[np.ndarray] = None,
                  act: int = 0, scale: float = 1.0, red: int = 0, eps: float = 1e-5,
-                 rows: Optional[Sequence[int]] = None) -> np.ndarray:
-    """float64 result for all rows of X, or for the listed ``rows`` only."""
+                 rows: Optional[Sequence[int]] = None, sub: Optional[np.ndarray] = None) -> np.ndarray:
+    """float64 result for all rows of X, or for the listed ``rows`` only.  ``sub`` is the
+    vector subtracted before the row mean of reduction 4 (mean-gelu-residual)."""
     lib = _load()
     M, K = X.shape
     N, K2 = W.shape
@@ -80,13 +81,14 @@ def fused_linear(X: np.ndarray, W: np.ndarray, b: Optional[np.ndarray] = None,
     ba, bp = _f32(b)
     ga, gp = _f32(gamma)
     bea, bep = _f32(beta)
+    sa, sp = _f32(sub)
     if rows is None:
         ra, rp, nrows = None, None, M
     else:
         ra = np.ascontiguousarray(rows, dtype=np.int64)
         rp, nrows = ra.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), int(ra.size)
-    out = np.empty((nrows,) if red in (1, 2) else (nrows, N), dtype=np.float64)
-    rc = lib.forge_oracle_fused_linear(M, N, K, Xp, Wp, bp, gp, bep, int(act), float(scale),
+    out = np.empty((nrows,) if red in (1, 2) else (nrows, K if red == 4 else N), dtype=np.float64)
+    rc = lib.forge_oracle_fused_linear(M, N, K, Xp, Wp, bp, gp, bep, sp, int(act), float(scale),
                                        int(red), float(eps), rp, nrows,
                                        out.ctypes.data_as(ctypes.POINTER(ctypes.c_double)))
     if rc != 0:

@@ -29,9 +29,9 @@ import numpy as np
 # depends on neither side.
 F32, BF16 = 0, 1
 ACT_IDENTITY, ACT_RELU, ACT_GELU_ERF, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3, 4
-RED_NONE, RED_SUM, RED_MAX, RED_LAYERNORM = 0, 1, 2, 3
+RED_NONE, RED_SUM, RED_MAX, RED_LAYERNORM, RED_MEAN_GELU_RESIDUAL = 0, 1, 2, 3, 4
 
-STREAM_X, STREAM_W, STREAM_B, STREAM_GAMMA, STREAM_BETA = 0, 1, 2, 3, 4
+STREAM_X, STREAM_W, STREAM_B, STREAM_GAMMA, STREAM_BETA, STREAM_SUB = 0, 1, 2, 3, 4, 5
 
 _MASK64 = np.uint64(0xFFFFFFFFFFFFFFFF)
 
@@ -138,6 +138,7 @@ class Workload:
     beta: Dist = Dist("none")
     seed: int = 0
     note: str = ""
+    sub: Dist = Dist("none")      # vector subtracted before the row mean (mean-gelu-residual only)
 
     @property
     def flops(self) -> int:
@@ -148,12 +149,19 @@ class Workload:
         return 4 if self.dtype == F32 else 2
 
     @property
+    def out_cols(self) -> int:
+        """Columns of the output matrix (0: the output is a vector of M floats)."""
+        if self.red in (RED_SUM, RED_MAX):
+            return 0
+        return self.K if self.red == RED_MEAN_GELU_RESIDUAL else self.N
+
+    @property
     def out_elems(self) -> int:
-        return self.M if self.red in (RED_SUM, RED_MAX) else self.M * self.N
+        return self.M * max(self.out_cols, 1)
 
     @property
     def out_bytes(self) -> int:
-        return self.M * 4 if self.red in (RED_SUM, RED_MAX) else self.M * self.N * self.elem_bytes
+        return self.M * 4 if self.out_cols == 0 else self.M * self.out_cols * self.elem_bytes
 
     @property
     def algorithmic_bytes(self) -> int:
@@ -164,6 +172,8 @@ class Workload:
             n += self.N
         if self.red == RED_LAYERNORM:
             n += 2 * self.N
+        if self.sub.kind != "none":
+            n += self.N
         return n * e + self.out_bytes
 
 
@@ -184,6 +194,14 @@ WORKLOADS: Dict[str, Workload] = {
                    Dist("normal", 1.0), Dist("normal", 0.02), Dist("normal", 0.02),
                    Dist("uniform", 0.9, 1.1), Dist("normal", 0.01),
                    note="bf16, GELU-tanh, LayerNorm over N"),
+}
+
+
+# Workloads beyond the five configurations: the paper's own case-study chain (Appendix B.1).
+EXTRA_WORKLOADS: Dict[str, Workload] = {
+    "n1": Workload("n1", F32, 4096, 4096, 4096, ACT_IDENTITY, RED_MEAN_GELU_RESIDUAL, 1.0, 0.0,
+                   Dist("normal", 1.0), Dist("uniform", -1 / 64, 1 / 64), Dist("uniform", -0.1, 0.1),
+                   note="fp32, subtract, row mean, GELU-erf, residual add", sub=Dist("uniform", -0.5, 0.5)),
 }
 
 
@@ -214,9 +232,10 @@ def make_inputs(wl: Workload, M: Optional[int] = None, row_offset: int = 0) -> D
     b = _draw(wl.bias, wl.seed, STREAM_B, wl.N)
     g = _draw(wl.gamma, wl.seed, STREAM_GAMMA, wl.N)
     be = _draw(wl.beta, wl.seed, STREAM_BETA, wl.N)
+    sb = _draw(wl.sub, wl.seed, STREAM_SUB, wl.N)
     r = lambda t: None if t is None else round_to_storage(t, wl.dtype)
     return {"X": r(x).reshape(rows, wl.K), "W": r(w).reshape(wl.N, wl.K),
-            "b": r(b), "gamma": r(g), "beta": r(be)}
+            "b": r(b), "gamma": r(g), "beta": r(be), "sub": r(sb)}
 
 
 def custom_workload(name: str, dtype: int, M: int, N: int, K: int, act: int, red: int,
@@ -229,7 +248,8 @@ def custom_workload(name: str, dtype: int, M: int, N: int, K: int, act: int, red
     return Workload(name, dtype, M, N, K, act, red, scale, ln_eps,
                     Dist("normal", 1.0), w, Dist("uniform", -0.1, 0.1) if has_bias else Dist("none"),
                     Dist("uniform", 0.9, 1.1) if ln else Dist("none"),
-                    Dist("normal", 0.01) if ln else Dist("none"), seed)
+                    Dist("normal", 0.01) if ln else Dist("none"), seed,
+                    sub=Dist("uniform", -0.5, 0.5) if red == RED_MEAN_GELU_RESIDUAL else Dist("none"))
 
 
 def sample_rows(M: int, tile: int = 128) -> np.ndarray:

@@ -40,13 +40,15 @@ def run_gpu(wl: wk.Workload, inp, check_status=True, op=None, repeats=1):
     own = op is None
     if own:
         op = B.FusedLinear(desc_of(wl, M))
-    if wl.red in (wk.RED_SUM, wk.RED_MAX):
+    if wl.out_cols == 0:
         out = torch.full((M,), float("nan"), dtype=torch.float32, device="cuda")
     else:
-        out = torch.full((M, wl.N), float("nan"), dtype=torch.float32 if wl.dtype == wk.F32 else torch.bfloat16,
+        out = torch.full((M, wl.out_cols), float("nan"), dtype=torch.float32 if wl.dtype == wk.F32 else torch.bfloat16,
                          device="cuda")
+    # the mean-gelu-residual chain takes its subtract vector in the gamma slot of the interface
+    aux = dev["sub"] if wl.red == wk.RED_MEAN_GELU_RESIDUAL else dev["gamma"]
     for _ in range(repeats):
-        op(dev["X"], dev["W"], dev["b"], dev["gamma"], dev["beta"], out)
+        op(dev["X"], dev["W"], dev["b"], aux, dev["beta"], out)
     torch.cuda.synchronize()
     if check_status:
         op.check()
@@ -59,7 +61,7 @@ def run_gpu(wl: wk.Workload, inp, check_status=True, op=None, repeats=1):
 def run_oracle(wl: wk.Workload, inp, rows=None):
     import oracle
     return oracle.fused_linear(inp["X"], inp["W"], inp["b"], inp["gamma"], inp["beta"], act=wl.act,
-                               scale=wl.scale, red=wl.red, eps=wl.ln_eps, rows=rows)
+                               scale=wl.scale, red=wl.red, eps=wl.ln_eps, rows=rows, sub=inp.get("sub"))
 
 
 def rel_err(g: np.ndarray, r: np.ndarray) -> float:

@@ -266,3 +266,55 @@ def test_bad_arguments_are_rejected():
         oracle.fused_linear(X, W, None, rows=[2])                    # row out of range
     with pytest.raises(ValueError):
         oracle.fused_linear(X, np.ones((4, 2), np.float32))          # K mismatch
+
+
+# ---- the case-study chain: Linear, subtract, row mean, GELU, residual add ---------------------
+def test_chain_worked_example():
+    g = _golden()
+    M, N, K = int(g["M"][0]), int(g["N"][0]), int(g["K"][0])
+    X, W, b = g["X"].reshape(M, K), g["W"].reshape(N, K), g["b"]
+    y = oracle.fused_linear(X, W, b, red=wk.RED_MEAN_GELU_RESIDUAL, sub=g["sub"])
+    assert y.shape == (M, K)
+    mean = g["rowmean_num"] / g["rowmean_den"]
+    want0 = X[0] + d_act(wk.ACT_GELU_ERF, float(Fraction(4, 3)))
+    np.testing.assert_allclose(y[0], want0, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(y[1], X[1] + g["gelu_of_minus_one"][0], rtol=0, atol=1e-15)
+    assert mean[1] == -1.0
+
+
+def test_chain_reduces_to_a_matrix_vector_product():
+    """The row mean of a linear map is linear: mean_n(X W^T + b - sub) = X wbar + mean(b - sub),
+    with wbar the mean of W's rows -- a float64 library GEMV plus the decimal GELU."""
+    rng = np.random.default_rng(21)
+    M, N, K = 9, 14, 11
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    b = rng.standard_normal(N).astype(np.float32)
+    sub = rng.standard_normal(N).astype(np.float32)
+    mu = X.astype(np.float64) @ W.astype(np.float64).mean(0) + (b.astype(np.float64) - sub.astype(np.float64)).mean()
+    want = X.astype(np.float64) + np.array([d_act(wk.ACT_GELU_ERF, float(v)) for v in mu])[:, None]
+    got = oracle.fused_linear(X, W, b, red=wk.RED_MEAN_GELU_RESIDUAL, sub=sub)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    # with an activation and a scale in front, the mean is taken of scale*act(Z) - sub
+    E = oracle.fused_linear(X, W, b, act=wk.ACT_RELU, scale=0.5)
+    mu2 = (E - sub.astype(np.float64)).mean(1)
+    want2 = X.astype(np.float64) + np.array([d_act(wk.ACT_GELU_ERF, float(v)) for v in mu2])[:, None]
+    got2 = oracle.fused_linear(X, W, b, act=wk.ACT_RELU, scale=0.5, red=wk.RED_MEAN_GELU_RESIDUAL, sub=sub)
+    np.testing.assert_allclose(got2, want2, rtol=0, atol=1e-12)
+
+
+def test_chain_special_cases():
+    rng = np.random.default_rng(22)
+    X = rng.standard_normal((4, 6)).astype(np.float32)
+    b = rng.standard_normal(5).astype(np.float32)
+    # zero weights and sub = b: the mean is exactly 0, gelu(0) = 0, the output is the input
+    y = oracle.fused_linear(X, np.zeros((5, 6), np.float32), b, red=wk.RED_MEAN_GELU_RESIDUAL, sub=b)
+    assert np.array_equal(y, X.astype(np.float64))
+    # no subtract vector means nothing is subtracted
+    W = rng.standard_normal((5, 6)).astype(np.float32)
+    y0 = oracle.fused_linear(X, W, b, red=wk.RED_MEAN_GELU_RESIDUAL)
+    y1 = oracle.fused_linear(X, W, b, red=wk.RED_MEAN_GELU_RESIDUAL, sub=np.zeros(5, np.float32))
+    assert np.array_equal(y0, y1)
+    # row subset
+    ys = oracle.fused_linear(X, W, b, red=wk.RED_MEAN_GELU_RESIDUAL, rows=[3, 1])
+    assert np.array_equal(ys, y0[[3, 1]])
