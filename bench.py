@@ -36,6 +36,7 @@ from paper_2511_01884_b200 import multigpu  # noqa: E402
 from paper_2511_01884_b200 import workloads as wk  # noqa: E402
 
 HEADLINE = "c3"
+ALL_WORKLOADS = {**wk.WORKLOADS, **wk.EXTRA_WORKLOADS}
 NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -140,10 +141,12 @@ def device_tensors(wl, inp, torch):
         return (t.to(torch.bfloat16) if wl.dtype == wk.BF16 else t).cuda()
     d = {k: dev(v) for k, v in inp.items()}
     M = inp["X"].shape[0]
-    if wl.red in (wk.RED_SUM, wk.RED_MAX):
+    if wl.out_cols == 0:
         d["out"] = torch.empty((M,), dtype=torch.float32, device="cuda")
     else:
-        d["out"] = torch.empty((M, wl.N), dtype=torch.bfloat16 if wl.dtype == wk.BF16 else torch.float32, device="cuda")
+        d["out"] = torch.empty((M, wl.out_cols), dtype=torch.bfloat16 if wl.dtype == wk.BF16 else torch.float32, device="cuda")
+    if wl.red == wk.RED_MEAN_GELU_RESIDUAL:
+        d["gamma"] = d["sub"]          # the chain's subtract vector travels in the gamma slot of the interface
     return d
 
 
@@ -252,7 +255,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    wl = wk.WORKLOADS[args.workload]
+    wl = ALL_WORKLOADS[args.workload]
     inp = wk.make_inputs(wl)
     per_step_target = max(1.0, min(10.0, 60.0 / max(1, args.steps + args.warmup)))
     first = oracle_sample(wl, inp, target_s=per_step_target)
@@ -286,7 +289,8 @@ def run_reference(args):
 def config_of(wl, n_gpus, extra=None):
     names = {wk.ACT_IDENTITY: "identity", wk.ACT_RELU: "relu", wk.ACT_GELU_ERF: "gelu_erf",
              wk.ACT_GELU_TANH: "gelu_tanh", wk.ACT_SILU: "silu"}
-    reds = {wk.RED_NONE: "none", wk.RED_SUM: "row_sum", wk.RED_MAX: "row_max", wk.RED_LAYERNORM: "layernorm"}
+    reds = {wk.RED_NONE: "none", wk.RED_SUM: "row_sum", wk.RED_MAX: "row_max", wk.RED_LAYERNORM: "layernorm",
+            wk.RED_MEAN_GELU_RESIDUAL: "subtract_rowmean_gelu_residual"}
     c = {"workload": f"{wl.name}: {wl.note}", "M_per_gpu": wl.M, "N": wl.N, "K": wl.K,
          "dtype": "bf16" if wl.dtype == wk.BF16 else "f32", "act": names[wl.act], "scale": wl.scale,
          "reduction": reds[wl.red], "seed": wl.seed, "parallelism": f"rows sharded over {n_gpus} gpu(s), no collective",
@@ -301,7 +305,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default=HEADLINE, choices=sorted(wk.WORKLOADS))
+    ap.add_argument("--workload", default=HEADLINE, choices=sorted(ALL_WORKLOADS))
     ap.add_argument("--impl", default="forge", choices=["forge", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the short runs of the other workloads")
     args = ap.parse_args()
@@ -327,7 +331,7 @@ def main():
 
     peaks = load_peaks()
     props = torch.cuda.get_device_properties(local)
-    wl = wk.WORKLOADS[args.workload]
+    wl = ALL_WORKLOADS[args.workload]
 
     # this rank's block of rows of the global [world * M, K] input; W, b, gamma, beta replicated
     rows, row_offset = multigpu.rank_rows_weak(wl, rank)
@@ -346,7 +350,7 @@ def main():
     # ---- end to end: pinned host buffers in, result out, through the host entry point ----
     e2e_steps = max(1, min(args.steps, 10))
     host = {}
-    for k in ("X", "W", "b", "gamma", "beta"):
+    for k in ("X", "W", "b", "gamma", "beta"):      # (gamma holds the subtract vector for the chain workload)
         host[k] = None if d[k] is None else d[k].cpu().pin_memory()
     host_out = torch.empty_like(d["out"], device="cpu").pin_memory()
     h2d = sum(v.numel() * v.element_size() for v in host.values() if v is not None)
@@ -383,17 +387,19 @@ def main():
         line["cpu_baseline"] = {k: v for k, v in oracle_sample(wl, inp).items() if k not in ("seconds", "rows")}
         if not args.no_extras:
             line["workloads"] = {}
-            for name in sorted(wk.WORKLOADS):
+            every = dict(wk.WORKLOADS)
+            every.update(wk.EXTRA_WORKLOADS)
+            for name in sorted(every):
                 if name == wl.name:
                     continue
-                w2 = wk.WORKLOADS[name]
+                w2 = every[name]
                 torch.cuda.empty_cache()
                 time.sleep(2.0)      # each workload is measured from the same (burst) power state, not in the wake of the previous one
                 i2 = wk.make_inputs(w2)
                 d2 = device_tensors(w2, i2, torch)
                 op2 = make_op(w2, w2.M, local)
                 fl = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device="cuda") if w2.algorithmic_bytes < 130e6 else None
-                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50}[name]
+                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50, "n1": 20}[name]
                 ms2 = time_steps(op2, d2, steps2, 3, torch, flush_buf=fl)
                 v2, u2 = unit_value(w2, ms2)
                 launches += steps2

@@ -5,6 +5,7 @@
  *     none:       Y[M,N]  = E
  *     sum / max:  out[M]  = sum_n E[m,n]  /  max_n E[m,n]
  *     layernorm:  Y[M,N]  = (E - mean_n E) / sqrt(var_n E + eps) * gamma[n] + beta[n]
+ *     mean-gelu-residual: Y[M,K] = X + gelu_erf(mean_n (E - sub[n]))   (see forge_red_t)
  *
  * The operation is the fused operator chain the paper's agents are asked to produce: one
  * kernel in place of a framework Linear (matmul + bias) followed by an element-wise
@@ -59,7 +60,13 @@ typedef enum {
     FORGE_RED_NONE = 0,
     FORGE_RED_SUM = 1,
     FORGE_RED_MAX = 2,
-    FORGE_RED_LAYERNORM = 3      /* population variance, eps inside the square root      */
+    FORGE_RED_LAYERNORM = 3,     /* population variance, eps inside the square root      */
+    FORGE_RED_MEAN_GELU_RESIDUAL = 4
+    /* The chain of the paper's Appendix B.1 case study (Linear, subtract, row mean, GELU,
+     * residual add of the layer's input, all in one kernel):
+     *     g[m] = gelu_erf(mean_n (E[m,n] - sub[n])),   Y[m,k] = X[m,k] + g[m]
+     * The output is Y [M,K] (the shape of X) in dtype.  run() takes the subtract vector sub[N]
+     * in its `gamma` argument (NULL: nothing is subtracted); `beta` is ignored.  fp32 only.   */
 } forge_red_t;
 
 typedef struct {
@@ -117,7 +124,8 @@ forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, 
  * Enqueue one evaluation on `cuda_stream` (a cudaStream_t; NULL = default stream).
  * DEVICE pointers, owned by the caller, 16-byte aligned, alive until the work completes:
  *   X [M,K], W [N,K], b [N] (may be NULL iff has_bias == 0), gamma, beta [N] (non-NULL iff
- *   layernorm), out: Y [M,N] in dtype (none, layernorm) or fp32 [M] (sum, max).
+ *   layernorm), out: Y [M,N] in dtype (none, layernorm), fp32 [M] (sum, max), or Y [M,K] in
+ *   dtype (mean-gelu-residual, whose subtract vector travels in `gamma`).
  * Allocates nothing and does not synchronise.  Returns only argument / launch errors;
  * device-side give-ups are reported by forge_fused_linear_last_status().  At most one run
  * per handle may be in flight (the workspace belongs to the handle).

@@ -15,7 +15,7 @@ constexpr size_t kStatusBytes = 256;     // status word lives alone in the first
 bool desc_enums_ok(const forge_fused_linear_desc_t &d)
 {
     return (d.dtype == FORGE_F32 || d.dtype == FORGE_BF16) && d.act >= FORGE_ACT_IDENTITY &&
-           d.act <= FORGE_ACT_SILU && d.red >= FORGE_RED_NONE && d.red <= FORGE_RED_LAYERNORM;
+           d.act <= FORGE_ACT_SILU && d.red >= FORGE_RED_NONE && d.red <= FORGE_RED_MEAN_GELU_RESIDUAL;
 }
 
 forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
@@ -30,6 +30,7 @@ forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_
         st = k1_plan(d, sm_count, info, wl);
     } else {
         if (d.K % 8 != 0 || d.N % 8 != 0) return FORGE_ERR_UNSUPPORTED;     // 16-byte row pitch for TMA
+        if (d.red == FORGE_RED_MEAN_GELU_RESIDUAL) return FORGE_ERR_UNSUPPORTED;   // fp32 only so far
         if (d.red == FORGE_RED_LAYERNORM) st = k4_plan(d, sm_count, info, wl);
         else if (d.M <= 16) st = k3_plan(d, sm_count, info, wl);
         else st = k2_plan(d, sm_count, info, wl);
@@ -59,8 +60,8 @@ struct DeviceGuard {
 size_t elem_bytes(const forge_fused_linear_desc_t &d) { return d.dtype == FORGE_F32 ? 4 : 2; }
 size_t out_bytes(const forge_fused_linear_desc_t &d)
 {
-    return (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) ? (size_t)d.M * 4
-                                                              : (size_t)d.M * (size_t)d.N * elem_bytes(d);
+    if (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) return (size_t)d.M * 4;
+    return (size_t)d.M * (size_t)(d.red == FORGE_RED_MEAN_GELU_RESIDUAL ? d.K : d.N) * elem_bytes(d);
 }
 
 forge_status_t check_run_args(const Handle &h, const RunArgs &a)
@@ -225,8 +226,11 @@ forge_status_t forge_fused_linear_run_host(forge_fused_linear_t hh, const void *
     if (ok && d.red == FORGE_RED_LAYERNORM)
         ok = cudaMemcpyAsync(h.hg, gamma, bn, cudaMemcpyHostToDevice, s) == cudaSuccess &&
              cudaMemcpyAsync(h.hbe, beta, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    const bool has_sub = d.red == FORGE_RED_MEAN_GELU_RESIDUAL && gamma;
+    if (ok && has_sub) ok = cudaMemcpyAsync(h.hg, gamma, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
     if (!ok) return FORGE_ERR_CUDA;
-    RunArgs a{h.hX, h.hW, d.has_bias ? h.hb : nullptr, h.hg, h.hbe, h.hout, s};
+    RunArgs a{h.hX, h.hW, d.has_bias ? h.hb : nullptr,
+              (d.red == FORGE_RED_LAYERNORM || has_sub) ? h.hg : nullptr, h.hbe, h.hout, s};
     const forge_status_t st = dispatch(h, a);
     if (st != FORGE_OK) return st;
     if (cudaMemcpyAsync(out, h.hout, bo, cudaMemcpyDeviceToHost, s) != cudaSuccess) return FORGE_ERR_CUDA;

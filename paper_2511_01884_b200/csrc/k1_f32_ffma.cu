@@ -31,6 +31,7 @@ struct K1Params {
     unsigned *counters;    // [tiles_m]
     int tiles_n;
     int out_vec4;          // Y rows can be written with 128-bit stores
+    int res_vec4;          // mean chain: X and Y rows ([M,K]) can be moved with 128-bit accesses
 };
 
 // One CTA-tile slab of 128 rows x 16 k from a K-major matrix into registers.
@@ -191,43 +192,72 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         return;
     }
 
-    if (RED == FORGE_RED_SUM || RED == FORGE_RED_MAX) {
+    if (RED == FORGE_RED_SUM || RED == FORGE_RED_MAX || RED == FORGE_RED_MEAN_GELU_RESIDUAL) {
+        constexpr bool ADD = RED != FORGE_RED_MAX;                       // row sum (also of the mean chain) or row max
+        constexpr bool CHAIN = RED == FORGE_RED_MEAN_GELU_RESIDUAL;      // subtract, row mean, GELU, residual add
+        float sub[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sub[j] = (CHAIN && p.gamma && cok[j]) ? __ldg(p.gamma + col[j]) : 0.f;
         // thread -> 16 lanes that share the row (shuffles) -> tile partial
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            float v = (RED == FORGE_RED_SUM) ? 0.f : -INFINITY;
+            float v = ADD ? 0.f : -INFINITY;
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                if (cok[j]) v = (RED == FORGE_RED_SUM) ? v + acc[i][j] : fmaxf(v, acc[i][j]);
+                if (cok[j]) v = ADD ? v + (acc[i][j] - sub[j]) : fmaxf(v, acc[i][j]);
 #pragma unroll
             for (int s = 8; s >= 1; s >>= 1) {
                 const float o = __shfl_xor_sync(0xffffffffu, v, s);
-                v = (RED == FORGE_RED_SUM) ? v + o : fmaxf(v, o);
+                v = ADD ? v + o : fmaxf(v, o);
             }
-            const int row = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
+            const int rl = ty * 4 + (i & 3) + (i >> 2) * 64;
+            const int row = m0 + rl;
             if (tx == 0 && row < M) {
-                if (p.tiles_n == 1) p.out[row] = v;
-                else p.partial[(size_t)tile_n * M + row] = v;
+                if (p.tiles_n > 1) p.partial[(size_t)tile_n * M + row] = v;
+                else if (CHAIN) s_mean[rl] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)N);
+                else p.out[row] = v;
             }
         }
-        if (p.tiles_n == 1) return;
-        // the last CTA to arrive at this row strip folds the partials in tile order
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) s_last = (atomicAdd(&p.counters[tile_m], 1u) == (unsigned)(p.tiles_n - 1));
-        __syncthreads();
-        if (!s_last) return;
-        __threadfence();
-        if (tid < K1_BM && m0 + tid < M) {
-            const int row = m0 + tid;
-            float v = __ldcg(&p.partial[row]);
-            for (int t = 1; t < p.tiles_n; ++t) {
-                const float o = __ldcg(&p.partial[(size_t)t * M + row]);
-                v = (RED == FORGE_RED_SUM) ? v + o : fmaxf(v, o);
+        if (p.tiles_n > 1) {
+            // the last CTA to arrive at this row strip folds the partials in tile order
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) s_last = (atomicAdd(&p.counters[tile_m], 1u) == (unsigned)(p.tiles_n - 1));
+            __syncthreads();
+            if (!s_last) return;
+            __threadfence();
+            if (tid < K1_BM && m0 + tid < M) {
+                const int row = m0 + tid;
+                float v = __ldcg(&p.partial[row]);
+                for (int t = 1; t < p.tiles_n; ++t) {
+                    const float o = __ldcg(&p.partial[(size_t)t * M + row]);
+                    v = ADD ? v + o : fmaxf(v, o);
+                }
+                if (CHAIN) s_mean[tid] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)N);
+                else p.out[row] = v;
             }
-            p.out[row] = v;
+            if (tid == 0) p.counters[tile_m] = 0u;     // ready for the next run
         }
-        if (tid == 0) p.counters[tile_m] = 0u;     // ready for the next run
+        if (CHAIN) {
+            // residual add: Y[row, :] = X[row, :] + gelu(mean) for the strip's rows, by the whole CTA
+            __syncthreads();
+            const int rows = min(K1_BM, M - m0);
+            if (p.res_vec4) {
+                const int k4 = K >> 2;
+                for (int e = tid; e < rows * k4; e += K1_THREADS) {
+                    const int r = e / k4, c = e - r * k4;
+                    float4 x = __ldg(reinterpret_cast<const float4 *>(p.X + (size_t)(m0 + r) * K) + c);
+                    const float g = s_mean[r];
+                    x.x += g; x.y += g; x.z += g; x.w += g;
+                    reinterpret_cast<float4 *>(p.out + (size_t)(m0 + r) * K)[c] = x;
+                }
+            } else {
+                for (int e = tid; e < rows * K; e += K1_THREADS) {
+                    const int r = e / K, c = e - r * K;
+                    p.out[(size_t)(m0 + r) * K + c] = __ldg(p.X + (size_t)(m0 + r) * K + c) + s_mean[r];
+                }
+            }
+        }
         return;
     }
 
@@ -305,7 +335,7 @@ forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     info->threads = K1_THREADS;
     info->grid = tiles_m * tiles_n;
     info->smem_bytes = 0;
-    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) && tiles_n > 1;
+    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL) && tiles_n > 1;
     wl->partial_floats = partials ? (size_t)tiles_n * (size_t)d.M : 0;
     wl->counters = partials ? (size_t)tiles_m : 0;
     return FORGE_OK;
@@ -351,6 +381,7 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
     p.counters = h.ws.counters;
     p.tiles_n = (int)((d.N + K1_BN - 1) / K1_BN);
     p.out_vec4 = (d.N % 4 == 0) && ((uintptr_t)a.out % 16 == 0);
+    p.res_vec4 = (d.K % 4 == 0) && ((uintptr_t)a.out % 16 == 0) && ((uintptr_t)a.X % 16 == 0);
     const dim3 grid((unsigned)p.tiles_n, (unsigned)((d.M + K1_BM - 1) / K1_BM));
     const bool vec = (d.K % 4 == 0) && ((uintptr_t)a.X % 16 == 0) && ((uintptr_t)a.W % 16 == 0);
 #define K1_CASE(R)                                                                      \
@@ -362,6 +393,7 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
         K1_CASE(FORGE_RED_SUM)
         K1_CASE(FORGE_RED_MAX)
         K1_CASE(FORGE_RED_LAYERNORM)
+        K1_CASE(FORGE_RED_MEAN_GELU_RESIDUAL)
     }
 #undef K1_CASE
     return FORGE_ERR_INVALID_ARG;
@@ -441,6 +473,7 @@ extern "C" forge_status_t forge_fused_linear_f32_reduce_static(int64_t M, int64_
     p.partial = (float *)((unsigned char *)scratch + counter_bytes);
     p.tiles_n = (int)tiles_n;
     p.out_vec4 = 0;
+    p.res_vec4 = 0;
     const dim3 grid((unsigned)tiles_n, (unsigned)tiles_m);
     const bool vec = (K % 4 == 0) && ((uintptr_t)X % 16 == 0) && ((uintptr_t)W % 16 == 0);
     if (red == FORGE_RED_SUM)

@@ -17,12 +17,13 @@ from . import workloads as wk
 
 def main() -> int:
     ap = argparse.ArgumentParser()
-    ap.add_argument("workload", choices=sorted(wk.WORKLOADS))
+    every = {**wk.WORKLOADS, **wk.EXTRA_WORKLOADS}
+    ap.add_argument("workload", choices=sorted(every))
     ap.add_argument("--launches", type=int, default=5)
     ap.add_argument("--rows", type=int, default=0, help="use only the first ROWS rows of X (smaller case)")
     args = ap.parse_args()
     import torch
-    wl = wk.WORKLOADS[args.workload]
+    wl = every[args.workload]
     M = args.rows or wl.M
     inp = wk.make_inputs(wl, M=M)
 
@@ -32,9 +33,11 @@ def main() -> int:
         t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
         return (t.to(torch.bfloat16) if wl.dtype == wk.BF16 else t).cuda()
     d = {k: dev(v) for k, v in inp.items()}
-    reduce = wl.red in (wk.RED_SUM, wk.RED_MAX)
-    out = torch.empty((M,) if reduce else (M, wl.N), device="cuda",
+    reduce = wl.out_cols == 0
+    out = torch.empty((M,) if reduce else (M, wl.out_cols), device="cuda",
                       dtype=torch.float32 if (reduce or wl.dtype == wk.F32) else torch.bfloat16)
+    if wl.red == wk.RED_MEAN_GELU_RESIDUAL:
+        d["gamma"] = d["sub"]          # the chain's subtract vector travels in the gamma slot
     op = B.FusedLinear(B.make_desc(M, wl.N, wl.K, wl.dtype, wl.act, wl.red, wl.scale, wl.ln_eps,
                                    wl.bias.kind != "none", 0))
     torch.cuda.synchronize()

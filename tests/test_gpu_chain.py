@@ -1,0 +1,64 @@
+"""GPU parity of the case-study chain (Linear, subtract, row mean, GELU, residual add) on the
+fp32 path against the CPU oracle."""
+import numpy as np
+import pytest
+
+from paper_2511_01884_b200 import binding as B
+from paper_2511_01884_b200 import workloads as wk
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+# one N-tile and several; ragged M, N, K; K not a multiple of 4 (scalar residual path)
+SHAPES = [(1, 1, 1), (5, 100, 7), (128, 128, 16), (130, 300, 36), (257, 1000, 64), (300, 96, 19), (1000, 2048, 128)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_shapes(M, N, K):
+    wl = wk.custom_workload(f"chain_{M}x{N}x{K}", wk.F32, M, N, K, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL, seed=M + N)
+    inp = wk.make_inputs(wl)
+    # spread the row means over the curved part of the GELU
+    inp["b"] = wk.round_to_storage(inp["b"] + np.linspace(-2, 2, N).astype(np.float32) * 0 + 0.7, wk.F32)
+    g, plan = pu.run_gpu(wl, inp)
+    assert g.shape == (M, K) and plan["kernel"] == B.FORGE_KERNEL_F32_FFMA
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_with_activation_scale_and_no_subtract_vector():
+    wl = wk.custom_workload("chain_act", wk.F32, 200, 260, 48, wk.ACT_RELU, wk.RED_MEAN_GELU_RESIDUAL, scale=3.0, seed=9)
+    inp = wk.make_inputs(wl)
+    inp["sub"] = None
+    g, _ = pu.run_gpu(wl, inp)
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_zero_mean_returns_the_input_bits():
+    wl = wk.custom_workload("chain_zero", wk.F32, 140, 256, 32, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL, seed=3)
+    inp = wk.make_inputs(wl)
+    inp["W"][:] = 0.0
+    inp["sub"] = inp["b"].copy()
+    g, _ = pu.run_gpu(wl, inp)
+    assert np.array_equal(g, inp["X"].astype(np.float64))
+
+
+def test_two_runs_on_one_handle_and_bf16_is_refused():
+    wl = wk.custom_workload("chain_rep", wk.F32, 300, 700, 64, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL, seed=4)
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op)
+    b, _ = pu.run_gpu(wl, inp, op=op, repeats=3)
+    op.close()
+    assert np.array_equal(a, b)
+    pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
+    st, _ = B.forge_fused_linear_query_plan(B.make_desc(64, 64, 64, wk.BF16, 0, wk.RED_MEAN_GELU_RESIDUAL))
+    assert st == B.FORGE_ERR_UNSUPPORTED
+
+
+def test_n1_sampled_rows_full_size():
+    wl = wk.EXTRA_WORKLOADS["n1"]
+    inp = wk.make_inputs(wl)
+    g, _ = pu.run_gpu(wl, inp)
+    rows = wk.sample_rows(wl.M)
+    pu.assert_parity(wl, g[rows], pu.run_oracle(wl, inp, rows))
+    assert np.isfinite(g).all()
