@@ -45,7 +45,7 @@ template <bool PAIR> struct K2Ring {
     static constexpr int STAGES = PAIR ? 6 : 4;
     static constexpr uint32_t BYTES = STAGES * STAGE_BYTES;      // 192 KiB either way
 };
-constexpr int K2_GROUP_M = 16;      // row tiles per rasterisation group (keeps a wave's operands in L2)
+constexpr int K2_GROUP_M = 16;      // 128-row tiles per rasterisation group (keeps a wave's operands in L2)
 
 struct K2Smem {
     uint64_t full[K2_MAX_STAGES];
@@ -72,21 +72,22 @@ struct K2Params {
     unsigned *counters;   // [tiles_m]
     int *status;
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
+    int group_m;          // row units per rasterisation group
     unsigned ln_target;   // layernorm: counter value at which a strip is complete in this run
 };
 
 template <bool LN>
-__device__ __forceinline__ void k2_tile_coords(int t, int tiles_m, int tiles_n, int &tm, int &tn)
+__device__ __forceinline__ void k2_tile_coords(int t, int tiles_m, int tiles_n, int group_m, int &tm, int &tn)
 {
     if (LN) {            // a strip's N-tiles are neighbours in the schedule
         tm = t / tiles_n;
         tn = t - tm * tiles_n;
         return;
     }
-    const int group_size = K2_GROUP_M * tiles_n;
+    const int group_size = group_m * tiles_n;
     const int g = t / group_size, r = t - g * group_size;
-    const int gm = min(K2_GROUP_M, tiles_m - g * K2_GROUP_M);
-    tm = g * K2_GROUP_M + r % gm;
+    const int gm = min(group_m, tiles_m - g * group_m);
+    tm = g * group_m + r % gm;
     tn = r / gm;
 }
 
@@ -157,7 +158,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             uint32_t phase = 0;
             for (int t = first_unit; t < total_tiles && ok; t += unit_stride) {
                 int tm, tn;
-                k2_tile_coords<LN>(t, unit_rows, p.tiles_n, tm, tn);
+                k2_tile_coords<LN>(t, unit_rows, p.tiles_n, p.group_m, tm, tn);
                 if (PAIR) tm = 2 * tm + (int)rank;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
@@ -225,7 +226,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                                             ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[1]), 0)};   // the leader's (PAIR)
         for (int t = first_unit; t < total_tiles; t += unit_stride) {
             int tm, tn;
-            k2_tile_coords<LN>(t, unit_rows, p.tiles_n, tm, tn);
+            k2_tile_coords<LN>(t, unit_rows, p.tiles_n, p.group_m, tm, tn);
             if (PAIR) tm = 2 * tm + (int)rank;
             const int m0 = tm * K2_BM, n0 = tn * K2_BN + h * HALF;
             const int part = 2 * tn + h;
@@ -542,7 +543,16 @@ static forge_status_t k2_launch_t(const Handle &h, const K2Params &p, cudaStream
         attr[n].val.clusterDim.z = 1;
         ++n;
     }
-    if (LN) {           // CTAs wait on one another: all of them must be resident
+    // CTAs wait on one another: a cooperative launch guarantees that all of them are resident.
+    // FORGE_K4_COOPERATIVE=0 drops the attribute (profilers refuse cooperative cluster launches);
+    // the grid never exceeds the SM count, and every wait is bounded, so the worst case on a GPU
+    // that is busy with other work is a reported time-out, not a hang.
+    static int coop = -1;
+    if (coop < 0) {
+        const char *e = std::getenv("FORGE_K4_COOPERATIVE");
+        coop = e ? (std::atoi(e) != 0) : 1;
+    }
+    if (LN && coop) {
         attr[n].id = cudaLaunchAttributeCooperative;
         attr[n].val.cooperative = 1;
         ++n;
@@ -581,6 +591,14 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     p.tiles_n = (int)((d.N + K2_BN - 1) / K2_BN);
     p.num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
     p.ln_target = 0;
+    {
+        static int env = -1;        // FORGE_K2_GROUP_M overrides the rasterisation group (tuning aid)
+        if (env < 0) {
+            const char *e = std::getenv("FORGE_K2_GROUP_M");
+            env = e ? std::atoi(e) : 0;
+        }
+        p.group_m = env > 0 ? env : (pair ? K2_GROUP_M / 2 : K2_GROUP_M);      // 2048 rows either way
+    }
     if (!ln) return pair ? k2_launch_t<false, true>(h, p, a.stream) : k2_launch_t<false, false>(h, p, a.stream);
     // Strip counters only ever grow: run r completes a strip at r * 2 * tiles_n arrivals (half tiles).
     h.run_gen += 1;
