@@ -83,14 +83,16 @@ typedef struct {
 /* Kernel families.  The choice is a pure function of the descriptor. */
 typedef enum {
     FORGE_KERNEL_F32_FFMA = 1,        /* fp32 register-tiled FFMA GEMM, fused epilogue        */
-    FORGE_KERNEL_BF16_TCGEN05 = 2,    /* bf16 TMA -> smem ring -> tcgen05.mma -> TMEM         */
+    FORGE_KERNEL_BF16_TCGEN05 = 2,    /* bf16 TMA -> smem ring -> tcgen05.mma -> TMEM; CTA     */
+                                      /* pairs (cta_group::2, 256x256 tiles) when M > 128      */
     FORGE_KERNEL_BF16_SKINNY = 3,     /* bf16, M <= 16: split-K over warps, HBM-bound          */
-    FORGE_KERNEL_BF16_TCGEN05_LN = 4  /* bf16 tcgen05 with a cluster-wide LayerNorm epilogue  */
+    FORGE_KERNEL_BF16_TCGEN05_LN = 4  /* bf16 tcgen05 whose epilogue merges row statistics    */
+                                      /* across the N-tiles of a row strip (LayerNorm)         */
 } forge_kernel_t;
 
 typedef struct {
     forge_kernel_t kernel;
-    int tile_m, tile_n, tile_k;  /* CTA tile                                              */
+    int tile_m, tile_n, tile_k;  /* CTA tile (cluster tile when cluster > 1)              */
     int stages;                  /* depth of the shared-memory ring (0: not ring-based)   */
     int cluster;                 /* CTAs per cluster (1: no cluster)                      */
     int threads;                 /* threads per CTA                                       */
@@ -106,8 +108,9 @@ typedef struct {
  * Kernel selection (Appendix B.1's point that the right fusion depends on whether the chain
  * is compute- or memory-bound): fp32 -> F32_FFMA; bf16 with M <= 16 and no LayerNorm ->
  * BF16_SKINNY; bf16 LayerNorm -> BF16_TCGEN05_LN; other bf16 -> BF16_TCGEN05.
- * Unsupported: bf16 with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); LayerNorm with N
- * larger than one cluster spans (bf16: 4096, fp32: 1024).
+ * Unsupported: bf16 with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); fp32 LayerNorm with
+ * N > 1024 (one 8-CTA cluster); bf16 LayerNorm with more 256-column tiles per row than
+ * clusters in the grid; the mean-gelu-residual chain in bf16.
  */
 forge_status_t forge_fused_linear_query_plan(const forge_fused_linear_desc_t *desc, int sm_count,
                                              forge_plan_info_t *info);
