@@ -1,0 +1,109 @@
+"""GPU-side behaviour of the C interface itself: argument checks in run(), the host-buffer entry
+point, unaligned fp32 operands, handles on a non-default stream, plan/launch bookkeeping."""
+import numpy as np
+import pytest
+
+from paper_2511_01884_b200 import binding as B
+from paper_2511_01884_b200 import workloads as wk
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def test_run_rejects_missing_and_misaligned_pointers():
+    import torch
+    wl = wk.custom_workload("iface_bf16", wk.BF16, 64, 64, 64, wk.ACT_RELU, wk.RED_LAYERNORM)
+    op = B.FusedLinear(pu.desc_of(wl))
+    t = torch.zeros(64 * 64 + 8, dtype=torch.bfloat16, device="cuda")
+    v = torch.zeros(64 + 8, dtype=torch.bfloat16, device="cuda")
+    ok = (t, t, v, v, v, t)
+    assert B.forge_fused_linear_run(op.h, *ok) == B.FORGE_OK
+    for i in range(6):                                             # each pointer missing in turn
+        args = list(ok)
+        args[i] = None
+        assert B.forge_fused_linear_run(op.h, *args) == B.FORGE_ERR_INVALID_ARG, i
+    off = t[1:]                                                    # 2-byte offset: not 16-byte aligned
+    assert B.forge_fused_linear_run(op.h, off, t, v, v, v, t) == B.FORGE_ERR_INVALID_ARG
+    assert B.forge_fused_linear_run(op.h, t, t, v, v, v, off) == B.FORGE_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    op.check()
+    op.close()
+    assert B.forge_fused_linear_launches_per_run(None) == 0
+
+
+def test_fp32_accepts_unaligned_operands_with_scalar_accesses():
+    import torch
+    wl = wk.custom_workload("iface_f32", wk.F32, 70, 50, 36, wk.ACT_SILU, wk.RED_NONE, seed=5)
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    assert B.forge_fused_linear_launches_per_run(op.h) == 1
+
+    def shifted(a):                                                # same values, 4-byte-aligned only
+        buf = torch.zeros(a.size + 1, dtype=torch.float32, device="cuda")
+        buf[1:] = torch.from_numpy(a.ravel())
+        return buf[1:]
+    X, W, b = shifted(inp["X"]), shifted(inp["W"]), shifted(inp["b"])
+    obuf = torch.full((70 * 50 + 1,), float("nan"), dtype=torch.float32, device="cuda")
+    out = obuf[1:]
+    assert X.data_ptr() % 16 != 0 and out.data_ptr() % 16 != 0
+    assert B.forge_fused_linear_run(op.h, X, W, b, None, None, out) == B.FORGE_OK
+    torch.cuda.synchronize()
+    op.close()
+    g = out.cpu().numpy().astype(np.float64).reshape(70, 50)
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+    assert np.isnan(obuf[0].item())                                # nothing written in front of the output
+
+
+@pytest.mark.parametrize("name", ["c1", "skinny", "ln", "plain", "chain"])
+def test_host_buffer_entry_point_matches_the_oracle(name):
+    import torch
+    wl = {"c1": wk.WORKLOADS["c1"],
+          "skinny": wk.custom_workload("h_skinny", wk.BF16, 16, 1024, 256, wk.ACT_GELU_ERF, wk.RED_MAX, w_std=0.05),
+          "ln": wk.custom_workload("h_ln", wk.BF16, 300, 520, 128, wk.ACT_GELU_TANH, wk.RED_LAYERNORM, w_std=0.05),
+          "plain": wk.custom_workload("h_plain", wk.BF16, 300, 520, 128, wk.ACT_SILU, wk.RED_NONE, w_std=0.05),
+          "chain": wk.custom_workload("h_chain", wk.F32, 150, 300, 40, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL)}[name]
+    inp = wk.make_inputs(wl)
+
+    def host(a):
+        if a is None:
+            return None
+        t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
+        return (t.to(torch.bfloat16) if wl.dtype == wk.BF16 else t).pin_memory()
+    h = {k: host(v) for k, v in inp.items()}
+    aux = h["sub"] if wl.red == wk.RED_MEAN_GELU_RESIDUAL else h["gamma"]
+    shape = (wl.M,) if wl.out_cols == 0 else (wl.M, wl.out_cols)
+    out = torch.zeros(shape, dtype=torch.float32 if (wl.out_cols == 0 or wl.dtype == wk.F32) else torch.bfloat16).pin_memory()
+    op = B.FusedLinear(pu.desc_of(wl))
+    for _ in range(2):                                             # second call reuses the staging buffers
+        op.run_host(h["X"], h["W"], h["b"], aux, h["beta"], out)
+    op.check()
+    op.close()
+    pu.assert_parity(wl, out.float().numpy().astype(np.float64), pu.run_oracle(wl, inp))
+
+
+def test_runs_on_a_side_stream():
+    import torch
+    wl = wk.custom_workload("iface_stream", wk.BF16, 512, 512, 256, wk.ACT_SILU, wk.RED_SUM, w_std=0.05, seed=7)
+    inp = wk.make_inputs(wl)
+    dev = {k: pu.to_device(v, wl.dtype) for k, v in inp.items()}
+    out = torch.zeros(512, dtype=torch.float32, device="cuda")
+    op = B.FusedLinear(pu.desc_of(wl))
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        op(dev["X"], dev["W"], dev["b"], None, None, out, stream=s.cuda_stream)
+    s.synchronize()
+    op.check()
+    op.close()
+    pu.assert_parity(wl, out.cpu().numpy().astype(np.float64), pu.run_oracle(wl, inp))
+
+
+def test_plans_report_the_kernel_families():
+    for wl, kernel, cluster in [(wk.WORKLOADS["c2"], B.FORGE_KERNEL_F32_FFMA, 1),
+                                (wk.WORKLOADS["c3"], B.FORGE_KERNEL_BF16_TCGEN05, 2),
+                                (wk.WORKLOADS["c4"], B.FORGE_KERNEL_BF16_SKINNY, 1),
+                                (wk.WORKLOADS["c5"], B.FORGE_KERNEL_BF16_TCGEN05_LN, 2)]:
+        st, p = B.forge_fused_linear_query_plan(pu.desc_of(wl))
+        assert st == B.FORGE_OK and p.kernel == kernel and p.cluster == cluster
+        assert p.grid <= 148 or kernel == B.FORGE_KERNEL_F32_FFMA          # the bf16 kernels are persistent
