@@ -193,6 +193,44 @@ def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
     return ms
 
 
+def eager_context_us(wl, d, torch, steps=10):
+    """PyTorch eager on the same GPU, the unfused operator chain in the workload's dtype: context
+    only (a library path, never part of this package's hot path).  Microseconds per call."""
+    import torch.nn.functional as F
+
+    def chain():
+        z = F.linear(d["X"], d["W"], d["b"])
+        if wl.act == wk.ACT_RELU:
+            z = F.relu(z)
+        elif wl.act == wk.ACT_GELU_ERF:
+            z = F.gelu(z)
+        elif wl.act == wk.ACT_GELU_TANH:
+            z = F.gelu(z, approximate="tanh")
+        elif wl.act == wk.ACT_SILU:
+            z = F.silu(z)
+        if wl.scale != 1.0:
+            z = z * wl.scale
+        if wl.red == wk.RED_SUM:
+            return z.sum(1, dtype=torch.float32)
+        if wl.red == wk.RED_MAX:
+            return z.amax(1).float()
+        if wl.red == wk.RED_LAYERNORM:
+            return F.layer_norm(z, (wl.N,), d["gamma"], d["beta"], wl.ln_eps)
+        if wl.red == wk.RED_MEAN_GELU_RESIDUAL:
+            return d["X"] + F.gelu((z - d["gamma"]).mean(1, keepdim=True))
+        return z
+    for _ in range(3):
+        chain()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        chain()
+    e1.record()
+    torch.cuda.synchronize()
+    return 1e3 * e0.elapsed_time(e1) / steps
+
+
 def roofline_of(wl, ms, peaks, kernel, sm_max_mhz, sm_count):
     """Roofline of the (single) kernel of a step: achieved = algorithmic work / measured time."""
     src = peaks["_source"]
@@ -380,6 +418,12 @@ def main():
             "roofline": roofline_of(wl, ms, peaks, op.plan.kernel, clocks.get("sm_max_mhz"), props.multi_processor_count),
             "nominal_frac": round((value / world) / (NOMINAL["hbm_gbs"] if wl.name == "c4" else NOMINAL["bf16_tflops"]), 4)
             if wl.dtype == wk.BF16 else None}
+    eager_us = None
+    if rank == 0 and world == 1:
+        time.sleep(2.0)
+        eager_us = eager_context_us(wl, d, torch)
+        line["torch_eager_context"] = {"us_per_call": round(eager_us, 1), "value": round(unit_value(wl, eager_us / 1e3)[0], 2),
+                                       "unit": unit, "what": "unfused F.linear + activation (+ reduction) in the same dtype, same GPU"}
     op.close()
     del d, host
 
@@ -403,7 +447,9 @@ def main():
                 ms2 = time_steps(op2, d2, steps2, 3, torch, flush_buf=fl)
                 v2, u2 = unit_value(w2, ms2)
                 launches += steps2
-                line["workloads"][name] = {"us_per_call": round(ms2 * 1e3, 2), "value": round(v2, 2), "unit": u2,
+                time.sleep(1.0)
+                eg = eager_context_us(w2, d2, torch, steps=5 if w2.flops > 1e11 else 50)
+                line["workloads"][name] = {"torch_eager_context_us": round(eg, 1), "us_per_call": round(ms2 * 1e3, 2), "value": round(v2, 2), "unit": u2,
                                            "steps": steps2, "l2": "flushed before every call" if fl is not None else "operands larger than L2",
                                            "kernel": op2.plan.as_dict()["kernel"],
                                            "roofline": roofline_of(w2, ms2, peaks, op2.plan.kernel, clocks.get("sm_max_mhz"),
