@@ -41,7 +41,7 @@ def _load():
         lib.forge_oracle_fused_linear.restype = ctypes.c_int
         lib.forge_oracle_fused_linear.argtypes = [
             ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, fp, fp, fp, fp, fp, fp,
-            ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_double,
+            ctypes.POINTER(ctypes.c_int32), ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_double,
             ctypes.POINTER(ctypes.c_int64), ctypes.c_int64, ctypes.POINTER(ctypes.c_double)]
         lib.forge_oracle_act.restype = ctypes.c_double
         lib.forge_oracle_act.argtypes = [ctypes.c_int, ctypes.c_double]
@@ -68,9 +68,11 @@ def act(kind: int, z: float) -> float:
 def fused_linear(X: np.ndarray, W: np.ndarray, b: Optional[np.ndarray] = None,
                  gamma: Optional[np.ndarray] = None, beta: Optional[np.ndarray] = None,
                  act: int = 0, scale: float = 1.0, red: int = 0, eps: float = 1e-5,
-                 rows: Optional[Sequence[int]] = None, sub: Optional[np.ndarray] = None) -> np.ndarray:
+                 rows: Optional[Sequence[int]] = None, sub: Optional[np.ndarray] = None,
+                 target: Optional[np.ndarray] = None) -> np.ndarray:
     """float64 result for all rows of X, or for the listed ``rows`` only.  ``sub`` is the
-    vector subtracted before the row mean of reduction 4 (mean-gelu-residual)."""
+    vector subtracted before the row mean of reduction 4 (mean-gelu-residual); ``target`` [M]
+    holds the class index of each row for reduction 6 (cross-entropy)."""
     lib = _load()
     M, K = X.shape
     N, K2 = W.shape
@@ -82,13 +84,15 @@ def fused_linear(X: np.ndarray, W: np.ndarray, b: Optional[np.ndarray] = None,
     ga, gp = _f32(gamma)
     bea, bep = _f32(beta)
     sa, sp = _f32(sub)
+    ta = None if target is None else np.ascontiguousarray(target, dtype=np.int32)
+    tp = None if ta is None else ta.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
     if rows is None:
         ra, rp, nrows = None, None, M
     else:
         ra = np.ascontiguousarray(rows, dtype=np.int64)
         rp, nrows = ra.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)), int(ra.size)
-    out = np.empty((nrows,) if red in (1, 2) else (nrows, K if red == 4 else N), dtype=np.float64)
-    rc = lib.forge_oracle_fused_linear(M, N, K, Xp, Wp, bp, gp, bep, sp, int(act), float(scale),
+    out = np.empty((nrows,) if red in (1, 2, 5, 6) else (nrows, K if red == 4 else N), dtype=np.float64)
+    rc = lib.forge_oracle_fused_linear(M, N, K, Xp, Wp, bp, gp, bep, sp, tp, int(act), float(scale),
                                        int(red), float(eps), rp, nrows,
                                        out.ctypes.data_as(ctypes.POINTER(ctypes.c_double)))
     if rc != 0:

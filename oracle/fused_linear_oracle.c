@@ -23,6 +23,10 @@
  *      mean-gelu-residual (the chain of the Appendix B.1 case study: Linear, subtract, row
  *                 mean, GELU, residual add of the layer's input):
  *                 g[m] = gelu_erf(mean_n (E[m,n] - sub[n])),  Y[m,k] = X[m,k] + g[m]   (Y is [M,K])
+ *      logsumexp: out[m] = log sum_n exp(E[m,n])   (the row statistic of a softmax; Section 4's
+ *                 case study replaces block-wide reductions of exactly this max / sum pair)
+ *      cross-entropy: out[m] = logsumexp_n E[m,:] - E[m, target[m]]   (Section 4: CrossEntropyLoss
+ *                 per row, before the mean over rows)
  *
  * All arithmetic is IEEE double.  Inputs arrive as float (values stored as fp32 or bf16 are
  * exactly representable in float and in double).  No blocking, no reordering: k runs
@@ -37,7 +41,8 @@
 #endif
 
 enum { ACT_IDENTITY = 0, ACT_RELU = 1, ACT_GELU_ERF = 2, ACT_GELU_TANH = 3, ACT_SILU = 4 };
-enum { RED_NONE = 0, RED_SUM = 1, RED_MAX = 2, RED_LAYERNORM = 3, RED_MEAN_GELU_RESIDUAL = 4 };
+enum { RED_NONE = 0, RED_SUM = 1, RED_MAX = 2, RED_LAYERNORM = 3, RED_MEAN_GELU_RESIDUAL = 4,
+       RED_LOGSUMEXP = 5, RED_CROSS_ENTROPY = 6 };
 
 /* Step 2: the activation, one value at a time. */
 double forge_oracle_act(int act, double z)
@@ -64,22 +69,26 @@ int forge_oracle_threads(void)
 /*
  * X [M,K], W [N,K], b [N] or NULL, gamma/beta [N] (layernorm only), all row-major float.
  * sub [N] (mean-gelu-residual only; NULL there means nothing is subtracted).
+ * target [M] column indices (cross-entropy only).
  * rows: nrows row indices into X (NULL means rows 0..nrows-1).
- * out:  double, [nrows,N] for none/layernorm, [nrows] for sum/max, [nrows,K] for mean-gelu-residual.
+ * out:  double, [nrows,N] for none/layernorm, [nrows] for sum/max/logsumexp/cross-entropy,
+ *       [nrows,K] for mean-gelu-residual.
  * Returns 0, or 1 on a bad argument.
  */
 int forge_oracle_fused_linear(int64_t M, int64_t N, int64_t K,
                               const float *X, const float *W, const float *b,
                               const float *gamma, const float *beta, const float *sub,
-                              int act, double scale, int red, double eps,
+                              const int32_t *target, int act, double scale, int red, double eps,
                               const int64_t *rows, int64_t nrows, double *out)
 {
     if (M <= 0 || N <= 0 || K <= 0 || nrows < 0 || !X || !W || !out) return 1;
-    if (act < ACT_IDENTITY || act > ACT_SILU || red < RED_NONE || red > RED_MEAN_GELU_RESIDUAL) return 1;
+    if (act < ACT_IDENTITY || act > ACT_SILU || red < RED_NONE || red > RED_CROSS_ENTROPY) return 1;
+    if (red == RED_CROSS_ENTROPY && !target) return 1;
     if (red == RED_LAYERNORM && (!gamma || !beta)) return 1;
     for (int64_t r = 0; r < nrows; ++r) {
         int64_t m = rows ? rows[r] : r;
         if (m < 0 || m >= M) return 1;
+        if (red == RED_CROSS_ENTROPY && (target[m] < 0 || target[m] >= N)) return 1;
     }
 
     int bad = 0;
@@ -110,6 +119,13 @@ int forge_oracle_fused_linear(int64_t M, int64_t N, int64_t K,
             double mx = E[0];
             for (int64_t n = 1; n < N; ++n) if (E[n] > mx) mx = E[n];
             out[r] = mx;
+        } else if (red == RED_LOGSUMEXP || red == RED_CROSS_ENTROPY) {
+            /* log sum exp, evaluated as mx + log sum exp(E - mx) so that no term overflows */
+            double mx = E[0], se = 0.0;
+            for (int64_t n = 1; n < N; ++n) if (E[n] > mx) mx = E[n];
+            for (int64_t n = 0; n < N; ++n) se += exp(E[n] - mx);
+            out[r] = mx + log(se);
+            if (red == RED_CROSS_ENTROPY) out[r] -= E[target[m]];
         } else if (red == RED_MEAN_GELU_RESIDUAL) {
             double mu = 0.0;
             for (int64_t n = 0; n < N; ++n) mu += E[n] - (sub ? (double)sub[n] : 0.0);

@@ -29,9 +29,10 @@ import numpy as np
 # depends on neither side.
 F32, BF16 = 0, 1
 ACT_IDENTITY, ACT_RELU, ACT_GELU_ERF, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3, 4
-RED_NONE, RED_SUM, RED_MAX, RED_LAYERNORM, RED_MEAN_GELU_RESIDUAL = 0, 1, 2, 3, 4
+RED_NONE, RED_SUM, RED_MAX, RED_LAYERNORM, RED_MEAN_GELU_RESIDUAL, RED_LOGSUMEXP, RED_CROSS_ENTROPY = 0, 1, 2, 3, 4, 5, 6
+VECTOR_OUT = (RED_SUM, RED_MAX, RED_LOGSUMEXP, RED_CROSS_ENTROPY)      # reductions whose output is fp32 [M]
 
-STREAM_X, STREAM_W, STREAM_B, STREAM_GAMMA, STREAM_BETA, STREAM_SUB = 0, 1, 2, 3, 4, 5
+STREAM_X, STREAM_W, STREAM_B, STREAM_GAMMA, STREAM_BETA, STREAM_SUB, STREAM_TARGET = 0, 1, 2, 3, 4, 5, 6
 
 _MASK64 = np.uint64(0xFFFFFFFFFFFFFFFF)
 
@@ -151,7 +152,7 @@ class Workload:
     @property
     def out_cols(self) -> int:
         """Columns of the output matrix (0: the output is a vector of M floats)."""
-        if self.red in (RED_SUM, RED_MAX):
+        if self.red in VECTOR_OUT:
             return 0
         return self.K if self.red == RED_MEAN_GELU_RESIDUAL else self.N
 
@@ -174,7 +175,7 @@ class Workload:
             n += 2 * self.N
         if self.sub.kind != "none":
             n += self.N
-        return n * e + self.out_bytes
+        return n * e + self.out_bytes + (4 * self.M if self.red == RED_CROSS_ENTROPY else 0)
 
 
 WORKLOADS: Dict[str, Workload] = {
@@ -202,6 +203,10 @@ EXTRA_WORKLOADS: Dict[str, Workload] = {
     "n1": Workload("n1", F32, 4096, 4096, 4096, ACT_IDENTITY, RED_MEAN_GELU_RESIDUAL, 1.0, 0.0,
                    Dist("normal", 1.0), Dist("uniform", -1 / 64, 1 / 64), Dist("uniform", -0.1, 0.1),
                    note="fp32, subtract, row mean, GELU-erf, residual add", sub=Dist("uniform", -0.5, 0.5)),
+    # the loss of a language-model head: logits never materialised (Section 4's CrossEntropyLoss case)
+    "n2": Workload("n2", BF16, 8192, 32768, 4096, ACT_IDENTITY, RED_CROSS_ENTROPY, 1.0, 0.0,
+                   Dist("normal", 1.0), Dist("normal", 0.02), Dist("normal", 0.02),
+                   note="bf16, per-row cross-entropy over 32768 classes"),
 }
 
 
@@ -234,8 +239,12 @@ def make_inputs(wl: Workload, M: Optional[int] = None, row_offset: int = 0) -> D
     be = _draw(wl.beta, wl.seed, STREAM_BETA, wl.N)
     sb = _draw(wl.sub, wl.seed, STREAM_SUB, wl.N)
     r = lambda t: None if t is None else round_to_storage(t, wl.dtype)
+    tg = None
+    if wl.red == RED_CROSS_ENTROPY:      # class index of every row: uniform over the N columns
+        u = uniform01(wl.seed, STREAM_TARGET, row_offset, rows)
+        tg = np.minimum((u * wl.N).astype(np.int32), wl.N - 1)
     return {"X": r(x).reshape(rows, wl.K), "W": r(w).reshape(wl.N, wl.K),
-            "b": r(b), "gamma": r(g), "beta": r(be), "sub": r(sb)}
+            "b": r(b), "gamma": r(g), "beta": r(be), "sub": r(sb), "target": tg}
 
 
 def custom_workload(name: str, dtype: int, M: int, N: int, K: int, act: int, red: int,

@@ -35,7 +35,7 @@ def run_gpu(wl: wk.Workload, inp, check_status=True, op=None, repeats=1):
     """``repeats`` calls through the C interface (no synchronisation between them); returns
     (float64 numpy result of the last one, plan dict)."""
     import torch
-    dev = {k: to_device(v, wl.dtype) for k, v in inp.items()}
+    dev = {k: to_device(v, wl.dtype) for k, v in inp.items() if k != "target"}
     M = inp["X"].shape[0]
     own = op is None
     if own:
@@ -45,8 +45,11 @@ def run_gpu(wl: wk.Workload, inp, check_status=True, op=None, repeats=1):
     else:
         out = torch.full((M, wl.out_cols), float("nan"), dtype=torch.float32 if wl.dtype == wk.F32 else torch.bfloat16,
                          device="cuda")
-    # the mean-gelu-residual chain takes its subtract vector in the gamma slot of the interface
+    # the mean-gelu-residual chain takes its subtract vector, and the cross-entropy its int32
+    # class indices, in the gamma slot of the interface
     aux = dev["sub"] if wl.red == wk.RED_MEAN_GELU_RESIDUAL else dev["gamma"]
+    if wl.red == wk.RED_CROSS_ENTROPY:
+        aux = torch.from_numpy(np.ascontiguousarray(inp["target"], dtype=np.int32)).cuda()
     for _ in range(repeats):
         op(dev["X"], dev["W"], dev["b"], aux, dev["beta"], out)
     torch.cuda.synchronize()
@@ -61,7 +64,8 @@ def run_gpu(wl: wk.Workload, inp, check_status=True, op=None, repeats=1):
 def run_oracle(wl: wk.Workload, inp, rows=None):
     import oracle
     return oracle.fused_linear(inp["X"], inp["W"], inp["b"], inp["gamma"], inp["beta"], act=wl.act,
-                               scale=wl.scale, red=wl.red, eps=wl.ln_eps, rows=rows, sub=inp.get("sub"))
+                               scale=wl.scale, red=wl.red, eps=wl.ln_eps, rows=rows, sub=inp.get("sub"),
+                               target=inp.get("target"))
 
 
 def rel_err(g: np.ndarray, r: np.ndarray) -> float:

@@ -318,3 +318,53 @@ def test_chain_special_cases():
     # row subset
     ys = oracle.fused_linear(X, W, b, red=wk.RED_MEAN_GELU_RESIDUAL, rows=[3, 1])
     assert np.array_equal(ys, y0[[3, 1]])
+
+
+# ---- log-sum-exp and per-row cross-entropy ---------------------------------------------------------
+def test_logsumexp_closed_forms():
+    # all logits equal to c: log(N e^c) = c + log N; identity weights make the logits X itself
+    N = 7
+    X = np.full((2, N), 1.25, np.float32)
+    got = oracle.fused_linear(X, np.eye(N, dtype=np.float32), None, red=wk.RED_LOGSUMEXP)
+    assert got == pytest.approx(np.full(2, 1.25 + float(Decimal(N).ln())), abs=1e-14)
+    # two logits a, b: log(e^a + e^b) in decimal arithmetic
+    X = np.array([[0.5, -1.5], [30.0, 29.0]], np.float32)
+    got = oracle.fused_linear(X, np.eye(2, dtype=np.float32), None, red=wk.RED_LOGSUMEXP)
+    want = [float((Decimal(a).exp() + Decimal(b).exp()).ln()) for a, b in X.tolist()]
+    assert got == pytest.approx(want, rel=1e-14)
+    # large logits must not overflow: exp(1000) is not representable, the result is
+    got = oracle.fused_linear(np.array([[1000.0, 1000.0]], np.float32), np.eye(2, dtype=np.float32), None, red=wk.RED_LOGSUMEXP)
+    assert got[0] == pytest.approx(1000.0 + math.log(2.0), rel=1e-15)
+
+
+def test_logsumexp_and_cross_entropy_reduce_to_library_routines():
+    import torch
+    from scipy.special import logsumexp as sp_lse
+    rng = np.random.default_rng(31)
+    M, N, K = 11, 23, 9
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    b = rng.standard_normal(N).astype(np.float32)
+    t = rng.integers(0, N, M).astype(np.int32)
+    E = oracle.fused_linear(X, W, b, act=wk.ACT_SILU, scale=2.0)
+    lse = oracle.fused_linear(X, W, b, act=wk.ACT_SILU, scale=2.0, red=wk.RED_LOGSUMEXP)
+    np.testing.assert_allclose(lse, sp_lse(E, axis=1), rtol=0, atol=1e-12)
+    ce = oracle.fused_linear(X, W, b, act=wk.ACT_SILU, scale=2.0, red=wk.RED_CROSS_ENTROPY, target=t)
+    want = torch.nn.functional.cross_entropy(torch.from_numpy(E), torch.from_numpy(t).long(), reduction="none").numpy()
+    np.testing.assert_allclose(ce, want, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(ce, lse - E[np.arange(M), t], rtol=0, atol=1e-13)
+    # invariants: shifting every logit of a row by c shifts lse by c and leaves the loss alone
+    ce2 = oracle.fused_linear(X, W, b + 3.0, red=wk.RED_CROSS_ENTROPY, target=t)
+    ce1 = oracle.fused_linear(X, W, b, red=wk.RED_CROSS_ENTROPY, target=t)
+    np.testing.assert_allclose(ce1, ce2, rtol=0, atol=1e-5)          # b + 3 is rounded to fp32 once
+    assert (ce >= 0).all() and (lse >= E.max(1)).all()
+    # row subset, and a dominant class has zero loss
+    sub = oracle.fused_linear(X, W, b, red=wk.RED_CROSS_ENTROPY, target=t, rows=[10, 2])
+    assert np.array_equal(sub, ce1[[10, 2]])
+    Xd = np.zeros((1, 3), np.float32)
+    bd = np.array([0.0, 200.0, 0.0], np.float32)
+    assert oracle.fused_linear(Xd, np.zeros((3, 3), np.float32), bd, red=wk.RED_CROSS_ENTROPY, target=[1])[0] == pytest.approx(0.0, abs=1e-80)
+    with pytest.raises(ValueError):
+        oracle.fused_linear(X, W, b, red=wk.RED_CROSS_ENTROPY)                      # targets missing
+    with pytest.raises(ValueError):
+        oracle.fused_linear(X, W, b, red=wk.RED_CROSS_ENTROPY, target=np.full(M, N))  # class out of range
