@@ -6,6 +6,7 @@
  *     sum / max:  out[M]  = sum_n E[m,n]  /  max_n E[m,n]
  *     layernorm:  Y[M,N]  = (E - mean_n E) / sqrt(var_n E + eps) * gamma[n] + beta[n]
  *     mean-gelu-residual: Y[M,K] = X + gelu_erf(mean_n (E - sub[n]))   (see forge_red_t)
+ *     logsumexp / cross-entropy: out[M] = log sum_n exp E  [ - E[m, target[m]] ]
  *
  * The operation is the fused operator chain the paper's agents are asked to produce: one
  * kernel in place of a framework Linear (matmul + bias) followed by an element-wise
@@ -61,12 +62,20 @@ typedef enum {
     FORGE_RED_SUM = 1,
     FORGE_RED_MAX = 2,
     FORGE_RED_LAYERNORM = 3,     /* population variance, eps inside the square root      */
-    FORGE_RED_MEAN_GELU_RESIDUAL = 4
+    FORGE_RED_MEAN_GELU_RESIDUAL = 4,
     /* The chain of the paper's Appendix B.1 case study (Linear, subtract, row mean, GELU,
      * residual add of the layer's input, all in one kernel):
      *     g[m] = gelu_erf(mean_n (E[m,n] - sub[n])),   Y[m,k] = X[m,k] + g[m]
      * The output is Y [M,K] (the shape of X) in dtype.  run() takes the subtract vector sub[N]
      * in its `gamma` argument (NULL: nothing is subtracted); `beta` is ignored.  fp32 only.   */
+    FORGE_RED_LOGSUMEXP = 5,
+    /* out[m] = log sum_n exp(E[m,n]), fp32 [M]: the row statistic of a softmax over N, merged
+     * across output tiles as (max, sum of exponentials) pairs; Y is never written (Section 4 of
+     * the paper: warp-shuffle max / sum reductions of a cross-entropy kernel).                */
+    FORGE_RED_CROSS_ENTROPY = 6
+    /* out[m] = logsumexp_n E[m,:] - E[m, target[m]], fp32 [M]: the per-row loss of a classifier
+     * head whose logits are never materialised.  run() takes the int32 class indices target[M]
+     * (device pointer, each in [0, N)) in its `gamma` argument; `beta` is ignored.             */
 } forge_red_t;
 
 typedef struct {
@@ -127,8 +136,9 @@ forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, 
  * Enqueue one evaluation on `cuda_stream` (a cudaStream_t; NULL = default stream).
  * DEVICE pointers, owned by the caller, 16-byte aligned, alive until the work completes:
  *   X [M,K], W [N,K], b [N] (may be NULL iff has_bias == 0), gamma, beta [N] (non-NULL iff
- *   layernorm), out: Y [M,N] in dtype (none, layernorm), fp32 [M] (sum, max), or Y [M,K] in
- *   dtype (mean-gelu-residual, whose subtract vector travels in `gamma`).
+ *   layernorm), out: Y [M,N] in dtype (none, layernorm), fp32 [M] (sum, max, logsumexp,
+ *   cross-entropy, whose int32 targets travel in `gamma`), or Y [M,K] in dtype
+ *   (mean-gelu-residual, whose subtract vector travels in `gamma`).
  * Allocates nothing and does not synchronise.  Returns only argument / launch errors;
  * device-side give-ups are reported by forge_fused_linear_last_status().  At most one run
  * per handle may be in flight (the workspace belongs to the handle).

@@ -15,7 +15,8 @@ LIB_PATH = os.path.join(_HERE, "libforge.so")
 FORGE_STATIC_SCRATCH_BYTES = 1 << 20
 FORGE_F32, FORGE_BF16 = 0, 1
 FORGE_ACT_IDENTITY, FORGE_ACT_RELU, FORGE_ACT_GELU_ERF, FORGE_ACT_GELU_TANH, FORGE_ACT_SILU = range(5)
-FORGE_RED_NONE, FORGE_RED_SUM, FORGE_RED_MAX, FORGE_RED_LAYERNORM, FORGE_RED_MEAN_GELU_RESIDUAL = range(5)
+(FORGE_RED_NONE, FORGE_RED_SUM, FORGE_RED_MAX, FORGE_RED_LAYERNORM, FORGE_RED_MEAN_GELU_RESIDUAL,
+ FORGE_RED_LOGSUMEXP, FORGE_RED_CROSS_ENTROPY) = range(7)
 FORGE_KERNEL_F32_FFMA, FORGE_KERNEL_BF16_TCGEN05, FORGE_KERNEL_BF16_SKINNY, FORGE_KERNEL_BF16_TCGEN05_LN = 1, 2, 3, 4
 
 EXPORTS = [

@@ -121,6 +121,23 @@ __device__ __forceinline__ RowStat shfl_xor_stat(RowStat s, int mask)
     return o;
 }
 
+// ---- log-sum-exp partials ---------------------------------------------------------------
+// A set of logits is summarised by (m, s) with m its maximum and s = sum exp(x - m); two
+// summaries combine to (max(m1, m2), s1 exp(m1 - m) + s2 exp(m2 - m)).  An empty set is
+// (-inf, 0) and must not contribute exp(-inf + inf).
+template <bool ACCURATE>
+__device__ __forceinline__ float lse_exp(float x) { return ACCURATE ? expf(x) : __expf(x); }
+
+template <bool ACCURATE>
+__device__ __forceinline__ void lse_merge(float &m, float &s, float om, float os)
+{
+    const float nm = fmaxf(m, om);
+    const float a = (m == -INFINITY) ? 0.f : s * lse_exp<ACCURATE>(m - nm);
+    const float b = (om == -INFINITY) ? 0.f : os * lse_exp<ACCURATE>(om - nm);
+    m = nm;
+    s = a + b;
+}
+
 // Order-preserving map float -> unsigned (for an order-independent atomic max).
 __device__ __forceinline__ unsigned float_to_ordered(float f)
 {

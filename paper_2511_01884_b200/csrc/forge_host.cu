@@ -15,7 +15,7 @@ constexpr size_t kStatusBytes = 256;     // status word lives alone in the first
 bool desc_enums_ok(const forge_fused_linear_desc_t &d)
 {
     return (d.dtype == FORGE_F32 || d.dtype == FORGE_BF16) && d.act >= FORGE_ACT_IDENTITY &&
-           d.act <= FORGE_ACT_SILU && d.red >= FORGE_RED_NONE && d.red <= FORGE_RED_MEAN_GELU_RESIDUAL;
+           d.act <= FORGE_ACT_SILU && d.red >= FORGE_RED_NONE && d.red <= FORGE_RED_CROSS_ENTROPY;
 }
 
 forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
@@ -32,7 +32,7 @@ forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_
         if (d.K % 8 != 0 || d.N % 8 != 0) return FORGE_ERR_UNSUPPORTED;     // 16-byte row pitch for TMA
         if (d.red == FORGE_RED_MEAN_GELU_RESIDUAL) return FORGE_ERR_UNSUPPORTED;   // fp32 only so far
         if (d.red == FORGE_RED_LAYERNORM) st = k4_plan(d, sm_count, info, wl);
-        else if (d.M <= 16) st = k3_plan(d, sm_count, info, wl);
+        else if (d.M <= 16 && d.red <= FORGE_RED_MAX) st = k3_plan(d, sm_count, info, wl);
         else st = k2_plan(d, sm_count, info, wl);
     }
     if (st != FORGE_OK) return st;
@@ -60,7 +60,8 @@ struct DeviceGuard {
 size_t elem_bytes(const forge_fused_linear_desc_t &d) { return d.dtype == FORGE_F32 ? 4 : 2; }
 size_t out_bytes(const forge_fused_linear_desc_t &d)
 {
-    if (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) return (size_t)d.M * 4;
+    if (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY)
+        return (size_t)d.M * 4;
     return (size_t)d.M * (size_t)(d.red == FORGE_RED_MEAN_GELU_RESIDUAL ? d.K : d.N) * elem_bytes(d);
 }
 
@@ -69,6 +70,7 @@ forge_status_t check_run_args(const Handle &h, const RunArgs &a)
     if (!a.X || !a.W || !a.out) return FORGE_ERR_INVALID_ARG;
     if (h.d.has_bias && !a.b) return FORGE_ERR_INVALID_ARG;
     if (h.d.red == FORGE_RED_LAYERNORM && (!a.gamma || !a.beta)) return FORGE_ERR_INVALID_ARG;
+    if (h.d.red == FORGE_RED_CROSS_ENTROPY && !a.gamma) return FORGE_ERR_INVALID_ARG;      // the targets
     const uintptr_t m = (uintptr_t)a.X | (uintptr_t)a.W | (uintptr_t)a.out | (uintptr_t)a.b |
                         (uintptr_t)a.gamma | (uintptr_t)a.beta;
     // bf16 operands travel by TMA and 128-bit accesses: 16-byte alignment is required.
@@ -203,15 +205,18 @@ forge_status_t forge_fused_linear_run_host(forge_fused_linear_t hh, const void *
     if (!hh) return FORGE_ERR_INVALID_ARG;
     Handle &h = *reinterpret_cast<Handle *>(hh);
     const forge_fused_linear_desc_t &d = h.d;
-    if (!X || !W || !out || (d.has_bias && !b) || (d.red == FORGE_RED_LAYERNORM && (!gamma || !beta)))
+    if (!X || !W || !out || (d.has_bias && !b) || (d.red == FORGE_RED_LAYERNORM && (!gamma || !beta)) ||
+        (d.red == FORGE_RED_CROSS_ENTROPY && !gamma))
         return FORGE_ERR_INVALID_ARG;
     DeviceGuard g(d.device);
     if (!g.ok) return FORGE_ERR_CUDA;
     const size_t e = elem_bytes(d);
     const size_t bx = (size_t)d.M * d.K * e, bw = (size_t)d.N * d.K * e, bn = (size_t)d.N * e, bo = out_bytes(d);
+    const size_t bt = (size_t)d.M * 4;                       // int32 targets of the cross-entropy
+    const size_t bg = bn > bt ? bn : bt;                     // the gamma slot holds either
     if (!h.hX) {
         if (cudaMalloc(&h.hX, bx) != cudaSuccess || cudaMalloc(&h.hW, bw) != cudaSuccess ||
-            cudaMalloc(&h.hb, bn) != cudaSuccess || cudaMalloc(&h.hg, bn) != cudaSuccess ||
+            cudaMalloc(&h.hb, bn) != cudaSuccess || cudaMalloc(&h.hg, bg) != cudaSuccess ||
             cudaMalloc(&h.hbe, bn) != cudaSuccess || cudaMalloc(&h.hout, bo) != cudaSuccess) {
             cudaGetLastError();
             cudaFree(h.hX); cudaFree(h.hW); cudaFree(h.hb); cudaFree(h.hg); cudaFree(h.hbe); cudaFree(h.hout);
@@ -228,9 +233,11 @@ forge_status_t forge_fused_linear_run_host(forge_fused_linear_t hh, const void *
              cudaMemcpyAsync(h.hbe, beta, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
     const bool has_sub = d.red == FORGE_RED_MEAN_GELU_RESIDUAL && gamma;
     if (ok && has_sub) ok = cudaMemcpyAsync(h.hg, gamma, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    const bool has_tgt = d.red == FORGE_RED_CROSS_ENTROPY;
+    if (ok && has_tgt) ok = cudaMemcpyAsync(h.hg, gamma, bt, cudaMemcpyHostToDevice, s) == cudaSuccess;
     if (!ok) return FORGE_ERR_CUDA;
     RunArgs a{h.hX, h.hW, d.has_bias ? h.hb : nullptr,
-              (d.red == FORGE_RED_LAYERNORM || has_sub) ? h.hg : nullptr, h.hbe, h.hout, s};
+              (d.red == FORGE_RED_LAYERNORM || has_sub || has_tgt) ? h.hg : nullptr, h.hbe, h.hout, s};
     const forge_status_t st = dispatch(h, a);
     if (st != FORGE_OK) return st;
     if (cudaMemcpyAsync(out, h.hout, bo, cudaMemcpyDeviceToHost, s) != cudaSuccess) return FORGE_ERR_CUDA;

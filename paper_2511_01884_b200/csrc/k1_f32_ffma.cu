@@ -261,6 +261,61 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         return;
     }
 
+    if (RED == FORGE_RED_LOGSUMEXP || RED == FORGE_RED_CROSS_ENTROPY) {
+        constexpr bool CE = RED == FORGE_RED_CROSS_ENTROPY;
+        const int *target = reinterpret_cast<const int *>(p.gamma);          // class index per row (CE)
+        float4 *part4 = reinterpret_cast<float4 *>(p.partial);               // (max, sum exp, target logit, -)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int row = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
+            float mx = -INFINITY, se = 0.f, tl = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (cok[j]) mx = fmaxf(mx, acc[i][j]);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (cok[j]) se += expf(acc[i][j] - mx);
+            if (CE && row < M) {
+                const int t = __ldg(target + row);
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (cok[j] && col[j] == t) tl = acc[i][j];
+            }
+            // the 16 lanes that share the row: shuffles, no block-wide barrier
+#pragma unroll
+            for (int s = 8; s >= 1; s >>= 1) {
+                const float om = __shfl_xor_sync(0xffffffffu, mx, s);
+                const float os = __shfl_xor_sync(0xffffffffu, se, s);
+                tl += __shfl_xor_sync(0xffffffffu, tl, s);                    // exactly one lane holds it
+                lse_merge<true>(mx, se, om, os);
+            }
+            if (tx == 0 && row < M) {
+                if (p.tiles_n == 1) p.out[row] = mx + logf(se) - tl;
+                else part4[(size_t)tile_n * M + row] = make_float4(mx, se, tl, 0.f);
+            }
+        }
+        if (p.tiles_n == 1) return;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) s_last = (atomicAdd(&p.counters[tile_m], 1u) == (unsigned)(p.tiles_n - 1));
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+        if (tid < K1_BM && m0 + tid < M) {
+            const int row = m0 + tid;
+            float4 f = __ldcg(&part4[row]);
+            float mx = f.x, se = f.y, tl = f.z;
+            for (int t = 1; t < p.tiles_n; ++t) {
+                f = __ldcg(&part4[(size_t)t * M + row]);
+                lse_merge<true>(mx, se, f.x, f.y);
+                tl += f.z;
+            }
+            p.out[row] = mx + logf(se) - tl;
+        }
+        if (tid == 0) p.counters[tile_m] = 0u;
+        return;
+    }
+
     if (RED == FORGE_RED_LAYERNORM) {
         cg::cluster_group cluster = cg::this_cluster();
         // per-thread statistics of its <= 8 columns of each row, two sweeps over registers
@@ -335,8 +390,9 @@ forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     info->threads = K1_THREADS;
     info->grid = tiles_m * tiles_n;
     info->smem_bytes = 0;
-    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL) && tiles_n > 1;
-    wl->partial_floats = partials ? (size_t)tiles_n * (size_t)d.M : 0;
+    const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;      // float4 partials
+    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL || lse) && tiles_n > 1;
+    wl->partial_floats = partials ? (lse ? 4 : 1) * (size_t)tiles_n * (size_t)d.M : 0;
     wl->counters = partials ? (size_t)tiles_m : 0;
     return FORGE_OK;
 }
@@ -394,6 +450,8 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
         K1_CASE(FORGE_RED_MAX)
         K1_CASE(FORGE_RED_LAYERNORM)
         K1_CASE(FORGE_RED_MEAN_GELU_RESIDUAL)
+        K1_CASE(FORGE_RED_LOGSUMEXP)
+        K1_CASE(FORGE_RED_CROSS_ENTROPY)
     }
 #undef K1_CASE
     return FORGE_ERR_INVALID_ARG;

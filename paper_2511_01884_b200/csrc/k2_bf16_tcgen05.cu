@@ -380,6 +380,67 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 continue;
             }
 
+            if (p.e.red == FORGE_RED_LOGSUMEXP || p.e.red == FORGE_RED_CROSS_ENTROPY) {
+                // online (max, sum exp) over this thread's row of the half tile; the target's logit
+                // is picked up on the way (cross-entropy); Y is never written
+                const int tgt = (p.e.red == FORGE_RED_CROSS_ENTROPY && row < p.M)
+                                    ? __ldg(reinterpret_cast<const int *>(p.gamma) + row) : -1;
+                float mx = -INFINITY, se = 0.f, tl = 0.f;
+#pragma unroll 1
+                for (int c = 0; c < CHUNKS; ++c) {
+                    const int col0 = n0 + c * 32;
+                    if (col0 >= p.N) break;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(taddr + c * 32, r);
+                    ptx::tmem_ld_wait();
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
+                    apply_act_array<false>(p.e.act, v, p.e.scale);
+                    const int nv = min(32, p.N - col0);
+                    float cm = -INFINITY;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) cm = j < nv ? fmaxf(cm, v[j]) : cm;
+                    const float nm = fmaxf(mx, cm);
+                    float cs = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) cs += j < nv ? __expf(v[j] - nm) : 0.f;
+                    se = (mx == -INFINITY ? 0.f : se * __expf(mx - nm)) + cs;
+                    mx = nm;
+                    if (tgt >= col0 && tgt < col0 + 32) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) tl = (col0 + j == tgt) ? v[j] : tl;
+                    }
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
+
+                float4 *part4 = reinterpret_cast<float4 *>(p.partial);
+                if (row < p.M) part4[(size_t)part * p.M + row] = make_float4(mx, se, tl, 0.f);
+                __threadfence();
+                epi_bar_sync(h);
+                if (et == 0) s.last_flag[h] = (atomicAdd(&p.counters[tm], 1u) == (unsigned)(parts - 1));
+                epi_bar_sync(h);
+                if (s.last_flag[h]) {
+                    // the group that arrives last at the strip merges the parts in order
+                    __threadfence();
+                    if (row < p.M) {
+                        float4 f = __ldcg(&part4[row]);
+                        mx = f.x; se = f.y; tl = f.z;
+                        for (int i = 1; i < parts; ++i) {
+                            f = __ldcg(&part4[(size_t)i * p.M + row]);
+                            lse_merge<false>(mx, se, f.x, f.y);
+                            tl += f.z;
+                        }
+                        reinterpret_cast<float *>(p.out)[row] = mx + __logf(se) - tl;
+                    }
+                    if (et == 0) p.counters[tm] = 0u;
+                }
+                if ((acc ^= 1) == 0) acc_phase ^= 1;
+                continue;
+            }
+
             float red = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY;
 #pragma unroll 1
             for (int c = 0; c < CHUNKS; ++c) {
@@ -486,8 +547,9 @@ forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
         info->grid = tiles_m * tiles_n < sm_count ? tiles_m * tiles_n : sm_count;
     }
     info->smem_bytes = (int64_t)K2_SMEM_BYTES;
-    const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX;      // one partial per row and half tile
-    wl->partial_floats = partials ? 2 * (size_t)tiles_n * (size_t)d.M : 0;
+    const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;      // float4 partials
+    const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || lse;         // one per row and half tile
+    wl->partial_floats = partials ? (lse ? 4 : 1) * 2 * (size_t)tiles_n * (size_t)d.M : 0;
     wl->counters = partials ? (size_t)tiles_m : 0;
     return FORGE_OK;
 }

@@ -45,7 +45,7 @@ def test_enums_match_the_workload_module():
 
 def test_invalid_descriptors():
     ok = dict(M=8, N=8, K=8, dtype=0, act=0, red=0)
-    for bad in (dict(M=0), dict(N=-1), dict(K=0), dict(dtype=2), dict(act=5), dict(act=-1), dict(red=5)):
+    for bad in (dict(M=0), dict(N=-1), dict(K=0), dict(dtype=2), dict(act=5), dict(act=-1), dict(red=7), dict(red=-1)):
         st, _ = B.forge_fused_linear_query_plan(B.make_desc(**{**ok, **bad}))
         assert st == B.FORGE_ERR_INVALID_ARG, bad
         st, h = B.forge_fused_linear_create(B.make_desc(**{**ok, **bad}))

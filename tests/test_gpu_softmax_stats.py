@@ -1,0 +1,68 @@
+"""GPU parity of the softmax row statistics -- log-sum-exp and per-row cross-entropy, merged
+across output tiles as (max, sum of exponentials) pairs -- on the fp32 and bf16 paths."""
+import numpy as np
+import pytest
+
+from paper_2511_01884_b200 import binding as B
+from paper_2511_01884_b200 import workloads as wk
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+REDS = [wk.RED_LOGSUMEXP, wk.RED_CROSS_ENTROPY]
+F32_SHAPES = [(1, 1, 1), (5, 100, 7), (128, 128, 16), (130, 300, 36), (257, 1000, 64), (64, 2500, 19)]
+BF16_SHAPES = [(17, 8, 8), (128, 256, 64), (16, 1024, 128), (300, 520, 200), (1000, 776, 328), (260, 4104, 64)]
+
+
+@pytest.mark.parametrize("M,N,K", F32_SHAPES)
+@pytest.mark.parametrize("red", REDS)
+def test_fp32(M, N, K, red):
+    wl = wk.custom_workload(f"lse_f32_{M}x{N}x{K}", wk.F32, M, N, K, wk.ACT_IDENTITY, red, scale=3.0, seed=M + N)
+    inp = wk.make_inputs(wl)
+    g, plan = pu.run_gpu(wl, inp)
+    assert g.shape == (M,) and plan["kernel"] == B.FORGE_KERNEL_F32_FFMA
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+@pytest.mark.parametrize("M,N,K", BF16_SHAPES)
+@pytest.mark.parametrize("red", REDS)
+def test_bf16(M, N, K, red):
+    wl = wk.custom_workload(f"lse_bf16_{M}x{N}x{K}", wk.BF16, M, N, K, wk.ACT_IDENTITY, red, scale=2.0, seed=M + N)
+    inp = wk.make_inputs(wl)
+    g, plan = pu.run_gpu(wl, inp)
+    assert plan["kernel"] == B.FORGE_KERNEL_BF16_TCGEN05          # also for M <= 16
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_large_logits_do_not_overflow_and_runs_repeat():
+    wl = wk.custom_workload("lse_big", wk.F32, 200, 700, 32, wk.ACT_IDENTITY, wk.RED_CROSS_ENTROPY, scale=40.0, seed=6)
+    inp = wk.make_inputs(wl)
+    ref = pu.run_oracle(wl, inp)
+    assert ref.max() > 50                                         # exp of these logits overflows fp32 without the max shift
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op)
+    b, _ = pu.run_gpu(wl, inp, op=op, repeats=3)
+    op.close()
+    assert np.array_equal(a, b) and np.isfinite(a).all()
+    pu.assert_parity(wl, a, ref)
+
+
+def test_cross_entropy_needs_its_targets():
+    import torch
+    wl = wk.custom_workload("lse_args", wk.BF16, 64, 64, 64, wk.ACT_IDENTITY, wk.RED_CROSS_ENTROPY)
+    op = B.FusedLinear(pu.desc_of(wl))
+    t = torch.zeros(64 * 64, dtype=torch.bfloat16, device="cuda")
+    o = torch.zeros(64, dtype=torch.float32, device="cuda")
+    assert B.forge_fused_linear_run(op.h, t, t, t, None, None, o) == B.FORGE_ERR_INVALID_ARG
+    op.close()
+
+
+def test_n2_sampled_rows_full_size():
+    wl = wk.EXTRA_WORKLOADS["n2"]
+    inp = wk.make_inputs(wl)
+    g, plan = pu.run_gpu(wl, inp)
+    assert plan["cluster"] == 2 and np.isfinite(g).all()
+    rows = wk.sample_rows(wl.M)[::2]
+    pu.assert_parity(wl, g[rows], pu.run_oracle(wl, inp, rows))
+    assert abs(g.mean() - np.log(wl.N)) < 1.0                     # near-uniform predictions: loss close to log N
