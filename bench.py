@@ -139,8 +139,10 @@ def device_tensors(wl, inp, torch):
             return None
         t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
         return (t.to(torch.bfloat16) if wl.dtype == wk.BF16 else t).cuda()
-    d = {k: dev(v) for k, v in inp.items()}
+    d = {k: dev(v) for k, v in inp.items() if k != "target"}
     M = inp["X"].shape[0]
+    if wl.red == wk.RED_CROSS_ENTROPY:     # the int32 class indices travel in the gamma slot of the interface
+        d["gamma"] = torch.from_numpy(np.ascontiguousarray(inp["target"], dtype=np.int32)).cuda()
     if wl.out_cols == 0:
         d["out"] = torch.empty((M,), dtype=torch.float32, device="cuda")
     else:
@@ -218,6 +220,10 @@ def eager_context_us(wl, d, torch, steps=10):
             return F.layer_norm(z, (wl.N,), d["gamma"], d["beta"], wl.ln_eps)
         if wl.red == wk.RED_MEAN_GELU_RESIDUAL:
             return d["X"] + F.gelu((z - d["gamma"]).mean(1, keepdim=True))
+        if wl.red == wk.RED_LOGSUMEXP:
+            return torch.logsumexp(z.float(), 1)
+        if wl.red == wk.RED_CROSS_ENTROPY:
+            return F.cross_entropy(z.float(), d["gamma"].long(), reduction="none")
         return z
     for _ in range(3):
         chain()
@@ -266,9 +272,10 @@ def oracle_sample(wl, inp, target_s=12.0, max_rows=None):
     M = inp["X"].shape[0]
     rows_all = wk.sample_rows(M)
     probe = rows_all[: min(len(rows_all), 4)]
+    extra = {"sub": inp.get("sub"), "target": inp.get("target")}
     t = time.perf_counter()
     oracle.fused_linear(inp["X"], inp["W"], inp["b"], inp["gamma"], inp["beta"], act=wl.act, scale=wl.scale,
-                        red=wl.red, eps=wl.ln_eps, rows=probe)
+                        red=wl.red, eps=wl.ln_eps, rows=probe, **extra)
     per_row = (time.perf_counter() - t) / len(probe)
     n = int(max(len(probe), min(M, target_s / max(per_row, 1e-9))))
     if max_rows:
@@ -276,7 +283,7 @@ def oracle_sample(wl, inp, target_s=12.0, max_rows=None):
     rows = np.arange(n, dtype=np.int64) * (M // n) if n < M else np.arange(M, dtype=np.int64)
     t = time.perf_counter()
     oracle.fused_linear(inp["X"], inp["W"], inp["b"], inp["gamma"], inp["beta"], act=wl.act, scale=wl.scale,
-                        red=wl.red, eps=wl.ln_eps, rows=rows)
+                        red=wl.red, eps=wl.ln_eps, rows=rows, **extra)
     dt = time.perf_counter() - t
     flops = 2.0 * len(rows) * wl.N * wl.K
     if wl.name == "c4":
@@ -304,7 +311,7 @@ def run_reference(args):
     for i in range(args.warmup + args.steps):
         t = time.perf_counter()
         oracle.fused_linear(inp["X"], inp["W"], inp["b"], inp["gamma"], inp["beta"], act=wl.act, scale=wl.scale,
-                            red=wl.red, eps=wl.ln_eps, rows=sel)
+                            red=wl.red, eps=wl.ln_eps, rows=sel, sub=inp.get("sub"), target=inp.get("target"))
         if i >= args.warmup:
             times.append(time.perf_counter() - t)
     ms = 1e3 * sum(times) / len(times)
@@ -328,7 +335,8 @@ def config_of(wl, n_gpus, extra=None):
     names = {wk.ACT_IDENTITY: "identity", wk.ACT_RELU: "relu", wk.ACT_GELU_ERF: "gelu_erf",
              wk.ACT_GELU_TANH: "gelu_tanh", wk.ACT_SILU: "silu"}
     reds = {wk.RED_NONE: "none", wk.RED_SUM: "row_sum", wk.RED_MAX: "row_max", wk.RED_LAYERNORM: "layernorm",
-            wk.RED_MEAN_GELU_RESIDUAL: "subtract_rowmean_gelu_residual"}
+            wk.RED_MEAN_GELU_RESIDUAL: "subtract_rowmean_gelu_residual", wk.RED_LOGSUMEXP: "row_logsumexp",
+            wk.RED_CROSS_ENTROPY: "row_cross_entropy"}
     c = {"workload": f"{wl.name}: {wl.note}", "M_per_gpu": wl.M, "N": wl.N, "K": wl.K,
          "dtype": "bf16" if wl.dtype == wk.BF16 else "f32", "act": names[wl.act], "scale": wl.scale,
          "reduction": reds[wl.red], "seed": wl.seed, "parallelism": f"rows sharded over {n_gpus} gpu(s), no collective",
@@ -443,7 +451,7 @@ def main():
                 d2 = device_tensors(w2, i2, torch)
                 op2 = make_op(w2, w2.M, local)
                 fl = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device="cuda") if w2.algorithmic_bytes < 130e6 else None
-                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50, "n1": 20}[name]
+                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50, "n1": 20, "n2": 10}[name]
                 ms2 = time_steps(op2, d2, steps2, 3, torch, flush_buf=fl)
                 v2, u2 = unit_value(w2, ms2)
                 launches += steps2

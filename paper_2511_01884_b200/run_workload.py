@@ -32,7 +32,9 @@ def main() -> int:
             return None
         t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
         return (t.to(torch.bfloat16) if wl.dtype == wk.BF16 else t).cuda()
-    d = {k: dev(v) for k, v in inp.items()}
+    d = {k: dev(v) for k, v in inp.items() if k != "target"}
+    if wl.red == wk.RED_CROSS_ENTROPY:     # int32 class indices travel in the gamma slot
+        d["gamma"] = torch.from_numpy(np.ascontiguousarray(inp["target"], dtype=np.int32)).cuda()
     reduce = wl.out_cols == 0
     out = torch.empty((M,) if reduce else (M, wl.out_cols), device="cuda",
                       dtype=torch.float32 if (reduce or wl.dtype == wk.F32) else torch.bfloat16)

@@ -55,14 +55,15 @@ def test_fp32_accepts_unaligned_operands_with_scalar_accesses():
     assert np.isnan(obuf[0].item())                                # nothing written in front of the output
 
 
-@pytest.mark.parametrize("name", ["c1", "skinny", "ln", "plain", "chain"])
+@pytest.mark.parametrize("name", ["c1", "skinny", "ln", "plain", "chain", "ce"])
 def test_host_buffer_entry_point_matches_the_oracle(name):
     import torch
     wl = {"c1": wk.WORKLOADS["c1"],
           "skinny": wk.custom_workload("h_skinny", wk.BF16, 16, 1024, 256, wk.ACT_GELU_ERF, wk.RED_MAX, w_std=0.05),
           "ln": wk.custom_workload("h_ln", wk.BF16, 300, 520, 128, wk.ACT_GELU_TANH, wk.RED_LAYERNORM, w_std=0.05),
           "plain": wk.custom_workload("h_plain", wk.BF16, 300, 520, 128, wk.ACT_SILU, wk.RED_NONE, w_std=0.05),
-          "chain": wk.custom_workload("h_chain", wk.F32, 150, 300, 40, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL)}[name]
+          "chain": wk.custom_workload("h_chain", wk.F32, 150, 300, 40, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL),
+          "ce": wk.custom_workload("h_ce", wk.BF16, 300, 1032, 128, wk.ACT_IDENTITY, wk.RED_CROSS_ENTROPY, w_std=0.05)}[name]
     inp = wk.make_inputs(wl)
 
     def host(a):
@@ -70,8 +71,10 @@ def test_host_buffer_entry_point_matches_the_oracle(name):
             return None
         t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
         return (t.to(torch.bfloat16) if wl.dtype == wk.BF16 else t).pin_memory()
-    h = {k: host(v) for k, v in inp.items()}
+    h = {k: host(v) for k, v in inp.items() if k != "target"}
     aux = h["sub"] if wl.red == wk.RED_MEAN_GELU_RESIDUAL else h["gamma"]
+    if wl.red == wk.RED_CROSS_ENTROPY:
+        aux = torch.from_numpy(np.ascontiguousarray(inp["target"], dtype=np.int32)).pin_memory()
     shape = (wl.M,) if wl.out_cols == 0 else (wl.M, wl.out_cols)
     out = torch.zeros(shape, dtype=torch.float32 if (wl.out_cols == 0 or wl.dtype == wk.F32) else torch.bfloat16).pin_memory()
     op = B.FusedLinear(pu.desc_of(wl))
