@@ -32,18 +32,21 @@ struct K1Params {
     int tiles_n;
     int out_vec4;          // Y rows can be written with 128-bit stores
     int res_vec4;          // mean chain: X and Y rows ([M,K]) can be moved with 128-bit accesses
+    int warm_l2;           // small grids: request the CTA's operand panels into L2 before the k loop
 };
 
-// One CTA-tile slab of 128 rows x 16 k from a K-major matrix into registers.
-template <bool VEC>
+// One CTA-tile slab (128 rows x 16 k, or 64 rows x 32 k) from a K-major matrix into registers:
+// two float4 per thread either way.
+template <bool VEC, int T>
 __device__ __forceinline__ void k1_fetch(const float *__restrict__ base, int rows_total, int K,
                                          int row0, int kt, int tid, float4 (&r)[2])
 {
+    constexpr int KQ = (T == 1 ? 32 : 16) / 4;          // float4 per row of the slab
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int idx = tid + i * K1_THREADS;
-        const int row = row0 + (idx >> 2);
-        const int k = kt + (idx & 3) * 4;
+        const int row = row0 + idx / KQ;
+        const int k = kt + (idx % KQ) * 4;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (row < rows_total) {
             const float *src = base + (size_t)row * K + k;
@@ -61,15 +64,17 @@ __device__ __forceinline__ void k1_fetch(const float *__restrict__ base, int row
 }
 
 // Registers -> shared memory, transposed to [k][row] so the inner product reads rows of 4.
-__device__ __forceinline__ void k1_stash(float (*S)[K1_BM + K1_PAD], int tid, const float4 (&r)[2])
+template <int T>
+__device__ __forceinline__ void k1_stash(float (*S)[64 * T + K1_PAD], int tid, const float4 (&r)[2])
 {
+    constexpr int KQ = (T == 1 ? 32 : 16) / 4;
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int idx = tid + i * K1_THREADS;
-        const int k = (idx & 3) * 4;
+        const int k = (idx % KQ) * 4;
         // rows of the k-groups 8..15 are stored with bit 3 of the row index flipped: the four
         // k-groups a warp writes at once then fall into four different bank octets
-        const int row = (idx >> 2) ^ (((k >> 3) & 1) << 3);
+        const int row = (idx / KQ) ^ (((k >> 3) & 1) << 3);
         S[k + 0][row] = r[i].x;
         S[k + 1][row] = r[i].y;
         S[k + 2][row] = r[i].z;
@@ -94,98 +99,119 @@ __device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
 
-template <bool VEC, int RED>
+// T = 2: 128x128 CTA tile, 8x8 accumulators per thread.  T = 1: 64x64 tile, 4x4 per thread, for
+// problems with too few 128x128 tiles to occupy the SMs (a grid of a handful of CTAs is bound by
+// the FMA rate of the few SMs it runs on, not by the GPU's).
+template <bool VEC, int RED, int T>
 __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Params p)
 {
-    __shared__ __align__(16) float As[2][K1_BK][K1_BM + K1_PAD];
-    __shared__ __align__(16) float Bs[2][K1_BK][K1_BN + K1_PAD];
-    __shared__ RowStat s_stat[K1_BM];
-    __shared__ float s_mean[K1_BM], s_rstd[K1_BM];
+    constexpr int BM = 64 * T, BN = 64 * T, R = 4 * T;       // tile and per-thread extent
+    constexpr int BK = T == 1 ? 32 : K1_BK;                  // the small tile takes longer k steps (fewer round trips)
+    __shared__ __align__(16) float As[2][BK][BM + K1_PAD];
+    __shared__ __align__(16) float Bs[2][BK][BN + K1_PAD];
+    __shared__ RowStat s_stat[BM];
+    __shared__ float s_mean[BM], s_rstd[BM];
     __shared__ int s_last;
 
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
     const int tile_n = blockIdx.x, tile_m = blockIdx.y;
-    const int m0 = tile_m * K1_BM, n0 = tile_n * K1_BN;
+    const int m0 = tile_m * BM, n0 = tile_n * BN;
     const int M = p.M, N = p.N, K = p.K;
 
-    unsigned long long acc2[8][4];       // acc2[i][j] = accumulators (i, 2j) and (i, 2j+1)
+    unsigned long long acc2[R][R / 2];   // acc2[i][j] = accumulators (i, 2j) and (i, 2j+1)
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < R; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc2[i][j] = 0ull;
+        for (int j = 0; j < R / 2; ++j) acc2[i][j] = 0ull;
 
+    if (p.warm_l2) {
+        // A small grid walks K with one tile of look-ahead, i.e. it pays the memory latency once
+        // per k-tile.  Asking L2 for both operand panels up front puts all of those requests in
+        // flight at once; the k loop then runs at L2 latency.
+        const int lines_per_row = (K * 4 + 127) / 128;
+        const int rows_a = min(BM, M - m0), rows_b = min(BN, N - n0);
+        for (int i = tid; i < (rows_a + rows_b) * lines_per_row; i += K1_THREADS) {
+            const int r = i / lines_per_row, c = i - r * lines_per_row;
+            const float *ptr = r < rows_a ? p.X + (size_t)(m0 + r) * K : p.W + (size_t)(n0 + r - rows_a) * K;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr + min(c * 32, K - 1)));
+        }
+    }
     float4 ra[2], rb[2];
-    k1_fetch<VEC>(p.X, M, K, m0, 0, tid, ra);
-    k1_fetch<VEC>(p.W, N, K, n0, 0, tid, rb);
-    k1_stash(As[0], tid, ra);
-    k1_stash(Bs[0], tid, rb);
+    k1_fetch<VEC, T>(p.X, M, K, m0, 0, tid, ra);
+    k1_fetch<VEC, T>(p.W, N, K, n0, 0, tid, rb);
+    k1_stash<T>(As[0], tid, ra);
+    k1_stash<T>(Bs[0], tid, rb);
     __syncthreads();
 
     int buf = 0;
-    for (int kt = 0; kt < K; kt += K1_BK) {
-        const bool more = kt + K1_BK < K;
+    for (int kt = 0; kt < K; kt += BK) {
+        const bool more = kt + BK < K;
         if (more) {
-            k1_fetch<VEC>(p.X, M, K, m0, kt + K1_BK, tid, ra);
-            k1_fetch<VEC>(p.W, N, K, n0, kt + K1_BK, tid, rb);
+            k1_fetch<VEC, T>(p.X, M, K, m0, kt + BK, tid, ra);
+            k1_fetch<VEC, T>(p.W, N, K, n0, kt + BK, tid, rb);
         }
 #pragma unroll
-        for (int k = 0; k < K1_BK; ++k) {
+        for (int k = 0; k < BK; ++k) {
             const int flip = ((k >> 3) & 1) << 3;          // see k1_stash
-            const float4 a0 = *reinterpret_cast<const float4 *>(&As[buf][k][(ty * 4) ^ flip]);
-            const float4 a1 = *reinterpret_cast<const float4 *>(&As[buf][k][64 + ((ty * 4) ^ flip)]);
-            const ulonglong2 b0 = *reinterpret_cast<const ulonglong2 *>(&Bs[buf][k][(tx * 4) ^ flip]);
-            const ulonglong2 b1 = *reinterpret_cast<const ulonglong2 *>(&Bs[buf][k][64 + ((tx * 4) ^ flip)]);
-            const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-            const unsigned long long b[4] = {b0.x, b0.y, b1.x, b1.y};      // column pairs as they lie in memory
+            float a[R];
+            unsigned long long b[R / 2];                    // column pairs as they lie in memory
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int q = 0; q < T; ++q) {
+                const float4 av = *reinterpret_cast<const float4 *>(&As[buf][k][64 * q + ((ty * 4) ^ flip)]);
+                const ulonglong2 bv = *reinterpret_cast<const ulonglong2 *>(&Bs[buf][k][64 * q + ((tx * 4) ^ flip)]);
+                a[4 * q + 0] = av.x; a[4 * q + 1] = av.y; a[4 * q + 2] = av.z; a[4 * q + 3] = av.w;
+                b[2 * q + 0] = bv.x; b[2 * q + 1] = bv.y;
+            }
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
                 const unsigned long long ai = pack2(a[i], a[i]);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) ffma2(acc2[i][j], ai, b[j]);
+                for (int j = 0; j < R / 2; ++j) ffma2(acc2[i][j], ai, b[j]);
             }
         }
         if (more) {
-            k1_stash(As[buf ^ 1], tid, ra);
-            k1_stash(Bs[buf ^ 1], tid, rb);
+            k1_stash<T>(As[buf ^ 1], tid, ra);
+            k1_stash<T>(Bs[buf ^ 1], tid, rb);
         }
         __syncthreads();
         buf ^= 1;
     }
 
-    float acc[8][8];
+    float acc[R][R];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < R; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) unpack2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
+        for (int j = 0; j < R / 2; ++j) unpack2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
 
     // ---- epilogue: bias, activation, scale, in registers --------------------------------
-    int col[8];
-    bool cok[8];
-    float bias[8];
+    int col[R];
+    bool cok[R];
+    float bias[R];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < R; ++j) {
         col[j] = n0 + tx * 4 + (j & 3) + (j >> 2) * 64;
         cok[j] = col[j] < N;
         bias[j] = (p.e.has_bias && cok[j]) ? __ldg(p.b + col[j]) : 0.f;
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < R; ++i)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = p.e.scale * apply_act<true>(p.e.act, acc[i][j] + bias[j]);
+        for (int j = 0; j < R; ++j) acc[i][j] = p.e.scale * apply_act<true>(p.e.act, acc[i][j] + bias[j]);
 
     if (RED == FORGE_RED_NONE) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < R; ++i) {
             const int row = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
             if (row >= M) continue;
             float *dst = p.out + (size_t)row * N;
             if (p.out_vec4) {
-                if (cok[0]) *reinterpret_cast<float4 *>(dst + col[0]) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-                if (cok[4]) *reinterpret_cast<float4 *>(dst + col[4]) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+#pragma unroll
+                for (int q = 0; q < T; ++q)
+                    if (cok[4 * q]) *reinterpret_cast<float4 *>(dst + col[4 * q]) = make_float4(acc[i][4 * q], acc[i][4 * q + 1], acc[i][4 * q + 2], acc[i][4 * q + 3]);
             } else {
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
+                for (int j = 0; j < R; ++j)
                     if (cok[j]) dst[col[j]] = acc[i][j];
             }
         }
@@ -195,15 +221,15 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
     if (RED == FORGE_RED_SUM || RED == FORGE_RED_MAX || RED == FORGE_RED_MEAN_GELU_RESIDUAL) {
         constexpr bool ADD = RED != FORGE_RED_MAX;                       // row sum (also of the mean chain) or row max
         constexpr bool CHAIN = RED == FORGE_RED_MEAN_GELU_RESIDUAL;      // subtract, row mean, GELU, residual add
-        float sub[8];
+        float sub[R];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) sub[j] = (CHAIN && p.gamma && cok[j]) ? __ldg(p.gamma + col[j]) : 0.f;
+        for (int j = 0; j < R; ++j) sub[j] = (CHAIN && p.gamma && cok[j]) ? __ldg(p.gamma + col[j]) : 0.f;
         // thread -> 16 lanes that share the row (shuffles) -> tile partial
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < R; ++i) {
             float v = ADD ? 0.f : -INFINITY;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j = 0; j < R; ++j)
                 if (cok[j]) v = ADD ? v + (acc[i][j] - sub[j]) : fmaxf(v, acc[i][j]);
 #pragma unroll
             for (int s = 8; s >= 1; s >>= 1) {
@@ -226,7 +252,7 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
             __syncthreads();
             if (!s_last) return;
             __threadfence();
-            if (tid < K1_BM && m0 + tid < M) {
+            if (tid < BM && m0 + tid < M) {
                 const int row = m0 + tid;
                 float v = __ldcg(&p.partial[row]);
                 for (int t = 1; t < p.tiles_n; ++t) {
@@ -241,7 +267,7 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         if (CHAIN) {
             // residual add: Y[row, :] = X[row, :] + gelu(mean) for the strip's rows, by the whole CTA
             __syncthreads();
-            const int rows = min(K1_BM, M - m0);
+            const int rows = min(BM, M - m0);
             if (p.res_vec4) {
                 const int k4 = K >> 2;
                 for (int e = tid; e < rows * k4; e += K1_THREADS) {
@@ -266,19 +292,19 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         const int *target = reinterpret_cast<const int *>(p.gamma);          // class index per row (CE)
         float4 *part4 = reinterpret_cast<float4 *>(p.partial);               // (max, sum exp, target logit, -)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < R; ++i) {
             const int row = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
             float mx = -INFINITY, se = 0.f, tl = 0.f;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j = 0; j < R; ++j)
                 if (cok[j]) mx = fmaxf(mx, acc[i][j]);
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j = 0; j < R; ++j)
                 if (cok[j]) se += expf(acc[i][j] - mx);
             if (CE && row < M) {
                 const int t = __ldg(target + row);
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
+                for (int j = 0; j < R; ++j)
                     if (cok[j] && col[j] == t) tl = acc[i][j];
             }
             // the 16 lanes that share the row: shuffles, no block-wide barrier
@@ -301,7 +327,7 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         __syncthreads();
         if (!s_last) return;
         __threadfence();
-        if (tid < K1_BM && m0 + tid < M) {
+        if (tid < BM && m0 + tid < M) {
             const int row = m0 + tid;
             float4 f = __ldcg(&part4[row]);
             float mx = f.x, se = f.y, tl = f.z;
@@ -320,24 +346,24 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         cg::cluster_group cluster = cg::this_cluster();
         // per-thread statistics of its <= 8 columns of each row, two sweeps over registers
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < R; ++i) {
             RowStat s;
             float sum = 0.f;
             s.n = 0.f;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j = 0; j < R; ++j)
                 if (cok[j]) { sum += acc[i][j]; s.n += 1.f; }
             s.mean = s.n > 0.f ? sum / s.n : 0.f;
             s.m2 = 0.f;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j = 0; j < R; ++j)
                 if (cok[j]) { const float d = acc[i][j] - s.mean; s.m2 = fmaf(d, d, s.m2); }
 #pragma unroll
             for (int sft = 1; sft <= 8; sft <<= 1) s = merge_stat(s, shfl_xor_stat(s, sft));
             if (tx == 0) s_stat[ty * 4 + (i & 3) + (i >> 2) * 64] = s;
         }
         cluster.sync();
-        if (tid < K1_BM) {
+        if (tid < BM) {
             const unsigned nranks = cluster.num_blocks();
             RowStat s = *cluster.map_shared_rank(&s_stat[tid], 0);
             for (unsigned r = 1; r < nranks; ++r) s = merge_stat(s, *cluster.map_shared_rank(&s_stat[tid], r));
@@ -345,28 +371,29 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
             s_rstd[tid] = rsqrtf(s.m2 / s.n + p.e.eps);
         }
         cluster.sync();      // also keeps every CTA's s_stat alive until all have read it
-        float g[8], be[8];
+        float g[R], be[R];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < R; ++j) {
             g[j] = cok[j] ? __ldg(p.gamma + col[j]) : 0.f;
             be[j] = cok[j] ? __ldg(p.beta + col[j]) : 0.f;
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < R; ++i) {
             const int rl = ty * 4 + (i & 3) + (i >> 2) * 64;
             const int row = m0 + rl;
             if (row >= M) continue;
             const float mu = s_mean[rl], rs = s_rstd[rl];
             float *dst = p.out + (size_t)row * N;
-            float y[8];
+            float y[R];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) y[j] = (acc[i][j] - mu) * rs * g[j] + be[j];
+            for (int j = 0; j < R; ++j) y[j] = (acc[i][j] - mu) * rs * g[j] + be[j];
             if (p.out_vec4) {
-                if (cok[0]) *reinterpret_cast<float4 *>(dst + col[0]) = make_float4(y[0], y[1], y[2], y[3]);
-                if (cok[4]) *reinterpret_cast<float4 *>(dst + col[4]) = make_float4(y[4], y[5], y[6], y[7]);
+#pragma unroll
+                for (int q = 0; q < T; ++q)
+                    if (cok[4 * q]) *reinterpret_cast<float4 *>(dst + col[4 * q]) = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
             } else {
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
+                for (int j = 0; j < R; ++j)
                     if (cok[j]) dst[col[j]] = y[j];
             }
         }
@@ -376,15 +403,19 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
 // ---- host side ---------------------------------------------------------------------------
 forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
-    (void)sm_count;
-    const int64_t tiles_m = (d.M + K1_BM - 1) / K1_BM, tiles_n = (d.N + K1_BN - 1) / K1_BN;
+    // 64x64 tiles when 128x128 tiles would leave most SMs idle (LayerNorm keeps the large tile:
+    // its cluster spans a row)
+    const bool small = d.red != FORGE_RED_LAYERNORM &&
+                       ((d.M + K1_BM - 1) / K1_BM) * ((d.N + K1_BN - 1) / K1_BN) * 2 <= sm_count;
+    const int bm = small ? K1_BM / 2 : K1_BM, bn = small ? K1_BN / 2 : K1_BN;
+    const int64_t tiles_m = (d.M + bm - 1) / bm, tiles_n = (d.N + bn - 1) / bn;
     if (tiles_m > 65535 || tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
     if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
     if (d.red == FORGE_RED_LAYERNORM && tiles_n > K1_LN_MAX_CLUSTER) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_F32_FFMA;
-    info->tile_m = K1_BM;
-    info->tile_n = K1_BN;
-    info->tile_k = K1_BK;
+    info->tile_m = bm;
+    info->tile_n = bn;
+    info->tile_k = small ? 32 : K1_BK;
     info->stages = 2;
     info->cluster = d.red == FORGE_RED_LAYERNORM ? (int)tiles_n : 1;
     info->threads = K1_THREADS;
@@ -399,7 +430,7 @@ forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
 
 forge_status_t k1_setup(Handle &) { return FORGE_OK; }
 
-template <bool VEC, int RED>
+template <bool VEC, int RED, int T = 2>
 static forge_status_t k1_launch_t(const K1Params &p, dim3 grid, int cluster, cudaStream_t stream)
 {
     cudaLaunchConfig_t cfg = {};
@@ -416,7 +447,7 @@ static forge_status_t k1_launch_t(const K1Params &p, dim3 grid, int cluster, cud
         cfg.attrs = attr;
         cfg.numAttrs = 1;
     }
-    return cudaLaunchKernelEx(&cfg, k1_f32_ffma_kernel<VEC, RED>, p) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, k1_f32_ffma_kernel<VEC, RED, T>, p) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
 }
 
 forge_status_t k1_launch(Handle &h, const RunArgs &a)
@@ -435,15 +466,19 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
     p.e = Epilogue{(int)d.act, (int)d.red, d.scale, d.ln_eps, d.has_bias};
     p.partial = h.ws.partial;
     p.counters = h.ws.counters;
-    p.tiles_n = (int)((d.N + K1_BN - 1) / K1_BN);
+    const int bm = h.info.tile_m, bn = h.info.tile_n;          // 128 or 64
+    p.warm_l2 = (h.info.grid < h.sm_count) && (d.K <= 4096);   // latency-bound grids with modest panels
+    p.tiles_n = (int)((d.N + bn - 1) / bn);
     p.out_vec4 = (d.N % 4 == 0) && ((uintptr_t)a.out % 16 == 0);
     p.res_vec4 = (d.K % 4 == 0) && ((uintptr_t)a.out % 16 == 0) && ((uintptr_t)a.X % 16 == 0);
-    const dim3 grid((unsigned)p.tiles_n, (unsigned)((d.M + K1_BM - 1) / K1_BM));
+    const dim3 grid((unsigned)p.tiles_n, (unsigned)((d.M + bm - 1) / bm));
     const bool vec = (d.K % 4 == 0) && ((uintptr_t)a.X % 16 == 0) && ((uintptr_t)a.W % 16 == 0);
-#define K1_CASE(R)                                                                      \
-    case R:                                                                             \
-        return vec ? k1_launch_t<true, R>(p, grid, h.info.cluster, a.stream)            \
-                   : k1_launch_t<false, R>(p, grid, h.info.cluster, a.stream);
+#define K1_CASE(R)                                                                                   \
+    case R:                                                                                          \
+        if (bm == K1_BM)                                                                             \
+            return vec ? k1_launch_t<true, R, 2>(p, grid, h.info.cluster, a.stream)                  \
+                       : k1_launch_t<false, R, 2>(p, grid, h.info.cluster, a.stream);                \
+        return vec ? k1_launch_t<true, R, 1>(p, grid, 1, a.stream) : k1_launch_t<false, R, 1>(p, grid, 1, a.stream);
     switch (d.red) {
         K1_CASE(FORGE_RED_NONE)
         K1_CASE(FORGE_RED_SUM)
@@ -532,6 +567,7 @@ extern "C" forge_status_t forge_fused_linear_f32_reduce_static(int64_t M, int64_
     p.tiles_n = (int)tiles_n;
     p.out_vec4 = 0;
     p.res_vec4 = 0;
+    p.warm_l2 = 0;
     const dim3 grid((unsigned)tiles_n, (unsigned)tiles_m);
     const bool vec = (K % 4 == 0) && ((uintptr_t)X % 16 == 0) && ((uintptr_t)W % 16 == 0);
     if (red == FORGE_RED_SUM)
