@@ -46,6 +46,8 @@ struct K3Smem {
     uint64_t empty[K3_STAGES];
     float4 red[K3_KSPLIT][K3_PAD_GROUPS][32];    // partial accumulators of the K-slices
     float rowred[K3_PAD_GROUPS][16];
+    float rowred_s[K3_PAD_GROUPS][16];           // softmax statistics: sum of exponentials ...
+    float rowred_t[K3_PAD_GROUPS][16];           // ... and the target's logit
     int last_flag;
     int abort_flag;
 };
@@ -56,7 +58,8 @@ struct K3Params {
     void *out;
     int M, N, K;
     Epilogue e;
-    float *partial;       // [grid][16]
+    const int *target;    // cross-entropy: class index per row
+    float *partial;       // [grid][16] floats, or [grid][16] float4 (softmax statistics)
     unsigned *counters;   // [1]
     int *status;
     int num_kb;
@@ -139,8 +142,12 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         const int ks = warp / K3_NSPLIT;    // which K-slice (ring stages with index % K3_KSPLIT == ks)
         const int t = threadIdx.x;          // 0..255
         const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX;
+        const bool softmax = p.e.red == FORGE_RED_LOGSUMEXP || p.e.red == FORGE_RED_CROSS_ENTROPY;
         bool ok = true;
-        float running = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY;     // threads 0..15: row t
+        float running = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY;     // threads 0..15: row t (for softmax: the max)
+        float running_s = 0.f, running_t = 0.f;                          // softmax: sum of exponentials, target logit
+        const int tgt0 = (p.e.red == FORGE_RED_CROSS_ENTROPY && (lane >> 2) < p.M) ? __ldg(p.target + (lane >> 2)) : -1;
+        const int tgt1 = (p.e.red == FORGE_RED_CROSS_ENTROPY && (lane >> 2) + 8 < p.M) ? __ldg(p.target + (lane >> 2) + 8) : -1;
 
         // ldmatrix lane addressing on the 128-byte-swizzled tiles (16-byte chunk c of row r
         // sits at r*128 + ((c ^ (r & 7)) << 4)).
@@ -237,6 +244,28 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                         s.rowred[g][r0] = m0;
                         s.rowred[g][r1] = m1;
                     }
+                } else if (softmax) {
+                    // (max, sum exp) of this thread's two columns of rows r0 and r1, merged over the
+                    // four lanes that share the rows; the target's logit rides along
+                    float m0 = live ? fmaxf(v[0], v[1]) : -INFINITY, m1 = live ? fmaxf(v[2], v[3]) : -INFINITY;
+                    float s0 = live ? __expf(v[0] - m0) + __expf(v[1] - m0) : 0.f;
+                    float s1 = live ? __expf(v[2] - m1) + __expf(v[3] - m1) : 0.f;
+                    float t0 = 0.f, t1 = 0.f;
+                    if (live) {
+                        t0 = col == tgt0 ? v[0] : (col + 1 == tgt0 ? v[1] : 0.f);
+                        t1 = col == tgt1 ? v[2] : (col + 1 == tgt1 ? v[3] : 0.f);
+                    }
+#pragma unroll
+                    for (int sh = 1; sh <= 2; sh <<= 1) {
+                        lse_merge<false>(m0, s0, __shfl_xor_sync(0xffffffffu, m0, sh), __shfl_xor_sync(0xffffffffu, s0, sh));
+                        lse_merge<false>(m1, s1, __shfl_xor_sync(0xffffffffu, m1, sh), __shfl_xor_sync(0xffffffffu, s1, sh));
+                        t0 += __shfl_xor_sync(0xffffffffu, t0, sh);
+                        t1 += __shfl_xor_sync(0xffffffffu, t1, sh);
+                    }
+                    if ((lane & 3) == 0) {
+                        s.rowred[g][r0] = m0; s.rowred_s[g][r0] = s0; s.rowred_t[g][r0] = t0;
+                        s.rowred[g][r1] = m1; s.rowred_s[g][r1] = s1; s.rowred_t[g][r1] = t1;
+                    }
                 } else if (live) {
                     __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(p.out);
                     if (r0 < p.M) *reinterpret_cast<uint32_t *>(Y + (size_t)r0 * p.N + col) = ptx::pack_bf16x2(v[0], v[1]);
@@ -250,8 +279,50 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                     running = p.e.red == FORGE_RED_SUM ? running + o : fmaxf(running, o);
                 }
             }
+            if (softmax && t < 16) {
+                for (int g = 0; g < K3_PAD_GROUPS; ++g) {
+                    lse_merge<false>(running, running_s, s.rowred[g][t], s.rowred_s[g][t]);
+                    running_t += s.rowred_t[g][t];
+                }
+            }
         }
         if (!ok) s.abort_flag = 1;
+
+        // ---- softmax statistics across CTAs: same last-arriver fold, on (max, sum exp, target) ----
+        if (softmax) {
+            float *out = reinterpret_cast<float *>(p.out);
+            float4 *part4 = reinterpret_cast<float4 *>(p.partial);
+            if (gridDim.x == 1) {
+                if (t < p.M) out[t] = running + __logf(running_s) - running_t;
+            } else {
+                if (t < 16) part4[(size_t)blockIdx.x * 16 + t] = make_float4(running, running_s, running_t, 0.f);
+                __threadfence();
+                k3_consumer_sync();
+                if (t == 0) s.last_flag = (atomicAdd(&p.counters[0], 1u) == gridDim.x - 1);
+                k3_consumer_sync();
+                if (s.last_flag) {
+                    __threadfence();
+                    const int row = t & 15, chunk = t >> 4;
+                    float mx = -INFINITY, se = 0.f, tl = 0.f;
+                    for (unsigned c = chunk; c < gridDim.x; c += 16) {
+                        const float4 f = __ldcg(&part4[(size_t)c * 16 + row]);
+                        lse_merge<false>(mx, se, f.x, f.y);
+                        tl += f.z;
+                    }
+                    s.rowred[chunk][row] = mx; s.rowred_s[chunk][row] = se; s.rowred_t[chunk][row] = tl;
+                    k3_consumer_sync();
+                    if (t < p.M) {
+                        mx = s.rowred[0][t]; se = s.rowred_s[0][t]; tl = s.rowred_t[0][t];
+                        for (int j = 1; j < 16; ++j) {
+                            lse_merge<false>(mx, se, s.rowred[j][t], s.rowred_s[j][t]);
+                            tl += s.rowred_t[j][t];
+                        }
+                        out[t] = mx + __logf(se) - tl;
+                    }
+                    if (t == 0) p.counters[0] = 0u;
+                }
+            }
+        }
 
         // ---- fold the CTAs' partials: the last CTA to arrive does it, in CTA order ----
         if (reduce) {
@@ -312,6 +383,7 @@ static int k3_box_groups(const forge_fused_linear_desc_t &d, int grid)
 forge_status_t k3_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
     if (d.M > 16 || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    if (d.red == FORGE_RED_LAYERNORM || d.red == FORGE_RED_MEAN_GELU_RESIDUAL) return FORGE_ERR_UNSUPPORTED;
     const int grid = k3_grid(d, sm_count);
     info->kernel = FORGE_KERNEL_BF16_SKINNY;
     info->tile_m = 16;
@@ -322,8 +394,9 @@ forge_status_t k3_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     info->threads = K3_THREADS;
     info->grid = grid;
     info->smem_bytes = (int64_t)K3_SMEM_BYTES;
-    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX) && grid > 1;
-    wl->partial_floats = partials ? (size_t)grid * 16 : 0;
+    const bool softmax = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;     // float4 partials
+    const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || softmax) && grid > 1;
+    wl->partial_floats = partials ? (size_t)grid * 16 * (softmax ? 4 : 1) : 0;
     wl->counters = partials ? 1 : 0;
     return FORGE_OK;
 }
@@ -348,6 +421,7 @@ forge_status_t k3_launch(Handle &h, const RunArgs &a)
     }
     K3Params p;
     p.b = (const __nv_bfloat16 *)a.b;
+    p.target = (const int *)a.gamma;
     p.out = a.out;
     p.M = (int)d.M;
     p.N = (int)d.N;

@@ -12,7 +12,8 @@ pytestmark = pytest.mark.gpu
 
 REDS = [wk.RED_LOGSUMEXP, wk.RED_CROSS_ENTROPY]
 F32_SHAPES = [(1, 1, 1), (5, 100, 7), (128, 128, 16), (130, 300, 36), (257, 1000, 64), (64, 2500, 19)]
-BF16_SHAPES = [(17, 8, 8), (128, 256, 64), (16, 1024, 128), (300, 520, 200), (1000, 776, 328), (260, 4104, 64)]
+BF16_SHAPES = [(17, 8, 8), (128, 256, 64), (16, 1024, 128), (300, 520, 200), (1000, 776, 328), (260, 4104, 64),
+               (1, 64, 16), (7, 20000, 264), (16, 148 * 8 * 17, 128), (3, 1184 * 13, 2048)]      # M <= 16: skinny kernel
 
 
 @pytest.mark.parametrize("M,N,K", F32_SHAPES)
@@ -31,7 +32,7 @@ def test_bf16(M, N, K, red):
     wl = wk.custom_workload(f"lse_bf16_{M}x{N}x{K}", wk.BF16, M, N, K, wk.ACT_IDENTITY, red, scale=2.0, seed=M + N)
     inp = wk.make_inputs(wl)
     g, plan = pu.run_gpu(wl, inp)
-    assert plan["kernel"] == B.FORGE_KERNEL_BF16_TCGEN05          # also for M <= 16
+    assert plan["kernel"] == (B.FORGE_KERNEL_BF16_SKINNY if M <= 16 else B.FORGE_KERNEL_BF16_TCGEN05)
     pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
 
 
@@ -56,6 +57,17 @@ def test_cross_entropy_needs_its_targets():
     o = torch.zeros(64, dtype=torch.float32, device="cuda")
     assert B.forge_fused_linear_run(op.h, t, t, t, None, None, o) == B.FORGE_ERR_INVALID_ARG
     op.close()
+
+
+def test_decode_step_of_a_language_model_head_full_oracle():
+    wl = wk.custom_workload("lse_decode", wk.BF16, 16, 32768, 4096, wk.ACT_IDENTITY, wk.RED_CROSS_ENTROPY, w_std=0.02, seed=12)
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, plan = pu.run_gpu(wl, inp, op=op)
+    b, _ = pu.run_gpu(wl, inp, op=op, repeats=3)
+    op.close()
+    assert plan["kernel"] == B.FORGE_KERNEL_BF16_SKINNY and np.array_equal(a, b)
+    pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
 
 
 def test_n2_sampled_rows_full_size():
