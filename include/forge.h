@@ -67,7 +67,7 @@ typedef enum {
      * residual add of the layer's input, all in one kernel):
      *     g[m] = gelu_erf(mean_n (E[m,n] - sub[n])),   Y[m,k] = X[m,k] + g[m]
      * The output is Y [M,K] (the shape of X) in dtype.  run() takes the subtract vector sub[N]
-     * in its `gamma` argument (NULL: nothing is subtracted); `beta` is ignored.  fp32 only.   */
+     * in its `gamma` argument (NULL: nothing is subtracted); `beta` is ignored.                */
     FORGE_RED_LOGSUMEXP = 5,
     /* out[m] = log sum_n exp(E[m,n]), fp32 [M]: the row statistic of a softmax over N, merged
      * across output tiles as (max, sum of exponentials) pairs; Y is never written (Section 4 of
@@ -119,7 +119,7 @@ typedef struct {
  * BF16_SKINNY; bf16 LayerNorm -> BF16_TCGEN05_LN; other bf16 -> BF16_TCGEN05.
  * Unsupported: bf16 with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); fp32 LayerNorm with
  * N > 1024 (one 8-CTA cluster); bf16 LayerNorm with more 256-column tiles per row than
- * clusters in the grid; the mean-gelu-residual chain in bf16.
+ * clusters in the grid.
  */
 forge_status_t forge_fused_linear_query_plan(const forge_fused_linear_desc_t *desc, int sm_count,
                                              forge_plan_info_t *info);

@@ -30,9 +30,8 @@ forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_
         st = k1_plan(d, sm_count, info, wl);
     } else {
         if (d.K % 8 != 0 || d.N % 8 != 0) return FORGE_ERR_UNSUPPORTED;     // 16-byte row pitch for TMA
-        if (d.red == FORGE_RED_MEAN_GELU_RESIDUAL) return FORGE_ERR_UNSUPPORTED;   // fp32 only so far
         if (d.red == FORGE_RED_LAYERNORM) st = k4_plan(d, sm_count, info, wl);
-        else if (d.M <= 16) st = k3_plan(d, sm_count, info, wl);
+        else if (d.M <= 16 && d.red != FORGE_RED_MEAN_GELU_RESIDUAL) st = k3_plan(d, sm_count, info, wl);
         else st = k2_plan(d, sm_count, info, wl);
     }
     if (st != FORGE_OK) return st;

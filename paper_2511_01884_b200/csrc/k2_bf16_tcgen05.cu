@@ -55,6 +55,7 @@ struct K2Smem {
     uint32_t tmem_base;
     int last_flag[2];
     int abort_flag;
+    float rowg[2][K2_BM];       // mean chain: gelu(mean) of the strip's rows, per epilogue group
     float bias[2][K2_BN];
     float gamma[2][K2_BN];
     float beta[2][K2_BN];
@@ -64,6 +65,7 @@ static_assert(K2Ring<false>::BYTES == K2Ring<true>::BYTES, "both ring layouts us
 
 struct K2Params {
     const __nv_bfloat16 *b;
+    const __nv_bfloat16 *X;     // mean chain only: the residual input
     void *out;
     int M, N, K;
     Epilogue e;
@@ -221,7 +223,9 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         const int parts = 2 * p.tiles_n;
         int acc = 0;
         uint32_t acc_phase = 0;
-        const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX;
+        const bool chain = p.e.red == FORGE_RED_MEAN_GELU_RESIDUAL;       // subtract, row mean, GELU, residual add
+        const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX || chain;
+        const bool add = p.e.red != FORGE_RED_MAX;
         const uint32_t acc_empty_addr[2] = {ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[0]), 0),
                                             ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[1]), 0)};   // the leader's (PAIR)
         for (int t = first_unit; t < total_tiles; t += unit_stride) {
@@ -238,6 +242,8 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 if (LN) {
                     sg[et] = in ? __bfloat162float(p.gamma[n0 + et]) : 0.f;
                     sbe[et] = in ? __bfloat162float(p.beta[n0 + et]) : 0.f;
+                } else if (chain) {          // the vector subtracted before the row mean
+                    sg[et] = (in && p.gamma) ? __bfloat162float(p.gamma[n0 + et]) : 0.f;
                 }
             }
             // the give-up decision must be taken by all threads of the group together
@@ -441,7 +447,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 continue;
             }
 
-            float red = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY;
+            float red = add ? 0.f : -INFINITY;
 #pragma unroll 1
             for (int c = 0; c < CHUNKS; ++c) {
                 const int col0 = n0 + c * 32;
@@ -454,9 +460,13 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
                 apply_act_array<false>(p.e.act, v, p.e.scale);
                 if (reduce) {
+                    if (chain) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] -= sg[c * 32 + j];
+                    }
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (col0 + j < p.N) red = p.e.red == FORGE_RED_SUM ? red + v[j] : fmaxf(red, v[j]);
+                        if (col0 + j < p.N) red = add ? red + v[j] : fmaxf(red, v[j]);
                 } else if (row < p.M) {
                     __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)row * p.N + col0;
 #pragma unroll
@@ -491,11 +501,31 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                         float v = __ldcg(&p.partial[row]);
                         for (int i = 1; i < parts; ++i) {
                             const float o = __ldcg(&p.partial[(size_t)i * p.M + row]);
-                            v = p.e.red == FORGE_RED_SUM ? v + o : fmaxf(v, o);
+                            v = add ? v + o : fmaxf(v, o);
                         }
-                        out[row] = v;
+                        if (chain) s.rowg[h][q * 32 + lane] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)p.N);
+                        else out[row] = v;
                     }
                     if (et == 0) p.counters[tm] = 0u;
+                    if (chain) {
+                        // residual add for the strip's rows, by the whole group, 16 bytes per access:
+                        // Y[row, :] = X[row, :] + gelu(mean)   (Y is [M,K])
+                        epi_bar_sync(h);
+                        const int rows = min(K2_BM, p.M - m0), k8 = p.K >> 3;
+                        const uint4 *Xs = reinterpret_cast<const uint4 *>(p.X + (size_t)m0 * p.K);
+                        uint4 *Ys = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)m0 * p.K);
+                        for (int e = et; e < rows * k8; e += K2_EPI_THREADS) {
+                            const float g = s.rowg[h][e / k8];
+                            uint4 x = __ldg(Xs + e);
+                            uint32_t *w = reinterpret_cast<uint32_t *>(&x);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float lo = __uint_as_float(w[i] << 16) + g, hi = __uint_as_float(w[i] & 0xffff0000u) + g;
+                                w[i] = ptx::pack_bf16x2(lo, hi);
+                            }
+                            Ys[e] = x;
+                        }
+                    }
                 }
             }
             if ((acc ^= 1) == 0) acc_phase ^= 1;
@@ -548,7 +578,7 @@ forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     }
     info->smem_bytes = (int64_t)K2_SMEM_BYTES;
     const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;      // float4 partials
-    const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || lse;         // one per row and half tile
+    const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL || lse;   // one per row and half tile
     wl->partial_floats = partials ? (lse ? 4 : 1) * 2 * (size_t)tiles_n * (size_t)d.M : 0;
     wl->counters = partials ? (size_t)tiles_m : 0;
     return FORGE_OK;
@@ -639,6 +669,7 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     }
     K2Params p;
     p.b = (const __nv_bfloat16 *)a.b;
+    p.X = (const __nv_bfloat16 *)a.X;
     p.gamma = (const __nv_bfloat16 *)a.gamma;
     p.beta = (const __nv_bfloat16 *)a.beta;
     p.out = a.out;

@@ -1,5 +1,5 @@
 """GPU parity of the case-study chain (Linear, subtract, row mean, GELU, residual add) on the
-fp32 path against the CPU oracle."""
+fp32 and bf16 paths against the CPU oracle."""
 import numpy as np
 import pytest
 
@@ -25,6 +25,32 @@ def test_shapes(M, N, K):
     pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
 
 
+BF16_SHAPES = [(17, 8, 8), (128, 256, 64), (130, 264, 72), (300, 1000, 200), (1000, 1536, 128), (16, 512, 64)]
+
+
+@pytest.mark.parametrize("M,N,K", BF16_SHAPES)
+def test_bf16_shapes(M, N, K):
+    wl = wk.custom_workload(f"chain_bf16_{M}x{N}x{K}", wk.BF16, M, N, K, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL,
+                            seed=M + N, w_std=0.1)
+    inp = wk.make_inputs(wl)
+    inp["b"] = wk.round_to_storage(inp["b"] + 0.7, wk.BF16)
+    g, plan = pu.run_gpu(wl, inp)
+    assert g.shape == (M, K) and plan["kernel"] == B.FORGE_KERNEL_BF16_TCGEN05          # also for M <= 16
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_bf16_repeats_and_no_subtract_vector():
+    wl = wk.custom_workload("chain_bf16_rep", wk.BF16, 700, 1304, 256, wk.ACT_SILU, wk.RED_MEAN_GELU_RESIDUAL, seed=4, w_std=0.1)
+    inp = wk.make_inputs(wl)
+    inp["sub"] = None
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op)
+    b, _ = pu.run_gpu(wl, inp, op=op, repeats=3)
+    op.close()
+    assert np.array_equal(a, b)
+    pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
+
+
 def test_with_activation_scale_and_no_subtract_vector():
     wl = wk.custom_workload("chain_act", wk.F32, 200, 260, 48, wk.ACT_RELU, wk.RED_MEAN_GELU_RESIDUAL, scale=3.0, seed=9)
     inp = wk.make_inputs(wl)
@@ -42,7 +68,7 @@ def test_zero_mean_returns_the_input_bits():
     assert np.array_equal(g, inp["X"].astype(np.float64))
 
 
-def test_two_runs_on_one_handle_and_bf16_is_refused():
+def test_two_runs_on_one_handle():
     wl = wk.custom_workload("chain_rep", wk.F32, 300, 700, 64, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL, seed=4)
     inp = wk.make_inputs(wl)
     op = B.FusedLinear(pu.desc_of(wl))
@@ -51,8 +77,6 @@ def test_two_runs_on_one_handle_and_bf16_is_refused():
     op.close()
     assert np.array_equal(a, b)
     pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
-    st, _ = B.forge_fused_linear_query_plan(B.make_desc(64, 64, 64, wk.BF16, 0, wk.RED_MEAN_GELU_RESIDUAL))
-    assert st == B.FORGE_ERR_UNSUPPORTED
 
 
 def test_n1_sampled_rows_full_size():
