@@ -172,6 +172,16 @@ forge_status_t forge_fused_linear_last_status(forge_fused_linear_t h);
  */
 forge_status_t forge_fused_linear_last_wait_detail(forge_fused_linear_t h, int detail[4]);
 
+/*
+ * Self-test of the bounded device-side wait that every kernel here uses (the paper's loop feeds
+ * runtime failures back to its Judge, Section 2.2; a kernel that waits for ever gives no feedback
+ * at all): runs a one-CTA kernel that waits on a barrier nothing signals, with a budget of
+ * `budget_ms` (1..1000).  The expected return value is FORGE_ERR_TIMEOUT with detail[0] = 1 (the
+ * operand-arrival wait), detail[1] = 0x5a5a, detail[2] = 0 (CTA), detail[3] = 32 (thread); the
+ * kernel ends by itself and the device stays usable.  Synchronous; allocates and frees 256 bytes.
+ */
+forge_status_t forge_selftest_bounded_wait(int device, int budget_ms, int detail[4]);
+
 /* Copy the plan chosen at create() into *info (host pointer). */
 forge_status_t forge_fused_linear_get_plan(forge_fused_linear_t h, forge_plan_info_t *info);
 

@@ -23,7 +23,7 @@ EXPORTS = [
     "forge_fused_linear_query_plan", "forge_fused_linear_create", "forge_fused_linear_run",
     "forge_fused_linear_run_host", "forge_fused_linear_last_status", "forge_fused_linear_get_plan",
     "forge_fused_linear_launches_per_run", "forge_fused_linear_destroy", "forge_fused_linear_last_wait_detail",
-    "forge_fused_linear_f32_reduce_static", "forge_status_string", "forge_kernel_name",
+    "forge_fused_linear_f32_reduce_static", "forge_selftest_bounded_wait", "forge_status_string", "forge_kernel_name",
 ]
 
 
@@ -77,7 +77,8 @@ def lib() -> ctypes.CDLL:
         L.forge_kernel_name.restype = ctypes.c_char_p
         L.forge_fused_linear_f32_reduce_static.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, i, i,
                                                            ctypes.c_float, vp, vp, vp, vp, vp]
-        for n in EXPORTS[:10]:
+        L.forge_selftest_bounded_wait.argtypes = [i, i, ctypes.POINTER(ctypes.c_int * 4)]
+        for n in EXPORTS[:11]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -140,6 +141,13 @@ def forge_fused_linear_last_wait_detail(h):
     if st != FORGE_OK:
         raise ForgeError(st, "last_wait_detail")
     return list(d)
+
+
+def forge_selftest_bounded_wait(device: int = 0, budget_ms: int = 50):
+    """(status, [site, detail, CTA, thread]) of the bounded-wait self-test (expects FORGE_ERR_TIMEOUT)."""
+    d = (ctypes.c_int * 4)()
+    st = lib().forge_selftest_bounded_wait(int(device), int(budget_ms), ctypes.byref(d))
+    return st, list(d)
 
 
 def forge_fused_linear_get_plan(h) -> PlanInfo:

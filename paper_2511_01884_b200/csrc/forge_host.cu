@@ -5,6 +5,7 @@
 
 #include "common.cuh"
 #include "plan.h"
+#include "sm100_ptx.cuh"
 
 namespace forge {
 
@@ -130,7 +131,45 @@ forge_status_t encode_tmap_bf16(CUtensorMap *tm, const void *ptr, uint64_t rows,
 
 using namespace forge;
 
+// One CTA, one barrier that nothing ever signals: the bounded wait must give up after
+// `budget_ns`, leave (FORGE_ERR_TIMEOUT, site, detail, CTA, thread) in the status area and
+// let the kernel end normally.
+__global__ void forge_wait_selftest_kernel(int *status, unsigned long long budget_ns, int detail)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 32) ptx::mbar_wait(&bar, 0, status, SITE_TMA_FULL, detail, budget_ns);
+}
+
 extern "C" {
+
+forge_status_t forge_selftest_bounded_wait(int device, int budget_ms, int detail[4])
+{
+    if (!detail || budget_ms <= 0 || budget_ms > 1000 || device < 0) return FORGE_ERR_INVALID_ARG;
+    DeviceGuard g(device);
+    if (!g.ok) return FORGE_ERR_CUDA;
+    int *status = nullptr;
+    if (cudaMalloc(&status, 256) != cudaSuccess) { cudaGetLastError(); return FORGE_ERR_ALLOC; }
+    forge_status_t st = FORGE_ERR_CUDA;
+    int word[4] = {0, 0, 0, 0};
+    if (cudaMemset(status, 0, 256) == cudaSuccess) {
+        forge_wait_selftest_kernel<<<1, 64>>>(status, (unsigned long long)budget_ms * 1000000ull, 0x5a5a);
+        if (cudaGetLastError() == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess &&
+            cudaMemcpy(word, status, sizeof(word), cudaMemcpyDeviceToHost) == cudaSuccess) {
+            st = (forge_status_t)(word[0] >> 16);
+            detail[0] = word[0] & 0xffff;
+            detail[1] = word[1];
+            detail[2] = word[2];
+            detail[3] = word[3];
+        }
+    }
+    cudaFree(status);
+    return st;
+}
 
 forge_status_t forge_fused_linear_query_plan(const forge_fused_linear_desc_t *desc, int sm_count, forge_plan_info_t *info)
 {

@@ -79,7 +79,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // wait returns false; callers then leave their loops and fall through to the teardown.
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;
 
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *status, int site, int detail = 0)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *status, int site, int detail = 0,
+                                          uint64_t budget_ns = kWaitBudgetNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;
@@ -89,7 +90,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *s
             if (*(volatile int *)status != 0) return false;
             const uint64_t t = globaltimer_ns();
             if (t0 == 0) t0 = t;
-            else if (t - t0 > kWaitBudgetNs) {
+            else if (t - t0 > budget_ns) {
                 report_timeout(status, site, detail);
                 return false;
             }

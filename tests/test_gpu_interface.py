@@ -110,3 +110,22 @@ def test_plans_report_the_kernel_families():
         st, p = B.forge_fused_linear_query_plan(pu.desc_of(wl))
         assert st == B.FORGE_OK and p.kernel == kernel and p.cluster == cluster
         assert p.grid <= 148 or kernel == B.FORGE_KERNEL_F32_FFMA          # the bf16 kernels are persistent
+
+
+def test_a_wait_that_nothing_satisfies_gives_up_and_reports():
+    """The give-up path of the bounded waits, exercised the safe way: a barrier nobody signals and a
+    50 ms budget.  The kernel must end by itself, report the time-out, and leave the GPU usable."""
+    import time
+    import torch
+    t = time.perf_counter()
+    st, detail = B.forge_selftest_bounded_wait(0, 50)
+    dt = time.perf_counter() - t
+    assert st == B.FORGE_ERR_TIMEOUT and detail == [1, 0x5A5A, 0, 32]
+    assert 0.04 < dt < 2.0
+    # the context is intact: an ordinary run right after it is correct
+    wl = wk.WORKLOADS["c1"]
+    inp = wk.make_inputs(wl)
+    g, _ = pu.run_gpu(wl, inp)
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+    assert B.forge_selftest_bounded_wait(0, 0)[0] == B.FORGE_ERR_INVALID_ARG
+    assert torch.cuda.is_available()
