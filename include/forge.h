@@ -47,7 +47,7 @@ typedef enum {
                                  /* forge_fused_linear_f32_reduce_static() holds          */
 } forge_status_t;
 
-typedef enum { FORGE_F32 = 0, FORGE_BF16 = 1 } forge_dtype_t;
+typedef enum { FORGE_F32 = 0, FORGE_BF16 = 1, FORGE_F16 = 2 } forge_dtype_t;   /* F16: IEEE half, same kernels as BF16 */
 
 typedef enum {
     FORGE_ACT_IDENTITY = 0,

@@ -15,7 +15,7 @@ constexpr size_t kStatusBytes = 256;     // status word lives alone in the first
 
 bool desc_enums_ok(const forge_fused_linear_desc_t &d)
 {
-    return (d.dtype == FORGE_F32 || d.dtype == FORGE_BF16) && d.act >= FORGE_ACT_IDENTITY &&
+    return (d.dtype == FORGE_F32 || d.dtype == FORGE_BF16 || d.dtype == FORGE_F16) && d.act >= FORGE_ACT_IDENTITY &&
            d.act <= FORGE_ACT_SILU && d.red >= FORGE_RED_NONE && d.red <= FORGE_RED_CROSS_ENTROPY;
 }
 
@@ -73,9 +73,9 @@ forge_status_t check_run_args(const Handle &h, const RunArgs &a)
     if (h.d.red == FORGE_RED_CROSS_ENTROPY && !a.gamma) return FORGE_ERR_INVALID_ARG;      // the targets
     const uintptr_t m = (uintptr_t)a.X | (uintptr_t)a.W | (uintptr_t)a.out | (uintptr_t)a.b |
                         (uintptr_t)a.gamma | (uintptr_t)a.beta;
-    // bf16 operands travel by TMA and 128-bit accesses: 16-byte alignment is required.
+    // 16-bit operands travel by TMA and 128-bit accesses: 16-byte alignment is required.
     // fp32 falls back to scalar accesses when unaligned, but still needs element alignment.
-    if (h.d.dtype == FORGE_BF16 ? (m % 16 != 0) : (m % 4 != 0)) return FORGE_ERR_INVALID_ARG;
+    if (h.d.dtype != FORGE_F32 ? (m % 16 != 0) : (m % 4 != 0)) return FORGE_ERR_INVALID_ARG;
     return FORGE_OK;
 }
 
@@ -96,8 +96,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-forge_status_t encode_tmap_bf16(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
-                                uint32_t box_rows, uint32_t box_cols)
+forge_status_t encode_tmap_16(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
+                              uint32_t box_rows, uint32_t box_cols, int f16)
 {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
@@ -122,7 +122,7 @@ forge_status_t encode_tmap_bf16(CUtensorMap *tm, const void *ptr, uint64_t rows,
                                       : promo == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
                                       : promo == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B
                                                      : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
-    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+    const CUresult r = fn(tm, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, l2, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? FORGE_OK : FORGE_ERR_CUDA;
 }

@@ -64,12 +64,13 @@ constexpr size_t K2_SMEM_BYTES = 1024 + (size_t)K2Ring<false>::BYTES + sizeof(K2
 static_assert(K2Ring<false>::BYTES == K2Ring<true>::BYTES, "both ring layouts use the same shared memory");
 
 struct K2Params {
-    const __nv_bfloat16 *b;
-    const __nv_bfloat16 *X;     // mean chain only: the residual input
+    int f16;                    // storage format of X, W, b, gamma, beta, Y: IEEE half (1) or bfloat16 (0)
+    const uint16_t *b;
+    const uint16_t *X;          // mean chain only: the residual input
     void *out;
     int M, N, K;
     Epilogue e;
-    const __nv_bfloat16 *gamma, *beta;
+    const uint16_t *gamma, *beta;
     float *partial;       // per half tile: sum/max [2*tiles_n][M] floats; layernorm [2*tiles_n][M] float4 triples
     unsigned *counters;   // [tiles_m]
     int *status;
@@ -184,7 +185,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if ((!PAIR || rank == 0) && ptx::elect_one()) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(PAIR ? 2 * K2_BM : K2_BM, K2_BN);
+            const uint32_t idesc = ptx::idesc_16_f32(PAIR ? 2 * K2_BM : K2_BM, K2_BN, p.f16);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             for (int t = first_unit; t < total_tiles && ok; t += unit_stride) {
@@ -238,12 +239,12 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             // bias (and gamma, beta) of this half tile -> shared memory as fp32, one value per thread
             {
                 const bool in = n0 + et < p.N;
-                sb[et] = (p.e.has_bias && in) ? __bfloat162float(p.b[n0 + et]) : 0.f;
+                sb[et] = (p.e.has_bias && in) ? ptx::load16(p.b, n0 + et, p.f16) : 0.f;
                 if (LN) {
-                    sg[et] = in ? __bfloat162float(p.gamma[n0 + et]) : 0.f;
-                    sbe[et] = in ? __bfloat162float(p.beta[n0 + et]) : 0.f;
+                    sg[et] = in ? ptx::load16(p.gamma, n0 + et, p.f16) : 0.f;
+                    sbe[et] = in ? ptx::load16(p.beta, n0 + et, p.f16) : 0.f;
                 } else if (chain) {          // the vector subtracted before the row mean
-                    sg[et] = (in && p.gamma) ? __bfloat162float(p.gamma[n0 + et]) : 0.f;
+                    sg[et] = (in && p.gamma) ? ptx::load16(p.gamma, n0 + et, p.f16) : 0.f;
                 }
             }
             // the give-up decision must be taken by all threads of the group together
@@ -370,10 +371,10 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                                     y[j] = fmaf(fmaf(__uint_as_float(r[i * 8 + j]), rstd, shift), sg[cc], sbe[cc]);
                                 }
                                 uint4 w;
-                                w.x = ptx::pack_bf16x2(y[0], y[1]);
-                                w.y = ptx::pack_bf16x2(y[2], y[3]);
-                                w.z = ptx::pack_bf16x2(y[4], y[5]);
-                                w.w = ptx::pack_bf16x2(y[6], y[7]);
+                                w.x = ptx::pack16x2(y[0], y[1], p.f16);
+                                w.y = ptx::pack16x2(y[2], y[3], p.f16);
+                                w.z = ptx::pack16x2(y[4], y[5], p.f16);
+                                w.w = ptx::pack16x2(y[6], y[7], p.f16);
                                 *reinterpret_cast<uint4 *>(dst + i * 8) = w;
                             }
                         }
@@ -473,10 +474,10 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                     for (int i = 0; i < 4; ++i) {
                         if (col0 + i * 8 < p.N) {
                             uint4 w;
-                            w.x = ptx::pack_bf16x2(v[i * 8 + 0], v[i * 8 + 1]);
-                            w.y = ptx::pack_bf16x2(v[i * 8 + 2], v[i * 8 + 3]);
-                            w.z = ptx::pack_bf16x2(v[i * 8 + 4], v[i * 8 + 5]);
-                            w.w = ptx::pack_bf16x2(v[i * 8 + 6], v[i * 8 + 7]);
+                            w.x = ptx::pack16x2(v[i * 8 + 0], v[i * 8 + 1], p.f16);
+                            w.y = ptx::pack16x2(v[i * 8 + 2], v[i * 8 + 3], p.f16);
+                            w.z = ptx::pack16x2(v[i * 8 + 4], v[i * 8 + 5], p.f16);
+                            w.w = ptx::pack16x2(v[i * 8 + 6], v[i * 8 + 7], p.f16);
                             *reinterpret_cast<uint4 *>(dst + i * 8) = w;
                         }
                     }
@@ -512,7 +513,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                         // Y[row, :] = X[row, :] + gelu(mean)   (Y is [M,K])
                         epi_bar_sync(h);
                         const int rows = min(K2_BM, p.M - m0), k8 = p.K >> 3;
-                        const uint4 *Xs = reinterpret_cast<const uint4 *>(p.X + (size_t)m0 * p.K);
+                        const uint4 *Xs = reinterpret_cast<const uint4 *>(p.X + (size_t)m0 * p.K);      // 16-bit elements
                         uint4 *Ys = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)m0 * p.K);
                         for (int e = et; e < rows * k8; e += K2_EPI_THREADS) {
                             const float g = s.rowg[h][e / k8];
@@ -520,8 +521,9 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                             uint32_t *w = reinterpret_cast<uint32_t *>(&x);
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
-                                const float lo = __uint_as_float(w[i] << 16) + g, hi = __uint_as_float(w[i] & 0xffff0000u) + g;
-                                w[i] = ptx::pack_bf16x2(lo, hi);
+                                float lo, hi;
+                                ptx::unpack16x2(w[i], p.f16, lo, hi);
+                                w[i] = ptx::pack16x2(lo + g, hi + g, p.f16);
                             }
                             Ys[e] = x;
                         }
@@ -660,18 +662,19 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     const bool pair = h.info.cluster == 2;
     forge_status_t st;
     if (h.tmX_ptr != a.X) {
-        if ((st = encode_tmap_bf16(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, K2_BM, K2_BK)) != FORGE_OK) return st;
+        if ((st = encode_tmap_16(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, K2_BM, K2_BK, d.dtype == FORGE_F16)) != FORGE_OK) return st;
         h.tmX_ptr = a.X;
     }
     if (h.tmW_ptr != a.W) {
-        if ((st = encode_tmap_bf16(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, pair ? K2_BN / 2 : K2_BN, K2_BK)) != FORGE_OK) return st;
+        if ((st = encode_tmap_16(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, pair ? K2_BN / 2 : K2_BN, K2_BK, d.dtype == FORGE_F16)) != FORGE_OK) return st;
         h.tmW_ptr = a.W;
     }
     K2Params p;
-    p.b = (const __nv_bfloat16 *)a.b;
-    p.X = (const __nv_bfloat16 *)a.X;
-    p.gamma = (const __nv_bfloat16 *)a.gamma;
-    p.beta = (const __nv_bfloat16 *)a.beta;
+    p.f16 = d.dtype == FORGE_F16;
+    p.b = (const uint16_t *)a.b;
+    p.X = (const uint16_t *)a.X;
+    p.gamma = (const uint16_t *)a.gamma;
+    p.beta = (const uint16_t *)a.beta;
     p.out = a.out;
     p.M = (int)d.M;
     p.N = (int)d.N;

@@ -54,7 +54,8 @@ struct K3Smem {
 constexpr size_t K3_SMEM_BYTES = 1024 + (size_t)K3_STAGES * K3_STAGE_BYTES + sizeof(K3Smem);
 
 struct K3Params {
-    const __nv_bfloat16 *b;
+    int f16;              // IEEE half (1) or bfloat16 (0) storage
+    const uint16_t *b;
     void *out;
     int M, N, K;
     Epilogue e;
@@ -77,6 +78,7 @@ struct K3Params {
 
 __device__ __forceinline__ void k3_consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(K3_CONSUMERS) : "memory"); }
 
+template <bool F16>
 __global__ void __launch_bounds__(K3_THREADS, 1)
 k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const K3Params p)
 {
@@ -185,8 +187,13 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                                 uint32_t b[4];
                                 const int r = g0 * 8 + b_row;
                                 ptx::ldmatrix_x4(b, wbase + j * wbox_bytes + r * 128 + (((2 * kk + b_chunk) ^ (r & 7)) << 4));
-                                ptx::mma_m16n8k16_bf16(acc[gp * 2], a, b[0], b[1]);
-                                ptx::mma_m16n8k16_bf16(acc[gp * 2 + 1], a, b[2], b[3]);
+                                if (F16) {
+                                    ptx::mma_m16n8k16_f16(acc[gp * 2], a, b[0], b[1]);
+                                    ptx::mma_m16n8k16_f16(acc[gp * 2 + 1], a, b[2], b[3]);
+                                } else {
+                                    ptx::mma_m16n8k16_bf16(acc[gp * 2], a, b[0], b[1]);
+                                    ptx::mma_m16n8k16_bf16(acc[gp * 2 + 1], a, b[2], b[3]);
+                                }
                             }
                         }
                     }
@@ -216,9 +223,7 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                 const bool live = g < ng && gbase + g < g_hi && col + 1 < p.N;   // in the box, in this CTA's share
                 float b0 = 0.f, b1 = 0.f;
                 if (live && p.e.has_bias) {
-                    const __nv_bfloat162 bb = *reinterpret_cast<const __nv_bfloat162 *>(p.b + col);
-                    b0 = __low2float(bb);
-                    b1 = __high2float(bb);
+                    ptx::unpack16x2(__ldg(reinterpret_cast<const uint32_t *>(p.b + col)), F16, b0, b1);
                 }
                 float v[4] = {z.x + b0, z.y + b1, z.z + b0, z.w + b1};
                 apply_act_array<false>(p.e.act, v, p.e.scale);
@@ -268,8 +273,8 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                     }
                 } else if (live) {
                     __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(p.out);
-                    if (r0 < p.M) *reinterpret_cast<uint32_t *>(Y + (size_t)r0 * p.N + col) = ptx::pack_bf16x2(v[0], v[1]);
-                    if (r1 < p.M) *reinterpret_cast<uint32_t *>(Y + (size_t)r1 * p.N + col) = ptx::pack_bf16x2(v[2], v[3]);
+                    if (r0 < p.M) *reinterpret_cast<uint32_t *>(Y + (size_t)r0 * p.N + col) = ptx::pack16x2(v[0], v[1], F16);
+                    if (r1 < p.M) *reinterpret_cast<uint32_t *>(Y + (size_t)r1 * p.N + col) = ptx::pack16x2(v[2], v[3], F16);
                 }
             }
             k3_consumer_sync();
@@ -403,7 +408,8 @@ forge_status_t k3_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
 
 forge_status_t k3_setup(Handle &)
 {
-    return cudaFuncSetAttribute(k3_bf16_skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K3_SMEM_BYTES) == cudaSuccess
+    return cudaFuncSetAttribute(k3_bf16_skinny_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K3_SMEM_BYTES) == cudaSuccess &&
+                   cudaFuncSetAttribute(k3_bf16_skinny_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K3_SMEM_BYTES) == cudaSuccess
                ? FORGE_OK : FORGE_ERR_CUDA;
 }
 
@@ -412,15 +418,16 @@ forge_status_t k3_launch(Handle &h, const RunArgs &a)
     const forge_fused_linear_desc_t &d = h.d;
     forge_status_t st;
     if (h.tmX_ptr != a.X) {
-        if ((st = encode_tmap_bf16(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, 16, K3_BK)) != FORGE_OK) return st;
+        if ((st = encode_tmap_16(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, 16, K3_BK, d.dtype == FORGE_F16)) != FORGE_OK) return st;
         h.tmX_ptr = a.X;
     }
     if (h.tmW_ptr != a.W) {
-        if ((st = encode_tmap_bf16(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, (uint32_t)h.info.tile_n, K3_BK)) != FORGE_OK) return st;
+        if ((st = encode_tmap_16(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, (uint32_t)h.info.tile_n, K3_BK, d.dtype == FORGE_F16)) != FORGE_OK) return st;
         h.tmW_ptr = a.W;
     }
     K3Params p;
-    p.b = (const __nv_bfloat16 *)a.b;
+    p.f16 = d.dtype == FORGE_F16;
+    p.b = (const uint16_t *)a.b;
     p.target = (const int *)a.gamma;
     p.out = a.out;
     p.M = (int)d.M;
@@ -443,7 +450,9 @@ forge_status_t k3_launch(Handle &h, const RunArgs &a)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k3_bf16_skinny_kernel, h.tmX, h.tmW, p) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+    const cudaError_t e = p.f16 ? cudaLaunchKernelEx(&cfg, k3_bf16_skinny_kernel<true>, h.tmX, h.tmW, p)
+                                : cudaLaunchKernelEx(&cfg, k3_bf16_skinny_kernel<false>, h.tmX, h.tmW, p);
+    return e == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
 }
 
 }  // namespace forge

@@ -62,9 +62,10 @@ forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
 forge_status_t k4_setup(Handle &h);
 forge_status_t k4_launch(Handle &h, const RunArgs &a);
 
-// Encode a 2-D row-major bf16 tensor map [rows, cols] with a [box_rows, box_cols] box and
-// the 128-byte shared-memory swizzle.  Host-only driver call.
-forge_status_t encode_tmap_bf16(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
-                                uint32_t box_rows, uint32_t box_cols);
+// Encode a 2-D row-major tensor map [rows, cols] of 16-bit elements (bfloat16, or IEEE half if
+// f16 != 0) with a [box_rows, box_cols] box and the 128-byte shared-memory swizzle.  Host-only
+// driver call.
+forge_status_t encode_tmap_16(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
+                              uint32_t box_rows, uint32_t box_cols, int f16);
 
 }  // namespace forge

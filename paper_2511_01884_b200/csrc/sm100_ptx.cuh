@@ -5,6 +5,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 
 #include "common.cuh"
@@ -160,10 +161,11 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(const void *tile)
     return d;
 }
 
-// Instruction descriptor: D fp32, A and B bf16, both K-major, dense, no negation.
-__host__ __device__ constexpr uint32_t idesc_bf16_f32(int m, int n)
+// Instruction descriptor: D fp32, A and B both bf16 (format 1) or both f16 (format 0) -- the two
+// operands of a kind::f16 MMA must have the same type --, both K-major, dense, no negation.
+__host__ __device__ constexpr uint32_t idesc_16_f32(int m, int n, int f16)
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+    return (1u << 4) | ((f16 ? 0u : 1u) << 7) | ((f16 ? 0u : 1u) << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // D[tmem] (+)= A[smem] * B[smem]; issued by one thread.
@@ -290,6 +292,13 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr)
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(saddr));
 }
+__device__ __forceinline__ void mma_m16n8k16_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ void mma_m16n8k16_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
     asm volatile(
@@ -303,6 +312,26 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// ---- the two 16-bit storage formats (f16 != 0: IEEE half, else bfloat16) --------------------
+// Round-to-nearest-even pack of two floats, and the exact widening of a stored value / pair.
+__device__ __forceinline__ uint32_t pack16x2(float lo, float hi, int f16) { return f16 ? pack_f16x2(lo, hi) : pack_bf16x2(lo, hi); }
+__device__ __forceinline__ float widen16(uint16_t v, int f16)
+{
+    return f16 ? __half2float(__ushort_as_half(v)) : __uint_as_float((uint32_t)v << 16);
+}
+__device__ __forceinline__ float load16(const uint16_t *base, size_t i, int f16) { return widen16(__ldg(base + i), f16); }
+__device__ __forceinline__ void unpack16x2(uint32_t w, int f16, float &lo, float &hi)
+{
+    lo = widen16((uint16_t)(w & 0xffffu), f16);
+    hi = widen16((uint16_t)(w >> 16), f16);
 }
 
 }  // namespace ptx

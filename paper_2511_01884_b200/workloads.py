@@ -27,7 +27,7 @@ import numpy as np
 
 # Enumerations of the public C interface, restated as plain integers so that this module
 # depends on neither side.
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 ACT_IDENTITY, ACT_RELU, ACT_GELU_ERF, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3, 4
 RED_NONE, RED_SUM, RED_MAX, RED_LAYERNORM, RED_MEAN_GELU_RESIDUAL, RED_LOGSUMEXP, RED_CROSS_ENTROPY = 0, 1, 2, 3, 4, 5, 6
 VECTOR_OUT = (RED_SUM, RED_MAX, RED_LOGSUMEXP, RED_CROSS_ENTROPY)      # reductions whose output is fp32 [M]
@@ -111,6 +111,8 @@ def round_to_storage(x: np.ndarray, dtype: int) -> np.ndarray:
     """Return float32 values that are exactly representable in the storage dtype."""
     if dtype == F32:
         return np.ascontiguousarray(x, dtype=np.float32)
+    if dtype == F16:          # IEEE half: numpy rounds to nearest even
+        return np.ascontiguousarray(x, dtype=np.float32).astype(np.float16).astype(np.float32)
     return bf16_bits_to_f32(f32_to_bf16_bits(x))
 
 

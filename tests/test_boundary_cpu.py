@@ -36,7 +36,7 @@ def test_no_vendor_gemm_library_is_linked():
 
 
 def test_enums_match_the_workload_module():
-    assert (B.FORGE_F32, B.FORGE_BF16) == (wk.F32, wk.BF16)
+    assert (B.FORGE_F32, B.FORGE_BF16, B.FORGE_F16) == (wk.F32, wk.BF16, wk.F16)
     assert (B.FORGE_ACT_IDENTITY, B.FORGE_ACT_RELU, B.FORGE_ACT_GELU_ERF, B.FORGE_ACT_GELU_TANH, B.FORGE_ACT_SILU) == \
            (wk.ACT_IDENTITY, wk.ACT_RELU, wk.ACT_GELU_ERF, wk.ACT_GELU_TANH, wk.ACT_SILU)
     assert (B.FORGE_RED_NONE, B.FORGE_RED_SUM, B.FORGE_RED_MAX, B.FORGE_RED_LAYERNORM) == \
@@ -45,7 +45,7 @@ def test_enums_match_the_workload_module():
 
 def test_invalid_descriptors():
     ok = dict(M=8, N=8, K=8, dtype=0, act=0, red=0)
-    for bad in (dict(M=0), dict(N=-1), dict(K=0), dict(dtype=2), dict(act=5), dict(act=-1), dict(red=7), dict(red=-1)):
+    for bad in (dict(M=0), dict(N=-1), dict(K=0), dict(dtype=3), dict(act=5), dict(act=-1), dict(red=7), dict(red=-1)):
         st, _ = B.forge_fused_linear_query_plan(B.make_desc(**{**ok, **bad}))
         assert st == B.FORGE_ERR_INVALID_ARG, bad
         st, h = B.forge_fused_linear_create(B.make_desc(**{**ok, **bad}))

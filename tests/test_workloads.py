@@ -29,6 +29,8 @@ def test_bf16_rounding_is_nearest_even():
     want = torch.from_numpy(x).to(torch.bfloat16).float().numpy()
     assert np.array_equal(wk.round_to_storage(x, wk.BF16), want)
     assert np.array_equal(wk.round_to_storage(x, wk.F32), x)
+    h = x[np.abs(x) < 6e4]
+    assert np.array_equal(wk.round_to_storage(h, wk.F16), torch.from_numpy(h).to(torch.float16).float().numpy())
 
 
 def test_workload_table_matches_the_five_configurations():
