@@ -94,7 +94,7 @@ typedef enum {
     FORGE_KERNEL_F32_FFMA = 1,        /* fp32 register-tiled FFMA GEMM, fused epilogue        */
     FORGE_KERNEL_BF16_TCGEN05 = 2,    /* bf16 TMA -> smem ring -> tcgen05.mma -> TMEM; CTA     */
                                       /* pairs (cta_group::2, 256x256 tiles) when M > 128      */
-    FORGE_KERNEL_BF16_SKINNY = 3,     /* bf16, M <= 16: split-K over warps, HBM-bound          */
+    FORGE_KERNEL_BF16_SKINNY = 3,     /* 16-bit, M <= 32: split-K over warps, HBM-bound        */
     FORGE_KERNEL_BF16_TCGEN05_LN = 4  /* bf16 tcgen05 whose epilogue merges row statistics    */
                                       /* across the N-tiles of a row strip (LayerNorm)         */
 } forge_kernel_t;
@@ -115,8 +115,9 @@ typedef struct {
  * `sm_count` multiprocessors.  Touches no device.  Returns FORGE_ERR_INVALID_ARG /
  * FORGE_ERR_UNSUPPORTED exactly as create() would for the same descriptor.
  * Kernel selection (Appendix B.1's point that the right fusion depends on whether the chain
- * is compute- or memory-bound): fp32 -> F32_FFMA; bf16 with M <= 16 and no LayerNorm ->
- * BF16_SKINNY; bf16 LayerNorm -> BF16_TCGEN05_LN; other bf16 -> BF16_TCGEN05.
+ * is compute- or memory-bound): fp32 -> F32_FFMA; 16-bit with M <= 32 and neither LayerNorm nor
+ * the mean-GELU-residual chain -> BF16_SKINNY; 16-bit LayerNorm -> BF16_TCGEN05_LN; other 16-bit
+ * -> BF16_TCGEN05.
  * Unsupported: bf16 with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); fp32 LayerNorm with
  * N > 1024 (one 8-CTA cluster); bf16 LayerNorm with more 256-column tiles per row than
  * clusters in the grid.

@@ -19,6 +19,21 @@ bool desc_enums_ok(const forge_fused_linear_desc_t &d)
            d.act <= FORGE_ACT_SILU && d.red >= FORGE_RED_NONE && d.red <= FORGE_RED_CROSS_ENTROPY;
 }
 
+// Largest M served by the skinny kernel.  Up to 32 rows it streams W a few percent faster than
+// the tensor-core tile kernel (148 CTAs against N/256 tiles); from there on its mma.sync rate,
+// not the stream, sets the time and the tile kernel wins.  FORGE_SKINNY_MAX_M (0..32) lowers the
+// limit, for comparing the two kernels on the same problem.
+int64_t skinny_max_m()
+{
+    static const int64_t v = [] {
+        const char *e = std::getenv("FORGE_SKINNY_MAX_M");
+        if (!e || !*e) return (int64_t)32;
+        const long x = std::strtol(e, nullptr, 10);
+        return (int64_t)(x < 0 ? 0 : x > 32 ? 32 : x);
+    }();
+    return v;
+}
+
 forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
     if (d.M <= 0 || d.N <= 0 || d.K <= 0 || !desc_enums_ok(d) || d.device < 0 || sm_count <= 0)
@@ -32,7 +47,7 @@ forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_
     } else {
         if (d.K % 8 != 0 || d.N % 8 != 0) return FORGE_ERR_UNSUPPORTED;     // 16-byte row pitch for TMA
         if (d.red == FORGE_RED_LAYERNORM) st = k4_plan(d, sm_count, info, wl);
-        else if (d.M <= 16 && d.red != FORGE_RED_MEAN_GELU_RESIDUAL) st = k3_plan(d, sm_count, info, wl);
+        else if (d.M <= skinny_max_m() && d.red != FORGE_RED_MEAN_GELU_RESIDUAL) st = k3_plan(d, sm_count, info, wl);
         else st = k2_plan(d, sm_count, info, wl);
     }
     if (st != FORGE_OK) return st;

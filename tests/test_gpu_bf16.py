@@ -37,7 +37,7 @@ def test_k_steps_inside_and_across_swizzle_atoms():
         pu.assert_parity(wl, g, pu.run_oracle(wl, inp), f"K={K}")
 
 
-SHAPES = [(17, 8, 8), (128, 256, 64), (129, 264, 72), (300, 520, 200), (1000, 776, 328), (2048, 1024, 512)]
+SHAPES = [(33, 8, 8), (128, 256, 64), (129, 264, 72), (300, 520, 200), (1000, 776, 328), (2048, 1024, 512)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)

@@ -28,7 +28,8 @@ def test_identity_weight_reproduces_x_in_half_precision():
     assert np.array_equal(g, inp["X"].astype(np.float64))
 
 
-@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (300, 520, 200), (1000, 776, 328), (16, 1192, 200), (5, 20000, 264)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (300, 520, 200), (1000, 776, 328), (16, 1192, 200), (5, 20000, 264),
+                                   (29, 20000, 264), (32, 1192, 200)])
 @pytest.mark.parametrize("red", REDS)
 def test_shapes_and_reductions(M, N, K, red):
     act = ACTS[(M + N + K + red) % len(ACTS)]

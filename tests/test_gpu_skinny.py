@@ -1,4 +1,4 @@
-"""GPU parity of the skinny-M bf16 path (M <= 16: split-K over warps, mma.sync from a TMA
+"""GPU parity of the skinny-M bf16 path (M <= 32: split-K over warps, mma.sync from a TMA
 ring, warp-shuffle row reductions) against the CPU oracle."""
 import numpy as np
 import pytest
@@ -30,8 +30,11 @@ def test_identity_weight_reproduces_x():
 # N/8 below, at and far above the SM count (1, several and many strips per CTA); K with a
 # ragged last block and fewer blocks than K-slices; M below 16
 # ... and K long enough for many passes over the shared-memory ring
+# ... and two 16-row tiles of X per CTA (M up to 32), full and ragged
 SHAPES = [(16, 8, 8), (1, 64, 16), (5, 1184, 72), (16, 1192, 200), (16, 4096, 1024), (7, 20000, 264),
-          (16, 148 * 8 * 17, 128), (16, 148 * 8 * 40 + 8, 64), (16, 2368, 4096), (3, 1184 * 13, 2048)]
+          (16, 148 * 8 * 17, 128), (16, 148 * 8 * 40 + 8, 64), (16, 2368, 4096), (3, 1184 * 13, 2048),
+          (17, 8, 8), (32, 1192, 200), (27, 20000, 264), (24, 4096, 1024), (32, 148 * 8 * 17, 128),
+          (19, 1184 * 13, 2048), (32, 2368, 4096)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -63,6 +66,14 @@ def test_repeatable_bits_and_back_to_back_runs():
     op.close()
     assert np.array_equal(a, b)
     pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
+
+
+def test_row_tiles_follow_m():
+    for M, rows in ((1, 16), (16, 16), (17, 32), (32, 32)):
+        st, plan = B.forge_fused_linear_query_plan(pu.desc_of(_case(M, 4096, 256, wk.ACT_RELU, wk.RED_SUM)))
+        assert st == B.FORGE_OK and plan.kernel == B.FORGE_KERNEL_BF16_SKINNY and plan.tile_m == rows
+    st, plan = B.forge_fused_linear_query_plan(pu.desc_of(_case(33, 4096, 256, wk.ACT_RELU, wk.RED_SUM)))
+    assert st == B.FORGE_OK and plan.kernel == B.FORGE_KERNEL_BF16_TCGEN05
 
 
 def test_c4_full():
