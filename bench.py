@@ -38,6 +38,7 @@ from paper_2511_01884_b200 import workloads as wk  # noqa: E402
 HEADLINE = "c3"
 ALL_WORKLOADS = {**wk.WORKLOADS, **wk.EXTRA_WORKLOADS}
 NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
+TF32_OVER_BF16 = 1.1 / 2.25          # nominal dense tensor peaks, TF32 : bf16
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel
@@ -64,7 +65,8 @@ def load_peaks():
 
 
 def kernel_source_hash(kernel: int) -> str:
-    name = {1: "k1_f32_ffma.cu", 2: "k2_bf16_tcgen05.cu", 3: "k3_bf16_skinny.cu", 4: "k2_bf16_tcgen05.cu"}[kernel]
+    name = {1: "k1_f32_ffma.cu", 2: "k2_bf16_tcgen05.cu", 3: "k3_bf16_skinny.cu", 4: "k2_bf16_tcgen05.cu",
+            5: "k5_f32_tf32x3.cu"}[kernel]
     with open(os.path.join(ROOT, "paper_2511_01884_b200", "csrc", name), "rb") as f:
         return hashlib.sha256(f.read()).hexdigest()[:16]
 
@@ -248,6 +250,11 @@ def roofline_of(wl, ms, peaks, kernel, sm_max_mhz, sm_count):
         ach = wl.flops / ms / 1e9
         peak, unit, bound = peaks["bf16_tflops"], "TFLOP/s", "tensor"
         note = f"2MNK = {wl.flops} flops per launch; peak = cuBLAS bf16 burst, of {src}"
+    elif wl.dtype == wk.F32_TF32X3:
+        ach = wl.flops / ms / 1e9
+        peak, unit, bound = peaks["bf16_tflops"] * TF32_OVER_BF16, "TFLOP/s", "tensor"
+        note = (f"2MNK = {wl.flops} algorithmic flops per launch, each product computed as three TF32 MMAs (ceiling of the "
+                f"scheme: a third of the peak); peak = cuBLAS bf16 burst, of {src}, x the nominal TF32/bf16 ratio 1.1/2.25")
     else:
         ach = wl.flops / ms / 1e9
         peak = sm_count * 128 * 2 * (sm_max_mhz or 1965.0) * 1e6 / 1e12
@@ -429,7 +436,7 @@ def main():
     eager_us = None
     if rank == 0 and world == 1:
         time.sleep(2.0)
-        eager_us = eager_context_us(wl, d, torch)
+        eager_us = eager_context_us(wl, d, torch, steps=args.steps)      # same number of back-to-back calls as the timed region
         line["torch_eager_context"] = {"us_per_call": round(eager_us, 1), "value": round(unit_value(wl, eager_us / 1e3)[0], 2),
                                        "unit": unit, "what": "unfused F.linear + activation (+ reduction) in the same dtype, same GPU"}
     op.close()
@@ -451,7 +458,7 @@ def main():
                 d2 = device_tensors(w2, i2, torch)
                 op2 = make_op(w2, w2.M, local)
                 fl = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device="cuda") if w2.algorithmic_bytes < 130e6 else None
-                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50, "n1": 20, "n2": 10}[name]
+                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50, "n1": 20, "n2": 10, "c2t": 50, "n1t": 50}[name]
                 ms2 = time_steps(op2, d2, steps2, 3, torch, flush_buf=fl)
                 v2, u2 = unit_value(w2, ms2)
                 launches += steps2

@@ -47,7 +47,18 @@ typedef enum {
                                  /* forge_fused_linear_f32_reduce_static() holds          */
 } forge_status_t;
 
-typedef enum { FORGE_F32 = 0, FORGE_BF16 = 1, FORGE_F16 = 2 } forge_dtype_t;   /* F16: IEEE half, same kernels as BF16 */
+typedef enum {
+    FORGE_F32 = 0,               /* fp32 storage, fp32 FFMA arithmetic                    */
+    FORGE_BF16 = 1,
+    FORGE_F16 = 2,               /* IEEE half, same kernels as BF16                       */
+    FORGE_F32_TF32X3 = 3
+    /* fp32 storage (every tensor exactly as for FORGE_F32), contraction on the tensor cores:
+     * each operand is split into a TF32 head and a TF32 tail and X W^T is accumulated in fp32
+     * from the three products head*head, head*tail, tail*head (relative error of a product
+     * about 2^-21), so the result stays within the 1e-4 of Section 2.2 with two orders of
+     * magnitude to spare.  Needs K % 4 == 0, N % 4 == 0 and 16-byte aligned pointers; LayerNorm
+     * is not served (FORGE_ERR_UNSUPPORTED).                                              */
+} forge_dtype_t;
 
 typedef enum {
     FORGE_ACT_IDENTITY = 0,
@@ -95,8 +106,10 @@ typedef enum {
     FORGE_KERNEL_BF16_TCGEN05 = 2,    /* bf16 TMA -> smem ring -> tcgen05.mma -> TMEM; CTA     */
                                       /* pairs (cta_group::2, 256x256 tiles) when M > 128      */
     FORGE_KERNEL_BF16_SKINNY = 3,     /* 16-bit, M <= 32: split-K over warps, HBM-bound        */
-    FORGE_KERNEL_BF16_TCGEN05_LN = 4  /* bf16 tcgen05 whose epilogue merges row statistics    */
+    FORGE_KERNEL_BF16_TCGEN05_LN = 4, /* bf16 tcgen05 whose epilogue merges row statistics    */
                                       /* across the N-tiles of a row strip (LayerNorm)         */
+    FORGE_KERNEL_F32_TF32X3 = 5       /* fp32 operands split in shared memory into TF32 head   */
+                                      /* and tail, three tcgen05.mma kind::tf32 per k-step     */
 } forge_kernel_t;
 
 typedef struct {
@@ -115,7 +128,7 @@ typedef struct {
  * `sm_count` multiprocessors.  Touches no device.  Returns FORGE_ERR_INVALID_ARG /
  * FORGE_ERR_UNSUPPORTED exactly as create() would for the same descriptor.
  * Kernel selection (Appendix B.1's point that the right fusion depends on whether the chain
- * is compute- or memory-bound): fp32 -> F32_FFMA; 16-bit with M <= 32 and neither LayerNorm nor
+ * is compute- or memory-bound): fp32 -> F32_FFMA; fp32 with TF32x3 arithmetic -> F32_TF32X3; 16-bit with M <= 32 and neither LayerNorm nor
  * the mean-GELU-residual chain -> BF16_SKINNY; 16-bit LayerNorm -> BF16_TCGEN05_LN; other 16-bit
  * -> BF16_TCGEN05.
  * Unsupported: bf16 with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); fp32 LayerNorm with

@@ -13,11 +13,12 @@ LIB_PATH = os.path.join(_HERE, "libforge.so")
 (FORGE_OK, FORGE_ERR_INVALID_ARG, FORGE_ERR_UNSUPPORTED, FORGE_ERR_CUDA, FORGE_ERR_ALLOC, FORGE_ERR_TIMEOUT,
  FORGE_ERR_SCRATCH_LIMIT) = range(7)
 FORGE_STATIC_SCRATCH_BYTES = 1 << 20
-FORGE_F32, FORGE_BF16, FORGE_F16 = 0, 1, 2
+FORGE_F32, FORGE_BF16, FORGE_F16, FORGE_F32_TF32X3 = 0, 1, 2, 3
 FORGE_ACT_IDENTITY, FORGE_ACT_RELU, FORGE_ACT_GELU_ERF, FORGE_ACT_GELU_TANH, FORGE_ACT_SILU = range(5)
 (FORGE_RED_NONE, FORGE_RED_SUM, FORGE_RED_MAX, FORGE_RED_LAYERNORM, FORGE_RED_MEAN_GELU_RESIDUAL,
  FORGE_RED_LOGSUMEXP, FORGE_RED_CROSS_ENTROPY) = range(7)
 FORGE_KERNEL_F32_FFMA, FORGE_KERNEL_BF16_TCGEN05, FORGE_KERNEL_BF16_SKINNY, FORGE_KERNEL_BF16_TCGEN05_LN = 1, 2, 3, 4
+FORGE_KERNEL_F32_TF32X3 = 5
 
 EXPORTS = [
     "forge_fused_linear_query_plan", "forge_fused_linear_create", "forge_fused_linear_run",

@@ -22,7 +22,7 @@ struct Epilogue {
 // Status word layout: 0 = ok; otherwise (FORGE_ERR_TIMEOUT << 16) | location code.
 enum WaitSite : int {
     SITE_TMA_FULL = 1, SITE_STAGE_EMPTY = 2, SITE_ACC_FULL = 3, SITE_ACC_EMPTY = 4,
-    SITE_ARRIVAL = 5, SITE_STORE = 6, SITE_CLUSTER = 7
+    SITE_ARRIVAL = 5, SITE_STORE = 6, SITE_CLUSTER = 7, SITE_SPLIT = 8
 };
 
 // Words 1..3 of the status area describe the first give-up: a caller-chosen detail word, the

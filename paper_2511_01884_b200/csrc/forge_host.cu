@@ -1,6 +1,7 @@
 // The C interface: descriptor validation, kernel selection, workspace, launches.
 #include <cstdlib>
 #include <cstring>
+#include <initializer_list>
 #include <new>
 
 #include "common.cuh"
@@ -15,7 +16,7 @@ constexpr size_t kStatusBytes = 256;     // status word lives alone in the first
 
 bool desc_enums_ok(const forge_fused_linear_desc_t &d)
 {
-    return (d.dtype == FORGE_F32 || d.dtype == FORGE_BF16 || d.dtype == FORGE_F16) && d.act >= FORGE_ACT_IDENTITY &&
+    return (d.dtype == FORGE_F32 || d.dtype == FORGE_BF16 || d.dtype == FORGE_F16 || d.dtype == FORGE_F32_TF32X3) && d.act >= FORGE_ACT_IDENTITY &&
            d.act <= FORGE_ACT_SILU && d.red >= FORGE_RED_NONE && d.red <= FORGE_RED_CROSS_ENTROPY;
 }
 
@@ -44,6 +45,8 @@ forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_
     forge_status_t st;
     if (d.dtype == FORGE_F32) {
         st = k1_plan(d, sm_count, info, wl);
+    } else if (d.dtype == FORGE_F32_TF32X3) {
+        st = k5_plan(d, sm_count, info, wl);
     } else {
         if (d.K % 8 != 0 || d.N % 8 != 0) return FORGE_ERR_UNSUPPORTED;     // 16-byte row pitch for TMA
         if (d.red == FORGE_RED_LAYERNORM) st = k4_plan(d, sm_count, info, wl);
@@ -72,7 +75,7 @@ struct DeviceGuard {
     }
 };
 
-size_t elem_bytes(const forge_fused_linear_desc_t &d) { return d.dtype == FORGE_F32 ? 4 : 2; }
+size_t elem_bytes(const forge_fused_linear_desc_t &d) { return (d.dtype == FORGE_F32 || d.dtype == FORGE_F32_TF32X3) ? 4 : 2; }
 size_t out_bytes(const forge_fused_linear_desc_t &d)
 {
     if (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY)
@@ -88,8 +91,8 @@ forge_status_t check_run_args(const Handle &h, const RunArgs &a)
     if (h.d.red == FORGE_RED_CROSS_ENTROPY && !a.gamma) return FORGE_ERR_INVALID_ARG;      // the targets
     const uintptr_t m = (uintptr_t)a.X | (uintptr_t)a.W | (uintptr_t)a.out | (uintptr_t)a.b |
                         (uintptr_t)a.gamma | (uintptr_t)a.beta;
-    // 16-bit operands travel by TMA and 128-bit accesses: 16-byte alignment is required.
-    // fp32 falls back to scalar accesses when unaligned, but still needs element alignment.
+    // Operands that travel by TMA and 128-bit accesses need 16-byte alignment.  The FFMA kernel
+    // falls back to scalar accesses when unaligned, but still needs element alignment.
     if (h.d.dtype != FORGE_F32 ? (m % 16 != 0) : (m % 4 != 0)) return FORGE_ERR_INVALID_ARG;
     return FORGE_OK;
 }
@@ -101,6 +104,7 @@ forge_status_t dispatch(Handle &h, const RunArgs &a)
     case FORGE_KERNEL_BF16_TCGEN05: return k2_launch(h, a);
     case FORGE_KERNEL_BF16_SKINNY: return k3_launch(h, a);
     case FORGE_KERNEL_BF16_TCGEN05_LN: return k4_launch(h, a);
+    case FORGE_KERNEL_F32_TF32X3: return k5_launch(h, a);
     }
     return FORGE_ERR_UNSUPPORTED;
 }
@@ -111,8 +115,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-forge_status_t encode_tmap_16(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
-                              uint32_t box_rows, uint32_t box_cols, int f16)
+static forge_status_t encode_tmap(CUtensorMap *tm, CUtensorMapDataType type, size_t elem, const void *ptr, uint64_t rows,
+                                  uint64_t cols, uint32_t box_rows, uint32_t box_cols)
 {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
@@ -124,7 +128,7 @@ forge_status_t encode_tmap_16(CUtensorMap *tm, const void *ptr, uint64_t rows, u
         fn = (EncodeTiledFn)sym;
     }
     const cuuint64_t dims[2] = {cols, rows};                  // innermost first
-    const cuuint64_t strides[1] = {cols * 2};                 // bytes, dimension 1
+    const cuuint64_t strides[1] = {cols * elem};              // bytes, dimension 1
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     // FORGE_TMA_L2_PROMOTION = 0 | 64 | 128 | 256 overrides the L2 fetch granularity (tuning aid)
@@ -137,9 +141,21 @@ forge_status_t encode_tmap_16(CUtensorMap *tm, const void *ptr, uint64_t rows, u
                                       : promo == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
                                       : promo == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B
                                                      : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
-    const CUresult r = fn(tm, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, l2, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    const CUresult r = fn(tm, type, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, l2, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? FORGE_OK : FORGE_ERR_CUDA;
+}
+
+forge_status_t encode_tmap_16(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
+                              uint32_t box_rows, uint32_t box_cols, int f16)
+{
+    return encode_tmap(tm, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, rows, cols, box_rows, box_cols);
+}
+
+forge_status_t encode_tmap_f32(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
+                               uint32_t box_rows, uint32_t box_cols)
+{
+    return encode_tmap(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ptr, rows, cols, box_rows, box_cols);
 }
 
 }  // namespace forge
@@ -233,6 +249,7 @@ forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, 
     case FORGE_KERNEL_BF16_TCGEN05: st = k2_setup(*h); break;
     case FORGE_KERNEL_BF16_SKINNY: st = k3_setup(*h); break;
     case FORGE_KERNEL_BF16_TCGEN05_LN: st = k4_setup(*h); break;
+    case FORGE_KERNEL_F32_TF32X3: st = k5_setup(*h); break;
     }
     if (st != FORGE_OK) { cudaFree(h->ws.base); delete h; return st; }
     *out = reinterpret_cast<forge_fused_linear_t>(h);
@@ -250,6 +267,65 @@ forge_status_t forge_fused_linear_run(forge_fused_linear_t hh, const void *X, co
     DeviceGuard g(h.d.device);
     if (!g.ok) return FORGE_ERR_CUDA;
     return dispatch(h, a);
+}
+
+// Block plan of the pipelined host path: 256-row multiples (whole CTA-pair tiles), at most
+// kHostPipeMaxBlocks blocks, and only when X is large enough for the overlap to matter.
+static int64_t host_block_rows(const forge_fused_linear_desc_t &d)
+{
+    static const int env = [] {          // FORGE_HOST_PIPELINE=0: one upload, one kernel, one download
+        const char *e = std::getenv("FORGE_HOST_PIPELINE");
+        return e ? std::atoi(e) : 1;
+    }();
+    const size_t bx = (size_t)d.M * (size_t)d.K * elem_bytes(d);
+    if (!env || d.M < 1024 || bx < ((size_t)8 << 20)) return 0;
+    const int64_t want = (d.M + kHostPipeMaxBlocks - 1) / kHostPipeMaxBlocks;
+    return ((want + 255) / 256) * 256;
+}
+
+static void pipeline_free(HostPipeline *p)
+{
+    if (!p) return;
+    if (p->block) forge_fused_linear_destroy(reinterpret_cast<forge_fused_linear_t>(p->block));
+    if (p->last) forge_fused_linear_destroy(reinterpret_cast<forge_fused_linear_t>(p->last));
+    for (int i = 0; i < kHostPipeMaxBlocks; ++i) {
+        if (p->landed[i]) cudaEventDestroy(p->landed[i]);
+        if (p->computed[i]) cudaEventDestroy(p->computed[i]);
+    }
+    if (p->s_in) cudaStreamDestroy(p->s_in);
+    if (p->s_run) cudaStreamDestroy(p->s_run);
+    if (p->s_out) cudaStreamDestroy(p->s_out);
+    delete p;
+}
+
+static forge_status_t pipeline_create(Handle &h, int64_t block_rows)
+{
+    HostPipeline *p = new (std::nothrow) HostPipeline();
+    if (!p) return FORGE_ERR_ALLOC;
+    p->block_rows = block_rows;
+    p->blocks = (int)((h.d.M + block_rows - 1) / block_rows);
+    forge_status_t st = FORGE_OK;
+    if (cudaStreamCreateWithFlags(&p->s_in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&p->s_run, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&p->s_out, cudaStreamNonBlocking) != cudaSuccess)
+        st = FORGE_ERR_CUDA;
+    for (int i = 0; i < p->blocks && st == FORGE_OK; ++i)
+        if (cudaEventCreateWithFlags(&p->landed[i], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&p->computed[i], cudaEventDisableTiming) != cudaSuccess)
+            st = FORGE_ERR_CUDA;
+    forge_fused_linear_desc_t d = h.d;
+    if (st == FORGE_OK) {
+        d.M = block_rows;
+        st = forge_fused_linear_create(&d, reinterpret_cast<forge_fused_linear_t *>(&p->block));
+    }
+    const int64_t rest = h.d.M - (int64_t)(p->blocks - 1) * block_rows;
+    if (st == FORGE_OK && rest != block_rows) {
+        d.M = rest;
+        st = forge_fused_linear_create(&d, reinterpret_cast<forge_fused_linear_t *>(&p->last));
+    }
+    if (st != FORGE_OK) { cudaGetLastError(); pipeline_free(p); return st; }
+    h.pipe = p;
+    return FORGE_OK;
 }
 
 forge_status_t forge_fused_linear_run_host(forge_fused_linear_t hh, const void *X, const void *W, const void *b,
@@ -276,25 +352,73 @@ forge_status_t forge_fused_linear_run_host(forge_fused_linear_t hh, const void *
             h.hX = h.hW = h.hb = h.hg = h.hbe = h.hout = nullptr;
             return FORGE_ERR_ALLOC;
         }
+        const int64_t block_rows = host_block_rows(d);
+        if (block_rows > 0 && block_rows < d.M) {
+            const forge_status_t st = pipeline_create(h, block_rows);
+            if (st != FORGE_OK) return st;
+        }
     }
-    cudaStream_t s = nullptr;
-    bool ok = cudaMemcpyAsync(h.hX, X, bx, cudaMemcpyHostToDevice, s) == cudaSuccess &&
-              cudaMemcpyAsync(h.hW, W, bw, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    HostPipeline *pp = h.pipe;
+    cudaStream_t s = pp ? pp->s_in : nullptr;
+    const bool has_sub = d.red == FORGE_RED_MEAN_GELU_RESIDUAL && gamma;
+    const bool has_tgt = d.red == FORGE_RED_CROSS_ENTROPY;
+    // everything but X first: the first block of rows needs all of W
+    bool ok = cudaMemcpyAsync(h.hW, W, bw, cudaMemcpyHostToDevice, s) == cudaSuccess;
     if (ok && d.has_bias) ok = cudaMemcpyAsync(h.hb, b, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
     if (ok && d.red == FORGE_RED_LAYERNORM)
         ok = cudaMemcpyAsync(h.hg, gamma, bn, cudaMemcpyHostToDevice, s) == cudaSuccess &&
              cudaMemcpyAsync(h.hbe, beta, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    const bool has_sub = d.red == FORGE_RED_MEAN_GELU_RESIDUAL && gamma;
     if (ok && has_sub) ok = cudaMemcpyAsync(h.hg, gamma, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    const bool has_tgt = d.red == FORGE_RED_CROSS_ENTROPY;
     if (ok && has_tgt) ok = cudaMemcpyAsync(h.hg, gamma, bt, cudaMemcpyHostToDevice, s) == cudaSuccess;
     if (!ok) return FORGE_ERR_CUDA;
-    RunArgs a{h.hX, h.hW, d.has_bias ? h.hb : nullptr,
-              (d.red == FORGE_RED_LAYERNORM || has_sub || has_tgt) ? h.hg : nullptr, h.hbe, h.hout, s};
-    const forge_status_t st = dispatch(h, a);
+    const void *aux = (d.red == FORGE_RED_LAYERNORM || has_sub || has_tgt) ? h.hg : nullptr;
+
+    if (!pp) {
+        if (cudaMemcpyAsync(h.hX, X, bx, cudaMemcpyHostToDevice, s) != cudaSuccess) return FORGE_ERR_CUDA;
+        RunArgs a{h.hX, h.hW, d.has_bias ? h.hb : nullptr, aux, h.hbe, h.hout, s};
+        const forge_status_t st = dispatch(h, a);
+        if (st != FORGE_OK) return st;
+        if (cudaMemcpyAsync(out, h.hout, bo, cudaMemcpyDeviceToHost, s) != cudaSuccess) return FORGE_ERR_CUDA;
+        return cudaStreamSynchronize(s) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+    }
+
+    // Blocks of rows: every reduction here runs along N, so a block of rows is a complete problem.
+    const size_t x_row = (size_t)d.K * e, o_row = bo / (size_t)d.M;
+    forge_status_t st = FORGE_OK;
+    for (int i = 0; i < pp->blocks && st == FORGE_OK; ++i) {
+        const int64_t r0 = (int64_t)i * pp->block_rows;
+        const int64_t rows = (i == pp->blocks - 1) ? d.M - r0 : pp->block_rows;
+        Handle &hb = (i == pp->blocks - 1 && pp->last) ? *pp->last : *pp->block;
+        char *xd = (char *)h.hX + (size_t)r0 * x_row, *od = (char *)h.hout + (size_t)r0 * o_row;
+        ok = cudaMemcpyAsync(xd, (const char *)X + (size_t)r0 * x_row, (size_t)rows * x_row, cudaMemcpyHostToDevice, pp->s_in) == cudaSuccess &&
+             cudaEventRecord(pp->landed[i], pp->s_in) == cudaSuccess &&
+             cudaStreamWaitEvent(pp->s_run, pp->landed[i], 0) == cudaSuccess;
+        if (!ok) { st = FORGE_ERR_CUDA; break; }
+        // per-row auxiliary data (the cross-entropy targets) moves with the block; per-column data does not
+        const void *aux_i = has_tgt ? (const void *)((const char *)h.hg + (size_t)r0 * 4) : aux;
+        RunArgs a{xd, h.hW, d.has_bias ? h.hb : nullptr, aux_i, h.hbe, od, pp->s_run};
+        st = dispatch(hb, a);
+        if (st != FORGE_OK) break;
+        ok = cudaEventRecord(pp->computed[i], pp->s_run) == cudaSuccess &&
+             cudaStreamWaitEvent(pp->s_out, pp->computed[i], 0) == cudaSuccess &&
+             cudaMemcpyAsync((char *)out + (size_t)r0 * o_row, od, (size_t)rows * o_row, cudaMemcpyDeviceToHost, pp->s_out) == cudaSuccess;
+        if (!ok) st = FORGE_ERR_CUDA;
+    }
+    // drain all three streams whatever happened, so that no copy still reads the caller's buffers
+    const bool drained = cudaStreamSynchronize(pp->s_in) == cudaSuccess && cudaStreamSynchronize(pp->s_run) == cudaSuccess &&
+                         cudaStreamSynchronize(pp->s_out) == cudaSuccess;
     if (st != FORGE_OK) return st;
-    if (cudaMemcpyAsync(out, h.hout, bo, cudaMemcpyDeviceToHost, s) != cudaSuccess) return FORGE_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return FORGE_ERR_CUDA;
+    if (!drained) return FORGE_ERR_CUDA;
+    // a give-up inside a block's kernel is recorded in the child's status word: fold it into this handle's
+    for (Handle *c : {pp->block, pp->last}) {
+        if (!c) continue;
+        int word = 0;
+        if (cudaMemcpy(&word, c->ws.status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return FORGE_ERR_CUDA;
+        if (word != 0) {
+            cudaMemcpy(h.ws.status, c->ws.status, 4 * sizeof(int), cudaMemcpyDeviceToDevice);
+            forge_fused_linear_last_status(reinterpret_cast<forge_fused_linear_t>(c));     // clears the child
+        }
+    }
     return FORGE_OK;
 }
 
@@ -344,6 +468,7 @@ forge_status_t forge_fused_linear_destroy(forge_fused_linear_t hh)
         DeviceGuard g(h->d.device);
         cudaFree(h->ws.base);
         cudaFree(h->hX); cudaFree(h->hW); cudaFree(h->hb); cudaFree(h->hg); cudaFree(h->hbe); cudaFree(h->hout);
+        pipeline_free(h->pipe);
     }
     delete h;
     return FORGE_OK;
@@ -370,6 +495,7 @@ const char *forge_kernel_name(forge_kernel_t k)
     case FORGE_KERNEL_BF16_TCGEN05: return "bf16_tcgen05_tma";
     case FORGE_KERNEL_BF16_SKINNY: return "bf16_skinny_splitk";
     case FORGE_KERNEL_BF16_TCGEN05_LN: return "bf16_tcgen05_tma_layernorm";
+    case FORGE_KERNEL_F32_TF32X3: return "f32_tf32x3_tcgen05_tma";
     }
     return "unknown kernel";
 }

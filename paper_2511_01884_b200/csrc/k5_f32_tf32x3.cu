@@ -1,0 +1,605 @@
+// K5: fp32 storage, contraction on the 5th-generation tensor cores as three TF32 products.
+//
+// A TF32 operand keeps the sign, the 8 exponent bits and the upper 10 fraction bits of an fp32
+// word.  Every fp32 input is split as x = hi + lo with hi = x with its 13 low fraction bits
+// cleared (a TF32 number) and lo = x - hi (exact in fp32; the tensor core keeps its upper 11
+// significant bits).  Then
+//     x w  =  hi_x hi_w + hi_x lo_w + lo_x hi_w  +  O(2^-21 |x w|),
+// three kind::tf32 MMAs per k-step accumulated in fp32 in TMEM, small terms first.  The split
+// error is two to three orders of magnitude inside the 1e-4 budget of the fp32 path, at about a
+// third of the TF32 tensor rate, which is still several times the FFMA rate of the SMs.
+//
+// The tensor core adds into its fp32 accumulator with truncation, not rounding to nearest, so
+// an accumulator that takes thousands of MMAs drifts towards zero by about 2^-24 per MMA
+// (measured: 7e-5 relative at K = 4096 with all 1536 MMAs of an output in one accumulator --
+// too close to the 1e-4 budget, and beyond it for same-sign data or larger K).  Therefore an
+// accumulator only ever takes one chunk of K (128 by default: 48 MMAs); the epilogue warps
+// drain each finished chunk out of TMEM and add it, rounding to nearest, to a running sum they
+// keep in registers (128 per thread), while the MMAs of the next chunk fill the other TMEM
+// buffer.  The drift is then bounded by the chunk length whatever K is.
+//
+// Persistent CTA pairs (cluster of two, tcgen05.mma.cta_group::2, 256x256 output tile per pair),
+// 512 threads per CTA in four warpgroups with different register shares (setmaxnreg):
+//   warp 0        TMA producer: this CTA's 128 rows of the X tile and its 128-row half of the W
+//                 tile (128x32 fp32 each, 128-byte swizzle) into a 3-stage ring, completion
+//                 counted on the CTA's own "full" barrier;
+//   warps 12..15  splitters: wait for the stage, compute lo of every raw word and write it at the
+//                 same offset of a second buffer (so the swizzle needs no thought; the raw words
+//                 themselves serve as hi, see K5_WRITE_HI), then fence towards the async proxy and
+//                 arrive on the leader's "split" barrier;
+//   warp 1        MMA issuer (leader CTA, one elected thread): waits for both CTAs' splitters,
+//                 issues 3 x 4 MMAs (256x256x8) per stage, commits to the "empty" barriers of
+//                 both CTAs and, per chunk of K, to the "accumulator full" barriers;
+//   warps 4..11   epilogue, two groups of four warps, one 128-column half of the tile each
+//                 (thread <-> output row): per chunk, tcgen05.ld and add to the running sum; after
+//                 the last chunk the sum goes back to TMEM and a rolled loop applies bias,
+//                 accurate fp32 activation and scale, then stores Y as float4, or forms the row
+//                 sum / max / (max, sum exp) / mean chain with per-half-tile partials folded by
+//                 the last group to arrive at a row strip.
+// TMEM holds two 128x256 fp32 accumulators per CTA, used alternately by the chunks, so the
+// draining (and the epilogue of tile i) overlaps the MMAs that follow.  No load is multicast;
+// every software wait is bounded.
+#include <cstdlib>
+
+#include "common.cuh"
+#include "plan.h"
+#include "sm100_ptx.cuh"
+
+namespace forge {
+
+constexpr int K5_BM = 128, K5_BN = 256, K5_BK = 32;     // rows per CTA, columns per pair tile, fp32 per 128-byte row
+constexpr int K5_STAGES = 3;
+constexpr int K5_THREADS = 512;
+constexpr int K5_EPI_WARP0 = 4, K5_SPLIT_WARP0 = 12;
+constexpr int K5_EPI_THREADS = 128;
+constexpr int K5_SPLIT_WARPS = 4, K5_SPLIT_THREADS = 32 * K5_SPLIT_WARPS;
+constexpr uint32_t K5_A_BYTES = K5_BM * K5_BK * 4;                 // 16 KiB: 128 rows of X
+constexpr uint32_t K5_B_BYTES = (K5_BN / 2) * K5_BK * 4;           // 16 KiB: this CTA's half of the W tile
+constexpr uint32_t K5_RAW_BYTES = K5_A_BYTES + K5_B_BYTES;         // what TMA writes per stage
+constexpr uint32_t K5_STAGE_BYTES = 2 * K5_RAW_BYTES;              // raw/hi, then lo
+constexpr uint32_t K5_RING_BYTES = K5_STAGES * K5_STAGE_BYTES;     // 192 KiB
+constexpr uint32_t K5_TMEM_COLS = 512;
+constexpr int K5_GROUP_M = 8;       // 256-row units per rasterisation group
+constexpr int K5_CHUNK_KB = 4;      // ring stages (32 k each) accumulated in TMEM before the epilogue drains them
+// Register shares after setmaxnreg: the epilogue warpgroups hold a 128-value running sum per
+// thread; producer, issuer and splitters need little.  The sum of the shares must not exceed the
+// registers the CTA was launched with (checked on the host before the first launch).
+constexpr int K5_REGS_EPI = 184, K5_REGS_OTHER = 64;
+constexpr int K5_REGS_NEEDED = 256 * K5_REGS_EPI + 256 * K5_REGS_OTHER;
+// A kind::tf32 MMA reading a full fp32 word uses its upper 19 bits and ignores the 13 low
+// fraction bits (measured on B200: with an identity weight and inputs that run through all 8192
+// tail patterns the result is exact, which it would not be if the word were rounded), so the raw
+// tile serves as hi.  K5_WRITE_HI = 1 instead stores hi explicitly (words that are TF32 numbers
+// whatever the hardware does with low bits) at the price of a third more shared-memory traffic
+// in the splitters: 717 us instead of 615 us on a 4096^3 problem.
+#ifndef K5_WRITE_HI
+#define K5_WRITE_HI 0
+#endif
+
+struct K5Smem {
+    uint64_t full[K5_STAGES];       // TMA -> splitters (this CTA)
+    uint64_t split[K5_STAGES];      // splitters of both CTAs -> MMA issuer (leader's copy is used)
+    uint64_t empty[K5_STAGES];      // MMA -> TMA producer (each CTA)
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint32_t tmem_base;
+    int last_flag[2];
+    int abort_flag;
+    float bias[2][K5_BN];
+    float sub[2][K5_BN];            // mean chain: the vector subtracted before the row mean
+};
+constexpr size_t K5_SMEM_BYTES = 1024 + (size_t)K5_RING_BYTES + sizeof(K5Smem);
+
+struct K5Params {
+    const float *b;
+    const float *X;             // mean chain only: the residual input
+    const void *aux;            // mean chain: sub[N] (float); cross-entropy: target[M] (int32)
+    void *out;
+    int M, N, K;
+    Epilogue e;
+    float *partial;             // per half tile: [2*tiles_n][M] floats (float4 for the softmax statistics)
+    unsigned *counters;         // [tiles_m]
+    float *rowg;                // mean chain: gelu(mean) per row, [M]
+    unsigned *strips_done;      // mean chain: strips whose rowg values are published; only ever grows
+    unsigned strips_target;     // ... and the value it reaches when this run's strips are all done
+    int *status;
+    int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
+    int group_m;
+    int chunk_kb;               // stages per TMEM accumulation chunk
+};
+
+template <int N> __device__ __forceinline__ void k5_reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void k5_reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+__device__ __forceinline__ void k5_tile_coords(int t, int units_m, int tiles_n, int group_m, int &um, int &tn)
+{
+    const int group_size = group_m * tiles_n;
+    const int g = t / group_size, r = t - g * group_size;
+    const int gm = min(group_m, units_m - g * group_m);
+    um = g * group_m + r % gm;
+    tn = r / gm;
+}
+
+__device__ __forceinline__ unsigned ld_acquire_gpu_u32(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void k5_epi_bar_sync(int g) { asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(K5_EPI_THREADS) : "memory"); }
+
+__global__ void __launch_bounds__(K5_THREADS, 1)
+k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const K5Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    K5Smem &s = *reinterpret_cast<K5Smem *>(tiles + (size_t)K5_RING_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();         // position in the pair; 0 leads
+    const int units_m = (p.tiles_m + 1) / 2;              // 256-row units
+    const int total_units = units_m * p.tiles_n;
+    const int first_unit = (int)(blockIdx.x >> 1), unit_stride = (int)(gridDim.x >> 1);
+    bool ok = true;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < K5_STAGES; ++i) {
+            ptx::mbar_init(&s.full[i], 1);
+            ptx::mbar_init(&s.split[i], 2 * K5_SPLIT_WARPS);
+            ptx::mbar_init(&s.empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) { ptx::mbar_init(&s.acc_full[i], 1); ptx::mbar_init(&s.acc_empty[i], 16); }
+        s.abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmX);
+        ptx::prefetch_tmap(&tmW);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(&s.tmem_base, K5_TMEM_COLS);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::cluster_sync_all();             // the peer's barriers exist before anything signals them
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = s.tmem_base;
+
+    if (warp < K5_EPI_WARP0) {
+        k5_reg_dec<K5_REGS_OTHER>();          // warpgroup 0: producer, issuer and two idle warps
+        if (warp == 0) {
+            // ---------------- TMA producer ----------------
+            if (ptx::elect_one()) {
+                int stage = 0;
+                uint32_t phase = 0;
+                for (int t = first_unit; t < total_units && ok; t += unit_stride) {
+                    int um, tn;
+                    k5_tile_coords(t, units_m, p.tiles_n, p.group_m, um, tn);
+                    const int tm = 2 * um + (int)rank;
+                    for (int kb = 0; kb < p.num_kb; ++kb) {
+                        if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
+                        uint8_t *a = tiles + (size_t)stage * K5_STAGE_BYTES;
+                        ptx::mbar_expect_tx(&s.full[stage], K5_RAW_BYTES);      // rows past M or N are zero fill and count in full
+                        ptx::tma_load_2d(a, &tmX, &s.full[stage], kb * K5_BK, tm * K5_BM);
+                        ptx::tma_load_2d(a + K5_A_BYTES, &tmW, &s.full[stage], kb * K5_BK, tn * K5_BN + (int)rank * (K5_BN / 2));
+                        if (++stage == K5_STAGES) { stage = 0; phase ^= 1; }
+                    }
+                }
+            }
+        } else if (warp == 1) {
+            // ---------------- MMA issuer (leader) ----------------
+            if (rank == 0 && ptx::elect_one()) {
+                const uint32_t idesc = ptx::idesc_tf32_f32(2 * K5_BM, K5_BN);
+                int stage = 0, acc = 0;
+                uint32_t phase = 0, acc_phase = 0;
+                for (int t = first_unit; t < total_units && ok; t += unit_stride) {
+                    for (int kb0 = 0; kb0 < p.num_kb && ok; kb0 += p.chunk_kb) {
+                        // one chunk of K into one TMEM buffer, starting from zero
+                        if (!ptx::mbar_wait(&s.acc_empty[acc], acc_phase ^ 1, p.status, SITE_ACC_EMPTY)) { ok = false; break; }
+                        ptx::tc_fence_after();
+                        const uint32_t d_tmem = tmem_base + (uint32_t)acc * K5_BN;
+                        const int kb1 = min(kb0 + p.chunk_kb, p.num_kb);
+                        for (int kb = kb0; kb < kb1; ++kb) {
+                            if (!ptx::mbar_wait(&s.split[stage], phase, p.status, SITE_SPLIT)) { ok = false; break; }
+                            ptx::tc_fence_after();
+                            const uint8_t *a = tiles + (size_t)stage * K5_STAGE_BYTES;
+                            const uint64_t a_hi = ptx::smem_desc_k_sw128(a), b_hi = ptx::smem_desc_k_sw128(a + K5_A_BYTES);
+                            const uint64_t a_lo = ptx::smem_desc_k_sw128(a + K5_RAW_BYTES);
+                            const uint64_t b_lo = ptx::smem_desc_k_sw128(a + K5_RAW_BYTES + K5_A_BYTES);
+#pragma unroll
+                            for (int k = 0; k < K5_BK / 8; ++k) {     // 8 fp32 = 32 bytes = 2 descriptor units
+                                ptx::umma_tf32_pair(d_tmem, a_lo + 2 * k, b_hi + 2 * k, idesc, (kb != kb0) | (k != 0));
+                                ptx::umma_tf32_pair(d_tmem, a_hi + 2 * k, b_lo + 2 * k, idesc, 1);
+                                ptx::umma_tf32_pair(d_tmem, a_hi + 2 * k, b_hi + 2 * k, idesc, 1);
+                            }
+                            ptx::umma_commit_pair(&s.empty[stage], 3);
+                            if (++stage == K5_STAGES) { stage = 0; phase ^= 1; }
+                        }
+                        if (!ok) break;
+                        ptx::umma_commit_pair(&s.acc_full[acc], 3);
+                        if ((acc ^= 1) == 0) acc_phase ^= 1;
+                    }
+                }
+            }
+        }
+    } else if (warp >= K5_SPLIT_WARP0) {
+        // ---------------- splitters ----------------
+        k5_reg_dec<K5_REGS_OTHER>();
+        const int st = threadIdx.x - 32 * K5_SPLIT_WARP0;   // 0..127
+        const uint32_t split_bar[K5_STAGES] = {ptx::mapa_u32(ptx::smem_u32(&s.split[0]), 0),
+                                               ptx::mapa_u32(ptx::smem_u32(&s.split[1]), 0),
+                                               ptx::mapa_u32(ptx::smem_u32(&s.split[2]), 0)};      // the leader's
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int t = first_unit; t < total_units && ok; t += unit_stride) {
+            for (int kb = 0; kb < p.num_kb; ++kb) {
+                if (!ptx::mbar_wait(&s.full[stage], phase, p.status, SITE_TMA_FULL)) { ok = false; break; }
+                float4 *raw = reinterpret_cast<float4 *>(tiles + (size_t)stage * K5_STAGE_BYTES);
+                float4 *lo = reinterpret_cast<float4 *>(tiles + (size_t)stage * K5_STAGE_BYTES + K5_RAW_BYTES);
+                constexpr int PER_THREAD = K5_RAW_BYTES / 16 / K5_SPLIT_THREADS;       // 16 float4
+#pragma unroll 4
+                for (int i = 0; i < PER_THREAD; ++i) {
+                    const int idx = i * K5_SPLIT_THREADS + st;
+                    const float4 v = raw[idx];
+                    float4 hi;
+                    hi.x = __uint_as_float(__float_as_uint(v.x) & 0xffffe000u);
+                    hi.y = __uint_as_float(__float_as_uint(v.y) & 0xffffe000u);
+                    hi.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
+                    hi.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
+                    lo[idx] = make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);
+                    if (K5_WRITE_HI) raw[idx] = hi;
+                }
+                ptx::fence_proxy_async_smem();      // these writes are read by the tensor core (async proxy)
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(split_bar[stage]);
+                if (++stage == K5_STAGES) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else {
+        // ---------------- epilogue ----------------
+        k5_reg_inc<K5_REGS_EPI>();
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int h = (warp - K5_EPI_WARP0) >> 2;     // column half
+        const int et = (threadIdx.x - 32 * K5_EPI_WARP0) & (K5_EPI_THREADS - 1);
+        constexpr int HALF = K5_BN / 2, CHUNKS = HALF / 32;
+        const int parts = 2 * p.tiles_n;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        const int red = p.e.red;
+        const bool chain = red == FORGE_RED_MEAN_GELU_RESIDUAL;
+        const bool lse = red == FORGE_RED_LOGSUMEXP || red == FORGE_RED_CROSS_ENTROPY;
+        const bool fold = red == FORGE_RED_SUM || red == FORGE_RED_MAX || chain;
+        const bool add = red != FORGE_RED_MAX;
+        const uint32_t acc_empty_addr[2] = {ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[0]), 0),
+                                            ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[1]), 0)};     // the leader's
+        int tile_parity = 0;            // bias / sub staging alternates per tile (a slow thread may still read the last one)
+        for (int t = first_unit; t < total_units; t += unit_stride, tile_parity ^= 1) {
+            int um, tn;
+            k5_tile_coords(t, units_m, p.tiles_n, p.group_m, um, tn);
+            const int tm = 2 * um + (int)rank;
+            const int m0 = tm * K5_BM, n0 = tn * K5_BN + h * HALF;
+            const int part = 2 * tn + h;
+            float *sb = s.bias[tile_parity] + h * HALF, *ss = s.sub[tile_parity] + h * HALF;
+            {
+                const bool in = n0 + et < p.N;
+                sb[et] = (p.e.has_bias && in) ? __ldg(p.b + n0 + et) : 0.f;
+                if (chain) ss[et] = (in && p.aux) ? __ldg(reinterpret_cast<const float *>(p.aux) + n0 + et) : 0.f;
+            }
+            const int row = m0 + q * 32 + lane;
+            const uint32_t lane_addr = tmem_base + (uint32_t)(h * HALF) + ((uint32_t)(q * 32) << 16);
+            // ---- chunks of K: drain every finished accumulator into the running sum (round to nearest) ----
+            float sum[HALF];
+#pragma unroll
+            for (int j = 0; j < HALF; ++j) sum[j] = 0.f;
+            const int nchunks = (p.num_kb + p.chunk_kb - 1) / p.chunk_kb;
+            for (int ch = 0; ch < nchunks; ++ch) {
+                // the give-up decision must be taken by all threads of the group together
+                if (!ptx::mbar_wait(&s.acc_full[acc], acc_phase, p.status, SITE_ACC_FULL)) s.abort_flag = 1;
+                k5_epi_bar_sync(h);
+                if (*(volatile int *)&s.abort_flag) { ok = false; break; }
+                ptx::tc_fence_after();
+                const bool last = ch == nchunks - 1;
+                if (m0 < p.M && nchunks > 1) {
+                    const uint32_t ca = lane_addr + (uint32_t)(acc * K5_BN);
+#pragma unroll
+                    for (int c = 0; c < CHUNKS; ++c) {
+                        uint32_t r[32];
+                        ptx::tmem_ld_32x32(ca + c * 32, r);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            sum[c * 32 + j] += __uint_as_float(r[j]);
+                            r[j] = __float_as_uint(sum[c * 32 + j]);
+                        }
+                        if (last) ptx::tmem_st_32x32(ca + c * 32, r);     // the total goes back for the rolled loop below
+                    }
+                    if (last) ptx::tmem_st_wait();
+                }
+                if (last) break;                 // this buffer is released after the final pass
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
+                if ((acc ^= 1) == 0) acc_phase ^= 1;
+            }
+            if (!ok) break;
+
+            const uint32_t taddr = lane_addr + (uint32_t)(acc * K5_BN);
+            if (m0 >= p.M) {
+                // this CTA's half of the last pair tile lies past M: nothing to publish
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
+                if ((acc ^= 1) == 0) acc_phase ^= 1;
+                continue;
+            }
+
+            const int tgt = (red == FORGE_RED_CROSS_ENTROPY && row < p.M) ? __ldg(reinterpret_cast<const int *>(p.aux) + row) : -1;
+            float acc_red = add ? 0.f : -INFINITY;        // row sum / max of this half tile
+            float mx = -INFINITY, se = 0.f, tl = 0.f;     // (max, sum exp) and the target's logit
+#pragma unroll 1
+            for (int c = 0; c < CHUNKS; ++c) {
+                const int col0 = n0 + c * 32;
+                if (col0 >= p.N) break;
+                uint32_t r[32];
+                ptx::tmem_ld_32x32(taddr + c * 32, r);
+                ptx::tmem_ld_wait();
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
+                apply_act_array<true>(p.e.act, v, p.e.scale);
+                const int nv = min(32, p.N - col0);
+                if (lse) {
+                    float cm = -INFINITY;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) cm = j < nv ? fmaxf(cm, v[j]) : cm;
+                    const float nm = fmaxf(mx, cm);
+                    float cs = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) cs += j < nv ? expf(v[j] - nm) : 0.f;
+                    se = (mx == -INFINITY ? 0.f : se * expf(mx - nm)) + cs;
+                    mx = nm;
+                    if (tgt >= col0 && tgt < col0 + 32) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) tl = (col0 + j == tgt) ? v[j] : tl;
+                    }
+                } else if (fold) {
+                    if (chain) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] -= ss[c * 32 + j];
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < nv) acc_red = add ? acc_red + v[j] : fmaxf(acc_red, v[j]);
+                } else if (row < p.M) {
+                    float *dst = reinterpret_cast<float *>(p.out) + (size_t)row * p.N + col0;      // N % 4 == 0: 16-byte aligned
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (i * 4 < nv) *reinterpret_cast<float4 *>(dst + i * 4) = make_float4(v[i * 4], v[i * 4 + 1], v[i * 4 + 2], v[i * 4 + 3]);
+                }
+            }
+            // accumulator drained: hand the TMEM buffer back to the MMA warp
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
+
+            if (lse || fold) {
+                // per-part row partials; the group that arrives last at the strip folds them in part order
+                float4 *part4 = reinterpret_cast<float4 *>(p.partial);
+                if (row < p.M) {
+                    if (lse) part4[(size_t)part * p.M + row] = make_float4(mx, se, tl, 0.f);
+                    else p.partial[(size_t)part * p.M + row] = acc_red;
+                }
+                __threadfence();
+                k5_epi_bar_sync(h);
+                if (et == 0) s.last_flag[h] = (atomicAdd(&p.counters[tm], 1u) == (unsigned)(parts - 1));
+                k5_epi_bar_sync(h);
+                if (s.last_flag[h]) {
+                    __threadfence();
+                    float *out = reinterpret_cast<float *>(p.out);
+                    if (row < p.M) {
+                        if (lse) {
+                            float4 f = __ldcg(&part4[row]);
+                            mx = f.x; se = f.y; tl = f.z;
+                            for (int i = 1; i < parts; ++i) {
+                                f = __ldcg(&part4[(size_t)i * p.M + row]);
+                                lse_merge<true>(mx, se, f.x, f.y);
+                                tl += f.z;
+                            }
+                            out[row] = mx + logf(se) - tl;
+                        } else {
+                            float v = __ldcg(&p.partial[row]);
+                            for (int i = 1; i < parts; ++i) {
+                                const float o = __ldcg(&p.partial[(size_t)i * p.M + row]);
+                                v = add ? v + o : fmaxf(v, o);
+                            }
+                            if (chain) p.rowg[row] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)p.N);
+                            else out[row] = v;
+                        }
+                    }
+                    if (et == 0) p.counters[tm] = 0u;
+                    if (chain) {
+                        // the strip's gelu(mean) values are published; the rows are written at the end, by the whole grid
+                        __threadfence();
+                        k5_epi_bar_sync(h);
+                        if (et == 0) atomicAdd(p.strips_done, 1u);
+                    }
+                }
+            }
+            if ((acc ^= 1) == 0) acc_phase ^= 1;
+        }
+    }
+
+    // ---------------- mean chain: residual rows ----------------
+    // Y[m, :] = X[m, :] + gelu(mean)[m] for all of Y ([M,K]) once every strip has published its
+    // values: 2 M K floats of traffic spread over the whole grid instead of being written strip by
+    // strip by whichever epilogue group finished a strip (which stalled that CTA's pipeline).
+    // CTAs wait on one another here: the launch is cooperative (all CTAs resident) and the wait is bounded.
+    if (p.e.red == FORGE_RED_MEAN_GELU_RESIDUAL) {
+        if (threadIdx.x == 0) {
+            uint64_t t0 = 0;
+            for (uint32_t it = 1; (int)(ld_acquire_gpu_u32(p.strips_done) - p.strips_target) < 0; ++it) {
+                __nanosleep(200);
+                if ((it & 0x3f) == 0) {
+                    if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
+                    const uint64_t now = ptx::globaltimer_ns();
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > ptx::kWaitBudgetNs) {
+                        report_timeout(p.status, SITE_ARRIVAL, (int)blockIdx.x);
+                        s.abort_flag = 1;
+                        break;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (!*(volatile int *)&s.abort_flag) {
+            const size_t k4 = (size_t)(p.K >> 2), total = (size_t)p.M * k4;
+            const float4 *X4 = reinterpret_cast<const float4 *>(p.X);
+            float4 *Y4 = reinterpret_cast<float4 *>(p.out);
+            for (size_t e = (size_t)blockIdx.x * K5_THREADS + threadIdx.x; e < total; e += (size_t)gridDim.x * K5_THREADS) {
+                const float g = __ldcg(p.rowg + e / k4);
+                float4 x = __ldg(X4 + e);
+                x.x += g; x.y += g; x.z += g; x.w += g;
+                Y4[e] = x;
+            }
+        } else {
+            ok = false;
+        }
+    }
+
+    // ---------------- teardown ----------------
+    if (!ok) __nanosleep(200000);      // give-up path: let copies and MMAs already in flight land
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::cluster_sync_all();           // the peer no longer reads this CTA's shared memory or signals its barriers
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc_pair(tmem_base, K5_TMEM_COLS);
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+forge_status_t k5_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
+{
+    if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    // 16-byte row pitch for TMA (K) and for the float4 stores of Y (N); pairs need two SMs;
+    // the row statistics of LayerNorm are not implemented on this kernel
+    if (d.K % 4 != 0 || d.N % 4 != 0 || sm_count < 2 || d.red == FORGE_RED_LAYERNORM) return FORGE_ERR_UNSUPPORTED;
+    const int64_t tiles_m = (d.M + K5_BM - 1) / K5_BM, tiles_n = (d.N + K5_BN - 1) / K5_BN;
+    if (tiles_m * tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    info->kernel = FORGE_KERNEL_F32_TF32X3;
+    info->tile_m = 2 * K5_BM;
+    info->tile_n = K5_BN;
+    info->tile_k = K5_BK;
+    info->stages = K5_STAGES;
+    info->cluster = 2;
+    info->threads = K5_THREADS;
+    const int64_t units = ((tiles_m + 1) / 2) * tiles_n, clusters = sm_count / 2;
+    info->grid = 2 * (units < clusters ? units : clusters);
+    info->smem_bytes = (int64_t)K5_SMEM_BYTES;
+    const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;
+    const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL || lse;
+    wl->partial_floats = partials ? (lse ? 4 : 1) * 2 * (size_t)tiles_n * (size_t)d.M : 0;
+    wl->counters = partials ? (size_t)tiles_m : 0;
+    if (d.red == FORGE_RED_MEAN_GELU_RESIDUAL) {      // gelu(mean) per row after the partials; one more counter
+        wl->partial_floats += (size_t)d.M;
+        wl->counters += 1;
+    }
+    return FORGE_OK;
+}
+
+forge_status_t k5_setup(Handle &h)
+{
+    // setmaxnreg.inc waits until the registers it asks for are free: the shares must fit into what
+    // a CTA is launched with, or the kernel is never launched
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, k5_f32_tf32x3_kernel) != cudaSuccess || fa.numRegs * K5_THREADS < K5_REGS_NEEDED)
+        return FORGE_ERR_CUDA;
+    if (cudaFuncSetAttribute(k5_f32_tf32x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K5_SMEM_BYTES) != cudaSuccess)
+        return FORGE_ERR_CUDA;
+    if (h.d.red == FORGE_RED_MEAN_GELU_RESIDUAL) {
+        // the CTAs of the mean chain wait on one another: they must all be resident at once
+        int coop = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h.d.device) != cudaSuccess || !coop) return FORGE_ERR_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k5_f32_tf32x3_kernel, K5_THREADS, K5_SMEM_BYTES) != cudaSuccess ||
+            (int64_t)per_sm * h.sm_count < h.info.grid)
+            return FORGE_ERR_CUDA;
+    }
+    return FORGE_OK;
+}
+
+forge_status_t k5_launch(Handle &h, const RunArgs &a)
+{
+    const forge_fused_linear_desc_t &d = h.d;
+    forge_status_t st;
+    if (h.tmX_ptr != a.X) {
+        if ((st = encode_tmap_f32(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, K5_BM, K5_BK)) != FORGE_OK) return st;
+        h.tmX_ptr = a.X;
+    }
+    if (h.tmW_ptr != a.W) {
+        if ((st = encode_tmap_f32(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, K5_BN / 2, K5_BK)) != FORGE_OK) return st;
+        h.tmW_ptr = a.W;
+    }
+    K5Params p;
+    p.b = (const float *)a.b;
+    p.X = (const float *)a.X;
+    p.aux = a.gamma;
+    p.out = a.out;
+    p.M = (int)d.M;
+    p.N = (int)d.N;
+    p.K = (int)d.K;
+    p.e = Epilogue{(int)d.act, (int)d.red, d.scale, d.ln_eps, d.has_bias};
+    p.partial = h.ws.partial;
+    p.counters = h.ws.counters;
+    p.status = h.ws.status;
+    p.tiles_m = (int)((d.M + K5_BM - 1) / K5_BM);
+    p.rowg = nullptr;
+    p.strips_done = nullptr;
+    p.strips_target = 0;
+    const bool chain = d.red == FORGE_RED_MEAN_GELU_RESIDUAL;
+    if (chain) {
+        const size_t tiles_n = (size_t)((d.N + K5_BN - 1) / K5_BN);
+        p.rowg = h.ws.partial + 2 * tiles_n * (size_t)d.M;
+        p.strips_done = h.ws.counters + p.tiles_m;
+        h.run_gen += 1;                                      // the counter only ever grows: run r ends at r * tiles_m
+        p.strips_target = h.run_gen * (unsigned)p.tiles_m;
+    }
+    p.tiles_n = (int)((d.N + K5_BN - 1) / K5_BN);
+    p.num_kb = (int)((d.K + K5_BK - 1) / K5_BK);
+    {
+        static int env = -1;        // FORGE_K5_GROUP_M overrides the rasterisation group (tuning aid)
+        if (env < 0) {
+            const char *e = std::getenv("FORGE_K5_GROUP_M");
+            env = e ? std::atoi(e) : 0;
+        }
+        p.group_m = env > 0 ? env : K5_GROUP_M;
+    }
+    {
+        static int env = -1;        // FORGE_K5_CHUNK_KB overrides the accumulation chunk (32 k per unit; tuning aid)
+        if (env < 0) {
+            const char *e = std::getenv("FORGE_K5_CHUNK_KB");
+            env = e ? std::atoi(e) : 0;
+        }
+        p.chunk_kb = env > 0 ? env : K5_CHUNK_KB;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)h.info.grid);
+    cfg.blockDim = dim3(K5_THREADS);
+    cfg.dynamicSmemBytes = K5_SMEM_BYTES;
+    cfg.stream = a.stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (chain && cooperative_launch_enabled()) {
+        attr[1].id = cudaLaunchAttributeCooperative;
+        attr[1].val.cooperative = 1;
+        cfg.numAttrs = 2;
+    }
+    return cudaLaunchKernelEx(&cfg, k5_f32_tf32x3_kernel, h.tmX, h.tmW, p) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+}
+
+}  // namespace forge

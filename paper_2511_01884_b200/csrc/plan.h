@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstdlib>
+
 #include "../../include/forge.h"
 
 namespace forge {
@@ -24,6 +26,16 @@ struct Workspace {
     size_t bytes = 0;
 };
 
+struct Handle;
+constexpr int kHostPipeMaxBlocks = 8;
+struct HostPipeline {
+    cudaStream_t s_in = nullptr, s_run = nullptr, s_out = nullptr;
+    cudaEvent_t landed[kHostPipeMaxBlocks] = {}, computed[kHostPipeMaxBlocks] = {};
+    Handle *block = nullptr, *last = nullptr;      // child handles (last: nullptr if all blocks are equal)
+    int64_t block_rows = 0;
+    int blocks = 0;
+};
+
 struct Handle {
     forge_fused_linear_desc_t d;
     forge_plan_info_t info;
@@ -33,10 +45,27 @@ struct Handle {
     Workspace ws;
     // staging buffers of run_host()
     void *hX = nullptr, *hW = nullptr, *hb = nullptr, *hg = nullptr, *hbe = nullptr, *hout = nullptr;
+    // run_host() on a large problem walks X in blocks of rows so that the upload of block i+1, the
+    // kernel on block i and the download of block i-1 overlap: three streams, one event pair per
+    // block, and a child handle planned for a block's rows (plus one for a shorter last block).
+    HostPipeline *pipe = nullptr;
     // cached TMA descriptors (bf16 kernels): re-encoded only when a pointer changes
     CUtensorMap tmX, tmW, tmY;
     const void *tmX_ptr = nullptr, *tmW_ptr = nullptr, *tmY_ptr = nullptr;
 };
+
+// Kernels whose CTAs wait on one another are launched cooperatively (all CTAs resident at once).
+// FORGE_K4_COOPERATIVE=0 drops the attribute: profilers refuse cooperative cluster launches.  The
+// grids never exceed the SM count and every wait is bounded, so the worst case on a GPU that is
+// busy with other work is a reported time-out, not a hang.
+inline bool cooperative_launch_enabled()
+{
+    static const int v = [] {
+        const char *e = std::getenv("FORGE_K4_COOPERATIVE");
+        return e ? (std::atoi(e) != 0) : 1;
+    }();
+    return v != 0;
+}
 
 // Layout of the workspace (element counts) for a plan; filled by the planners.
 struct WorkspaceLayout {
@@ -62,10 +91,18 @@ forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
 forge_status_t k4_setup(Handle &h);
 forge_status_t k4_launch(Handle &h, const RunArgs &a);
 
+forge_status_t k5_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl);
+forge_status_t k5_setup(Handle &h);
+forge_status_t k5_launch(Handle &h, const RunArgs &a);
+
 // Encode a 2-D row-major tensor map [rows, cols] of 16-bit elements (bfloat16, or IEEE half if
 // f16 != 0) with a [box_rows, box_cols] box and the 128-byte shared-memory swizzle.  Host-only
 // driver call.
 forge_status_t encode_tmap_16(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
                               uint32_t box_rows, uint32_t box_cols, int f16);
+
+// The same for fp32 elements (box_cols = 32 gives the 128-byte rows of the swizzle).
+forge_status_t encode_tmap_f32(CUtensorMap *tm, const void *ptr, uint64_t rows, uint64_t cols,
+                               uint32_t box_rows, uint32_t box_cols);
 
 }  // namespace forge

@@ -37,7 +37,7 @@ def main() -> int:
         d["gamma"] = torch.from_numpy(np.ascontiguousarray(inp["target"], dtype=np.int32)).cuda()
     reduce = wl.out_cols == 0
     out = torch.empty((M,) if reduce else (M, wl.out_cols), device="cuda",
-                      dtype=torch.float32 if (reduce or wl.dtype == wk.F32) else torch.bfloat16)
+                      dtype=torch.float32 if (reduce or wl.dtype != wk.BF16) else torch.bfloat16)
     if wl.red == wk.RED_MEAN_GELU_RESIDUAL:
         d["gamma"] = d["sub"]          # the chain's subtract vector travels in the gamma slot
     op = B.FusedLinear(B.make_desc(M, wl.N, wl.K, wl.dtype, wl.act, wl.red, wl.scale, wl.ln_eps,

@@ -27,7 +27,7 @@ import numpy as np
 
 # Enumerations of the public C interface, restated as plain integers so that this module
 # depends on neither side.
-F32, BF16, F16 = 0, 1, 2
+F32, BF16, F16, F32_TF32X3 = 0, 1, 2, 3      # F32_TF32X3: fp32 storage, tensor-core arithmetic
 ACT_IDENTITY, ACT_RELU, ACT_GELU_ERF, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3, 4
 RED_NONE, RED_SUM, RED_MAX, RED_LAYERNORM, RED_MEAN_GELU_RESIDUAL, RED_LOGSUMEXP, RED_CROSS_ENTROPY = 0, 1, 2, 3, 4, 5, 6
 VECTOR_OUT = (RED_SUM, RED_MAX, RED_LOGSUMEXP, RED_CROSS_ENTROPY)      # reductions whose output is fp32 [M]
@@ -109,7 +109,7 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 
 def round_to_storage(x: np.ndarray, dtype: int) -> np.ndarray:
     """Return float32 values that are exactly representable in the storage dtype."""
-    if dtype == F32:
+    if dtype in (F32, F32_TF32X3):
         return np.ascontiguousarray(x, dtype=np.float32)
     if dtype == F16:          # IEEE half: numpy rounds to nearest even
         return np.ascontiguousarray(x, dtype=np.float32).astype(np.float16).astype(np.float32)
@@ -149,7 +149,7 @@ class Workload:
 
     @property
     def elem_bytes(self) -> int:
-        return 4 if self.dtype == F32 else 2
+        return 4 if self.dtype in (F32, F32_TF32X3) else 2
 
     @property
     def out_cols(self) -> int:
@@ -200,7 +200,8 @@ WORKLOADS: Dict[str, Workload] = {
 }
 
 
-# Workloads beyond the five configurations: the paper's own case-study chain (Appendix B.1).
+# Workloads beyond the five configurations: the paper's own case-study chain (Appendix B.1), the
+# loss of a classifier head, and C2 / the chain again with the contraction on the tensor cores.
 EXTRA_WORKLOADS: Dict[str, Workload] = {
     "n1": Workload("n1", F32, 4096, 4096, 4096, ACT_IDENTITY, RED_MEAN_GELU_RESIDUAL, 1.0, 0.0,
                    Dist("normal", 1.0), Dist("uniform", -1 / 64, 1 / 64), Dist("uniform", -0.1, 0.1),
@@ -209,7 +210,11 @@ EXTRA_WORKLOADS: Dict[str, Workload] = {
     "n2": Workload("n2", BF16, 8192, 32768, 4096, ACT_IDENTITY, RED_CROSS_ENTROPY, 1.0, 0.0,
                    Dist("normal", 1.0), Dist("normal", 0.02), Dist("normal", 0.02),
                    note="bf16, per-row cross-entropy over 32768 classes"),
+    "c2t": dataclasses.replace(WORKLOADS["c2"], name="c2t", dtype=F32_TF32X3,
+                               note="C2's tensors, contraction as three TF32 tensor-core products"),
 }
+EXTRA_WORKLOADS["n1t"] = dataclasses.replace(EXTRA_WORKLOADS["n1"], name="n1t", dtype=F32_TF32X3,
+                                             note="n1's tensors, contraction as three TF32 tensor-core products")
 
 
 def _draw(d: Dist, seed: int, stream: int, n: int) -> Optional[np.ndarray]:

@@ -14,7 +14,7 @@ from paper_2511_01884_b200 import binding as B
 from paper_2511_01884_b200 import workloads as wk
 
 # fp16 storage: output rounding is 2^-11, the approximate activations dominate (see the error budget in the design doc)
-TOL = {wk.F32: 1e-4, wk.BF16: 2e-2, wk.F16: 5e-3}
+TOL = {wk.F32: 1e-4, wk.BF16: 2e-2, wk.F16: 5e-3, wk.F32_TF32X3: 1e-4}
 
 
 def to_device(a, dtype):
@@ -46,7 +46,7 @@ def run_gpu(wl: wk.Workload, inp, check_status=True, op=None, repeats=1):
     if wl.out_cols == 0:
         out = torch.full((M,), float("nan"), dtype=torch.float32, device="cuda")
     else:
-        out = torch.full((M, wl.out_cols), float("nan"), dtype={wk.F32: torch.float32, wk.BF16: torch.bfloat16, wk.F16: torch.float16}[wl.dtype],
+        out = torch.full((M, wl.out_cols), float("nan"), dtype={wk.F32: torch.float32, wk.BF16: torch.bfloat16, wk.F16: torch.float16, wk.F32_TF32X3: torch.float32}[wl.dtype],
                          device="cuda")
     # the mean-gelu-residual chain takes its subtract vector, and the cross-entropy its int32
     # class indices, in the gamma slot of the interface

@@ -36,7 +36,7 @@ def test_no_vendor_gemm_library_is_linked():
 
 
 def test_enums_match_the_workload_module():
-    assert (B.FORGE_F32, B.FORGE_BF16, B.FORGE_F16) == (wk.F32, wk.BF16, wk.F16)
+    assert (B.FORGE_F32, B.FORGE_BF16, B.FORGE_F16, B.FORGE_F32_TF32X3) == (wk.F32, wk.BF16, wk.F16, wk.F32_TF32X3)
     assert (B.FORGE_ACT_IDENTITY, B.FORGE_ACT_RELU, B.FORGE_ACT_GELU_ERF, B.FORGE_ACT_GELU_TANH, B.FORGE_ACT_SILU) == \
            (wk.ACT_IDENTITY, wk.ACT_RELU, wk.ACT_GELU_ERF, wk.ACT_GELU_TANH, wk.ACT_SILU)
     assert (B.FORGE_RED_NONE, B.FORGE_RED_SUM, B.FORGE_RED_MAX, B.FORGE_RED_LAYERNORM) == \
@@ -45,7 +45,7 @@ def test_enums_match_the_workload_module():
 
 def test_invalid_descriptors():
     ok = dict(M=8, N=8, K=8, dtype=0, act=0, red=0)
-    for bad in (dict(M=0), dict(N=-1), dict(K=0), dict(dtype=3), dict(act=5), dict(act=-1), dict(red=7), dict(red=-1)):
+    for bad in (dict(M=0), dict(N=-1), dict(K=0), dict(dtype=4), dict(dtype=-1), dict(act=5), dict(act=-1), dict(red=7), dict(red=-1)):
         st, _ = B.forge_fused_linear_query_plan(B.make_desc(**{**ok, **bad}))
         assert st == B.FORGE_ERR_INVALID_ARG, bad
         st, h = B.forge_fused_linear_create(B.make_desc(**{**ok, **bad}))
@@ -68,6 +68,19 @@ def test_unsupported_is_reported_not_rerouted():
         assert st == B.FORGE_ERR_UNSUPPORTED
     st, _ = B.forge_fused_linear_query_plan(B.make_desc(64, 1025, 8, wk.F32, 0, wk.RED_LAYERNORM))
     assert st == B.FORGE_ERR_UNSUPPORTED
+    # fp32 on the tensor cores: 16-byte pitch of X, W and Y rows, no LayerNorm
+    for M, N, K, red in ((64, 64, 66, wk.RED_NONE), (64, 66, 64, wk.RED_NONE), (64, 64, 64, wk.RED_LAYERNORM)):
+        st, _ = B.forge_fused_linear_query_plan(B.make_desc(M, N, K, wk.F32_TF32X3, 0, red))
+        assert st == B.FORGE_ERR_UNSUPPORTED
+
+
+def test_tf32x3_plan():
+    wl = wk.EXTRA_WORKLOADS["c2t"]
+    st, p = B.forge_fused_linear_query_plan(B.make_desc(wl.M, wl.N, wl.K, wl.dtype, wl.act, wl.red, wl.scale))
+    assert st == B.FORGE_OK and p.kernel == B.FORGE_KERNEL_F32_TF32X3
+    assert (p.tile_m, p.tile_n, p.tile_k, p.cluster, p.grid, p.threads) == (256, 256, 32, 2, 148, 448)
+    assert p.smem_bytes <= 227 * 1024
+    assert "tf32" in B.kernel_name(B.FORGE_KERNEL_F32_TF32X3)
 
 
 def test_status_and_kernel_strings():

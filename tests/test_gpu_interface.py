@@ -85,6 +85,46 @@ def test_host_buffer_entry_point_matches_the_oracle(name):
     pu.assert_parity(wl, out.float().numpy().astype(np.float64), pu.run_oracle(wl, inp))
 
 
+@pytest.mark.parametrize("name", ["plain", "ln", "ce", "f32_sum", "f32_chain"])
+def test_host_entry_point_in_row_blocks_matches_the_oracle(name):
+    """Large X: the host entry point uploads, computes and downloads in blocks of rows on three
+    streams (here 4 blocks of 512 rows and a last one of 252)."""
+    import torch
+    M = 2300
+    wl = {"plain": wk.custom_workload("hp_plain", wk.BF16, M, 520, 2048, wk.ACT_SILU, wk.RED_NONE, w_std=0.03),
+          "ln": wk.custom_workload("hp_ln", wk.BF16, M, 520, 2048, wk.ACT_GELU_TANH, wk.RED_LAYERNORM, w_std=0.03),
+          "ce": wk.custom_workload("hp_ce", wk.BF16, M, 1032, 2048, wk.ACT_IDENTITY, wk.RED_CROSS_ENTROPY, w_std=0.03),
+          "f32_sum": wk.custom_workload("hp_sum", wk.F32, M, 300, 1024, wk.ACT_RELU, wk.RED_SUM),
+          "f32_chain": wk.custom_workload("hp_chain", wk.F32, M, 200, 1024, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL)}[name]
+    inp = wk.make_inputs(wl)
+
+    def host(a):
+        if a is None:
+            return None
+        t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
+        return (t.to(torch.bfloat16) if wl.dtype == wk.BF16 else t).pin_memory()
+    h = {k: host(v) for k, v in inp.items() if k != "target"}
+    aux = h["sub"] if wl.red == wk.RED_MEAN_GELU_RESIDUAL else h["gamma"]
+    if wl.red == wk.RED_CROSS_ENTROPY:
+        aux = torch.from_numpy(np.ascontiguousarray(inp["target"], dtype=np.int32)).pin_memory()
+    shape = (M,) if wl.out_cols == 0 else (M, wl.out_cols)
+    out = torch.full(shape, float("nan"), dtype=torch.float32 if (wl.out_cols == 0 or wl.dtype == wk.F32) else torch.bfloat16).pin_memory()
+    op = B.FusedLinear(pu.desc_of(wl))
+    for _ in range(2):
+        op.run_host(h["X"], h["W"], h["b"], aux, h["beta"], out)
+    op.check()
+    # the same handle's device entry point on the whole problem gives the same bits
+    dev = {k: (None if v is None else v.cuda()) for k, v in h.items()}
+    dout = torch.empty(shape, dtype=out.dtype, device="cuda")
+    op(dev["X"], dev["W"], dev["b"], None if aux is None else aux.cuda(), dev["beta"], dout)
+    torch.cuda.synchronize()
+    op.check()
+    op.close()
+    assert torch.equal(dout.cpu(), out)
+    rows = np.unique(np.concatenate([np.arange(0, M, 97), np.array([511, 512, 2047, 2048, M - 1])]))
+    pu.assert_parity(wl, out.float().numpy().astype(np.float64)[rows], pu.run_oracle(wl, inp, rows=rows))
+
+
 def test_runs_on_a_side_stream():
     import torch
     wl = wk.custom_workload("iface_stream", wk.BF16, 512, 512, 256, wk.ACT_SILU, wk.RED_SUM, w_std=0.05, seed=7)
