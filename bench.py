@@ -45,10 +45,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # from the ncu captures summarised under profiles/, keyed by workload, with the sha256 of the
 # kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
 NCU_TRAFFIC = {
-    "c2": {"bytes": 395_432_960, "sha": "cac102579ae7490f"},
-    "c3": {"bytes": 1_142_733_824, "sha": "fc05604e4ad9ee5c"},
-    "c4": {"bytes": 272_649_728, "sha": "2d971fa9a500e610"},
-    "c5": {"bytes": 281_256_960, "sha": "fc05604e4ad9ee5c"},
+    "c2": {"bytes": 549_508_608, "sha": "b4b97b469603ec83"},
+    "c3": {"bytes": 1_294_669_808, "sha": "2c86a6abc8b62959"},
+    "c4": {"bytes": 273_142_272, "sha": "6c195e10916ae16e"},
+    "c5": {"bytes": 305_444_864, "sha": "2c86a6abc8b62959"},
+    "c2t": {"bytes": 347_831_040, "sha": "cdb418cf86d3d76c"},
 }
 
 
