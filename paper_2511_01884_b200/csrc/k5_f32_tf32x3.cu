@@ -39,6 +39,13 @@
 // TMEM holds two 128x256 fp32 accumulators per CTA, used alternately by the chunks, so the
 // draining (and the epilogue of tile i) overlaps the MMAs that follow.  No load is multicast;
 // every software wait is bounded.
+//
+// Last, partly filled wave: when the tiles left over after the full waves are fewer than half the
+// clusters, each of them is cut along K into S parts that run on S clusters at once.  Parts 1..S-1
+// leave their running sums (the registers above) in a scratch area and count themselves in; part 0
+// waits for them (bounded), adds them to its own sum in part order and runs the epilogue.  Nothing
+// else changes: a part is just a tile with a shorter K range.  A 4096^3 problem (256 tiles on 74
+// clusters) takes 3.5 tile times instead of 4.
 #include <cstdlib>
 
 #include "common.cuh"
@@ -106,7 +113,50 @@ struct K5Params {
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     int group_m;
     int chunk_kb;               // stages per TMEM accumulation chunk
+    // K split of the last wave's tiles (tail_parts = 1: none)
+    int tail_parts;             // S
+    int tail_kb;                // k-blocks per part
+    float4 *tail_scratch;       // [tail tile][part - 1][rank][column half][32][128] float4
+    unsigned *tail_flags;       // [tail tile][rank][column half]; only ever grow
+    unsigned tail_target;       // value a flag reaches when parts 1..S-1 of this run have arrived
 };
+
+// One unit of work of a cluster: a pair tile and a range of k-blocks.  Cluster c takes the whole
+// tiles c, c + C, ... of the full waves and then at most one item of the last wave.
+struct K5Item {
+    int um, tn;                 // 256-row unit, 256-column tile
+    int kb_lo, kb_hi;           // k-blocks [kb_lo, kb_hi)
+    int part, tail;             // part of the K split (0 leads), index of the tile among the split ones (-1: whole tile)
+};
+
+__device__ __forceinline__ void k5_tile_coords(int t, int units_m, int tiles_n, int group_m, int &um, int &tn);
+
+__device__ __forceinline__ bool k5_item(const K5Params &p, int j, int cluster, int clusters, int units_m, K5Item &w)
+{
+    const int total = units_m * p.tiles_n, full = total / clusters, rest = total - full * clusters;
+    int t;
+    w.kb_lo = 0;
+    w.kb_hi = p.num_kb;
+    w.part = 0;
+    w.tail = -1;
+    if (j < full) {
+        t = j * clusters + cluster;
+    } else if (j == full && p.tail_parts <= 1) {
+        if (cluster >= rest) return false;
+        t = full * clusters + cluster;
+    } else if (j == full) {
+        if (cluster >= rest * p.tail_parts) return false;
+        w.tail = cluster / p.tail_parts;
+        w.part = cluster - w.tail * p.tail_parts;
+        t = full * clusters + w.tail;
+        w.kb_lo = w.part * p.tail_kb;
+        w.kb_hi = min(w.kb_lo + p.tail_kb, p.num_kb);
+    } else {
+        return false;
+    }
+    k5_tile_coords(t, units_m, p.tiles_n, p.group_m, w.um, w.tn);
+    return true;
+}
 
 template <int N> __device__ __forceinline__ void k5_reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void k5_reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -139,8 +189,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();         // position in the pair; 0 leads
     const int units_m = (p.tiles_m + 1) / 2;              // 256-row units
-    const int total_units = units_m * p.tiles_n;
-    const int first_unit = (int)(blockIdx.x >> 1), unit_stride = (int)(gridDim.x >> 1);
+    const int cluster = (int)(blockIdx.x >> 1), clusters = (int)(gridDim.x >> 1);
     bool ok = true;
 
     if (threadIdx.x == 0) {
@@ -172,11 +221,10 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             if (ptx::elect_one()) {
                 int stage = 0;
                 uint32_t phase = 0;
-                for (int t = first_unit; t < total_units && ok; t += unit_stride) {
-                    int um, tn;
-                    k5_tile_coords(t, units_m, p.tiles_n, p.group_m, um, tn);
-                    const int tm = 2 * um + (int)rank;
-                    for (int kb = 0; kb < p.num_kb; ++kb) {
+                K5Item w;
+                for (int j = 0; ok && k5_item(p, j, cluster, clusters, units_m, w); ++j) {
+                    const int tm = 2 * w.um + (int)rank, tn = w.tn;
+                    for (int kb = w.kb_lo; kb < w.kb_hi; ++kb) {
                         if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
                         uint8_t *a = tiles + (size_t)stage * K5_STAGE_BYTES;
                         ptx::mbar_expect_tx(&s.full[stage], K5_RAW_BYTES);      // rows past M or N are zero fill and count in full
@@ -192,13 +240,14 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const uint32_t idesc = ptx::idesc_tf32_f32(2 * K5_BM, K5_BN);
                 int stage = 0, acc = 0;
                 uint32_t phase = 0, acc_phase = 0;
-                for (int t = first_unit; t < total_units && ok; t += unit_stride) {
-                    for (int kb0 = 0; kb0 < p.num_kb && ok; kb0 += p.chunk_kb) {
+                K5Item w;
+                for (int j = 0; ok && k5_item(p, j, cluster, clusters, units_m, w); ++j) {
+                    for (int kb0 = w.kb_lo; kb0 < w.kb_hi && ok; kb0 += p.chunk_kb) {
                         // one chunk of K into one TMEM buffer, starting from zero
                         if (!ptx::mbar_wait(&s.acc_empty[acc], acc_phase ^ 1, p.status, SITE_ACC_EMPTY)) { ok = false; break; }
                         ptx::tc_fence_after();
                         const uint32_t d_tmem = tmem_base + (uint32_t)acc * K5_BN;
-                        const int kb1 = min(kb0 + p.chunk_kb, p.num_kb);
+                        const int kb1 = min(kb0 + p.chunk_kb, w.kb_hi);
                         for (int kb = kb0; kb < kb1; ++kb) {
                             if (!ptx::mbar_wait(&s.split[stage], phase, p.status, SITE_SPLIT)) { ok = false; break; }
                             ptx::tc_fence_after();
@@ -231,8 +280,9 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                                                ptx::mapa_u32(ptx::smem_u32(&s.split[2]), 0)};      // the leader's
         int stage = 0;
         uint32_t phase = 0;
-        for (int t = first_unit; t < total_units && ok; t += unit_stride) {
-            for (int kb = 0; kb < p.num_kb; ++kb) {
+        K5Item w;
+        for (int j = 0; ok && k5_item(p, j, cluster, clusters, units_m, w); ++j) {
+            for (int kb = w.kb_lo; kb < w.kb_hi; ++kb) {
                 if (!ptx::mbar_wait(&s.full[stage], phase, p.status, SITE_TMA_FULL)) { ok = false; break; }
                 float4 *raw = reinterpret_cast<float4 *>(tiles + (size_t)stage * K5_STAGE_BYTES);
                 float4 *lo = reinterpret_cast<float4 *>(tiles + (size_t)stage * K5_STAGE_BYTES + K5_RAW_BYTES);
@@ -273,10 +323,9 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         const uint32_t acc_empty_addr[2] = {ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[0]), 0),
                                             ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[1]), 0)};     // the leader's
         int tile_parity = 0;            // bias / sub staging alternates per tile (a slow thread may still read the last one)
-        for (int t = first_unit; t < total_units; t += unit_stride, tile_parity ^= 1) {
-            int um, tn;
-            k5_tile_coords(t, units_m, p.tiles_n, p.group_m, um, tn);
-            const int tm = 2 * um + (int)rank;
+        K5Item w;
+        for (int j = 0; k5_item(p, j, cluster, clusters, units_m, w); ++j, tile_parity ^= 1) {
+            const int tn = w.tn, tm = 2 * w.um + (int)rank;
             const int m0 = tm * K5_BM, n0 = tn * K5_BN + h * HALF;
             const int part = 2 * tn + h;
             float *sb = s.bias[tile_parity] + h * HALF, *ss = s.sub[tile_parity] + h * HALF;
@@ -291,7 +340,8 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             float sum[HALF];
 #pragma unroll
             for (int j = 0; j < HALF; ++j) sum[j] = 0.f;
-            const int nchunks = (p.num_kb + p.chunk_kb - 1) / p.chunk_kb;
+            const int nchunks = (w.kb_hi - w.kb_lo + p.chunk_kb - 1) / p.chunk_kb;
+            const bool split = w.tail >= 0;           // this item is one of S parts of a tile
             for (int ch = 0; ch < nchunks; ++ch) {
                 // the give-up decision must be taken by all threads of the group together
                 if (!ptx::mbar_wait(&s.acc_full[acc], acc_phase, p.status, SITE_ACC_FULL)) s.abort_flag = 1;
@@ -299,7 +349,8 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
                 ptx::tc_fence_after();
                 const bool last = ch == nchunks - 1;
-                if (m0 < p.M && nchunks > 1) {
+                if (m0 < p.M && (nchunks > 1 || split)) {
+                    const bool put_back = last && !split;      // a split tile's total is formed below
                     const uint32_t ca = lane_addr + (uint32_t)(acc * K5_BN);
 #pragma unroll
                     for (int c = 0; c < CHUNKS; ++c) {
@@ -311,9 +362,9 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                             sum[c * 32 + j] += __uint_as_float(r[j]);
                             r[j] = __float_as_uint(sum[c * 32 + j]);
                         }
-                        if (last) ptx::tmem_st_32x32(ca + c * 32, r);     // the total goes back for the rolled loop below
+                        if (put_back) ptx::tmem_st_32x32(ca + c * 32, r);     // the total goes back for the rolled loop below
                     }
-                    if (last) ptx::tmem_st_wait();
+                    if (put_back) ptx::tmem_st_wait();
                 }
                 if (last) break;                 // this buffer is released after the final pass
                 ptx::tc_fence_before();
@@ -324,6 +375,59 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             if (!ok) break;
 
             const uint32_t taddr = lane_addr + (uint32_t)(acc * K5_BN);
+            if (split && m0 < p.M) {
+                // ---- K split of a last-wave tile: parts 1.. hand their sums over, part 0 collects them ----
+                unsigned *flag = p.tail_flags + ((size_t)w.tail * 2 + rank) * 2 + h;
+                if (w.part > 0) {
+                    float4 *dst = p.tail_scratch + ((((size_t)w.tail * (p.tail_parts - 1) + (w.part - 1)) * 2 + rank) * 2 + h) * (32 * K5_EPI_THREADS);
+#pragma unroll
+                    for (int i = 0; i < HALF / 4; ++i)
+                        dst[i * K5_EPI_THREADS + et] = make_float4(sum[4 * i], sum[4 * i + 1], sum[4 * i + 2], sum[4 * i + 3]);
+                    __threadfence();
+                    k5_epi_bar_sync(h);
+                    if (et == 0) atomicAdd(flag, 1u);
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
+                    if ((acc ^= 1) == 0) acc_phase ^= 1;
+                    continue;
+                }
+                if (et == 0) {
+                    uint64_t t0 = 0;
+                    for (uint32_t it = 1; (int)(ld_acquire_gpu_u32(flag) - p.tail_target) < 0; ++it) {
+                        __nanosleep(100);
+                        if ((it & 0x3f) == 0) {
+                            if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
+                            const uint64_t now = ptx::globaltimer_ns();
+                            if (t0 == 0) t0 = now;
+                            else if (now - t0 > ptx::kWaitBudgetNs) {
+                                report_timeout(p.status, SITE_ARRIVAL, w.tail);
+                                s.abort_flag = 1;
+                                break;
+                            }
+                        }
+                    }
+                }
+                k5_epi_bar_sync(h);
+                if (*(volatile int *)&s.abort_flag) { ok = false; break; }
+                __threadfence();
+                for (int pp = 1; pp < p.tail_parts; ++pp) {
+                    const float4 *src = p.tail_scratch + ((((size_t)w.tail * (p.tail_parts - 1) + (pp - 1)) * 2 + rank) * 2 + h) * (32 * K5_EPI_THREADS);
+#pragma unroll
+                    for (int i = 0; i < HALF / 4; ++i) {
+                        const float4 o = __ldcg(src + i * K5_EPI_THREADS + et);
+                        sum[4 * i] += o.x; sum[4 * i + 1] += o.y; sum[4 * i + 2] += o.z; sum[4 * i + 3] += o.w;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < CHUNKS; ++c) {
+                    uint32_t r[32];
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) r[jj] = __float_as_uint(sum[c * 32 + jj]);
+                    ptx::tmem_st_32x32(taddr + c * 32, r);
+                }
+                ptx::tmem_st_wait();
+            }
             if (m0 >= p.M) {
                 // this CTA's half of the last pair tile lies past M: nothing to publish
                 ptx::tc_fence_before();
@@ -479,14 +583,65 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 }
 
 // ---- host side ---------------------------------------------------------------------------
+// Grid, K split of the last wave and workspace layout: a pure function of the problem and the SM count,
+// used by the planner and by the launcher.
+constexpr int K5_TAIL_MAX_PARTS = 8;      // bounds the scratch area and the serial adds of part 0
+constexpr int K5_TAIL_MIN_KB = 16;        // a part is worth its hand-over only with 512 k or more
+struct K5Layout {
+    int64_t tiles_m, tiles_n, units, clusters, grid;
+    int tail_parts, tail_kb, tail_tiles;
+    size_t fold_floats;       // per half tile row partials of the row reductions
+    size_t rowg_off;          // mean chain: gelu(mean) per row (float offset into the partial area)
+    size_t scratch_off;       // K split: hand-over area (float offset, multiple of 4)
+    size_t partial_floats;
+    size_t strips_done_idx, tail_flags_idx, counters;
+};
+
+static K5Layout k5_layout(const forge_fused_linear_desc_t &d, int sm_count)
+{
+    K5Layout L = {};
+    L.tiles_m = (d.M + K5_BM - 1) / K5_BM;
+    L.tiles_n = (d.N + K5_BN - 1) / K5_BN;
+    L.units = ((L.tiles_m + 1) / 2) * L.tiles_n;
+    L.clusters = sm_count / 2;
+    const int64_t full = L.units / L.clusters, rest = L.units % L.clusters;
+    const int num_kb = (int)((d.K + K5_BK - 1) / K5_BK);
+    static const int env = [] {          // FORGE_K5_TAIL_SPLIT=0: never cut the last wave's tiles along K
+        const char *e = std::getenv("FORGE_K5_TAIL_SPLIT");
+        return e ? std::atoi(e) : 1;
+    }();
+    int parts = 1;
+    if (env && rest > 0) {
+        int64_t s = L.clusters / rest;
+        if (s > K5_TAIL_MAX_PARTS) s = K5_TAIL_MAX_PARTS;
+        if (s > num_kb / K5_TAIL_MIN_KB) s = num_kb / K5_TAIL_MIN_KB;
+        parts = s < 1 ? 1 : (int)s;
+    }
+    L.tail_kb = (num_kb + parts - 1) / parts;
+    L.tail_parts = (num_kb + L.tail_kb - 1) / L.tail_kb;       // no empty part
+    L.tail_tiles = L.tail_parts > 1 ? (int)rest : 0;
+    L.grid = 2 * (full > 0 ? L.clusters : rest * L.tail_parts);
+    const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;
+    const bool chain = d.red == FORGE_RED_MEAN_GELU_RESIDUAL;
+    const bool fold = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || chain || lse;
+    L.fold_floats = fold ? (lse ? 4 : 1) * 2 * (size_t)L.tiles_n * (size_t)d.M : 0;
+    L.rowg_off = L.fold_floats;
+    L.scratch_off = (L.rowg_off + (chain ? (size_t)d.M : 0) + 3) / 4 * 4;
+    L.partial_floats = L.scratch_off + (size_t)L.tail_tiles * (L.tail_parts - 1) * 2 * 2 * (4 * 32 * K5_EPI_THREADS);
+    L.strips_done_idx = fold ? (size_t)L.tiles_m : 0;
+    L.tail_flags_idx = L.strips_done_idx + (chain ? 1 : 0);
+    L.counters = L.tail_flags_idx + (size_t)L.tail_tiles * 4;
+    return L;
+}
+
 forge_status_t k5_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
     if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
     // 16-byte row pitch for TMA (K) and for the float4 stores of Y (N); pairs need two SMs;
     // the row statistics of LayerNorm are not implemented on this kernel
     if (d.K % 4 != 0 || d.N % 4 != 0 || sm_count < 2 || d.red == FORGE_RED_LAYERNORM) return FORGE_ERR_UNSUPPORTED;
-    const int64_t tiles_m = (d.M + K5_BM - 1) / K5_BM, tiles_n = (d.N + K5_BN - 1) / K5_BN;
-    if (tiles_m * tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    const K5Layout L = k5_layout(d, sm_count);
+    if (L.tiles_m * L.tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_F32_TF32X3;
     info->tile_m = 2 * K5_BM;
     info->tile_n = K5_BN;
@@ -494,19 +649,15 @@ forge_status_t k5_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     info->stages = K5_STAGES;
     info->cluster = 2;
     info->threads = K5_THREADS;
-    const int64_t units = ((tiles_m + 1) / 2) * tiles_n, clusters = sm_count / 2;
-    info->grid = 2 * (units < clusters ? units : clusters);
+    info->grid = L.grid;
     info->smem_bytes = (int64_t)K5_SMEM_BYTES;
-    const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;
-    const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL || lse;
-    wl->partial_floats = partials ? (lse ? 4 : 1) * 2 * (size_t)tiles_n * (size_t)d.M : 0;
-    wl->counters = partials ? (size_t)tiles_m : 0;
-    if (d.red == FORGE_RED_MEAN_GELU_RESIDUAL) {      // gelu(mean) per row after the partials; one more counter
-        wl->partial_floats += (size_t)d.M;
-        wl->counters += 1;
-    }
+    wl->partial_floats = L.partial_floats;
+    wl->counters = L.counters;
     return FORGE_OK;
 }
+
+// CTAs wait on one another in the mean chain (all strips) and in the K split (part 0 on the others).
+static bool k5_ctas_wait(const Handle &h) { return h.d.red == FORGE_RED_MEAN_GELU_RESIDUAL || k5_layout(h.d, h.sm_count).tail_parts > 1; }
 
 forge_status_t k5_setup(Handle &h)
 {
@@ -517,8 +668,8 @@ forge_status_t k5_setup(Handle &h)
         return FORGE_ERR_CUDA;
     if (cudaFuncSetAttribute(k5_f32_tf32x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)K5_SMEM_BYTES) != cudaSuccess)
         return FORGE_ERR_CUDA;
-    if (h.d.red == FORGE_RED_MEAN_GELU_RESIDUAL) {
-        // the CTAs of the mean chain wait on one another: they must all be resident at once
+    if (k5_ctas_wait(h)) {
+        // CTAs that wait on one another must all be resident at once
         int coop = 0, per_sm = 0;
         if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h.d.device) != cudaSuccess || !coop) return FORGE_ERR_CUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k5_f32_tf32x3_kernel, K5_THREADS, K5_SMEM_BYTES) != cudaSuccess ||
@@ -553,17 +704,16 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
     p.counters = h.ws.counters;
     p.status = h.ws.status;
     p.tiles_m = (int)((d.M + K5_BM - 1) / K5_BM);
-    p.rowg = nullptr;
-    p.strips_done = nullptr;
-    p.strips_target = 0;
-    const bool chain = d.red == FORGE_RED_MEAN_GELU_RESIDUAL;
-    if (chain) {
-        const size_t tiles_n = (size_t)((d.N + K5_BN - 1) / K5_BN);
-        p.rowg = h.ws.partial + 2 * tiles_n * (size_t)d.M;
-        p.strips_done = h.ws.counters + p.tiles_m;
-        h.run_gen += 1;                                      // the counter only ever grows: run r ends at r * tiles_m
-        p.strips_target = h.run_gen * (unsigned)p.tiles_m;
-    }
+    const K5Layout L = k5_layout(d, h.sm_count);
+    h.run_gen += 1;                                          // the wait counters only ever grow: run r ends at r * arrivals per run
+    p.rowg = h.ws.partial + L.rowg_off;
+    p.strips_done = h.ws.counters + L.strips_done_idx;
+    p.strips_target = h.run_gen * (unsigned)p.tiles_m;
+    p.tail_parts = L.tail_parts;
+    p.tail_kb = L.tail_kb;
+    p.tail_scratch = reinterpret_cast<float4 *>(h.ws.partial + L.scratch_off);
+    p.tail_flags = h.ws.counters + L.tail_flags_idx;
+    p.tail_target = h.run_gen * (unsigned)(L.tail_parts - 1);
     p.tiles_n = (int)((d.N + K5_BN - 1) / K5_BN);
     p.num_kb = (int)((d.K + K5_BK - 1) / K5_BK);
     {
@@ -594,7 +744,7 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (chain && cooperative_launch_enabled()) {
+    if (k5_ctas_wait(h) && cooperative_launch_enabled()) {
         attr[1].id = cudaLaunchAttributeCooperative;
         attr[1].val.cooperative = 1;
         cfg.numAttrs = 2;

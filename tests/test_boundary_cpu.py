@@ -78,9 +78,18 @@ def test_tf32x3_plan():
     wl = wk.EXTRA_WORKLOADS["c2t"]
     st, p = B.forge_fused_linear_query_plan(B.make_desc(wl.M, wl.N, wl.K, wl.dtype, wl.act, wl.red, wl.scale))
     assert st == B.FORGE_OK and p.kernel == B.FORGE_KERNEL_F32_TF32X3
-    assert (p.tile_m, p.tile_n, p.tile_k, p.cluster, p.grid, p.threads) == (256, 256, 32, 2, 148, 448)
+    assert (p.tile_m, p.tile_n, p.tile_k, p.cluster, p.grid, p.threads) == (256, 256, 32, 2, 148, 512)
     assert p.smem_bytes <= 227 * 1024
     assert "tf32" in B.kernel_name(B.FORGE_KERNEL_F32_TF32X3)
+    # 256 pair tiles on 74 clusters leave 34 for the last wave: each is cut in two along K, and the
+    # workspace holds one 256x256 fp32 hand-over area per cut tile
+    assert p.workspace_bytes >= 34 * 256 * 256 * 4
+    # a problem of 4 tiles and 128 k-blocks is cut into 8 parts per tile: 32 clusters
+    st, p = B.forge_fused_linear_query_plan(B.make_desc(512, 512, 4096, wl.dtype, 0, 0))
+    assert st == B.FORGE_OK and p.grid == 2 * 4 * 8
+    # short K: no cut
+    st, p = B.forge_fused_linear_query_plan(B.make_desc(512, 512, 256, wl.dtype, 0, 0))
+    assert st == B.FORGE_OK and p.grid == 2 * 4
 
 
 def test_status_and_kernel_strings():

@@ -101,6 +101,23 @@ def test_repeatable_bits_no_bias_and_workspace_reuse():
     pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
 
 
+@pytest.mark.parametrize("red", [wk.RED_NONE, wk.RED_MAX, wk.RED_MEAN_GELU_RESIDUAL, wk.RED_CROSS_ENTROPY])
+def test_tiles_of_the_last_wave_cut_along_k(red):
+    """6 pair tiles on 74 clusters, K = 2048: every tile is computed by 4 clusters, a quarter of K each,
+    and put together by the first of them.  Same bits on every run (the arrival flags only ever grow)."""
+    wl = wk.custom_workload("t_ksplit", T, 300, 520, 2048, wk.ACT_GELU_ERF, red, seed=11)
+    st, plan = B.forge_fused_linear_query_plan(pu.desc_of(wl))
+    assert st == B.FORGE_OK and plan.grid == 2 * 6 * 4
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op, repeats=3)
+    b, _ = pu.run_gpu(wl, inp, op=op)
+    op.close()
+    assert np.array_equal(a, b)
+    e = pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
+    assert e <= 1e-5, e
+
+
 def test_agrees_with_the_ffma_kernel_far_inside_the_tolerance():
     base = wk.custom_workload("t_vs_ffma", wk.F32, 512, 768, 2048, wk.ACT_GELU_ERF, wk.RED_NONE, seed=5)
     inp = wk.make_inputs(base)
