@@ -459,7 +459,7 @@ def main():
                 d2 = device_tensors(w2, i2, torch)
                 op2 = make_op(w2, w2.M, local)
                 fl = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device="cuda") if w2.algorithmic_bytes < 130e6 else None
-                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50, "n1": 20, "n2": 10, "c2t": 50, "n1t": 50}[name]
+                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50, "n1": 20, "n2": 10, "c2t": 50, "n1t": 50, "n1b": 50}[name]
                 ms2 = time_steps(op2, d2, steps2, 3, torch, flush_buf=fl)
                 v2, u2 = unit_value(w2, ms2)
                 launches += steps2

@@ -57,7 +57,7 @@ typedef enum {
      * from the three products head*head, head*tail, tail*head (relative error of a product
      * about 2^-21), so the result stays within the 1e-4 of Section 2.2 with two orders of
      * magnitude to spare.  Needs K % 4 == 0, N % 4 == 0 and 16-byte aligned pointers; LayerNorm
-     * is not served (FORGE_ERR_UNSUPPORTED).                                              */
+     * needs ceil(N / 256) to be at most the number of CTA pairs of the grid (74 on a B200).  */
 } forge_dtype_t;
 
 typedef enum {

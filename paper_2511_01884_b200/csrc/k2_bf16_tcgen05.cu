@@ -55,7 +55,6 @@ struct K2Smem {
     uint32_t tmem_base;
     int last_flag[2];
     int abort_flag;
-    float rowg[2][K2_BM];       // mean chain: gelu(mean) of the strip's rows, per epilogue group
     float bias[2][K2_BN];
     float gamma[2][K2_BN];
     float beta[2][K2_BN];
@@ -77,6 +76,9 @@ struct K2Params {
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     int group_m;          // row units per rasterisation group
     unsigned ln_target;   // layernorm: counter value at which a strip is complete in this run
+    float *rowg;              // mean chain: gelu(mean) per row, [M]
+    unsigned *strips_done;    // mean chain: strips whose rowg values are published; only ever grows
+    unsigned strips_target;   // ... and the value it reaches when this run's strips are all done
 };
 
 template <bool LN>
@@ -504,33 +506,63 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                             const float o = __ldcg(&p.partial[(size_t)i * p.M + row]);
                             v = add ? v + o : fmaxf(v, o);
                         }
-                        if (chain) s.rowg[h][q * 32 + lane] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)p.N);
+                        if (chain) p.rowg[row] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)p.N);
                         else out[row] = v;
                     }
                     if (et == 0) p.counters[tm] = 0u;
                     if (chain) {
-                        // residual add for the strip's rows, by the whole group, 16 bytes per access:
-                        // Y[row, :] = X[row, :] + gelu(mean)   (Y is [M,K])
+                        // the strip's gelu(mean) values are published; the rows are written at the end, by the whole grid
+                        __threadfence();
                         epi_bar_sync(h);
-                        const int rows = min(K2_BM, p.M - m0), k8 = p.K >> 3;
-                        const uint4 *Xs = reinterpret_cast<const uint4 *>(p.X + (size_t)m0 * p.K);      // 16-bit elements
-                        uint4 *Ys = reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)m0 * p.K);
-                        for (int e = et; e < rows * k8; e += K2_EPI_THREADS) {
-                            const float g = s.rowg[h][e / k8];
-                            uint4 x = __ldg(Xs + e);
-                            uint32_t *w = reinterpret_cast<uint32_t *>(&x);
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                float lo, hi;
-                                ptx::unpack16x2(w[i], p.f16, lo, hi);
-                                w[i] = ptx::pack16x2(lo + g, hi + g, p.f16);
-                            }
-                            Ys[e] = x;
-                        }
+                        if (et == 0) atomicAdd(p.strips_done, 1u);
                     }
                 }
             }
             if ((acc ^= 1) == 0) acc_phase ^= 1;
+        }
+    }
+
+    // ---------------- mean chain: residual rows ----------------
+    // Y[m, :] = X[m, :] + gelu(mean)[m] for all of Y ([M,K]) once every strip has published its
+    // values, spread over the whole grid, 16 bytes per access (a strip written by the epilogue group
+    // that finished it would stall that CTA's pipeline for the duration).  CTAs wait on one another
+    // here: the launch is cooperative (all CTAs resident) and the wait is bounded.
+    if (!LN && p.e.red == FORGE_RED_MEAN_GELU_RESIDUAL) {
+        if (threadIdx.x == 0) {
+            uint64_t t0 = 0;
+            for (uint32_t it = 1; (int)(ld_acquire_u32(p.strips_done) - p.strips_target) < 0; ++it) {
+                __nanosleep(200);
+                if ((it & 0x3f) == 0) {
+                    if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
+                    const uint64_t now = ptx::globaltimer_ns();
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > ptx::kWaitBudgetNs) {
+                        report_timeout(p.status, SITE_ARRIVAL, (int)blockIdx.x);
+                        s.abort_flag = 1;
+                        break;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (!*(volatile int *)&s.abort_flag) {
+            const size_t k8 = (size_t)(p.K >> 3), total = (size_t)p.M * k8;
+            const uint4 *X8 = reinterpret_cast<const uint4 *>(p.X);
+            uint4 *Y8 = reinterpret_cast<uint4 *>(p.out);
+            for (size_t e = (size_t)blockIdx.x * K2_THREADS + threadIdx.x; e < total; e += (size_t)gridDim.x * K2_THREADS) {
+                const float g = __ldcg(p.rowg + e / k8);
+                uint4 x = __ldg(X8 + e);
+                uint32_t *w = reinterpret_cast<uint32_t *>(&x);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float lo, hi;
+                    ptx::unpack16x2(w[i], p.f16, lo, hi);
+                    w[i] = ptx::pack16x2(lo + g, hi + g, p.f16);
+                }
+                Y8[e] = x;
+            }
+        } else {
+            ok = false;
         }
     }
 
@@ -583,6 +615,10 @@ forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL || lse;   // one per row and half tile
     wl->partial_floats = partials ? (lse ? 4 : 1) * 2 * (size_t)tiles_n * (size_t)d.M : 0;
     wl->counters = partials ? (size_t)tiles_m : 0;
+    if (d.red == FORGE_RED_MEAN_GELU_RESIDUAL) {      // gelu(mean) per row after the partials; one more counter
+        wl->partial_floats += (size_t)d.M;
+        wl->counters += 1;
+    }
     return FORGE_OK;
 }
 
@@ -593,7 +629,26 @@ static forge_status_t k2_prepare()
                                 (int)K2_SMEM_BYTES) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
 }
 
-forge_status_t k2_setup(Handle &h) { return h.info.cluster == 2 ? k2_prepare<false, true>() : k2_prepare<false, false>(); }
+// Kernels whose CTAs wait on one another (LayerNorm strips, the mean chain's residual phase) need the
+// whole grid resident at once.
+template <bool LN, bool PAIR>
+static forge_status_t k2_check_residency(const Handle &h)
+{
+    int coop = 0, per_sm = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h.d.device) != cudaSuccess || !coop) return FORGE_ERR_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2_bf16_tcgen05_kernel<LN, PAIR>, K2_THREADS, K2_SMEM_BYTES) != cudaSuccess ||
+        (int64_t)per_sm * h.sm_count < h.info.grid)
+        return FORGE_ERR_CUDA;
+    return FORGE_OK;
+}
+
+forge_status_t k2_setup(Handle &h)
+{
+    const bool pair = h.info.cluster == 2;
+    if ((pair ? k2_prepare<false, true>() : k2_prepare<false, false>()) != FORGE_OK) return FORGE_ERR_CUDA;
+    if (h.d.red != FORGE_RED_MEAN_GELU_RESIDUAL) return FORGE_OK;
+    return pair ? k2_check_residency<false, true>(h) : k2_check_residency<false, false>(h);
+}
 
 forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
@@ -612,12 +667,7 @@ forge_status_t k4_setup(Handle &h)
 {
     const bool pair = h.info.cluster == 2;
     if ((pair ? k2_prepare<true, true>() : k2_prepare<true, false>()) != FORGE_OK) return FORGE_ERR_CUDA;
-    int coop = 0, per_sm = 0;
-    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h.d.device) != cudaSuccess || !coop) return FORGE_ERR_CUDA;
-    const cudaError_t e = pair ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2_bf16_tcgen05_kernel<true, true>, K2_THREADS, K2_SMEM_BYTES)
-                               : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2_bf16_tcgen05_kernel<true, false>, K2_THREADS, K2_SMEM_BYTES);
-    if (e != cudaSuccess || (int64_t)per_sm * h.sm_count < h.info.grid) return FORGE_ERR_CUDA;
-    return FORGE_OK;
+    return pair ? k2_check_residency<true, true>(h) : k2_check_residency<true, false>(h);
 }
 
 template <bool LN, bool PAIR>
@@ -637,16 +687,8 @@ static forge_status_t k2_launch_t(const Handle &h, const K2Params &p, cudaStream
         attr[n].val.clusterDim.z = 1;
         ++n;
     }
-    // CTAs wait on one another: a cooperative launch guarantees that all of them are resident.
-    // FORGE_K4_COOPERATIVE=0 drops the attribute (profilers refuse cooperative cluster launches);
-    // the grid never exceeds the SM count, and every wait is bounded, so the worst case on a GPU
-    // that is busy with other work is a reported time-out, not a hang.
-    static int coop = -1;
-    if (coop < 0) {
-        const char *e = std::getenv("FORGE_K4_COOPERATIVE");
-        coop = e ? (std::atoi(e) != 0) : 1;
-    }
-    if (LN && coop) {
+    // CTAs that wait on one another: a cooperative launch guarantees that all of them are resident
+    if ((LN || p.e.red == FORGE_RED_MEAN_GELU_RESIDUAL) && cooperative_launch_enabled()) {
         attr[n].id = cudaLaunchAttributeCooperative;
         attr[n].val.cooperative = 1;
         ++n;
@@ -694,6 +736,15 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
             env = e ? std::atoi(e) : 0;
         }
         p.group_m = env > 0 ? env : (pair ? K2_GROUP_M / 2 : K2_GROUP_M);      // 2048 rows either way
+    }
+    p.rowg = nullptr;
+    p.strips_done = nullptr;
+    p.strips_target = 0;
+    if (d.red == FORGE_RED_MEAN_GELU_RESIDUAL) {
+        p.rowg = h.ws.partial + 2 * (size_t)p.tiles_n * (size_t)d.M;
+        p.strips_done = h.ws.counters + p.tiles_m;
+        h.run_gen += 1;                                      // the counter only ever grows: run r ends at r * tiles_m
+        p.strips_target = h.run_gen * (unsigned)p.tiles_m;
     }
     if (!ln) return pair ? k2_launch_t<false, true>(h, p, a.stream) : k2_launch_t<false, false>(h, p, a.stream);
     // Strip counters only ever grow: run r completes a strip at r * 2 * tiles_n arrivals (half tiles).

@@ -93,14 +93,17 @@ struct K5Smem {
     int last_flag[2];
     int abort_flag;
     float bias[2][K5_BN];
-    float sub[2][K5_BN];            // mean chain: the vector subtracted before the row mean
+    float sub[2][K5_BN];            // mean chain: the vector subtracted before the row mean; LayerNorm: gamma
+    float beta[2][K5_BN];           // LayerNorm: beta
 };
 constexpr size_t K5_SMEM_BYTES = 1024 + (size_t)K5_RING_BYTES + sizeof(K5Smem);
 
 struct K5Params {
     const float *b;
     const float *X;             // mean chain only: the residual input
-    const void *aux;            // mean chain: sub[N] (float); cross-entropy: target[M] (int32)
+    const void *aux;            // mean chain: sub[N] (float); cross-entropy: target[M] (int32); LayerNorm: gamma[N]
+    const float *beta;          // LayerNorm
+    unsigned ln_target;         // LayerNorm: value a strip's counter reaches when all its half tiles of this run are in
     void *out;
     int M, N, K;
     Epilogue e;
@@ -163,6 +166,11 @@ template <int N> __device__ __forceinline__ void k5_reg_inc() { asm volatile("se
 
 __device__ __forceinline__ void k5_tile_coords(int t, int units_m, int tiles_n, int group_m, int &um, int &tn)
 {
+    if (group_m <= 0) {          // LayerNorm: the N-tiles of a row strip are neighbours in the schedule
+        um = t / tiles_n;
+        tn = t - um * tiles_n;
+        return;
+    }
     const int group_size = group_m * tiles_n;
     const int g = t / group_size, r = t - g * group_size;
     const int gm = min(group_m, units_m - g * group_m);
@@ -317,6 +325,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         uint32_t acc_phase = 0;
         const int red = p.e.red;
         const bool chain = red == FORGE_RED_MEAN_GELU_RESIDUAL;
+        const bool ln = red == FORGE_RED_LAYERNORM;
         const bool lse = red == FORGE_RED_LOGSUMEXP || red == FORGE_RED_CROSS_ENTROPY;
         const bool fold = red == FORGE_RED_SUM || red == FORGE_RED_MAX || chain;
         const bool add = red != FORGE_RED_MAX;
@@ -333,6 +342,10 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 const bool in = n0 + et < p.N;
                 sb[et] = (p.e.has_bias && in) ? __ldg(p.b + n0 + et) : 0.f;
                 if (chain) ss[et] = (in && p.aux) ? __ldg(reinterpret_cast<const float *>(p.aux) + n0 + et) : 0.f;
+                if (ln) {
+                    ss[et] = in ? __ldg(reinterpret_cast<const float *>(p.aux) + n0 + et) : 0.f;
+                    s.beta[tile_parity][h * HALF + et] = in ? __ldg(p.beta + n0 + et) : 0.f;
+                }
             }
             const int row = m0 + q * 32 + lane;
             const uint32_t lane_addr = tmem_base + (uint32_t)(h * HALF) + ((uint32_t)(q * 32) << 16);
@@ -430,6 +443,116 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             }
             if (m0 >= p.M) {
                 // this CTA's half of the last pair tile lies past M: nothing to publish
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
+                if ((acc ^= 1) == 0) acc_phase ^= 1;
+                continue;
+            }
+
+            if (ln) {
+                // ---- LayerNorm over N: row statistics merged across the half tiles of the strip ----
+                // sweep 1: activated values back to TMEM, (n, mean, M2) of this half tile by 32-column chunks
+                const float *sbe = s.beta[tile_parity] + h * HALF;
+                RowStat rs{0.f, 0.f, 0.f};
+#pragma unroll 1
+                for (int c = 0; c < CHUNKS; ++c) {
+                    const int col0 = n0 + c * 32;
+                    if (col0 >= p.N) break;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(taddr + c * 32, r);
+                    ptx::tmem_ld_wait();
+                    float v[32];
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) v[jj] = __uint_as_float(r[jj]) + sb[c * 32 + jj];
+                    apply_act_array<true>(p.e.act, v, p.e.scale);
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) r[jj] = __float_as_uint(v[jj]);
+                    ptx::tmem_st_32x32(taddr + c * 32, r);
+                    const int nv = min(32, p.N - col0);
+                    RowStat cs;
+                    cs.n = (float)nv;
+                    float csum = 0.f;
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) csum += jj < nv ? v[jj] : 0.f;
+                    cs.mean = csum / cs.n;
+                    cs.m2 = 0.f;
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) {
+                        const float dlt = jj < nv ? v[jj] - cs.mean : 0.f;
+                        cs.m2 = fmaf(dlt, dlt, cs.m2);
+                    }
+                    rs = merge_stat(rs, cs);
+                }
+                ptx::tmem_st_wait();
+                float4 *stats = reinterpret_cast<float4 *>(p.partial);
+                if (row < p.M) stats[(size_t)part * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
+                // publish, then wait (bounded) for the other half tiles of the strip
+                __threadfence();
+                k5_epi_bar_sync(h);
+                if (et == 0) {
+                    atomicAdd(&p.counters[tm], 1u);
+                    uint64_t t0 = 0;
+                    for (uint32_t it = 1; (int)(ld_acquire_gpu_u32(&p.counters[tm]) - p.ln_target) < 0; ++it) {
+                        if ((it & 0xff) == 0) {
+                            if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
+                            const uint64_t now = ptx::globaltimer_ns();
+                            if (t0 == 0) t0 = now;
+                            else if (now - t0 > ptx::kWaitBudgetNs) {
+                                report_timeout(p.status, SITE_ARRIVAL, tm);
+                                s.abort_flag = 1;
+                                break;
+                            }
+                        }
+                    }
+                }
+                k5_epi_bar_sync(h);
+                if (*(volatile int *)&s.abort_flag) { ok = false; break; }
+                __threadfence();
+                // the strip's parts combined in part order: mean = sum n_i mean_i / sum n_i, M2 = sum (M2_i + n_i (mean_i - mean)^2)
+                float rstd = 0.f, shift = 0.f;
+                if (row < p.M) {
+                    float cnt = 0.f, wsum = 0.f;
+                    for (int i = 0; i < parts; ++i) {
+                        const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
+                        cnt += o.x;
+                        wsum = fmaf(o.x, o.y, wsum);
+                    }
+                    const float mean = wsum / cnt;
+                    float m2 = 0.f;
+                    for (int i = 0; i < parts; ++i) {
+                        const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
+                        const float dm = o.y - mean;
+                        m2 += fmaf(o.x * dm, dm, o.z);
+                    }
+                    rstd = 1.0f / sqrtf(m2 / cnt + p.e.eps);
+                    shift = -mean * rstd;
+                }
+                // sweep 2: normalise out of TMEM and store
+#pragma unroll 1
+                for (int c = 0; c < CHUNKS; ++c) {
+                    const int col0 = n0 + c * 32;
+                    if (col0 >= p.N) break;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(taddr + c * 32, r);
+                    ptx::tmem_ld_wait();
+                    if (row < p.M) {
+                        const int nv = min(32, p.N - col0);
+                        float *dst = reinterpret_cast<float *>(p.out) + (size_t)row * p.N + col0;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            if (i * 4 < nv) {
+                                float y[4];
+#pragma unroll
+                                for (int jj = 0; jj < 4; ++jj) {
+                                    const int cc = c * 32 + i * 4 + jj;
+                                    y[jj] = fmaf(fmaf(__uint_as_float(r[i * 4 + jj]), rstd, shift), ss[cc], sbe[cc]);
+                                }
+                                *reinterpret_cast<float4 *>(dst + i * 4) = make_float4(y[0], y[1], y[2], y[3]);
+                            }
+                        }
+                    }
+                }
                 ptx::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
@@ -610,8 +733,9 @@ static K5Layout k5_layout(const forge_fused_linear_desc_t &d, int sm_count)
         const char *e = std::getenv("FORGE_K5_TAIL_SPLIT");
         return e ? std::atoi(e) : 1;
     }();
+    const bool ln = d.red == FORGE_RED_LAYERNORM;
     int parts = 1;
-    if (env && rest > 0) {
+    if (env && rest > 0 && !ln) {        // LayerNorm: a tile already waits for its strip; no second dependency
         int64_t s = L.clusters / rest;
         if (s > K5_TAIL_MAX_PARTS) s = K5_TAIL_MAX_PARTS;
         if (s > num_kb / K5_TAIL_MIN_KB) s = num_kb / K5_TAIL_MIN_KB;
@@ -623,8 +747,8 @@ static K5Layout k5_layout(const forge_fused_linear_desc_t &d, int sm_count)
     L.grid = 2 * (full > 0 ? L.clusters : rest * L.tail_parts);
     const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;
     const bool chain = d.red == FORGE_RED_MEAN_GELU_RESIDUAL;
-    const bool fold = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || chain || lse;
-    L.fold_floats = fold ? (lse ? 4 : 1) * 2 * (size_t)L.tiles_n * (size_t)d.M : 0;
+    const bool fold = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || chain || lse || ln;
+    L.fold_floats = fold ? ((lse || ln) ? 4 : 1) * 2 * (size_t)L.tiles_n * (size_t)d.M : 0;
     L.rowg_off = L.fold_floats;
     L.scratch_off = (L.rowg_off + (chain ? (size_t)d.M : 0) + 3) / 4 * 4;
     L.partial_floats = L.scratch_off + (size_t)L.tail_tiles * (L.tail_parts - 1) * 2 * 2 * (4 * 32 * K5_EPI_THREADS);
@@ -637,11 +761,12 @@ static K5Layout k5_layout(const forge_fused_linear_desc_t &d, int sm_count)
 forge_status_t k5_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
     if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
-    // 16-byte row pitch for TMA (K) and for the float4 stores of Y (N); pairs need two SMs;
-    // the row statistics of LayerNorm are not implemented on this kernel
-    if (d.K % 4 != 0 || d.N % 4 != 0 || sm_count < 2 || d.red == FORGE_RED_LAYERNORM) return FORGE_ERR_UNSUPPORTED;
+    // 16-byte row pitch for TMA (K) and for the float4 stores of Y (N); pairs need two SMs
+    if (d.K % 4 != 0 || d.N % 4 != 0 || sm_count < 2) return FORGE_ERR_UNSUPPORTED;
     const K5Layout L = k5_layout(d, sm_count);
     if (L.tiles_m * L.tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
+    // LayerNorm: the tiles of a strip wait for one another, so they must all be resident at once
+    if (d.red == FORGE_RED_LAYERNORM && L.tiles_n > L.clusters) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_F32_TF32X3;
     info->tile_m = 2 * K5_BM;
     info->tile_n = K5_BN;
@@ -657,7 +782,10 @@ forge_status_t k5_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
 }
 
 // CTAs wait on one another in the mean chain (all strips) and in the K split (part 0 on the others).
-static bool k5_ctas_wait(const Handle &h) { return h.d.red == FORGE_RED_MEAN_GELU_RESIDUAL || k5_layout(h.d, h.sm_count).tail_parts > 1; }
+static bool k5_ctas_wait(const Handle &h)
+{
+    return h.d.red == FORGE_RED_MEAN_GELU_RESIDUAL || h.d.red == FORGE_RED_LAYERNORM || k5_layout(h.d, h.sm_count).tail_parts > 1;
+}
 
 forge_status_t k5_setup(Handle &h)
 {
@@ -691,7 +819,7 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
         if ((st = encode_tmap_f32(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, K5_BN / 2, K5_BK)) != FORGE_OK) return st;
         h.tmW_ptr = a.W;
     }
-    K5Params p;
+    K5Params p = {};
     p.b = (const float *)a.b;
     p.X = (const float *)a.X;
     p.aux = a.gamma;
@@ -714,6 +842,8 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
     p.tail_scratch = reinterpret_cast<float4 *>(h.ws.partial + L.scratch_off);
     p.tail_flags = h.ws.counters + L.tail_flags_idx;
     p.tail_target = h.run_gen * (unsigned)(L.tail_parts - 1);
+    p.beta = (const float *)a.beta;
+    p.ln_target = h.run_gen * 2u * (unsigned)L.tiles_n;      // strip counters only ever grow under LayerNorm
     p.tiles_n = (int)((d.N + K5_BN - 1) / K5_BN);
     p.num_kb = (int)((d.K + K5_BK - 1) / K5_BK);
     {
@@ -722,7 +852,7 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
             const char *e = std::getenv("FORGE_K5_GROUP_M");
             env = e ? std::atoi(e) : 0;
         }
-        p.group_m = env > 0 ? env : K5_GROUP_M;
+        p.group_m = d.red == FORGE_RED_LAYERNORM ? 0 : (env > 0 ? env : K5_GROUP_M);
     }
     {
         static int env = -1;        // FORGE_K5_CHUNK_KB overrides the accumulation chunk (32 k per unit; tuning aid)

@@ -210,6 +210,9 @@ EXTRA_WORKLOADS: Dict[str, Workload] = {
     "n2": Workload("n2", BF16, 8192, 32768, 4096, ACT_IDENTITY, RED_CROSS_ENTROPY, 1.0, 0.0,
                    Dist("normal", 1.0), Dist("normal", 0.02), Dist("normal", 0.02),
                    note="bf16, per-row cross-entropy over 32768 classes"),
+    "n1b": Workload("n1b", BF16, 8192, 8192, 8192, ACT_IDENTITY, RED_MEAN_GELU_RESIDUAL, 1.0, 0.0,
+                    Dist("normal", 1.0), Dist("normal", 0.02), Dist("normal", 0.02),
+                    note="bf16, subtract, row mean, GELU-erf, residual add", sub=Dist("uniform", -0.5, 0.5)),
     "c2t": dataclasses.replace(WORKLOADS["c2"], name="c2t", dtype=F32_TF32X3,
                                note="C2's tensors, contraction as three TF32 tensor-core products"),
 }

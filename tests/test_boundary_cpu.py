@@ -68,8 +68,8 @@ def test_unsupported_is_reported_not_rerouted():
         assert st == B.FORGE_ERR_UNSUPPORTED
     st, _ = B.forge_fused_linear_query_plan(B.make_desc(64, 1025, 8, wk.F32, 0, wk.RED_LAYERNORM))
     assert st == B.FORGE_ERR_UNSUPPORTED
-    # fp32 on the tensor cores: 16-byte pitch of X, W and Y rows, no LayerNorm
-    for M, N, K, red in ((64, 64, 66, wk.RED_NONE), (64, 66, 64, wk.RED_NONE), (64, 64, 64, wk.RED_LAYERNORM)):
+    # fp32 on the tensor cores: 16-byte pitch of X, W and Y rows; LayerNorm rows of at most 74 tiles
+    for M, N, K, red in ((64, 64, 66, wk.RED_NONE), (64, 66, 64, wk.RED_NONE), (64, 256 * 74 + 4, 64, wk.RED_LAYERNORM)):
         st, _ = B.forge_fused_linear_query_plan(B.make_desc(M, N, K, wk.F32_TF32X3, 0, red))
         assert st == B.FORGE_ERR_UNSUPPORTED
 

@@ -1,5 +1,7 @@
 """GPU parity of the fp32-storage path whose contraction runs on the tensor cores as three TF32
 products (head*head + head*tail + tail*head) against the CPU oracle, at the fp32 tolerance."""
+import dataclasses
+
 import numpy as np
 import pytest
 
@@ -12,7 +14,7 @@ pytestmark = pytest.mark.gpu
 
 T = wk.F32_TF32X3
 ACTS = [wk.ACT_IDENTITY, wk.ACT_RELU, wk.ACT_GELU_ERF, wk.ACT_GELU_TANH, wk.ACT_SILU]
-REDS = [wk.RED_NONE, wk.RED_SUM, wk.RED_MAX, wk.RED_MEAN_GELU_RESIDUAL, wk.RED_LOGSUMEXP, wk.RED_CROSS_ENTROPY]
+REDS = [wk.RED_NONE, wk.RED_SUM, wk.RED_MAX, wk.RED_LAYERNORM, wk.RED_MEAN_GELU_RESIDUAL, wk.RED_LOGSUMEXP, wk.RED_CROSS_ENTROPY]
 
 
 def test_identity_weight_reproduces_full_fp32_mantissas():
@@ -122,13 +124,39 @@ def test_agrees_with_the_ffma_kernel_far_inside_the_tolerance():
     base = wk.custom_workload("t_vs_ffma", wk.F32, 512, 768, 2048, wk.ACT_GELU_ERF, wk.RED_NONE, seed=5)
     inp = wk.make_inputs(base)
     f, pf = pu.run_gpu(base, inp)
-    import dataclasses
     t, pt = pu.run_gpu(dataclasses.replace(base, dtype=T), inp)
     assert pf["kernel"] == B.FORGE_KERNEL_F32_FFMA and pt["kernel"] == B.FORGE_KERNEL_F32_TF32X3
     assert pu.rel_err(t, f) <= 1e-5
 
 
+def test_layernorm_rows_wider_than_the_ffma_kernel_serves():
+    """N = 4096 (16 tiles per row strip, far beyond the 1024 of the FFMA kernel's cluster), many strips,
+    several launches on one handle (the strip counters only ever grow)."""
+    wl = wk.custom_workload("t_ln_wide", T, 1500, 4096, 256, wk.ACT_GELU_TANH, wk.RED_LAYERNORM, seed=6)
+    st, _ = B.forge_fused_linear_query_plan(pu.desc_of(dataclasses.replace(wl, dtype=wk.F32)))
+    assert st == B.FORGE_ERR_UNSUPPORTED
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op, repeats=3)
+    b, _ = pu.run_gpu(wl, inp, op=op)
+    op.close()
+    assert np.array_equal(a, b)
+    rows = wk.sample_rows(wl.M)
+    e = pu.assert_parity(wl, a[rows], pu.run_oracle(wl, inp, rows))
+    assert e <= 2e-5, e
+
+
+def test_layernorm_constant_rows_give_beta():
+    wl = wk.custom_workload("t_ln_const", T, 5, 520, 12, wk.ACT_RELU, wk.RED_LAYERNORM, seed=1)
+    inp = wk.make_inputs(wl)
+    inp["X"][:] = -np.abs(inp["X"])
+    inp["W"][:] = np.abs(inp["W"])
+    inp["b"][:] = -0.5                      # every pre-activation negative: ReLU output is all zero
+    g, _ = pu.run_gpu(wl, inp)
+    assert np.array_equal(g, np.tile(inp["beta"].astype(np.float64), (5, 1)))
+
+
 def test_what_the_kernel_does_not_serve_is_refused():
-    for M, N, K, red in [(64, 64, 66, wk.RED_NONE), (64, 66, 64, wk.RED_NONE), (64, 64, 64, wk.RED_LAYERNORM)]:
+    for M, N, K, red in [(64, 64, 66, wk.RED_NONE), (64, 66, 64, wk.RED_NONE), (64, 256 * 74 + 4, 64, wk.RED_LAYERNORM)]:
         st, _ = B.forge_fused_linear_query_plan(B.make_desc(M, N, K, T, 0, red))
         assert st == B.FORGE_ERR_UNSUPPORTED
