@@ -46,10 +46,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
 NCU_TRAFFIC = {
     "c2": {"bytes": 549_508_608, "sha": "b4b97b469603ec83"},
-    "c3": {"bytes": 1_294_669_808, "sha": "2c86a6abc8b62959"},
+    "c3": {"bytes": 1_215_054_288, "sha": "fb517b2a9e0efcbf"},
     "c4": {"bytes": 273_142_272, "sha": "6c195e10916ae16e"},
-    "c5": {"bytes": 305_444_864, "sha": "2c86a6abc8b62959"},
-    "c2t": {"bytes": 347_831_040, "sha": "cdb418cf86d3d76c"},
+    "c5": {"bytes": 299_930_368, "sha": "fb517b2a9e0efcbf"},
+    "c2t": {"bytes": 349_515_776, "sha": "23334c3c03030526"},
 }
 
 
