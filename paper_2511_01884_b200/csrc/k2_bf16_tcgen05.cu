@@ -76,6 +76,13 @@ struct K2Params {
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     int group_m;          // row units per rasterisation group
     unsigned ln_target;   // layernorm: counter value at which a strip is complete in this run
+    // K split of the last wave's tiles (tail_parts = 1: none)
+    int tail_parts;           // S
+    int tail_kb;              // k-blocks per part
+    float4 *tail_scratch;     // [tail tile][part - 1][rank][column half][32][128] float4: raw accumulators
+    unsigned *tail_flags;     // [tail tile][rank][column half]; only ever grow
+    unsigned tail_target;     // value a flag reaches when parts 1..S-1 of this run have arrived
+    int cooperative;          // host only: CTAs of this launch wait on one another
     float *rowg;              // mean chain: gelu(mean) per row, [M]
     unsigned *strips_done;    // mean chain: strips whose rowg values are published; only ever grows
     unsigned strips_target;   // ... and the value it reaches when this run's strips are all done
@@ -94,6 +101,47 @@ __device__ __forceinline__ void k2_tile_coords(int t, int tiles_m, int tiles_n, 
     const int gm = min(group_m, tiles_m - g * group_m);
     tm = g * group_m + r % gm;
     tn = r / gm;
+}
+
+// One unit of work of a CTA (or CTA pair): a tile and a range of k-blocks.  Unit c of C takes the whole
+// tiles c, c + C, ... of the full waves and then at most one item of the last wave.  When the tiles
+// left for the last wave are at most half the units, each is cut along K into S parts that run on S
+// units at once: parts 1..S-1 leave their raw accumulators in a scratch area and count themselves
+// in; part 0 waits for them (bounded), adds them into its accumulator in part order and runs the
+// epilogue.  The same cut lets a problem with fewer tiles than SMs (M <= 128 with a few thousand
+// columns, say) stream its weights with most of the GPU.
+struct K2Item {
+    int tm, tn;                 // row unit, 256-column tile
+    int kb_lo, kb_hi;           // k-blocks [kb_lo, kb_hi)
+    int part, tail;             // part of the K split (0 leads), index of the tile among the split ones (-1: whole tile)
+};
+
+template <bool LN>
+__device__ __forceinline__ bool k2_item(const K2Params &p, int j, int unit, int units, int unit_rows, K2Item &w)
+{
+    const int total = unit_rows * p.tiles_n, full = total / units, rest = total - full * units;
+    int t;
+    w.kb_lo = 0;
+    w.kb_hi = p.num_kb;
+    w.part = 0;
+    w.tail = -1;
+    if (j < full) {
+        t = j * units + unit;
+    } else if (j == full && p.tail_parts <= 1) {
+        if (unit >= rest) return false;
+        t = full * units + unit;
+    } else if (j == full) {
+        if (unit >= rest * p.tail_parts) return false;
+        w.tail = unit / p.tail_parts;
+        w.part = unit - w.tail * p.tail_parts;
+        t = full * units + w.tail;
+        w.kb_lo = w.part * p.tail_kb;
+        w.kb_hi = min(w.kb_lo + p.tail_kb, p.num_kb);
+    } else {
+        return false;
+    }
+    k2_tile_coords<LN>(t, unit_rows, p.tiles_n, p.group_m, w.tm, w.tn);
+    return true;
 }
 
 // named barrier of epilogue group g (ids 1 and 2; 0 is __syncthreads)
@@ -128,9 +176,8 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
     const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;        // position in the pair; 0 leads
     // work units: tiles (one CTA each) or 256-row pair tiles (one cluster each)
     const int unit_rows = PAIR ? (p.tiles_m + 1) / 2 : p.tiles_m;
-    const int total_tiles = unit_rows * p.tiles_n;
-    const int first_unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-    const int unit_stride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // this CTA's (pair's) place among ...
+    const int units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;        // ... the units that share the work
     bool ok = true;
 
     if (threadIdx.x == 0) {
@@ -161,11 +208,10 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         if (ptx::elect_one()) {
             int stage = 0;
             uint32_t phase = 0;
-            for (int t = first_unit; t < total_tiles && ok; t += unit_stride) {
-                int tm, tn;
-                k2_tile_coords<LN>(t, unit_rows, p.tiles_n, p.group_m, tm, tn);
-                if (PAIR) tm = 2 * tm + (int)rank;
-                for (int kb = 0; kb < p.num_kb; ++kb) {
+            K2Item w;
+            for (int j = 0; ok && k2_item<LN>(p, j, unit, units, unit_rows, w); ++j) {
+                const int tm = PAIR ? 2 * w.tm + (int)rank : w.tm, tn = w.tn;
+                for (int kb = w.kb_lo; kb < w.kb_hi; ++kb) {
                     if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
                     uint8_t *a = tiles + (size_t)stage * STAGE_BYTES;
                     if (PAIR) {
@@ -190,11 +236,12 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             const uint32_t idesc = ptx::idesc_16_f32(PAIR ? 2 * K2_BM : K2_BM, K2_BN, p.f16);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
-            for (int t = first_unit; t < total_tiles && ok; t += unit_stride) {
+            K2Item w;
+            for (int j = 0; ok && k2_item<LN>(p, j, unit, units, unit_rows, w); ++j) {
                 if (!ptx::mbar_wait(&s.acc_empty[acc], acc_phase ^ 1, p.status, SITE_ACC_EMPTY)) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * K2_BN;
-                for (int kb = 0; kb < p.num_kb; ++kb) {
+                for (int kb = w.kb_lo; kb < w.kb_hi; ++kb) {
                     if (!ptx::mbar_wait(&s.full[stage], phase, p.status, SITE_TMA_FULL)) { ok = false; break; }
                     ptx::tc_fence_after();
                     const uint8_t *a = tiles + (size_t)stage * STAGE_BYTES;
@@ -202,8 +249,8 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                     const uint64_t bdesc = ptx::smem_desc_k_sw128(a + K2_A_BYTES);
 #pragma unroll
                     for (int k = 0; k < K2_BK / 16; ++k) {     // 16 bf16 = 32 bytes = 2 descriptor units
-                        if (PAIR) ptx::umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
-                        else ptx::umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                        if (PAIR) ptx::umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb != w.kb_lo) | (k != 0));
+                        else ptx::umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb != w.kb_lo) | (k != 0));
                     }
                     if (PAIR) ptx::umma_commit_pair(&s.empty[stage], 3);
                     else ptx::umma_commit(&s.empty[stage]);
@@ -231,10 +278,9 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         const bool add = p.e.red != FORGE_RED_MAX;
         const uint32_t acc_empty_addr[2] = {ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[0]), 0),
                                             ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[1]), 0)};   // the leader's (PAIR)
-        for (int t = first_unit; t < total_tiles; t += unit_stride) {
-            int tm, tn;
-            k2_tile_coords<LN>(t, unit_rows, p.tiles_n, p.group_m, tm, tn);
-            if (PAIR) tm = 2 * tm + (int)rank;
+        K2Item w;
+        for (int j = 0; k2_item<LN>(p, j, unit, units, unit_rows, w); ++j) {
+            const int tm = PAIR ? 2 * w.tm + (int)rank : w.tm, tn = w.tn;
             const int m0 = tm * K2_BM, n0 = tn * K2_BN + h * HALF;
             const int part = 2 * tn + h;
             float *sb = s.bias[acc] + h * HALF, *sg = s.gamma[acc] + h * HALF, *sbe = s.beta[acc] + h * HALF;
@@ -264,6 +310,71 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
                 if ((acc ^= 1) == 0) acc_phase ^= 1;
                 continue;
+            }
+
+            if (!LN && w.tail >= 0 && m0 < p.M) {
+                // ---- K split of a last-wave tile: parts 1.. hand their accumulators over, part 0 collects them ----
+                unsigned *flag = p.tail_flags + ((size_t)w.tail * 2 + rank) * 2 + h;
+                const size_t slot = 32 * K2_EPI_THREADS;        // float4 per (tile, part, rank, half)
+                if (w.part > 0) {
+                    float4 *dst = p.tail_scratch + ((((size_t)w.tail * (p.tail_parts - 1) + (w.part - 1)) * 2 + rank) * 2 + h) * slot;
+#pragma unroll 1
+                    for (int c = 0; c < CHUNKS; ++c) {
+                        uint32_t r[32];
+                        ptx::tmem_ld_32x32(taddr + c * 32, r);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            dst[(c * 8 + i) * K2_EPI_THREADS + et] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
+                                                                                 __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+                    }
+                    __threadfence();
+                    epi_bar_sync(h);
+                    if (et == 0) atomicAdd(flag, 1u);
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
+                    if ((acc ^= 1) == 0) acc_phase ^= 1;
+                    continue;
+                }
+                if (et == 0) {
+                    uint64_t t0 = 0;
+                    for (uint32_t it = 1; (int)(ld_acquire_u32(flag) - p.tail_target) < 0; ++it) {
+                        __nanosleep(100);
+                        if ((it & 0x3f) == 0) {
+                            if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
+                            const uint64_t now = ptx::globaltimer_ns();
+                            if (t0 == 0) t0 = now;
+                            else if (now - t0 > ptx::kWaitBudgetNs) {
+                                report_timeout(p.status, SITE_ARRIVAL, w.tail);
+                                s.abort_flag = 1;
+                                break;
+                            }
+                        }
+                    }
+                }
+                epi_bar_sync(h);
+                if (*(volatile int *)&s.abort_flag) { ok = false; break; }
+                __threadfence();
+#pragma unroll 1
+                for (int c = 0; c < CHUNKS; ++c) {
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(taddr + c * 32, r);
+                    ptx::tmem_ld_wait();
+                    for (int pp = 1; pp < p.tail_parts; ++pp) {
+                        const float4 *src = p.tail_scratch + ((((size_t)w.tail * (p.tail_parts - 1) + (pp - 1)) * 2 + rank) * 2 + h) * slot;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float4 o = __ldcg(src + (c * 8 + i) * K2_EPI_THREADS + et);
+                            r[4 * i] = __float_as_uint(__uint_as_float(r[4 * i]) + o.x);
+                            r[4 * i + 1] = __float_as_uint(__uint_as_float(r[4 * i + 1]) + o.y);
+                            r[4 * i + 2] = __float_as_uint(__uint_as_float(r[4 * i + 2]) + o.z);
+                            r[4 * i + 3] = __float_as_uint(__uint_as_float(r[4 * i + 3]) + o.w);
+                        }
+                    }
+                    ptx::tmem_st_32x32(taddr + c * 32, r);
+                }
+                ptx::tmem_st_wait();
             }
 
             if (LN) {
@@ -591,36 +702,78 @@ static bool k2_use_pair(const forge_fused_linear_desc_t &d, int sm_count)
     return env && d.M > K2_BM && sm_count >= 2;
 }
 
+// Grid, K split of the last wave and workspace layout of the non-LayerNorm kernel: a pure function of
+// the problem and the SM count, used by the planner and by the launcher.
+constexpr int K2_TAIL_MAX_PARTS = 8;      // bounds the scratch area and the serial adds of part 0
+constexpr int K2_TAIL_MIN_KB = 16;        // a part is worth its hand-over only with 1024 k or more
+struct K2Layout {
+    bool pair;
+    int64_t tiles_m, tiles_n, units, slots, grid;      // slots: CTAs (or CTA pairs) the GPU offers
+    int tail_parts, tail_kb, tail_tiles;
+    size_t rowg_off, scratch_off, partial_floats;      // float offsets into the partial area
+    size_t strips_done_idx, tail_flags_idx, counters;
+};
+
+static K2Layout k2_layout(const forge_fused_linear_desc_t &d, int sm_count)
+{
+    K2Layout L = {};
+    L.pair = k2_use_pair(d, sm_count);
+    L.tiles_m = (d.M + K2_BM - 1) / K2_BM;
+    L.tiles_n = (d.N + K2_BN - 1) / K2_BN;
+    L.units = (L.pair ? (L.tiles_m + 1) / 2 : L.tiles_m) * L.tiles_n;
+    L.slots = L.pair ? sm_count / 2 : sm_count;
+    const int64_t full = L.units / L.slots, rest = L.units % L.slots;
+    const int num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
+    static const int env = [] {          // FORGE_K2_TAIL_SPLIT=0: never cut the last wave's tiles along K
+        const char *e = std::getenv("FORGE_K2_TAIL_SPLIT");
+        return e ? std::atoi(e) : 1;
+    }();
+    int parts = 1;
+    if (env && rest > 0 && d.red != FORGE_RED_LAYERNORM) {
+        int64_t s = L.slots / rest;
+        if (s > K2_TAIL_MAX_PARTS) s = K2_TAIL_MAX_PARTS;
+        if (s > num_kb / K2_TAIL_MIN_KB) s = num_kb / K2_TAIL_MIN_KB;
+        parts = s < 1 ? 1 : (int)s;
+    }
+    L.tail_kb = (num_kb + parts - 1) / parts;
+    L.tail_parts = (num_kb + L.tail_kb - 1) / L.tail_kb;       // no empty part
+    L.tail_tiles = L.tail_parts > 1 ? (int)rest : 0;
+    const int64_t ctas = full > 0 ? L.slots : rest * L.tail_parts;
+    L.grid = L.pair ? 2 * ctas : ctas;
+    const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;      // float4 partials
+    const bool chain = d.red == FORGE_RED_MEAN_GELU_RESIDUAL;
+    const bool fold = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || chain || lse;      // one partial per row and half tile
+    const size_t fold_floats = fold ? (lse ? 4 : 1) * 2 * (size_t)L.tiles_n * (size_t)d.M : 0;
+    L.rowg_off = fold_floats;                                  // mean chain: gelu(mean) per row after the partials
+    L.scratch_off = (L.rowg_off + (chain ? (size_t)d.M : 0) + 3) / 4 * 4;
+    L.partial_floats = L.scratch_off + (size_t)L.tail_tiles * (L.tail_parts - 1) * 2 * 2 * (4 * 32 * K2_EPI_THREADS);
+    L.strips_done_idx = fold ? (size_t)L.tiles_m : 0;
+    L.tail_flags_idx = L.strips_done_idx + (chain ? 1 : 0);
+    L.counters = L.tail_flags_idx + (size_t)L.tail_tiles * 4;
+    return L;
+}
+
 forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
     if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
-    const int64_t tiles_m = (d.M + K2_BM - 1) / K2_BM, tiles_n = (d.N + K2_BN - 1) / K2_BN;
-    if (tiles_m * tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
-    const bool pair = k2_use_pair(d, sm_count);
+    const K2Layout L = k2_layout(d, sm_count);
+    if (L.tiles_m * L.tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_BF16_TCGEN05;
-    info->tile_m = pair ? 2 * K2_BM : K2_BM;
+    info->tile_m = L.pair ? 2 * K2_BM : K2_BM;
     info->tile_n = K2_BN;
     info->tile_k = K2_BK;
-    info->stages = pair ? K2Ring<true>::STAGES : K2Ring<false>::STAGES;
-    info->cluster = pair ? 2 : 1;
+    info->stages = L.pair ? K2Ring<true>::STAGES : K2Ring<false>::STAGES;
+    info->cluster = L.pair ? 2 : 1;
     info->threads = K2_THREADS;
-    if (pair) {
-        const int64_t units = ((tiles_m + 1) / 2) * tiles_n, clusters = sm_count / 2;
-        info->grid = 2 * (units < clusters ? units : clusters);
-    } else {
-        info->grid = tiles_m * tiles_n < sm_count ? tiles_m * tiles_n : sm_count;
-    }
+    info->grid = L.grid;
     info->smem_bytes = (int64_t)K2_SMEM_BYTES;
-    const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;      // float4 partials
-    const bool partials = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL || lse;   // one per row and half tile
-    wl->partial_floats = partials ? (lse ? 4 : 1) * 2 * (size_t)tiles_n * (size_t)d.M : 0;
-    wl->counters = partials ? (size_t)tiles_m : 0;
-    if (d.red == FORGE_RED_MEAN_GELU_RESIDUAL) {      // gelu(mean) per row after the partials; one more counter
-        wl->partial_floats += (size_t)d.M;
-        wl->counters += 1;
-    }
+    wl->partial_floats = L.partial_floats;
+    wl->counters = L.counters;
     return FORGE_OK;
 }
+
+// CTAs wait on one another in the mean chain (all strips) and in the K split (part 0 on the others).
+static bool k2_ctas_wait(const Handle &h) { return h.d.red == FORGE_RED_MEAN_GELU_RESIDUAL || k2_layout(h.d, h.sm_count).tail_parts > 1; }
 
 template <bool LN, bool PAIR>
 static forge_status_t k2_prepare()
@@ -646,7 +799,7 @@ forge_status_t k2_setup(Handle &h)
 {
     const bool pair = h.info.cluster == 2;
     if ((pair ? k2_prepare<false, true>() : k2_prepare<false, false>()) != FORGE_OK) return FORGE_ERR_CUDA;
-    if (h.d.red != FORGE_RED_MEAN_GELU_RESIDUAL) return FORGE_OK;
+    if (!k2_ctas_wait(h)) return FORGE_OK;
     return pair ? k2_check_residency<false, true>(h) : k2_check_residency<false, false>(h);
 }
 
@@ -688,7 +841,7 @@ static forge_status_t k2_launch_t(const Handle &h, const K2Params &p, cudaStream
         ++n;
     }
     // CTAs that wait on one another: a cooperative launch guarantees that all of them are resident
-    if ((LN || p.e.red == FORGE_RED_MEAN_GELU_RESIDUAL) && cooperative_launch_enabled()) {
+    if (p.cooperative && cooperative_launch_enabled()) {
         attr[n].id = cudaLaunchAttributeCooperative;
         attr[n].val.cooperative = 1;
         ++n;
@@ -711,7 +864,7 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
         if ((st = encode_tmap_16(&h.tmW, a.W, (uint64_t)d.N, (uint64_t)d.K, pair ? K2_BN / 2 : K2_BN, K2_BK, d.dtype == FORGE_F16)) != FORGE_OK) return st;
         h.tmW_ptr = a.W;
     }
-    K2Params p;
+    K2Params p = {};
     p.f16 = d.dtype == FORGE_F16;
     p.b = (const uint16_t *)a.b;
     p.X = (const uint16_t *)a.X;
@@ -737,19 +890,26 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
         }
         p.group_m = env > 0 ? env : (pair ? K2_GROUP_M / 2 : K2_GROUP_M);      // 2048 rows either way
     }
-    p.rowg = nullptr;
-    p.strips_done = nullptr;
-    p.strips_target = 0;
-    if (d.red == FORGE_RED_MEAN_GELU_RESIDUAL) {
-        p.rowg = h.ws.partial + 2 * (size_t)p.tiles_n * (size_t)d.M;
-        p.strips_done = h.ws.counters + p.tiles_m;
-        h.run_gen += 1;                                      // the counter only ever grows: run r ends at r * tiles_m
-        p.strips_target = h.run_gen * (unsigned)p.tiles_m;
-    }
-    if (!ln) return pair ? k2_launch_t<false, true>(h, p, a.stream) : k2_launch_t<false, false>(h, p, a.stream);
-    // Strip counters only ever grow: run r completes a strip at r * 2 * tiles_n arrivals (half tiles).
+    // The counters that CTAs wait on only ever grow: run r is complete at r times the arrivals of one run
+    // (mean chain: strips; K split: parts 1..S-1 of a tile; LayerNorm: half tiles of a strip).
     h.run_gen += 1;
-    p.ln_target = h.run_gen * 2u * (unsigned)p.tiles_n;
+    if (!ln) {
+        const K2Layout L = k2_layout(d, h.sm_count);
+        p.rowg = h.ws.partial + L.rowg_off;
+        p.strips_done = h.ws.counters + L.strips_done_idx;
+        p.strips_target = h.run_gen * (unsigned)p.tiles_m;
+        p.tail_parts = L.tail_parts;
+        p.tail_kb = L.tail_kb;
+        p.tail_scratch = reinterpret_cast<float4 *>(h.ws.partial + L.scratch_off);
+        p.tail_flags = h.ws.counters + L.tail_flags_idx;
+        p.tail_target = h.run_gen * (unsigned)(L.tail_parts - 1);
+        p.cooperative = d.red == FORGE_RED_MEAN_GELU_RESIDUAL || L.tail_parts > 1;
+        return pair ? k2_launch_t<false, true>(h, p, a.stream) : k2_launch_t<false, false>(h, p, a.stream);
+    }
+    p.tail_parts = 1;
+    p.tail_kb = p.num_kb;
+    p.cooperative = 1;
+    p.ln_target = h.run_gen * 2u * (unsigned)p.tiles_n;      // half tiles of a strip
     return pair ? k2_launch_t<true, true>(h, p, a.stream) : k2_launch_t<true, false>(h, p, a.stream);
 }
 

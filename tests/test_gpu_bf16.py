@@ -97,3 +97,21 @@ def test_c3_sampled_rows_full_size():
     assert np.isfinite(g).all()
     rows = wk.sample_rows(wl.M)
     pu.assert_parity(wl, g[rows], pu.run_oracle(wl, inp, rows))
+
+
+@pytest.mark.parametrize("M,N,K,grid", [(64, 2048, 4096, 8 * 4), (300, 520, 4096, 2 * 6 * 4), (128, 16384, 2048, 64 * 2)])
+@pytest.mark.parametrize("red", [wk.RED_NONE, wk.RED_SUM, wk.RED_MEAN_GELU_RESIDUAL, wk.RED_CROSS_ENTROPY])
+def test_tiles_of_the_last_wave_cut_along_k(M, N, K, grid, red):
+    """Fewer tiles than CTAs (or CTA pairs): every tile is computed by several of them, a slice of K
+    each, and put together by the first.  Same bits on every run (the arrival flags only ever grow)."""
+    wl = wk.custom_workload(f"bf16_ksplit_{M}", wk.BF16, M, N, K, wk.ACT_GELU_TANH, red, seed=M + red, w_std=0.02)
+    st, plan = B.forge_fused_linear_query_plan(pu.desc_of(wl))
+    assert st == B.FORGE_OK and plan.kernel == B.FORGE_KERNEL_BF16_TCGEN05 and plan.grid == grid
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op, repeats=3)
+    b, _ = pu.run_gpu(wl, inp, op=op)
+    op.close()
+    assert np.array_equal(a, b)
+    rows = np.unique(np.concatenate([np.arange(0, M, 7), [M - 1]]))
+    pu.assert_parity(wl, a[rows], pu.run_oracle(wl, inp, rows))

@@ -113,14 +113,15 @@ def test_host_entry_point_in_row_blocks_matches_the_oracle(name):
     for _ in range(2):
         op.run_host(h["X"], h["W"], h["b"], aux, h["beta"], out)
     op.check()
-    # the same handle's device entry point on the whole problem gives the same bits
+    # the same handle's device entry point on the whole problem agrees far inside the tolerance (not to the
+    # bit: a block of rows has fewer tiles than the whole problem, so its K range may be cut differently)
     dev = {k: (None if v is None else v.cuda()) for k, v in h.items()}
     dout = torch.empty(shape, dtype=out.dtype, device="cuda")
     op(dev["X"], dev["W"], dev["b"], None if aux is None else aux.cuda(), dev["beta"], dout)
     torch.cuda.synchronize()
     op.check()
     op.close()
-    assert torch.equal(dout.cpu(), out)
+    assert pu.rel_err(out.float().numpy().astype(np.float64), dout.float().cpu().numpy().astype(np.float64)) <= pu.TOL[wl.dtype] / 10
     rows = np.unique(np.concatenate([np.arange(0, M, 97), np.array([511, 512, 2047, 2048, M - 1])]))
     pu.assert_parity(wl, out.float().numpy().astype(np.float64)[rows], pu.run_oracle(wl, inp, rows=rows))
 
