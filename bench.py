@@ -46,9 +46,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
 NCU_TRAFFIC = {
     "c2": {"bytes": 549_508_608, "sha": "b4b97b469603ec83"},
-    "c3": {"bytes": 1_215_054_288, "sha": "fb517b2a9e0efcbf"},
+    "c3": {"bytes": 1_403_875_920, "sha": "3772f5ccb7e73774"},
     "c4": {"bytes": 273_142_272, "sha": "6c195e10916ae16e"},
-    "c5": {"bytes": 299_930_368, "sha": "fb517b2a9e0efcbf"},
+    "c5": {"bytes": 302_728_192, "sha": "3772f5ccb7e73774"},
     "c2t": {"bytes": 349_515_776, "sha": "23334c3c03030526"},
 }
 
