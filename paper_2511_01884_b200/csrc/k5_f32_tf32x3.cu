@@ -710,6 +710,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 // used by the planner and by the launcher.
 constexpr int K5_TAIL_MAX_PARTS = 8;      // bounds the scratch area and the serial adds of part 0
 constexpr int K5_TAIL_MIN_KB = 16;        // a part is worth its hand-over only with 512 k or more
+constexpr int K5_TAIL_MAX_FULL_WAVES = 8; // after that many full waves the last one is too small a share to matter
 struct K5Layout {
     int64_t tiles_m, tiles_n, units, clusters, grid;
     int tail_parts, tail_kb, tail_tiles;
@@ -735,7 +736,7 @@ static K5Layout k5_layout(const forge_fused_linear_desc_t &d, int sm_count)
     }();
     const bool ln = d.red == FORGE_RED_LAYERNORM;
     int parts = 1;
-    if (env && rest > 0 && !ln) {        // LayerNorm: a tile already waits for its strip; no second dependency
+    if (env && rest > 0 && full < K5_TAIL_MAX_FULL_WAVES && !ln) {        // LayerNorm: a tile already waits for its strip; no second dependency
         int64_t s = L.clusters / rest;
         if (s > K5_TAIL_MAX_PARTS) s = K5_TAIL_MAX_PARTS;
         if (s > num_kb / K5_TAIL_MIN_KB) s = num_kb / K5_TAIL_MIN_KB;

@@ -170,3 +170,30 @@ def test_a_wait_that_nothing_satisfies_gives_up_and_reports():
     pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
     assert B.forge_selftest_bounded_wait(0, 0)[0] == B.FORGE_ERR_INVALID_ARG
     assert torch.cuda.is_available()
+
+
+def test_two_handles_on_two_streams_do_not_disturb_each_other():
+    """Every handle owns its workspace (partials, counters, hand-over areas), so launches of different
+    handles may overlap on the GPU; the kernels whose CTAs wait on one another are launched
+    cooperatively and simply take turns."""
+    import torch
+    cases = [wk.custom_workload("two_a", wk.BF16, 300, 520, 4096, wk.ACT_SILU, wk.RED_SUM, w_std=0.02, seed=1),      # K split, CTA pairs
+             wk.custom_workload("two_b", wk.BF16, 700, 1032, 256, wk.ACT_GELU_TANH, wk.RED_LAYERNORM, w_std=0.05, seed=2),
+             wk.custom_workload("two_c", wk.F32_TF32X3, 300, 520, 2048, wk.ACT_RELU, wk.RED_MAX, seed=3),
+             wk.custom_workload("two_d", wk.F32, 200, 300, 96, wk.ACT_GELU_ERF, wk.RED_SUM, seed=4)]
+    work = []
+    for wl in cases:
+        inp = wk.make_inputs(wl)
+        dev = {k: pu.to_device(v, wl.dtype) for k, v in inp.items() if k != "target"}
+        shape = (wl.M,) if wl.out_cols == 0 else (wl.M, wl.out_cols)
+        odt = torch.float32 if (wl.out_cols == 0 or wl.dtype != wk.BF16) else torch.bfloat16
+        work.append((wl, inp, dev, torch.full(shape, float("nan"), dtype=odt, device="cuda"), B.FusedLinear(pu.desc_of(wl)), torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    for _ in range(5):
+        for wl, inp, dev, out, op, st in work:
+            op(dev["X"], dev["W"], dev["b"], dev["gamma"], dev["beta"], out, stream=st.cuda_stream)
+    torch.cuda.synchronize()
+    for wl, inp, dev, out, op, st in work:
+        op.check()
+        op.close()
+        pu.assert_parity(wl, out.float().cpu().numpy().astype(np.float64), pu.run_oracle(wl, inp), wl.name)
