@@ -46,10 +46,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
 NCU_TRAFFIC = {
     "c2": {"bytes": 549_508_608, "sha": "b4b97b469603ec83"},
-    "c3": {"bytes": 1_403_875_920, "sha": "3772f5ccb7e73774"},
+    "c3": {"bytes": 1180000152, "sha": "3617f4f76dcefcef"},
     "c4": {"bytes": 273_142_272, "sha": "6c195e10916ae16e"},
-    "c5": {"bytes": 302_728_192, "sha": "3772f5ccb7e73774"},
-    "c2t": {"bytes": 349_515_776, "sha": "23334c3c03030526"},
+    "c5": {"bytes": 301247488, "sha": "3617f4f76dcefcef"},
+    "c2t": {"bytes": 351503104, "sha": "42e26b9e51b85263"},
 }
 
 
