@@ -13,7 +13,7 @@ import numpy as np
 from paper_2511_01884_b200 import binding as B
 from paper_2511_01884_b200 import workloads as wk
 
-# fp16 storage: output rounding is 2^-11, the approximate activations dominate (see the error budget in the design doc)
+# fp16 storage: output rounding is 2^-11, the approximate activations dominate
 TOL = {wk.F32: 1e-4, wk.BF16: 2e-2, wk.F16: 5e-3, wk.F32_TF32X3: 1e-4}
 
 
