@@ -434,6 +434,14 @@ def main():
             "roofline": roofline_of(wl, ms, peaks, op.plan.kernel, clocks.get("sm_max_mhz"), props.multi_processor_count),
             "nominal_frac": round((value / world) / (NOMINAL["hbm_gbs"] if wl.name == "c4" else NOMINAL["bf16_tflops"]), 4)
             if wl.dtype == wk.BF16 else None}
+    # the static half of the paper's hardware feedback (Section 2.3): what the device is
+    line["gpu_spec"] = {"name": props.name, "compute_capability": f"{props.major}.{props.minor}",
+                        "sms": props.multi_processor_count, "l2_bytes": getattr(props, "L2_cache_size", None),
+                        "hbm_bytes": props.total_memory,
+                        "shared_memory_per_sm": getattr(props, "shared_memory_per_multiprocessor", None),
+                        "registers_per_sm": getattr(props, "regs_per_multiprocessor", None),
+                        "measured_peaks": {k: peaks.get(k) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained")},
+                        "peaks_source": peaks["_source"]}
     eager_us = None
     if rank == 0 and world == 1:
         time.sleep(2.0)
