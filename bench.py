@@ -164,9 +164,11 @@ def make_op(wl, M, device):
 def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
     """Average device milliseconds per step over exactly `steps` steps (CUDA events on the
     launching stream).  With flush_buf every step is bracketed by its own events and L2 is
-    overwritten before it."""
+    overwritten before it.  The calls go through a pre-bound forge_fused_linear_run (pointers
+    marshalled once), so the host side of a step is one foreign-function call."""
+    step = op.bind(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
     for _ in range(warmup):
-        op(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
+        step()
     torch.cuda.synchronize()
     op.check()
     if barrier:
@@ -176,7 +178,7 @@ def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
-            op(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
+            step()
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / steps
@@ -186,7 +188,7 @@ def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
             flush_buf.fill_(1.0)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            op(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
+            step()
             e1.record()
             torch.cuda.synchronize()
             tot += e0.elapsed_time(e1)
@@ -196,6 +198,23 @@ def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
     torch.cuda.synchronize()
     op.check()
     return ms
+
+
+def back_to_back_us(op, d, torch, calls=1000):
+    """Microseconds per call of `calls` calls issued without anything in between (operands stay in
+    L2): what a latency-bound problem costs inside a stream of work."""
+    step = op.bind(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
+    for _ in range(20):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(calls):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    op.check()
+    return 1e3 * e0.elapsed_time(e1) / calls
 
 
 def eager_context_us(wl, d, torch, steps=10):
@@ -471,10 +490,15 @@ def main():
                 ms2 = time_steps(op2, d2, steps2, 3, torch, flush_buf=fl)
                 v2, u2 = unit_value(w2, ms2)
                 launches += steps2
+                b2b = None
+                if fl is not None:            # latency-bound workload: also the figure without the flush
+                    b2b = back_to_back_us(op2, d2, torch)
+                    launches += 1020
                 time.sleep(1.0)
                 eg = eager_context_us(w2, d2, torch, steps=5 if w2.flops > 1e11 else 50)
                 line["workloads"][name] = {"torch_eager_context_us": round(eg, 1), "us_per_call": round(ms2 * 1e3, 2), "value": round(v2, 2), "unit": u2,
                                            "steps": steps2, "l2": "flushed before every call" if fl is not None else "operands larger than L2",
+                                           **({"us_per_call_back_to_back_warm_l2": round(b2b, 2)} if b2b is not None else {}),
                                            "kernel": op2.plan.as_dict()["kernel"],
                                            "roofline": roofline_of(w2, ms2, peaks, op2.plan.kernel, clocks.get("sm_max_mhz"),
                                                                    props.multi_processor_count)}

@@ -194,6 +194,24 @@ class FusedLinear:
             raise ForgeError(st, "forge_fused_linear_run")
         return out
 
+    def bind(self, X, W, b=None, gamma=None, beta=None, out=None, stream=None):
+        """A zero-argument callable that issues ``forge_fused_linear_run`` on these buffers: the
+        pointers and the stream are marshalled once, so a call costs one foreign-function call (for
+        launch-latency-bound problems the per-call argument handling of ``__call__`` is a visible
+        share of the time).  The buffers must stay alive and in place while the callable is used."""
+        if stream is None:
+            import torch
+            stream = torch.cuda.current_stream().cuda_stream
+        vp = ctypes.c_void_p
+        args = (self.h, vp(_ptr(X)), vp(_ptr(W)), vp(_ptr(b)), vp(_ptr(gamma)), vp(_ptr(beta)), vp(_ptr(out)), vp(stream))
+        fn = lib().forge_fused_linear_run
+
+        def call():
+            st = fn(*args)
+            if st != FORGE_OK:
+                raise ForgeError(st, "forge_fused_linear_run")
+        return call
+
     def run_host(self, X, W, b=None, gamma=None, beta=None, out=None):
         st = forge_fused_linear_run_host(self.h, X, W, b, gamma, beta, out)
         if st != FORGE_OK:

@@ -197,3 +197,22 @@ def test_two_handles_on_two_streams_do_not_disturb_each_other():
         op.check()
         op.close()
         pu.assert_parity(wl, out.float().cpu().numpy().astype(np.float64), pu.run_oracle(wl, inp), wl.name)
+
+
+def test_bound_call_is_the_same_call():
+    import torch
+    wl = wk.WORKLOADS["c1"]
+    inp = wk.make_inputs(wl)
+    dev = {k: pu.to_device(v, wl.dtype) for k, v in inp.items() if k != "target"}
+    a = torch.zeros(wl.M, device="cuda")
+    b = torch.zeros(wl.M, device="cuda")
+    op = B.FusedLinear(pu.desc_of(wl))
+    op(dev["X"], dev["W"], dev["b"], None, None, a)
+    step = op.bind(dev["X"], dev["W"], dev["b"], None, None, b)
+    step()
+    step()
+    torch.cuda.synchronize()
+    op.check()
+    op.close()
+    assert torch.equal(a, b)
+    pu.assert_parity(wl, b.cpu().numpy().astype(np.float64), pu.run_oracle(wl, inp))
