@@ -102,7 +102,8 @@ def test_status_and_kernel_strings():
 def test_fp32_plan():
     st, p = B.forge_fused_linear_query_plan(pu_desc("c1"))
     assert st == B.FORGE_OK and p.kernel == B.FORGE_KERNEL_F32_FFMA
-    assert (p.tile_m, p.tile_n, p.grid) == (64, 64, 16) and p.workspace_bytes >= 8 * 128 * 4     # few tiles: the small tile
+    # few tiles: the small tile, and K = 256 cut into 4 slices of 64 so that 64 CTAs take part
+    assert (p.tile_m, p.tile_n, p.grid) == (64, 64, 16 * 4) and p.workspace_bytes >= 8 * 128 * 4 + 16 * 4 * 64 * 64 * 4
     st, p = B.forge_fused_linear_query_plan(pu_desc("c2"))
     assert st == B.FORGE_OK and p.grid == 32 * 32 and p.cluster == 1 and p.tile_m == 128
 

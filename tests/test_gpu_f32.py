@@ -97,3 +97,25 @@ def test_repeatable_bits_and_workspace_reuse():
     op.close()
     assert np.array_equal(a, b)
     pu.assert_parity(wl, a, pu.run_oracle(wl, inp))
+
+
+# few 64x64 tiles and a long K: K is cut into slices that run on different SMs and are summed, in slice
+# order, by the CTA that arrives last (ragged last slice, scalar loads when K % 4 != 0)
+SLICED = [(100, 200, 520), (7, 70, 1000), (33, 65, 333), (128, 512, 256)]
+
+
+@pytest.mark.parametrize("M,N,K", SLICED)
+@pytest.mark.parametrize("red", [wk.RED_NONE, wk.RED_SUM, wk.RED_MAX, wk.RED_MEAN_GELU_RESIDUAL, wk.RED_LOGSUMEXP, wk.RED_CROSS_ENTROPY])
+def test_small_grids_cut_along_k(M, N, K, red):
+    act = ACTS[(M + red) % len(ACTS)]
+    wl = wk.custom_workload(f"f32_sl_{M}x{N}x{K}", wk.F32, M, N, K, act, red, scale=1.5, seed=K + red)
+    st, plan = B.forge_fused_linear_query_plan(pu.desc_of(wl))
+    tiles = -(-M // 64) * -(-N // 64)
+    assert st == B.FORGE_OK and plan.tile_m == 64 and plan.grid > tiles
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op, repeats=3)
+    b, _ = pu.run_gpu(wl, inp, op=op)
+    op.close()
+    assert np.array_equal(a, b)                 # fixed summation order, counters back at zero
+    pu.assert_parity(wl, a, pu.run_oracle(wl, inp), f"act={act} red={red}")
