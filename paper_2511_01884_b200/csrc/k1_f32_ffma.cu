@@ -33,17 +33,47 @@ struct K1Params {
     int out_vec4;          // Y rows can be written with 128-bit stores
     int res_vec4;          // mean chain: X and Y rows ([M,K]) can be moved with 128-bit accesses
     int warm_l2;           // small grids: request the CTA's operand panels into L2 before the k loop
-    // small grids only: K is cut into k_slices ranges of k_per (a multiple of the k-tile), one CTA each
-    // (blockIdx.z); the CTA that arrives last at the tile's counter sums the slices in slice order
-    int k_slices, k_per;
-    float *slice_partial;      // [tile][slice][thread][R*R] raw accumulators
-    unsigned *slice_counters;  // [tile]
+    // (Small grids: K is cut into gridDim.z slices, one CTA each; the slice length and the hand-over
+    // area follow from the fields above -- see k1_slice_len() -- so that this structure, whose size
+    // the code generated for the large tile turned out to be sensitive to, stays as it is.)
 };
+
+// Length of a K slice when K is cut into `slices`: a multiple of the small tile's 32-wide k-tile.
+__host__ __device__ inline int k1_slice_len(int K, int slices) { return ((K + slices - 1) / slices + 31) / 32 * 32; }
 
 // One CTA-tile slab (128 rows x 16 k, or 64 rows x 32 k) from a K-major matrix into registers:
 // two float4 per thread either way.
 template <bool VEC, int T>
 __device__ __forceinline__ void k1_fetch(const float *__restrict__ base, int rows_total, int K,
+                                         int row0, int kt, int tid, float4 (&r)[2])
+{
+    constexpr int KQ = (T == 1 ? 32 : 16) / 4;          // float4 per row of the slab
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int idx = tid + i * K1_THREADS;
+        const int row = row0 + idx / KQ;
+        const int k = kt + (idx % KQ) * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row < rows_total) {
+            const float *src = base + (size_t)row * K + k;
+            if (VEC) {
+                if (k < K) v = __ldg(reinterpret_cast<const float4 *>(src));
+            } else {
+                if (k + 0 < K) v.x = __ldg(src + 0);
+                if (k + 1 < K) v.y = __ldg(src + 1);
+                if (k + 2 < K) v.z = __ldg(src + 2);
+                if (k + 3 < K) v.w = __ldg(src + 3);
+            }
+        }
+        r[i] = v;
+    }
+}
+
+// The same with an explicit end of the k range (K slices of the small tile).
+// One CTA-tile slab (128 rows x 16 k, or 64 rows x 32 k) from a K-major matrix into registers:
+// two float4 per thread either way.
+template <bool VEC, int T>
+__device__ __forceinline__ void k1_fetch_range(const float *__restrict__ base, int rows_total, int K,
                                          int row0, int kt, int tid, float4 (&r)[2], int k_end)
 {
     constexpr int KQ = (T == 1 ? 32 : 16) / 4;          // float4 per row of the slab
@@ -130,61 +160,118 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
 #pragma unroll
         for (int j = 0; j < R / 2; ++j) acc2[i][j] = 0ull;
 
-    if (p.warm_l2) {
-        // A small grid walks K with one tile of look-ahead, i.e. it pays the memory latency once
-        // per k-tile.  Asking L2 for both operand panels up front puts all of those requests in
-        // flight at once; the k loop then runs at L2 latency.
-        const int w_lo = T == 1 ? (int)blockIdx.z * p.k_per : 0, w_len = (T == 1 ? min(K, w_lo + p.k_per) : K) - w_lo;
-        const int lines_per_row = (w_len * 4 + 127) / 128;
-        const int rows_a = min(BM, M - m0), rows_b = min(BN, N - n0);
-        for (int i = tid; i < (rows_a + rows_b) * lines_per_row; i += K1_THREADS) {
-            const int r = i / lines_per_row, c = i - r * lines_per_row;
-            const float *ptr = r < rows_a ? p.X + (size_t)(m0 + r) * K : p.W + (size_t)(n0 + r - rows_a) * K;
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr + w_lo + min(c * 32, w_len - 1)));
-        }
-    }
-    // this CTA's range of k (the whole of K unless a small grid is cut into slices)
-    const int k_lo = T == 1 ? (int)blockIdx.z * p.k_per : 0;
-    const int k_hi = T == 1 ? min(K, k_lo + p.k_per) : K;
-    float4 ra[2], rb[2];
-    k1_fetch<VEC, T>(p.X, M, K, m0, k_lo, tid, ra, k_hi);
-    k1_fetch<VEC, T>(p.W, N, K, n0, k_lo, tid, rb, k_hi);
-    k1_stash<T>(As[0], tid, ra);
-    k1_stash<T>(Bs[0], tid, rb);
-    __syncthreads();
-
-    int buf = 0;
-    for (int kt = k_lo; kt < k_hi; kt += BK) {
-        const bool more = kt + BK < k_hi;
-        if (more) {
-            k1_fetch<VEC, T>(p.X, M, K, m0, kt + BK, tid, ra, k_hi);
-            k1_fetch<VEC, T>(p.W, N, K, n0, kt + BK, tid, rb, k_hi);
-        }
-#pragma unroll
-        for (int k = 0; k < BK; ++k) {
-            const int flip = ((k >> 3) & 1) << 3;          // see k1_stash
-            float a[R];
-            unsigned long long b[R / 2];                    // column pairs as they lie in memory
-#pragma unroll
-            for (int q = 0; q < T; ++q) {
-                const float4 av = *reinterpret_cast<const float4 *>(&As[buf][k][64 * q + ((ty * 4) ^ flip)]);
-                const ulonglong2 bv = *reinterpret_cast<const ulonglong2 *>(&Bs[buf][k][64 * q + ((tx * 4) ^ flip)]);
-                a[4 * q + 0] = av.x; a[4 * q + 1] = av.y; a[4 * q + 2] = av.z; a[4 * q + 3] = av.w;
-                b[2 * q + 0] = bv.x; b[2 * q + 1] = bv.y;
-            }
-#pragma unroll
-            for (int i = 0; i < R; ++i) {
-                const unsigned long long ai = pack2(a[i], a[i]);
-#pragma unroll
-                for (int j = 0; j < R / 2; ++j) ffma2(acc2[i][j], ai, b[j]);
+    if (T == 1) {
+        // small tile: this CTA may own only a slice of K (blockIdx.z of gridDim.z slices)
+        if (p.warm_l2) {
+            // A small grid walks K with one tile of look-ahead, i.e. it pays the memory latency once
+            // per k-tile.  Asking L2 for both operand panels up front puts all of those requests in
+            // flight at once; the k loop then runs at L2 latency.
+            const int w_per = k1_slice_len(K, (int)gridDim.z), w_lo = (int)blockIdx.z * w_per, w_len = min(K, w_lo + w_per) - w_lo;
+            const int lines_per_row = (w_len * 4 + 127) / 128;
+            const int rows_a = min(BM, M - m0), rows_b = min(BN, N - n0);
+            for (int i = tid; i < (rows_a + rows_b) * lines_per_row; i += K1_THREADS) {
+                const int r = i / lines_per_row, c = i - r * lines_per_row;
+                const float *ptr = r < rows_a ? p.X + (size_t)(m0 + r) * K : p.W + (size_t)(n0 + r - rows_a) * K;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr + w_lo + min(c * 32, w_len - 1)));
             }
         }
-        if (more) {
-            k1_stash<T>(As[buf ^ 1], tid, ra);
-            k1_stash<T>(Bs[buf ^ 1], tid, rb);
-        }
+        // this CTA's range of k (the whole of K unless a small grid is cut into slices)
+        const int k_per = k1_slice_len(K, (int)gridDim.z), k_lo = (int)blockIdx.z * k_per, k_hi = min(K, k_lo + k_per);
+        float4 ra[2], rb[2];
+        k1_fetch_range<VEC, T>(p.X, M, K, m0, k_lo, tid, ra, k_hi);
+        k1_fetch_range<VEC, T>(p.W, N, K, n0, k_lo, tid, rb, k_hi);
+        k1_stash<T>(As[0], tid, ra);
+        k1_stash<T>(Bs[0], tid, rb);
         __syncthreads();
-        buf ^= 1;
+
+        int buf = 0;
+        for (int kt = k_lo; kt < k_hi; kt += BK) {
+            const bool more = kt + BK < k_hi;
+            if (more) {
+                k1_fetch_range<VEC, T>(p.X, M, K, m0, kt + BK, tid, ra, k_hi);
+                k1_fetch_range<VEC, T>(p.W, N, K, n0, kt + BK, tid, rb, k_hi);
+            }
+#pragma unroll
+            for (int k = 0; k < BK; ++k) {
+                const int flip = ((k >> 3) & 1) << 3;          // see k1_stash
+                float a[R];
+                unsigned long long b[R / 2];                    // column pairs as they lie in memory
+#pragma unroll
+                for (int q = 0; q < T; ++q) {
+                    const float4 av = *reinterpret_cast<const float4 *>(&As[buf][k][64 * q + ((ty * 4) ^ flip)]);
+                    const ulonglong2 bv = *reinterpret_cast<const ulonglong2 *>(&Bs[buf][k][64 * q + ((tx * 4) ^ flip)]);
+                    a[4 * q + 0] = av.x; a[4 * q + 1] = av.y; a[4 * q + 2] = av.z; a[4 * q + 3] = av.w;
+                    b[2 * q + 0] = bv.x; b[2 * q + 1] = bv.y;
+                }
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    const unsigned long long ai = pack2(a[i], a[i]);
+#pragma unroll
+                    for (int j = 0; j < R / 2; ++j) ffma2(acc2[i][j], ai, b[j]);
+                }
+            }
+            if (more) {
+                k1_stash<T>(As[buf ^ 1], tid, ra);
+                k1_stash<T>(Bs[buf ^ 1], tid, rb);
+            }
+            __syncthreads();
+            buf ^= 1;
+        }
+
+    } else {
+        if (p.warm_l2) {
+            // A small grid walks K with one tile of look-ahead, i.e. it pays the memory latency once
+            // per k-tile.  Asking L2 for both operand panels up front puts all of those requests in
+            // flight at once; the k loop then runs at L2 latency.
+            const int lines_per_row = (K * 4 + 127) / 128;
+            const int rows_a = min(BM, M - m0), rows_b = min(BN, N - n0);
+            for (int i = tid; i < (rows_a + rows_b) * lines_per_row; i += K1_THREADS) {
+                const int r = i / lines_per_row, c = i - r * lines_per_row;
+                const float *ptr = r < rows_a ? p.X + (size_t)(m0 + r) * K : p.W + (size_t)(n0 + r - rows_a) * K;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr + min(c * 32, K - 1)));
+            }
+        }
+        float4 ra[2], rb[2];
+        k1_fetch<VEC, T>(p.X, M, K, m0, 0, tid, ra);
+        k1_fetch<VEC, T>(p.W, N, K, n0, 0, tid, rb);
+        k1_stash<T>(As[0], tid, ra);
+        k1_stash<T>(Bs[0], tid, rb);
+        __syncthreads();
+
+        int buf = 0;
+        for (int kt = 0; kt < K; kt += BK) {
+            const bool more = kt + BK < K;
+            if (more) {
+                k1_fetch<VEC, T>(p.X, M, K, m0, kt + BK, tid, ra);
+                k1_fetch<VEC, T>(p.W, N, K, n0, kt + BK, tid, rb);
+            }
+#pragma unroll
+            for (int k = 0; k < BK; ++k) {
+                const int flip = ((k >> 3) & 1) << 3;          // see k1_stash
+                float a[R];
+                unsigned long long b[R / 2];                    // column pairs as they lie in memory
+#pragma unroll
+                for (int q = 0; q < T; ++q) {
+                    const float4 av = *reinterpret_cast<const float4 *>(&As[buf][k][64 * q + ((ty * 4) ^ flip)]);
+                    const ulonglong2 bv = *reinterpret_cast<const ulonglong2 *>(&Bs[buf][k][64 * q + ((tx * 4) ^ flip)]);
+                    a[4 * q + 0] = av.x; a[4 * q + 1] = av.y; a[4 * q + 2] = av.z; a[4 * q + 3] = av.w;
+                    b[2 * q + 0] = bv.x; b[2 * q + 1] = bv.y;
+                }
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    const unsigned long long ai = pack2(a[i], a[i]);
+#pragma unroll
+                    for (int j = 0; j < R / 2; ++j) ffma2(acc2[i][j], ai, b[j]);
+                }
+            }
+            if (more) {
+                k1_stash<T>(As[buf ^ 1], tid, ra);
+                k1_stash<T>(Bs[buf ^ 1], tid, rb);
+            }
+            __syncthreads();
+            buf ^= 1;
+        }
+
     }
 
     float acc[R][R];
@@ -193,17 +280,24 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
 #pragma unroll
         for (int j = 0; j < R / 2; ++j) unpack2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
 
-    if (T == 1 && p.k_slices > 1) {
+    if (T == 1 && gridDim.z > 1) {
         // ---- K slices of one tile: raw accumulators to the workspace, summed by the last to arrive ----
+        // the hand-over area and its counters lie behind the row partials and the strip counters
+        constexpr bool LSE = RED == FORGE_RED_LOGSUMEXP || RED == FORGE_RED_CROSS_ENTROPY;
+        const bool row_partials = p.tiles_n > 1 && (RED == FORGE_RED_SUM || RED == FORGE_RED_MAX || RED == FORGE_RED_MEAN_GELU_RESIDUAL || LSE);
+        const size_t row_floats = row_partials ? (LSE ? 4 : 1) * (size_t)p.tiles_n * (size_t)M : 0;
+        float4 *slice_partial = reinterpret_cast<float4 *>(p.partial + (row_floats + 3) / 4 * 4);
+        unsigned *slice_counters = p.counters + (row_partials ? gridDim.y : 0);
+        const int k_slices = (int)gridDim.z;
         const int tile = tile_m * (int)gridDim.x + tile_n;
-        float4 *mine = reinterpret_cast<float4 *>(p.slice_partial) + (((size_t)tile * p.k_slices + blockIdx.z) * K1_THREADS + tid) * (R * R / 4);
+        float4 *mine = slice_partial + (((size_t)tile * k_slices + blockIdx.z) * K1_THREADS + tid) * (R * R / 4);
 #pragma unroll
         for (int i = 0; i < R; ++i)
 #pragma unroll
             for (int j = 0; j < R / 4; ++j) mine[i * (R / 4) + j] = make_float4(acc[i][4 * j], acc[i][4 * j + 1], acc[i][4 * j + 2], acc[i][4 * j + 3]);
         __threadfence();
         __syncthreads();
-        if (tid == 0) s_last = (atomicAdd(&p.slice_counters[tile], 1u) == (unsigned)(p.k_slices - 1));
+        if (tid == 0) s_last = (atomicAdd(&slice_counters[tile], 1u) == (unsigned)(k_slices - 1));
         __syncthreads();
         if (!s_last) return;
         __threadfence();
@@ -211,8 +305,8 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         for (int i = 0; i < R; ++i)
 #pragma unroll
             for (int j = 0; j < R; ++j) acc[i][j] = 0.f;
-        for (int sl = 0; sl < p.k_slices; ++sl) {         // slice order, whichever CTA got here last
-            const float4 *src = reinterpret_cast<const float4 *>(p.slice_partial) + (((size_t)tile * p.k_slices + sl) * K1_THREADS + tid) * (R * R / 4);
+        for (int sl = 0; sl < k_slices; ++sl) {           // slice order, whichever CTA got here last
+            const float4 *src = slice_partial + (((size_t)tile * k_slices + sl) * K1_THREADS + tid) * (R * R / 4);
 #pragma unroll
             for (int i = 0; i < R; ++i)
 #pragma unroll
@@ -222,7 +316,7 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
                 }
         }
         __syncthreads();                                   // s_last is reused by the row reductions below
-        if (tid == 0) p.slice_counters[tile] = 0u;         // ready for the next run
+        if (tid == 0) slice_counters[tile] = 0u;           // ready for the next run
     }
 
     // ---- epilogue: bias, activation, scale, in registers --------------------------------
@@ -445,16 +539,19 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
 // Small grids (64x64 tiles, at most half an SM's worth of tiles each): K is cut into up to 8 slices of
 // at least 64 k so that more SMs take part; a grid of 16 CTAs otherwise spends its time in the k loop
 // of 16 SMs.  Returns the slice count and sets the slice length (a multiple of the 32-wide k-tile).
-static int k1_slices(const forge_fused_linear_desc_t &d, int sm_count, int64_t tiles, int *k_per)
+static int k1_slices(const forge_fused_linear_desc_t &d, int sm_count, int64_t tiles)
 {
     int64_t s = sm_count / (tiles > 0 ? tiles : 1);
     if (s > 8) s = 8;
     if (s > d.K / 64) s = d.K / 64;
     if (s < 1) s = 1;
-    int64_t per = (d.K + s - 1) / s;
-    per = (per + 31) / 32 * 32;
-    *k_per = (int)per;
-    return (int)((d.K + per - 1) / per);
+    // the kernel derives the slice length from the slice count: settle on a count that reproduces itself
+    for (;;) {
+        const int per = k1_slice_len((int)d.K, (int)s);
+        const int64_t need = (d.K + per - 1) / per;
+        if (need == s) return (int)s;
+        s = need;
+    }
 }
 
 forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
@@ -475,8 +572,7 @@ forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     info->stages = 2;
     info->cluster = d.red == FORGE_RED_LAYERNORM ? (int)tiles_n : 1;
     info->threads = K1_THREADS;
-    int k_per = 0;
-    const int slices = small ? k1_slices(d, sm_count, tiles_m * tiles_n, &k_per) : 1;
+    const int slices = small ? k1_slices(d, sm_count, tiles_m * tiles_n) : 1;
     info->grid = tiles_m * tiles_n * slices;
     info->smem_bytes = 0;
     const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;      // float4 partials
@@ -534,21 +630,8 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
     p.out_vec4 = (d.N % 4 == 0) && ((uintptr_t)a.out % 16 == 0);
     p.res_vec4 = (d.K % 4 == 0) && ((uintptr_t)a.out % 16 == 0) && ((uintptr_t)a.X % 16 == 0);
     const int64_t tiles_m = (d.M + bm - 1) / bm;
-    p.k_slices = 1;
-    p.k_per = (int)d.K;
-    p.slice_partial = nullptr;
-    p.slice_counters = nullptr;
-    if (bm != K1_BM) {
-        p.k_slices = k1_slices(d, h.sm_count, tiles_m * p.tiles_n, &p.k_per);
-        if (p.k_slices > 1) {
-            const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;
-            const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL || lse) && p.tiles_n > 1;
-            const size_t row_floats = partials ? (lse ? 4 : 1) * (size_t)p.tiles_n * (size_t)d.M : 0;
-            p.slice_partial = h.ws.partial + (row_floats + 3) / 4 * 4;
-            p.slice_counters = h.ws.counters + (partials ? (size_t)tiles_m : 0);
-        }
-    }
-    const dim3 grid((unsigned)p.tiles_n, (unsigned)tiles_m, (unsigned)p.k_slices);
+    const int k_slices = bm != K1_BM ? k1_slices(d, h.sm_count, tiles_m * p.tiles_n) : 1;
+    const dim3 grid((unsigned)p.tiles_n, (unsigned)tiles_m, (unsigned)k_slices);
     const bool vec = (d.K % 4 == 0) && ((uintptr_t)a.X % 16 == 0) && ((uintptr_t)a.W % 16 == 0);
 #define K1_CASE(R)                                                                                   \
     case R:                                                                                          \
@@ -645,10 +728,6 @@ extern "C" forge_status_t forge_fused_linear_f32_reduce_static(int64_t M, int64_
     p.out_vec4 = 0;
     p.res_vec4 = 0;
     p.warm_l2 = 0;
-    p.k_slices = 1;
-    p.k_per = (int)K;
-    p.slice_partial = nullptr;
-    p.slice_counters = nullptr;
     const dim3 grid((unsigned)tiles_n, (unsigned)tiles_m);
     const bool vec = (K % 4 == 0) && ((uintptr_t)X % 16 == 0) && ((uintptr_t)W % 16 == 0);
     if (red == FORGE_RED_SUM)
