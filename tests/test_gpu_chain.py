@@ -86,3 +86,16 @@ def test_n1_sampled_rows_full_size():
     rows = wk.sample_rows(wl.M)
     pu.assert_parity(wl, g[rows], pu.run_oracle(wl, inp, rows))
     assert np.isfinite(g).all()
+
+
+@pytest.mark.parametrize("name", ["n1t", "n1b"])
+def test_chain_on_the_tensor_core_kernels_sampled_rows_full_size(name):
+    """The bench's launch configurations: the residual rows are written by the whole grid after all
+    strips have published gelu(mean) (cooperative launch); n1t also cuts its last wave along K."""
+    wl = wk.EXTRA_WORKLOADS[name]
+    inp = wk.make_inputs(wl)
+    g, plan = pu.run_gpu(wl, inp, repeats=2)
+    assert plan["cluster"] == 2
+    rows = wk.sample_rows(wl.M)
+    pu.assert_parity(wl, g[rows], pu.run_oracle(wl, inp, rows))
+    assert np.isfinite(g).all()
