@@ -18,8 +18,6 @@ LIB = os.path.join(HERE, "libforge.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
          "-Xcompiler", "-fPIC"]
-if os.environ.get("FORGE_DEBUG_BOUNDS"):            # range-check indices inside the kernels
-    FLAGS.append("-DFORGE_DEBUG_BOUNDS")
 
 
 def _stale(target: str, deps) -> bool:

@@ -216,3 +216,38 @@ def test_bound_call_is_the_same_call():
     op.close()
     assert torch.equal(a, b)
     pu.assert_parity(wl, b.cpu().numpy().astype(np.float64), pu.run_oracle(wl, inp))
+
+
+@pytest.mark.parametrize("case", ["f32", "f32_sliced", "tf32x3", "tf32x3_ln", "bf16_pair", "bf16_ksplit", "bf16_ln", "skinny", "f16", "chain_bf16"])
+def test_nothing_is_written_outside_the_output(case):
+    """Every kernel family on a ragged shape, with the output in the middle of a larger buffer whose
+    guard zones must keep their pattern (stores past a row end, a tile edge or the last row would
+    land there)."""
+    import torch
+    M, N, K, dt, act, red = {
+        "f32": (129, 257, 33, wk.F32, wk.ACT_GELU_ERF, wk.RED_NONE),
+        "f32_sliced": (100, 204, 520, wk.F32, wk.ACT_RELU, wk.RED_NONE),
+        "tf32x3": (300, 516, 132, wk.F32_TF32X3, wk.ACT_SILU, wk.RED_NONE),
+        "tf32x3_ln": (300, 516, 132, wk.F32_TF32X3, wk.ACT_GELU_TANH, wk.RED_LAYERNORM),
+        "bf16_pair": (300, 520, 136, wk.BF16, wk.ACT_SILU, wk.RED_NONE),
+        "bf16_ksplit": (100, 520, 4096, wk.BF16, wk.ACT_GELU_TANH, wk.RED_NONE),
+        "bf16_ln": (300, 520, 136, wk.BF16, wk.ACT_GELU_TANH, wk.RED_LAYERNORM),
+        "skinny": (20, 1032, 520, wk.BF16, wk.ACT_GELU_ERF, wk.RED_NONE),
+        "f16": (150, 264, 72, wk.F16, wk.ACT_RELU, wk.RED_NONE),
+        "chain_bf16": (300, 520, 136, wk.BF16, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL),
+    }[case]
+    wl = wk.custom_workload("guard_" + case, dt, M, N, K, act, red, seed=len(case), w_std=0.05 if dt in (wk.BF16, wk.F16) else None)
+    inp = wk.make_inputs(wl)
+    dev = {k: pu.to_device(v, wl.dtype) for k, v in inp.items() if k != "target"}
+    odt = {wk.F32: torch.float32, wk.F32_TF32X3: torch.float32, wk.BF16: torch.bfloat16, wk.F16: torch.float16}[dt]
+    n_out, guard = M * wl.out_cols, 4096
+    buf = torch.full((guard + n_out + guard,), 12345.0, dtype=odt, device="cuda")
+    out = buf[guard:guard + n_out].view(M, wl.out_cols)
+    aux = dev["sub"] if red == wk.RED_MEAN_GELU_RESIDUAL else dev["gamma"]
+    op = B.FusedLinear(pu.desc_of(wl))
+    op(dev["X"], dev["W"], dev["b"], aux, dev["beta"], out)
+    torch.cuda.synchronize()
+    op.check()
+    op.close()
+    assert bool((buf[:guard] == 12345.0).all()) and bool((buf[guard + n_out:] == 12345.0).all())
+    pu.assert_parity(wl, out.float().cpu().numpy().astype(np.float64), pu.run_oracle(wl, inp))
