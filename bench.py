@@ -358,6 +358,83 @@ def run_reference(args):
     return 0
 
 
+def run_column_sharded(args, wl, torch, dist, rank, world, local, peaks, props):
+    """--shard cols: the rows of W (and the slice of b) are split over the ranks, X is replicated, every
+    rank runs the fused kernel on its slice and the partial out[M] are combined by one all-reduce of M
+    floats per step (inside the timed region).  Strong scaling of one skinny-M problem."""
+    import dataclasses
+    if wl.red not in multigpu.COLUMN_SHARDABLE:
+        raise SystemExit("--shard cols needs a row-sum or row-max workload (c4)")
+    lo, hi = multigpu.rank_cols(wl, rank, world)
+    inp = wk.make_inputs(wl)
+    inp["W"] = np.ascontiguousarray(inp["W"][lo:hi])
+    if inp["b"] is not None:
+        inp["b"] = np.ascontiguousarray(inp["b"][lo:hi])
+    wl_r = dataclasses.replace(wl, N=hi - lo)
+    d = device_tensors(wl_r, inp, torch)
+    op = make_op(wl_r, wl.M, local)
+    step = op.bind(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
+    grp = dist if world > 1 else None
+
+    def one():
+        step()
+        multigpu.combine_column_partials(d["out"], wl.red, grp)
+    for _ in range(args.warmup):
+        one()
+    torch.cuda.synchronize()
+    op.check()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as cs:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            one()
+        e1.record()
+        torch.cuda.synchronize()
+    ms = multigpu.max_over_ranks(e0.elapsed_time(e1) / args.steps, grp, device="cuda")
+    op.check()
+    value = wl.algorithmic_bytes / ms / 1e6            # the one global problem's bytes: strong scaling
+    # end to end: this rank's slice from pinned host memory, the combined result back
+    host = {k: (None if d[k] is None else d[k].cpu().pin_memory()) for k in ("X", "W", "b")}
+    host_out = torch.empty_like(d["out"], device="cpu").pin_memory()
+    op.run_host(host["X"], host["W"], host["b"], None, None, host_out)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    n = max(1, min(args.steps, 10))
+    for _ in range(n):
+        op.run_host(host["X"], host["W"], host["b"], None, None, host_out)
+        if world > 1:
+            t = host_out.cuda()
+            multigpu.combine_column_partials(t, wl.red, grp)
+            host_out.copy_(t)
+    torch.cuda.synchronize()
+    e2e_ms = multigpu.max_over_ranks(1e3 * (time.perf_counter() - t0) / n, grp, device="cuda")
+    line = {"metric": f"fused-op GB/s ({wl.name})", "value": round(value, 2), "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 5), "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "bf16" if wl.dtype == wk.BF16 else "f32", "data": "synthetic",
+            "config": config_of(wl, world, {"kernel": op.plan.as_dict(),
+                                            "parallelism": f"rows of W sharded over {world} gpu(s), X replicated, one all-reduce of M floats per step"}),
+            "clocks": cs.summary(),
+            "e2e": {"value": round(wl.algorithmic_bytes / e2e_ms / 1e6, 3), "unit": "GB/s",
+                    "h2d_bytes_per_step": sum(v.numel() * v.element_size() for v in host.values() if v is not None),
+                    "d2h_bytes_per_step": host_out.numel() * host_out.element_size(), "steps": n, "ms_per_step": round(e2e_ms, 3)},
+            "gpu_launches": args.steps,
+            "roofline": {"bound": "hbm", "achieved": round(value / world, 2), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": round(value / world / peaks["hbm_gbs"], 4), "traffic": None,
+                         "note": f"per GPU: the global problem's {wl.algorithmic_bytes} bytes / {world} ranks; peak = copy bandwidth, of {peaks['_source']}"}}
+    op.close()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
 def config_of(wl, n_gpus, extra=None):
     names = {wk.ACT_IDENTITY: "identity", wk.ACT_RELU: "relu", wk.ACT_GELU_ERF: "gelu_erf",
              wk.ACT_GELU_TANH: "gelu_tanh", wk.ACT_SILU: "silu"}
@@ -381,6 +458,9 @@ def main():
     ap.add_argument("--workload", default=HEADLINE, choices=sorted(ALL_WORKLOADS))
     ap.add_argument("--impl", default="forge", choices=["forge", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the short runs of the other workloads")
+    ap.add_argument("--shard", default="rows", choices=["rows", "cols"],
+                    help="rows: every rank its own rows of X (weak scaling, no collective); cols: the rows of W of one "
+                         "skinny-M problem over the ranks, partial out[M] combined by an all-reduce (strong scaling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -405,6 +485,9 @@ def main():
     peaks = load_peaks()
     props = torch.cuda.get_device_properties(local)
     wl = ALL_WORKLOADS[args.workload]
+
+    if args.shard == "cols":
+        return run_column_sharded(args, wl, torch, dist, rank, world, local, peaks, props)
 
     # this rank's block of rows of the global [world * M, K] input; W, b, gamma, beta replicated
     rows, row_offset = multigpu.rank_rows_weak(wl, rank)

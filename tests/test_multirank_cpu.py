@@ -76,3 +76,44 @@ def test_single_process_helpers():
     wl = wk.WORKLOADS["c3"]
     assert multigpu.rank_rows_weak(wl, 3) == (8192, 3 * 8192)
     assert multigpu.rank_rows_strong(wl, 1, 4) == (2048, 2048)
+
+
+def _col_worker(rank, world, port, red, q):
+    import oracle
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = wk.custom_workload("mc", wk.F32, 9, 40, 24, wk.ACT_GELU_ERF, red, seed=3)
+    inp = wk.make_inputs(wl)
+    lo, hi = multigpu.rank_cols(wl, rank, world)
+    part = oracle.fused_linear(inp["X"], inp["W"][lo:hi], inp["b"][lo:hi], act=wl.act, scale=wl.scale, red=wl.red)
+    out = multigpu.combine_column_partials(torch.from_numpy(np.ascontiguousarray(part)), red, dist)
+    if rank == 0:
+        q.put(((lo, hi), out.numpy()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_column_shards_combine_to_the_unsharded_result():
+    """W split by rows over two ranks; the per-rank row sums / maxima (here from the
+    oracle) combined by the small collective give the unsharded operator's output."""
+    import oracle
+    for red in multigpu.COLUMN_SHARDABLE:
+        ctx = mp.get_context("spawn")
+        q = ctx.SimpleQueue()
+        port = _free_port()
+        procs = [ctx.Process(target=_col_worker, args=(r, 2, port, red, q)) for r in range(2)]
+        for p in procs:
+            p.start()
+        (lo, hi), got = q.get()
+        for p in procs:
+            p.join(60)
+            assert p.exitcode == 0
+        assert (lo, hi) == (0, 24)                           # 5 groups of 8 columns: 3 + 2
+        wl = wk.custom_workload("mc", wk.F32, 9, 40, 24, wk.ACT_GELU_ERF, red, seed=3)
+        inp = wk.make_inputs(wl)
+        want = oracle.fused_linear(inp["X"], inp["W"], inp["b"], act=wl.act, scale=wl.scale, red=wl.red)
+        assert np.allclose(got, want, rtol=1e-13, atol=1e-13), red
+    wl = wk.WORKLOADS["c4"]
+    assert [multigpu.rank_cols(wl, r, 8) for r in (0, 7)] == [(0, 2048), (14336, 16384)]
+    with np.testing.assert_raises(ValueError):
+        multigpu.combine_column_partials(torch.zeros(3), wk.RED_LAYERNORM)
