@@ -298,7 +298,7 @@ def oracle_sample(wl, inp, target_s=12.0, max_rows=None):
     import oracle
     M = inp["X"].shape[0]
     rows_all = wk.sample_rows(M)
-    probe = rows_all[: min(len(rows_all), 4)]
+    probe = rows_all[: min(len(rows_all), max(4, 2 * oracle.threads()))]      # enough rows to occupy every thread
     extra = {"sub": inp.get("sub"), "target": inp.get("target")}
     per_row = 0.0
     for _ in range(2):          # the first call pays for thread start-up and first touches; estimate from the second
