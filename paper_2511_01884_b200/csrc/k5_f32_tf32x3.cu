@@ -40,12 +40,19 @@
 // draining (and the epilogue of tile i) overlaps the MMAs that follow.  No load is multicast;
 // every software wait is bounded.
 //
-// Last, partly filled wave: when the tiles left over after the full waves are fewer than half the
-// clusters, each of them is cut along K into S parts that run on S clusters at once.  Parts 1..S-1
+// Last, partly filled wave: when the tiles left over after the full waves are at most half the
+// clusters (and at most 8 full waves precede them), each of them is cut along K into S parts of at
+// least 512 k that run on S clusters at once.  Parts 1..S-1
 // leave their running sums (the registers above) in a scratch area and count themselves in; part 0
 // waits for them (bounded), adds them to its own sum in part order and runs the epilogue.  Nothing
 // else changes: a part is just a tile with a shorter K range.  A 4096^3 problem (256 tiles on 74
 // clusters) takes 3.5 tile times instead of 4.
+//
+// LayerNorm over N: as on the bf16 kernel, the N-tiles of a row strip are neighbours in the schedule;
+// each half tile writes its activated values back to TMEM, publishes (n, mean, M2) per row, waits
+// (bounded) for the strip's other half tiles, combines the statistics in part order and normalises
+// out of TMEM.  The mean chain publishes gelu(mean) per row and the whole grid writes the residual
+// rows at the end.  In both, and with the K cut, CTAs wait on one another: the launch is cooperative.
 #include <cstdlib>
 
 #include "common.cuh"
