@@ -390,7 +390,15 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
             if (tid < BM && m0 + tid < M) {
                 const int row = m0 + tid;
                 float v = __ldcg(&p.partial[row]);
-                for (int t = 1; t < p.tiles_n; ++t) {
+                int t = 1;
+                for (; t + 8 <= p.tiles_n; t += 8) {      // 8 independent loads in flight
+                    float o[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) o[u] = __ldcg(&p.partial[(size_t)(t + u) * M + row]);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v = ADD ? v + o[u] : fmaxf(v, o[u]);
+                }
+                for (; t < p.tiles_n; ++t) {
                     const float o = __ldcg(&p.partial[(size_t)t * M + row]);
                     v = ADD ? v + o : fmaxf(v, o);
                 }
@@ -466,7 +474,18 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
             const int row = m0 + tid;
             float4 f = __ldcg(&part4[row]);
             float mx = f.x, se = f.y, tl = f.z;
-            for (int t = 1; t < p.tiles_n; ++t) {
+            int t = 1;
+            for (; t + 8 <= p.tiles_n; t += 8) {      // 8 independent loads in flight, then the chain of merges
+                float4 g[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) g[u] = __ldcg(&part4[(size_t)(t + u) * M + row]);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    lse_merge<true>(mx, se, g[u].x, g[u].y);
+                    tl += g[u].z;
+                }
+            }
+            for (; t < p.tiles_n; ++t) {
                 f = __ldcg(&part4[(size_t)t * M + row]);
                 lse_merge<true>(mx, se, f.x, f.y);
                 tl += f.z;

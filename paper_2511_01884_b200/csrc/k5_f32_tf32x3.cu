@@ -634,7 +634,18 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                         if (lse) {
                             float4 f = __ldcg(&part4[row]);
                             mx = f.x; se = f.y; tl = f.z;
-                            for (int i = 1; i < parts; ++i) {
+                            int i = 1;
+                            for (; i + 8 <= parts; i += 8) {      // 8 independent loads in flight, then the chain of merges
+                                float4 g[8];
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) g[u] = __ldcg(&part4[(size_t)(i + u) * p.M + row]);
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) {
+                                    lse_merge<true>(mx, se, g[u].x, g[u].y);
+                                    tl += g[u].z;
+                                }
+                            }
+                            for (; i < parts; ++i) {
                                 f = __ldcg(&part4[(size_t)i * p.M + row]);
                                 lse_merge<true>(mx, se, f.x, f.y);
                                 tl += f.z;
@@ -642,7 +653,15 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                             out[row] = mx + logf(se) - tl;
                         } else {
                             float v = __ldcg(&p.partial[row]);
-                            for (int i = 1; i < parts; ++i) {
+                            int i = 1;
+                            for (; i + 8 <= parts; i += 8) {      // 8 independent loads in flight
+                                float o[8];
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) o[u] = __ldcg(&p.partial[(size_t)(i + u) * p.M + row]);
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) v = add ? v + o[u] : fmaxf(v, o[u]);
+                            }
+                            for (; i < parts; ++i) {
                                 const float o = __ldcg(&p.partial[(size_t)i * p.M + row]);
                                 v = add ? v + o : fmaxf(v, o);
                             }
