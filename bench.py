@@ -46,11 +46,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # from the ncu captures summarised under profiles/, keyed by workload, with the sha256 of the
 # kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
 NCU_TRAFFIC = {
-    "c2": {"bytes": 547829504, "sha": "3a89491b5c100d43"},
-    "c3": {"bytes": 1180000152, "sha": "9bec398f3dab02da"},
+    "c2": {"bytes": 539106048, "sha": "83c493efb815777f"},
+    "c3": {"bytes": 1243247040, "sha": "8f87836249bf05fe"},
     "c4": {"bytes": 273_142_272, "sha": "d1f4e9fb22aed839"},
-    "c5": {"bytes": 301247488, "sha": "9bec398f3dab02da"},
-    "c2t": {"bytes": 351503104, "sha": "2a56462ae982f3d9"},
+    "c5": {"bytes": 300177664, "sha": "8f87836249bf05fe"},
+    "c2t": {"bytes": 351129088, "sha": "a34344002eb31ab1"},
 }
 
 
