@@ -12,6 +12,14 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200, sm_100a)")
 
 
+def pytest_sessionstart(session):
+    """The CUDA library is built in-tree and kept out of version control: compile it when a fresh
+    checkout has none (nvcc cross-compiles without a GPU)."""
+    from paper_2511_01884_b200 import binding, build
+    if not os.path.exists(binding.LIB_PATH):
+        build.build()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
