@@ -47,9 +47,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
 NCU_TRAFFIC = {
     "c2": {"bytes": 539106048, "sha": "83c493efb815777f"},
-    "c3": {"bytes": 1243247040, "sha": "8f87836249bf05fe"},
+    "c3": {"bytes": 1150823328, "sha": "b0fa426747d03e58"},
     "c4": {"bytes": 273_142_272, "sha": "d1f4e9fb22aed839"},
-    "c5": {"bytes": 300177664, "sha": "8f87836249bf05fe"},
+    "c5": {"bytes": 304678656, "sha": "b0fa426747d03e58"},
     "c2t": {"bytes": 351129088, "sha": "a34344002eb31ab1"},
 }
 

@@ -101,6 +101,7 @@ __device__ __forceinline__ void k2_tile_coords(int t, int tiles_m, int tiles_n, 
     const int gm = min(group_m, tiles_m - g * group_m);
     tm = g * group_m + r % gm;
     tn = r / gm;
+    if (g & 1) tn = tiles_n - 1 - tn;      // every other group walks the N-tiles backwards: the W panels last used are still in L2
 }
 
 // One unit of work of a CTA (or CTA pair): a tile and a range of k-blocks.  Unit c of C takes the whole
