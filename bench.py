@@ -66,17 +66,19 @@ def load_peaks():
     return p
 
 
-def kernel_source_hash(kernel: int) -> str:
-    """Hash of the kernel's source with comments and blank space removed: a reworded comment does not
+def source_digest(text: str) -> str:
+    """Hash of a source text with comments and blank space removed: a reworded comment does not
     make the traffic counters stale, a changed statement does."""
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    text = re.sub(r"//[^\n]*", "", text)
+    return hashlib.sha256("".join(text.split()).encode()).hexdigest()[:16]
+
+
+def kernel_source_hash(kernel: int) -> str:
     name = {1: "k1_f32_ffma.cu", 2: "k2_bf16_tcgen05.cu", 3: "k3_bf16_skinny.cu", 4: "k2_bf16_tcgen05.cu",
             5: "k5_f32_tf32x3.cu"}[kernel]
     with open(os.path.join(ROOT, "paper_2511_01884_b200", "csrc", name), "r") as f:
-        text = f.read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    text = re.sub(r"//[^\n]*", "", text)
-    text = "".join(text.split())
-    return hashlib.sha256(text.encode()).hexdigest()[:16]
+        return source_digest(f.read())
 
 
 # ---- clocks during the timed region (NVML; nvidia-smi as a fallback) -------------------------
