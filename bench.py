@@ -50,7 +50,7 @@ NCU_TRAFFIC = {
     "c3": {"bytes": 1150823328, "sha": "b0fa426747d03e58"},
     "c4": {"bytes": 273_142_272, "sha": "d1f4e9fb22aed839"},
     "c5": {"bytes": 304678656, "sha": "b0fa426747d03e58"},
-    "c2t": {"bytes": 351129088, "sha": "a34344002eb31ab1"},
+    "c2t": {"bytes": 353031168, "sha": "cb0f91a3d90a1e4c"},
 }
 
 

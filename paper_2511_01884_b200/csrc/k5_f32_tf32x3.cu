@@ -302,7 +302,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 float4 *raw = reinterpret_cast<float4 *>(tiles + (size_t)stage * K5_STAGE_BYTES);
                 float4 *lo = reinterpret_cast<float4 *>(tiles + (size_t)stage * K5_STAGE_BYTES + K5_RAW_BYTES);
                 constexpr int PER_THREAD = K5_RAW_BYTES / 16 / K5_SPLIT_THREADS;       // 16 float4
-#pragma unroll 4
+#pragma unroll 8
                 for (int i = 0; i < PER_THREAD; ++i) {
                     const int idx = i * K5_SPLIT_THREADS + st;
                     const float4 v = raw[idx];
