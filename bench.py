@@ -12,8 +12,15 @@ rows of a global X (rows are independent: no collective on the data path) and th
 the aggregate over ranks of work / max-over-ranks time.
 
 Timing: CUDA events on the stream the kernels are launched on, after >= 3 warm-up steps,
-barrier + synchronize on both sides.  L2: the operands of C2..C5 exceed the 126 MB L2; C1
-fits and is timed with an L2 flush (a 256 MiB write) before every call.
+barrier + synchronize on both sides.  L2: the operands of C2, C3, C5 exceed the 126 MB L2 and
+those kernels are compute-bound; C4 (HBM-bound: the whole cost is streaming W once) rotates
+through three distinct copies of W (768 MiB) so that no byte of a W can still be in L2 when it
+is read again; C1 fits in L2 and is timed with an L2 flush (a 256 MiB write) before every call.
+
+    python bench.py --workload c5 --kernel-only --steps 4 [--rows R]
+
+launches the workload's kernel a few times (each launch timed alone) and nothing else: the
+fixed launch sequence to put under a profiler, R rows of X for a small case.
 """
 from __future__ import annotations
 
@@ -170,16 +177,55 @@ def make_op(wl, M, device):
                                      wl.bias.kind != "none", device))
 
 
-def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
+class Rotation:
+    """The step callables of one workload.  Normally one handle bound to one set of buffers.  For the
+    HBM-bound workload: `copies` handles, each bound to its own copy of W (its tensor map is encoded
+    once), called in turn, so that a W is read again only after the other copies -- several times the
+    L2 -- have streamed through."""
+
+    def __init__(self, wl, d, device, torch, copies=1):
+        self.ops, self.steps, self.keep = [], [], []
+        for i in range(copies):
+            W = d["W"] if i == 0 else d["W"].clone()
+            op = make_op(wl, d["X"].shape[0], device)
+            self.ops.append(op)
+            self.keep.append(W)
+            self.steps.append(op.bind(d["X"], W, d["b"], d["gamma"], d["beta"], d["out"]))
+        self.w_bytes = sum(w.numel() * w.element_size() for w in self.keep)
+        self.i = 0
+
+    def step(self):
+        self.steps[self.i]()
+        self.i = (self.i + 1) % len(self.steps)
+
+    def check(self):
+        for op in self.ops:
+            op.check()
+
+    def close(self):
+        for op in self.ops:
+            op.close()
+        self.keep = []
+
+    @property
+    def plan(self):
+        return self.ops[0].plan
+
+
+def w_copies(wl):
+    """Distinct copies of W the timed loop rotates through (only the HBM-bound workload needs more than one)."""
+    return 3 if wl.name == "c4" else 1
+
+
+def time_steps(rot, steps, warmup, torch, flush_buf=None, barrier=None):
     """Average device milliseconds per step over exactly `steps` steps (CUDA events on the
     launching stream).  With flush_buf every step is bracketed by its own events and L2 is
     overwritten before it.  The calls go through a pre-bound forge_fused_linear_run (pointers
     marshalled once), so the host side of a step is one foreign-function call."""
-    step = op.bind(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
     for _ in range(warmup):
-        step()
+        rot.step()
     torch.cuda.synchronize()
-    op.check()
+    rot.check()
     if barrier:
         barrier()
     torch.cuda.synchronize()
@@ -187,7 +233,7 @@ def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
-            step()
+            rot.step()
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / steps
@@ -197,7 +243,7 @@ def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
             flush_buf.fill_(1.0)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            step()
+            rot.step()
             e1.record()
             torch.cuda.synchronize()
             tot += e0.elapsed_time(e1)
@@ -205,24 +251,67 @@ def time_steps(op, d, steps, warmup, torch, flush_buf=None, barrier=None):
     if barrier:
         barrier()
     torch.cuda.synchronize()
-    op.check()
+    rot.check()
     return ms
 
 
-def back_to_back_us(op, d, torch, calls=1000):
+def isolated_us(rot, torch, calls=30):
+    """Microseconds of one call with nothing before or after it on the device (a synchronise after every
+    call): no overlap with a neighbour's start-up or tail.  Median and minimum over `calls` calls."""
+    ts = []
+    for _ in range(calls):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        rot.step()
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(1e3 * e0.elapsed_time(e1))
+    rot.check()
+    return statistics.median(ts), min(ts)
+
+
+def sustained_block(rot, wl, peaks, local, torch, seconds=2.5):
+    """Back-to-back launches for `seconds` of device time: what the kernel holds once the GPU has settled
+    at the clock its power limit allows, with the clocks sampled meanwhile."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(20):
+        rot.step()
+    e1.record()
+    torch.cuda.synchronize()
+    n = max(50, int(seconds * 1e3 / max(e0.elapsed_time(e1) / 20, 1e-3)))
+    with ClockSampler(local, period_s=0.02) as cs:
+        e0.record()
+        for _ in range(n):
+            rot.step()
+        e1.record()
+        torch.cuda.synchronize()
+    rot.check()
+    ms = e0.elapsed_time(e1) / n
+    v, u = unit_value(wl, ms)
+    key = "hbm_gbs" if wl.name == "c4" else "bf16_tflops_sustained"
+    blk = {"steps": n, "seconds": round(ms * n / 1e3, 3), "ms_per_step": round(ms, 5), "value": round(v, 2), "unit": u,
+           "clocks": cs.summary()}
+    if wl.dtype == wk.BF16 and peaks.get(key):
+        blk["frac_of_sustained_peak"] = round(v / peaks[key], 4)
+        blk["peak"] = peaks[key]
+        blk["note"] = f"peak = {key} of {peaks['_source']}"
+    return blk, n
+
+
+def back_to_back_us(rot, torch, calls=1000):
     """Microseconds per call of `calls` calls issued without anything in between (operands stay in
     L2): what a latency-bound problem costs inside a stream of work."""
-    step = op.bind(d["X"], d["W"], d["b"], d["gamma"], d["beta"], d["out"])
     for _ in range(20):
-        step()
+        rot.step()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(calls):
-        step()
+        rot.step()
     e1.record()
     torch.cuda.synchronize()
-    op.check()
+    rot.check()
     return 1e3 * e0.elapsed_time(e1) / calls
 
 
@@ -268,7 +357,7 @@ def eager_context_us(wl, d, torch, steps=10):
     return 1e3 * e0.elapsed_time(e1) / steps
 
 
-def roofline_of(wl, ms, peaks, kernel, sm_max_mhz, sm_count):
+def roofline_of(wl, ms, peaks, kernel, sm_max_mhz, sm_count, alu_peak=None):
     """Roofline of the (single) kernel of a step: achieved = algorithmic work / measured time."""
     src = peaks["_source"]
     if wl.name == "c4":
@@ -286,9 +375,15 @@ def roofline_of(wl, ms, peaks, kernel, sm_max_mhz, sm_count):
                 f"scheme: a third of the peak); peak = cuBLAS bf16 burst, of {src}, x the nominal TF32/bf16 ratio 1.1/2.25")
     else:
         ach = wl.flops / ms / 1e9
-        peak = sm_count * 128 * 2 * (sm_max_mhz or 1965.0) * 1e6 / 1e12
+        derived = sm_count * 128 * 2 * (sm_max_mhz or 1965.0) * 1e6 / 1e12
         unit, bound = "TFLOP/s", "alu"
-        note = "fp32 FFMA peak = SMs x 128 lanes x 2 flop x max SM clock (derived, not measured)"
+        if alu_peak:
+            peak = alu_peak
+            note = (f"fp32 FFMA peak measured on this GPU with a register-only FMA loop (forge_selftest_ffma_rate); "
+                    f"SMs x 128 lanes x 2 flop x max SM clock would be {derived:.2f}")
+        else:
+            peak = derived
+            note = "fp32 FFMA peak = SMs x 128 lanes x 2 flop x max SM clock (derived, not measured)"
     key = NCU_TRAFFIC.get(wl.name)
     traffic = key["bytes"] if key and key["sha"] == kernel_source_hash(kernel) else None
     return {"bound": bound, "achieved": round(ach, 2), "peak": round(peak, 2), "unit": unit,
@@ -296,9 +391,10 @@ def roofline_of(wl, ms, peaks, kernel, sm_max_mhz, sm_count):
 
 
 def unit_value(wl, ms, n_units=1):
+    """Whole-job rate: the units (bytes or flops of one workload) all ranks processed / the slowest rank's time."""
     if wl.name == "c4":
-        return n_units * wl.algorithmic_bytes / ms / 1e6, "GB/s"
-    return n_units * wl.flops / ms / 1e9, "TFLOP/s"
+        return multigpu.aggregate_rate(wl.algorithmic_bytes, n_units, ms) / 1e9, "GB/s"
+    return multigpu.aggregate_rate(wl.flops, n_units, ms) / 1e12, "TFLOP/s"
 
 
 # ---- CPU oracle leg -------------------------------------------------------------------------------
@@ -455,10 +551,76 @@ def config_of(wl, n_gpus, extra=None):
     c = {"workload": f"{wl.name}: {wl.note}", "M_per_gpu": wl.M, "N": wl.N, "K": wl.K,
          "dtype": "bf16" if wl.dtype == wk.BF16 else "f32", "act": names[wl.act], "scale": wl.scale,
          "reduction": reds[wl.red], "seed": wl.seed, "parallelism": f"rows sharded over {n_gpus} gpu(s), no collective",
-         "l2": "operands larger than L2 (126 MB): no flush" if wl.algorithmic_bytes > 130e6 else "L2 flushed before every call"}
+         "l2": l2_policy(wl)}
     if extra:
         c.update(extra)
     return c
+
+
+EXTRA_STEPS = {"c1": 200, "c2": 20, "c4": 300, "c5": 50, "c3": 50, "n1": 20, "n2": 10, "c2t": 50, "n1t": 50, "n1b": 50}
+
+
+def measure_extra(w2, local, torch, peaks, props, alu_peak):
+    """One of the other workloads, measured the same way as the headline (shorter), with its own clock
+    record.  Returns (entry, launches)."""
+    i2 = wk.make_inputs(w2)
+    d2 = device_tensors(w2, i2, torch)
+    rot = Rotation(w2, d2, local, torch, copies=w_copies(w2))
+    fl = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device="cuda") if w2.algorithmic_bytes < 130e6 else None
+    steps2 = EXTRA_STEPS[w2.name]
+    with ClockSampler(local, period_s=0.001) as cs:
+        ms2 = time_steps(rot, steps2, 3, torch, flush_buf=fl)
+    clocks2 = cs.summary()
+    v2, u2 = unit_value(w2, ms2)
+    launches = steps2 + 3
+    entry = {"us_per_call": round(ms2 * 1e3, 2), "value": round(v2, 2), "unit": u2, "steps": steps2,
+             "l2": l2_policy(w2), "clocks": clocks2, "kernel": rot.plan.as_dict()["kernel"]}
+    if fl is not None:            # latency-bound workload: also the figure without the flush
+        entry["us_per_call_back_to_back_warm_l2"] = round(back_to_back_us(rot, torch), 2)
+        launches += 1020
+    if w2.name == "c4":           # HBM-bound: one call alone on the device, beside the back-to-back figure
+        med, best = isolated_us(rot, torch)
+        entry["us_per_call_isolated"] = {"median": round(med, 2), "min": round(best, 2), "calls": 30,
+                                         "how": "a synchronise after every call; W copies rotated as in the timed loop"}
+        entry["w_copies"] = {"count": len(rot.steps), "bytes": rot.w_bytes}
+        launches += 30
+    entry["roofline"] = roofline_of(w2, ms2, peaks, rot.plan.kernel, clocks2.get("sm_max_mhz"), props.multi_processor_count, alu_peak)
+    time.sleep(1.0)
+    entry["torch_eager_context_us"] = round(eager_context_us(w2, d2, torch, steps=5 if w2.flops > 1e11 else 50), 1)
+    rot.close()
+    return entry, launches
+
+
+def run_kernel_only(args, wl, torch, local):
+    """--kernel-only: `steps` launches of the workload's kernel on (the first --rows rows of) its seeded
+    input, each timed alone, nothing else on the device: the launch sequence to profile."""
+    from paper_2511_01884_b200 import binding as B
+    M = args.rows or wl.M
+    inp = wk.make_inputs(wl, M=M)
+    d = device_tensors(wl, inp, torch)
+    rot = Rotation(wl, d, local, torch, copies=1)
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        rot.step()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(round(1e3 * e0.elapsed_time(e1), 1))
+    rot.check()
+    print(json.dumps({"kernel_only": True, "workload": wl.name, "M": M, "N": wl.N, "K": wl.K,
+                      "kernel": B.kernel_name(rot.plan.kernel), "plan": rot.plan.as_dict(), "us_per_launch": times}), flush=True)
+    rot.close()
+    return 0
+
+
+def l2_policy(wl):
+    if wl.name == "c4":
+        return "HBM-bound: three distinct copies of W (768 MiB) rotated, no byte of a W is in L2 when it is read again"
+    if wl.algorithmic_bytes > 130e6:
+        return "operands larger than L2 (126 MB), compute-bound: no flush"
+    return "L2 flushed (256 MiB write) before every call"
 
 
 def main():
@@ -468,12 +630,19 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=HEADLINE, choices=sorted(ALL_WORKLOADS))
     ap.add_argument("--impl", default="forge", choices=["forge", "reference"])
-    ap.add_argument("--no-extras", action="store_true", help="skip the short runs of the other workloads")
+    ap.add_argument("--no-extras", action="store_true", help="skip the sustained block and the short runs of the other workloads")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="only launch the workload's kernel --steps times, each timed alone (for use under a profiler)")
+    ap.add_argument("--rows", type=int, default=0, help="with --kernel-only: use only the first ROWS rows of X (a smaller case)")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="with --shard rows and N > 1: weak = every rank runs the whole workload on its own rows of a global X; "
+                         "strong = the workload's M rows are split over the ranks")
     ap.add_argument("--shard", default="rows", choices=["rows", "cols"],
                     help="rows: every rank its own rows of X (weak scaling, no collective); cols: the rows of W of one "
                          "skinny-M problem over the ranks, partial out[M] combined by an all-reduce (strong scaling)")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3)
+    if not args.kernel_only:
+        args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         return run_reference(args)
 
@@ -500,19 +669,25 @@ def main():
     if args.shard == "cols":
         return run_column_sharded(args, wl, torch, dist, rank, world, local, peaks, props)
 
+    if args.kernel_only:
+        return run_kernel_only(args, wl, torch, local)
+
     # this rank's block of rows of the global [world * M, K] input; W, b, gamma, beta replicated
-    rows, row_offset = multigpu.rank_rows_weak(wl, rank)
+    strong = args.scaling == "strong"       # one workload's rows split over the ranks instead of one workload per rank
+    rows, row_offset = multigpu.rank_rows_strong(wl, rank, world) if strong else multigpu.rank_rows_weak(wl, rank)
+    n_units = 1 if strong else world
     inp = wk.make_inputs(wl, M=rows, row_offset=row_offset)
     d = device_tensors(wl, inp, torch)
-    op = make_op(wl, wl.M, local)
+    rot = Rotation(wl, d, local, torch, copies=w_copies(wl))
     flush = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device="cuda") if wl.algorithmic_bytes < 130e6 else None
 
-    with ClockSampler(local) as cs:
-        ms = time_steps(op, d, args.steps, args.warmup, torch, flush_buf=flush, barrier=barrier)
+    with ClockSampler(local, period_s=0.001) as cs:
+        ms = time_steps(rot, args.steps, args.warmup, torch, flush_buf=flush, barrier=barrier)
     clocks = cs.summary()
     ms_max = multigpu.max_over_ranks(ms, dist if world > 1 else None, device="cuda")
-    value, unit = unit_value(wl, ms_max, n_units=world)
+    value, unit = unit_value(wl, ms_max, n_units=n_units)
     launches = args.steps * 1
+    op = rot.ops[0]
 
     # ---- end to end: pinned host buffers in, result out, through the host entry point ----
     e2e_steps = max(1, min(args.steps, 10))
@@ -531,22 +706,33 @@ def main():
     torch.cuda.synchronize()
     e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
     e2e_ms = multigpu.max_over_ranks(e2e_ms, dist if world > 1 else None, device="cuda")
-    e2e_val, _ = unit_value(wl, e2e_ms, n_units=world)
+    e2e_val, _ = unit_value(wl, e2e_ms, n_units=n_units)
     same = bool(torch.equal(host_out.cuda(), d["out"]))
     op.check()
 
+    # the measured fp32 ceiling: a register-only FMA loop on every SM
+    alu_peak = None
+    if rank == 0 and world == 1:
+        from paper_2511_01884_b200 import binding as B
+        time.sleep(1.0)
+        st, tf, mhz = B.forge_selftest_ffma_rate(local, 200)
+        if st == B.FORGE_OK:
+            alu_peak = tf
     line = {"metric": f"fused-op {unit} ({wl.name})", "value": round(value, 2), "unit": unit, "n_gpus": n_gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_max, 5), "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == wk.BF16 else "f32",
-            "data": "synthetic", "config": config_of(wl, n_gpus, {"kernel": op.plan.as_dict()}),
+            "scaling": args.scaling, "vs_baseline": None, "dtype": "bf16" if wl.dtype == wk.BF16 else "f32",
+            "data": "synthetic", "config": config_of(wl, n_gpus, {"kernel": op.plan.as_dict(), "M_per_gpu": rows}),
             "clocks": clocks,
             "e2e": {"value": round(e2e_val, 3), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": round(e2e_ms, 3),
                     "matches_device_run": same, "how": "forge_fused_linear_run_host, pinned host buffers, wall clock"},
             "gpu_launches": launches,
-            "roofline": roofline_of(wl, ms, peaks, op.plan.kernel, clocks.get("sm_max_mhz"), props.multi_processor_count),
+            "roofline": roofline_of(wl, ms * wl.M / rows, peaks, op.plan.kernel, clocks.get("sm_max_mhz"), props.multi_processor_count, alu_peak),
             "nominal_frac": round((value / world) / (NOMINAL["hbm_gbs"] if wl.name == "c4" else NOMINAL["bf16_tflops"]), 4)
             if wl.dtype == wk.BF16 else None}
+    if alu_peak:
+        line["alu_peak_measured"] = {"value": round(alu_peak, 2), "unit": "TFLOP/s", "effective_sm_mhz": round(mhz, 1),
+                                     "how": "forge_selftest_ffma_rate: 200 ms of independent register-to-register fma.rn.f32x2 on every SM, CUDA events"}
     # the static half of the paper's hardware feedback (Section 2.3): what the device is
     line["gpu_spec"] = {"name": props.name, "compute_capability": f"{props.major}.{props.minor}",
                         "sms": props.multi_processor_count, "l2_bytes": getattr(props, "L2_cache_size", None),
@@ -555,49 +741,30 @@ def main():
                         "registers_per_sm": getattr(props, "regs_per_multiprocessor", None),
                         "measured_peaks": {k: peaks.get(k) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained")},
                         "peaks_source": peaks["_source"]}
-    eager_us = None
     if rank == 0 and world == 1:
         time.sleep(2.0)
         eager_us = eager_context_us(wl, d, torch, steps=args.steps)      # same number of back-to-back calls as the timed region
         line["torch_eager_context"] = {"us_per_call": round(eager_us, 1), "value": round(unit_value(wl, eager_us / 1e3)[0], 2),
                                        "unit": unit, "what": "unfused F.linear + activation (+ reduction) in the same dtype, same GPU"}
-    op.close()
+        if not args.no_extras:
+            # seconds of back-to-back launches: the clock the power limit allows, not the burst clock
+            time.sleep(1.0)
+            line["sustained"], n_sus = sustained_block(rot, wl, peaks, local, torch)
+            launches += n_sus + 20
+    rot.close()
     del d, host
 
     if rank == 0 and world == 1:
         line["cpu_baseline"] = {k: v for k, v in oracle_sample(wl, inp).items() if k not in ("seconds", "rows")}
         if not args.no_extras:
             line["workloads"] = {}
-            every = dict(wk.WORKLOADS)
-            every.update(wk.EXTRA_WORKLOADS)
-            for name in sorted(every):
+            for name in sorted(ALL_WORKLOADS):
                 if name == wl.name:
                     continue
-                w2 = every[name]
                 torch.cuda.empty_cache()
                 time.sleep(2.0)      # each workload is measured from the same (burst) power state, not in the wake of the previous one
-                i2 = wk.make_inputs(w2)
-                d2 = device_tensors(w2, i2, torch)
-                op2 = make_op(w2, w2.M, local)
-                fl = torch.empty(64 * 1024 * 1024, dtype=torch.float32, device="cuda") if w2.algorithmic_bytes < 130e6 else None
-                steps2 = {"c1": 200, "c2": 20, "c4": 200, "c5": 50, "c3": 50, "n1": 20, "n2": 10, "c2t": 50, "n1t": 50, "n1b": 50}[name]
-                ms2 = time_steps(op2, d2, steps2, 3, torch, flush_buf=fl)
-                v2, u2 = unit_value(w2, ms2)
-                launches += steps2
-                b2b = None
-                if fl is not None:            # latency-bound workload: also the figure without the flush
-                    b2b = back_to_back_us(op2, d2, torch)
-                    launches += 1020
-                time.sleep(1.0)
-                eg = eager_context_us(w2, d2, torch, steps=5 if w2.flops > 1e11 else 50)
-                line["workloads"][name] = {"torch_eager_context_us": round(eg, 1), "us_per_call": round(ms2 * 1e3, 2), "value": round(v2, 2), "unit": u2,
-                                           "steps": steps2, "l2": "flushed before every call" if fl is not None else "operands larger than L2",
-                                           **({"us_per_call_back_to_back_warm_l2": round(b2b, 2)} if b2b is not None else {}),
-                                           "kernel": op2.plan.as_dict()["kernel"],
-                                           "roofline": roofline_of(w2, ms2, peaks, op2.plan.kernel, clocks.get("sm_max_mhz"),
-                                                                   props.multi_processor_count)}
-                op2.close()
-                del d2, i2, fl
+                line["workloads"][name], n2 = measure_extra(ALL_WORKLOADS[name], local, torch, peaks, props, alu_peak)
+                launches += n2
             line["gpu_launches_all_workloads"] = launches
     if rank == 0:
         print(json.dumps(line), flush=True)

@@ -24,7 +24,8 @@ EXPORTS = [
     "forge_fused_linear_query_plan", "forge_fused_linear_create", "forge_fused_linear_run",
     "forge_fused_linear_run_host", "forge_fused_linear_last_status", "forge_fused_linear_get_plan",
     "forge_fused_linear_launches_per_run", "forge_fused_linear_destroy", "forge_fused_linear_last_wait_detail",
-    "forge_fused_linear_f32_reduce_static", "forge_selftest_bounded_wait", "forge_status_string", "forge_kernel_name",
+    "forge_fused_linear_f32_reduce_static", "forge_selftest_bounded_wait", "forge_selftest_ffma_rate",
+    "forge_status_string", "forge_kernel_name", "forge_fused_linear_kernel_name",
 ]
 
 
@@ -79,7 +80,10 @@ def lib() -> ctypes.CDLL:
         L.forge_fused_linear_f32_reduce_static.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, i, i,
                                                            ctypes.c_float, vp, vp, vp, vp, vp]
         L.forge_selftest_bounded_wait.argtypes = [i, i, ctypes.POINTER(ctypes.c_int * 4)]
-        for n in EXPORTS[:11]:
+        L.forge_selftest_ffma_rate.argtypes = [i, i, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+        L.forge_fused_linear_kernel_name.argtypes = [vp]
+        L.forge_fused_linear_kernel_name.restype = ctypes.c_char_p
+        for n in EXPORTS[:12]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -149,6 +153,17 @@ def forge_selftest_bounded_wait(device: int = 0, budget_ms: int = 50):
     d = (ctypes.c_int * 4)()
     st = lib().forge_selftest_bounded_wait(int(device), int(budget_ms), ctypes.byref(d))
     return st, list(d)
+
+
+def forge_selftest_ffma_rate(device: int = 0, milliseconds: int = 200):
+    """(status, TFLOP/s, effective SM MHz) of the register-only FMA loop: the measured fp32 ceiling."""
+    t, f = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    st = lib().forge_selftest_ffma_rate(int(device), int(milliseconds), ctypes.byref(t), ctypes.byref(f))
+    return st, t.value, f.value
+
+
+def forge_fused_linear_kernel_name(h) -> str:
+    return lib().forge_fused_linear_kernel_name(h).decode()
 
 
 def forge_fused_linear_get_plan(h) -> PlanInfo:

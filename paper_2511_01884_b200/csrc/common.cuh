@@ -22,7 +22,7 @@ struct Epilogue {
 // Status word layout: 0 = ok; otherwise (FORGE_ERR_TIMEOUT << 16) | location code.
 enum WaitSite : int {
     SITE_TMA_FULL = 1, SITE_STAGE_EMPTY = 2, SITE_ACC_FULL = 3, SITE_ACC_EMPTY = 4,
-    SITE_ARRIVAL = 5, SITE_STORE = 6, SITE_CLUSTER = 7, SITE_SPLIT = 8
+    SITE_ARRIVAL = 5, SITE_SPLIT = 8
 };
 
 // Words 1..3 of the status area describe the first give-up: a caller-chosen detail word, the
@@ -138,15 +138,63 @@ __device__ __forceinline__ void lse_merge(float &m, float &s, float om, float os
     s = a + b;
 }
 
-// Order-preserving map float -> unsigned (for an order-independent atomic max).
-__device__ __forceinline__ unsigned float_to_ordered(float f)
+// ---- counters that CTAs of one launch wait on --------------------------------------------------
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
 {
-    const unsigned u = __float_as_uint(f);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
-__device__ __forceinline__ float ordered_to_float(unsigned u)
+
+__device__ __forceinline__ uint64_t wait_clock_ns()
 {
-    return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Budget of every device-side wait: about two seconds of wall clock.
+constexpr uint64_t kWaitBudgetNs = 2000000000ull;
+
+// Poll until *counter has reached `target` (counters only ever grow; the difference is taken
+// modulo 2^32).  Gives up -- returning false -- when another thread has already recorded a give-up
+// in the status word or when the budget is spent, in which case the give-up is recorded with
+// `site` and `detail`.  SLEEP_NS > 0 backs off between polls.
+template <int SLEEP_NS>
+__device__ __forceinline__ bool wait_counter(const unsigned *counter, unsigned target, int *status, int site, int detail)
+{
+    uint64_t t0 = 0;
+    for (uint32_t it = 1; (int)(ld_acquire_u32(counter) - target) < 0; ++it) {
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+        if ((it & 0x3f) == 0) {
+            if (*(volatile int *)status != 0) return false;
+            const uint64_t now = wait_clock_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitBudgetNs) {
+                report_timeout(status, site, detail);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// Run index of a launch whose CTAs wait on one another's arrival counters.  Those counters are
+// never reset: every run adds a fixed number of arrivals to each, so run r is complete at r times
+// that number.  r itself lives in device memory -- gen[0] = runs completed, gen[1] = CTAs of the
+// current run that have finished -- so that nothing about a launch depends on how many launches
+// the host has issued before (a launch that failed, or one replayed from a captured graph, sees
+// the right index).  Every CTA reads the index when it starts and reports when it ends; the CTA
+// that ends last publishes the new count.  One run per handle in flight.
+__device__ __forceinline__ unsigned run_index_begin(const unsigned *gen) { return ld_acquire_u32(gen) + 1u; }
+__device__ __forceinline__ void run_index_end(unsigned *gen, unsigned run)
+{
+    __threadfence();
+    if (atomicAdd(gen + 1, 1u) == gridDim.x - 1) {
+        gen[1] = 0u;
+        __threadfence();
+        *(volatile unsigned *)gen = run;
+    }
 }
 
 constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }

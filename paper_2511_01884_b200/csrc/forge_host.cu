@@ -22,18 +22,13 @@ bool desc_enums_ok(const forge_fused_linear_desc_t &d)
 
 // Largest M served by the skinny kernel.  Up to 32 rows it streams W a few percent faster than
 // the tensor-core tile kernel (148 CTAs against N/256 tiles); from there on its mma.sync rate,
-// not the stream, sets the time and the tile kernel wins.  FORGE_SKINNY_MAX_M (0..32) lowers the
-// limit, for comparing the two kernels on the same problem.
-int64_t skinny_max_m()
-{
-    static const int64_t v = [] {
-        const char *e = std::getenv("FORGE_SKINNY_MAX_M");
-        if (!e || !*e) return (int64_t)32;
-        const long x = std::strtol(e, nullptr, 10);
-        return (int64_t)(x < 0 ? 0 : x > 32 ? 32 : x);
-    }();
-    return v;
-}
+// not the stream, sets the time and the tile kernel wins.  A tuning build may lower the limit
+// (-DFORGE_SKINNY_MAX_M=0..32) to compare the two kernels on the same problem.
+#ifndef FORGE_SKINNY_MAX_M
+#define FORGE_SKINNY_MAX_M 32
+#endif
+static_assert(FORGE_SKINNY_MAX_M >= 0 && FORGE_SKINNY_MAX_M <= 32, "the skinny kernel carries at most 32 rows");
+constexpr int64_t skinny_max_m() { return FORGE_SKINNY_MAX_M; }
 
 forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
@@ -131,12 +126,12 @@ static forge_status_t encode_tmap(CUtensorMap *tm, CUtensorMapDataType type, siz
     const cuuint64_t strides[1] = {cols * elem};              // bytes, dimension 1
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    // FORGE_TMA_L2_PROMOTION = 0 | 64 | 128 | 256 overrides the L2 fetch granularity (tuning aid)
-    static int promo = -1;
-    if (promo < 0) {
-        const char *e = std::getenv("FORGE_TMA_L2_PROMOTION");
-        promo = e ? std::atoi(e) : 256;
-    }
+    // L2 fetch granularity of the tensor maps: 256 bytes measured best; a tuning build may set
+    // -DFORGE_TMA_L2_PROMOTION=0|64|128|256
+#ifndef FORGE_TMA_L2_PROMOTION
+#define FORGE_TMA_L2_PROMOTION 256
+#endif
+    constexpr int promo = FORGE_TMA_L2_PROMOTION;
     const CUtensorMapL2promotion l2 = promo == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
                                       : promo == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
                                       : promo == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B
@@ -176,7 +171,72 @@ __global__ void forge_wait_selftest_kernel(int *status, unsigned long long budge
     if (threadIdx.x == 32) ptx::mbar_wait(&bar, 0, status, SITE_TMA_FULL, detail, budget_ns);
 }
 
+// Register-only fused multiply-add loop: 16 independent packed-pair chains per thread, nothing but
+// FMA-pipe work in the loop body.  What it sustains is the ceiling of any FFMA kernel on this device
+// at the clock the device actually holds under that load.
+__global__ void __launch_bounds__(512, 2) forge_ffma_rate_kernel(float *sink, float a0, float b0, int iters)
+{
+    unsigned long long acc[16], a, b;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(a) : "f"(a0));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(b) : "f"(b0));
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float v = (float)(threadIdx.x + i);
+        asm("mov.b64 %0, {%1, %1};" : "=l"(acc[i]) : "f"(v));
+    }
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int i = 0; i < 16; ++i) asm volatile("fma.rn.f32x2 %0, %0, %1, %2;" : "+l"(acc[i]) : "l"(a), "l"(b));
+    }
+    unsigned long long x = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x ^= acc[i];
+    if (x == 0x7ff0dead7ff0beefull) sink[0] = 1.f;      // keeps the chains alive; practically never true
+}
+
 extern "C" {
+
+forge_status_t forge_selftest_ffma_rate(int device, int milliseconds, double *tflops, double *sm_mhz_effective)
+{
+    if (!tflops || milliseconds <= 0 || milliseconds > 2000 || device < 0) return FORGE_ERR_INVALID_ARG;
+    DeviceGuard g(device);
+    if (!g.ok) return FORGE_ERR_CUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms <= 0) return FORGE_ERR_CUDA;
+    float *sink = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaMalloc(&sink, 256) != cudaSuccess) { cudaGetLastError(); return FORGE_ERR_ALLOC; }
+    forge_status_t st = FORGE_ERR_CUDA;
+    if (cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess) {
+        const int grid = 2 * sms, threads = 512;
+        // calibrate on a short launch, then size one launch for the requested duration
+        int iters = 2048;
+        float ms = 0.f;
+        bool ok = true;
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+            ok = cudaEventRecord(e0) == cudaSuccess;
+            forge_ffma_rate_kernel<<<grid, threads>>>(sink, 0.999f, 1e-3f, iters);
+            ok = ok && cudaGetLastError() == cudaSuccess && cudaEventRecord(e1) == cudaSuccess &&
+                 cudaEventSynchronize(e1) == cudaSuccess && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess && ms > 0.f;
+            if (ok && pass == 0) {
+                const double want = (double)iters * milliseconds / ms;
+                iters = want > 1e8 ? 100000000 : (want < 1024 ? 1024 : (int)want);
+            }
+        }
+        if (ok) {
+            const double fmas = (double)grid * threads * (double)iters * 4 * 16 * 2;      // two lanes per packed instruction
+            *tflops = 2.0 * fmas / (ms * 1e-3) / 1e12;
+            if (sm_mhz_effective) *sm_mhz_effective = fmas / (ms * 1e-3) / ((double)sms * 128.0) / 1e6;
+            st = FORGE_OK;
+        }
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(sink);
+    return st;
+}
 
 forge_status_t forge_selftest_bounded_wait(int device, int budget_ms, int detail[4])
 {
@@ -273,12 +333,8 @@ forge_status_t forge_fused_linear_run(forge_fused_linear_t hh, const void *X, co
 // kHostPipeMaxBlocks blocks, and only when X is large enough for the overlap to matter.
 static int64_t host_block_rows(const forge_fused_linear_desc_t &d)
 {
-    static const int env = [] {          // FORGE_HOST_PIPELINE=0: one upload, one kernel, one download
-        const char *e = std::getenv("FORGE_HOST_PIPELINE");
-        return e ? std::atoi(e) : 1;
-    }();
     const size_t bx = (size_t)d.M * (size_t)d.K * elem_bytes(d);
-    if (!env || d.M < 1024 || bx < ((size_t)8 << 20)) return 0;
+    if (d.M < 1024 || bx < ((size_t)8 << 20)) return 0;
     const int64_t want = (d.M + kHostPipeMaxBlocks - 1) / kHostPipeMaxBlocks;
     return ((want + 255) / 256) * 256;
 }
@@ -370,16 +426,20 @@ forge_status_t forge_fused_linear_run_host(forge_fused_linear_t hh, const void *
              cudaMemcpyAsync(h.hbe, beta, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
     if (ok && has_sub) ok = cudaMemcpyAsync(h.hg, gamma, bn, cudaMemcpyHostToDevice, s) == cudaSuccess;
     if (ok && has_tgt) ok = cudaMemcpyAsync(h.hg, gamma, bt, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (!ok) return FORGE_ERR_CUDA;
+    // after the first enqueue no path returns before the stream has drained: a copy still in flight
+    // would go on reading the caller's buffers (or writing `out`) after the call has returned
+    if (!ok) { cudaStreamSynchronize(s); return FORGE_ERR_CUDA; }
     const void *aux = (d.red == FORGE_RED_LAYERNORM || has_sub || has_tgt) ? h.hg : nullptr;
 
     if (!pp) {
-        if (cudaMemcpyAsync(h.hX, X, bx, cudaMemcpyHostToDevice, s) != cudaSuccess) return FORGE_ERR_CUDA;
-        RunArgs a{h.hX, h.hW, d.has_bias ? h.hb : nullptr, aux, h.hbe, h.hout, s};
-        const forge_status_t st = dispatch(h, a);
-        if (st != FORGE_OK) return st;
-        if (cudaMemcpyAsync(out, h.hout, bo, cudaMemcpyDeviceToHost, s) != cudaSuccess) return FORGE_ERR_CUDA;
-        return cudaStreamSynchronize(s) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+        forge_status_t st = cudaMemcpyAsync(h.hX, X, bx, cudaMemcpyHostToDevice, s) == cudaSuccess ? FORGE_OK : FORGE_ERR_CUDA;
+        if (st == FORGE_OK) {
+            RunArgs a{h.hX, h.hW, d.has_bias ? h.hb : nullptr, aux, h.hbe, h.hout, s};
+            st = dispatch(h, a);
+        }
+        if (st == FORGE_OK && cudaMemcpyAsync(out, h.hout, bo, cudaMemcpyDeviceToHost, s) != cudaSuccess) st = FORGE_ERR_CUDA;
+        const bool drained = cudaStreamSynchronize(s) == cudaSuccess;
+        return st != FORGE_OK ? st : (drained ? FORGE_OK : FORGE_ERR_CUDA);
     }
 
     // Blocks of rows: every reduction here runs along N, so a block of rows is a complete problem.
@@ -434,7 +494,6 @@ forge_status_t forge_fused_linear_last_status(forge_fused_linear_t hh)
     if (word != 0) {
         // a give-up may have left arrival counters half way: clear the whole workspace
         cudaMemset(h.ws.base, 0, h.ws.bytes);
-        h.run_gen = 0;
         return (forge_status_t)(word >> 16);
     }
     return FORGE_OK;
@@ -459,6 +518,11 @@ forge_status_t forge_fused_linear_get_plan(forge_fused_linear_t hh, forge_plan_i
 }
 
 int forge_fused_linear_launches_per_run(forge_fused_linear_t hh) { return hh ? 1 : 0; }
+
+const char *forge_fused_linear_kernel_name(forge_fused_linear_t hh)
+{
+    return hh ? forge_kernel_name(reinterpret_cast<Handle *>(hh)->info.kernel) : "no handle";
+}
 
 forge_status_t forge_fused_linear_destroy(forge_fused_linear_t hh)
 {

@@ -21,8 +21,6 @@
 // through global memory; the un-normalised tile never leaves the SM.  The wait is hidden
 // behind the MMAs of the next tile (other TMEM buffer).  CTAs wait on one another, so the
 // launch is cooperative and a strip may not have more tiles than there are CTAs.
-#include <cstdlib>
-
 #include "common.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
@@ -45,7 +43,17 @@ template <bool PAIR> struct K2Ring {
     static constexpr int STAGES = PAIR ? 6 : 4;
     static constexpr uint32_t BYTES = STAGES * STAGE_BYTES;      // 192 KiB either way
 };
-constexpr int K2_GROUP_M = 16;      // 128-row tiles per rasterisation group (keeps a wave's operands in L2)
+// Tuning builds may override these three (-DFORGE_K2_GROUP_M=.. and so on); the defaults are the measured best.
+#ifndef FORGE_K2_GROUP_M
+#define FORGE_K2_GROUP_M 16
+#endif
+#ifndef FORGE_K2_PAIR
+#define FORGE_K2_PAIR 1            // 0: one CTA per tile, never CTA pairs
+#endif
+#ifndef FORGE_K2_TAIL_SPLIT
+#define FORGE_K2_TAIL_SPLIT 1      // 0: never cut the last wave's tiles along K
+#endif
+constexpr int K2_GROUP_M = FORGE_K2_GROUP_M;      // 128-row tiles per rasterisation group (keeps a wave's operands in L2)
 
 struct K2Smem {
     uint64_t full[K2_MAX_STAGES];
@@ -75,17 +83,15 @@ struct K2Params {
     int *status;
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     int group_m;          // row units per rasterisation group
-    unsigned ln_target;   // layernorm: counter value at which a strip is complete in this run
+    unsigned *gen;        // launches whose CTAs wait on one another: run index (see run_index_begin)
     // K split of the last wave's tiles (tail_parts = 1: none)
     int tail_parts;           // S
     int tail_kb;              // k-blocks per part
     float4 *tail_scratch;     // [tail tile][part - 1][rank][column half][32][128] float4: raw accumulators
-    unsigned *tail_flags;     // [tail tile][rank][column half]; only ever grow
-    unsigned tail_target;     // value a flag reaches when parts 1..S-1 of this run have arrived
-    int cooperative;          // host only: CTAs of this launch wait on one another
+    unsigned *tail_flags;     // [tail tile][rank][column half]; only ever grow: tail_parts - 1 arrivals per run
+    int cooperative;          // CTAs of this launch wait on one another
     float *rowg;              // mean chain: gelu(mean) per row, [M]
-    unsigned *strips_done;    // mean chain: strips whose rowg values are published; only ever grows
-    unsigned strips_target;   // ... and the value it reaches when this run's strips are all done
+    unsigned *strips_done;    // mean chain: strips whose rowg values are published; only ever grows: tiles_m per run
 };
 
 template <bool LN>
@@ -148,13 +154,6 @@ __device__ __forceinline__ bool k2_item(const K2Params &p, int j, int unit, int 
 // named barrier of epilogue group g (ids 1 and 2; 0 is __syncthreads)
 __device__ __forceinline__ void epi_bar_sync(int g) { asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(K2_EPI_THREADS) : "memory"); }
 
-__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
-{
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-
 // PAIR: the kernel runs as clusters of two CTAs on one TPC.  A pair owns a 256x256 output tile:
 // CTA `rank` loads rows [128 rank, 128 rank + 128) of the X tile and of the W tile; the leader
 // (rank 0) issues tcgen05.mma.cta_group::2, which accumulates 128 rows x 256 columns in the TMEM
@@ -180,6 +179,8 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
     const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // this CTA's (pair's) place among ...
     const int units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;        // ... the units that share the work
     bool ok = true;
+    // counters that CTAs wait on only ever grow: this run is complete at `run` times the arrivals of one run
+    const unsigned run = p.cooperative ? run_index_begin(p.gen) : 0u;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&s.full[i], 1); ptx::mbar_init(&s.empty[i], 1); }
@@ -338,22 +339,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                     if ((acc ^= 1) == 0) acc_phase ^= 1;
                     continue;
                 }
-                if (et == 0) {
-                    uint64_t t0 = 0;
-                    for (uint32_t it = 1; (int)(ld_acquire_u32(flag) - p.tail_target) < 0; ++it) {
-                        __nanosleep(100);
-                        if ((it & 0x3f) == 0) {
-                            if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
-                            const uint64_t now = ptx::globaltimer_ns();
-                            if (t0 == 0) t0 = now;
-                            else if (now - t0 > ptx::kWaitBudgetNs) {
-                                report_timeout(p.status, SITE_ARRIVAL, w.tail);
-                                s.abort_flag = 1;
-                                break;
-                            }
-                        }
-                    }
-                }
+                if (et == 0 && !wait_counter<100>(flag, run * (unsigned)(p.tail_parts - 1), p.status, SITE_ARRIVAL, w.tail)) s.abort_flag = 1;
                 epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
                 __threadfence();
@@ -428,19 +414,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 epi_bar_sync(h);
                 if (et == 0) {
                     atomicAdd(&p.counters[tm], 1u);
-                    uint64_t t0 = 0;
-                    for (uint32_t it = 1; (int)(ld_acquire_u32(&p.counters[tm]) - p.ln_target) < 0; ++it) {
-                        if ((it & 0xff) == 0) {
-                            if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
-                            const uint64_t now = ptx::globaltimer_ns();
-                            if (t0 == 0) t0 = now;
-                            else if (now - t0 > ptx::kWaitBudgetNs) {
-                                report_timeout(p.status, SITE_ARRIVAL, tm);
-                                s.abort_flag = 1;
-                                break;
-                            }
-                        }
-                    }
+                    if (!wait_counter<0>(&p.counters[tm], run * (unsigned)parts, p.status, SITE_ARRIVAL, tm)) s.abort_flag = 1;
                 }
                 epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
@@ -659,22 +633,8 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
     // that finished it would stall that CTA's pipeline for the duration).  CTAs wait on one another
     // here: the launch is cooperative (all CTAs resident) and the wait is bounded.
     if (!LN && p.e.red == FORGE_RED_MEAN_GELU_RESIDUAL) {
-        if (threadIdx.x == 0) {
-            uint64_t t0 = 0;
-            for (uint32_t it = 1; (int)(ld_acquire_u32(p.strips_done) - p.strips_target) < 0; ++it) {
-                __nanosleep(200);
-                if ((it & 0x3f) == 0) {
-                    if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
-                    const uint64_t now = ptx::globaltimer_ns();
-                    if (t0 == 0) t0 = now;
-                    else if (now - t0 > ptx::kWaitBudgetNs) {
-                        report_timeout(p.status, SITE_ARRIVAL, (int)blockIdx.x);
-                        s.abort_flag = 1;
-                        break;
-                    }
-                }
-            }
-        }
+        if (threadIdx.x == 0 && !wait_counter<200>(p.strips_done, run * (unsigned)p.tiles_m, p.status, SITE_ARRIVAL, (int)blockIdx.x))
+            s.abort_flag = 1;
         __syncthreads();
         if (!*(volatile int *)&s.abort_flag) {
             const size_t k8 = (size_t)(p.K >> 3), total = (size_t)p.M * k8;
@@ -707,19 +667,15 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         if (PAIR) ptx::tmem_dealloc_pair(tmem_base, K2_TMEM_COLS);
         else ptx::tmem_dealloc(tmem_base, K2_TMEM_COLS);
     }
+    if (p.cooperative && threadIdx.x == 0) run_index_end(p.gen, run);
 }
 
 // ---- host side ---------------------------------------------------------------------------
-// CTA pairs need at least two 128-row strips and two SMs.  FORGE_K2_PAIR=0 forces one CTA per
-// tile (tuning aid).
+// CTA pairs need at least two 128-row strips and two SMs (a tuning build with -DFORGE_K2_PAIR=0
+// runs one CTA per tile throughout).
 static bool k2_use_pair(const forge_fused_linear_desc_t &d, int sm_count)
 {
-    static int env = -1;
-    if (env < 0) {
-        const char *e = std::getenv("FORGE_K2_PAIR");
-        env = e ? (std::atoi(e) != 0) : 1;
-    }
-    return env && d.M > K2_BM && sm_count >= 2;
+    return FORGE_K2_PAIR != 0 && d.M > K2_BM && sm_count >= 2;
 }
 
 // Grid, K split of the last wave and workspace layout of the non-LayerNorm kernel: a pure function of
@@ -733,7 +689,7 @@ struct K2Layout {
     int64_t tiles_m, tiles_n, units, slots, grid;      // slots: CTAs (or CTA pairs) the GPU offers
     int tail_parts, tail_kb, tail_tiles;
     size_t rowg_off, scratch_off, partial_floats;      // float offsets into the partial area
-    size_t strips_done_idx, tail_flags_idx, counters;
+    size_t strips_done_idx, tail_flags_idx, gen_idx, counters;
 };
 
 static K2Layout k2_layout(const forge_fused_linear_desc_t &d, int sm_count)
@@ -746,10 +702,7 @@ static K2Layout k2_layout(const forge_fused_linear_desc_t &d, int sm_count)
     L.slots = L.pair ? sm_count / 2 : sm_count;
     const int64_t full = L.units / L.slots, rest = L.units % L.slots;
     const int num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
-    static const int env = [] {          // FORGE_K2_TAIL_SPLIT=0: never cut the last wave's tiles along K
-        const char *e = std::getenv("FORGE_K2_TAIL_SPLIT");
-        return e ? std::atoi(e) : 1;
-    }();
+    constexpr bool env = FORGE_K2_TAIL_SPLIT != 0;
     int parts = 1;
     if (env && rest > 0 && full < K2_TAIL_MAX_FULL_WAVES && d.red != FORGE_RED_LAYERNORM) {
         int64_t s = L.slots / rest;
@@ -771,7 +724,8 @@ static K2Layout k2_layout(const forge_fused_linear_desc_t &d, int sm_count)
     L.partial_floats = L.scratch_off + (size_t)L.tail_tiles * (L.tail_parts - 1) * 2 * 2 * (4 * 32 * K2_EPI_THREADS);
     L.strips_done_idx = fold ? (size_t)L.tiles_m : 0;
     L.tail_flags_idx = L.strips_done_idx + (chain ? 1 : 0);
-    L.counters = L.tail_flags_idx + (size_t)L.tail_tiles * 4;
+    L.gen_idx = L.tail_flags_idx + (size_t)L.tail_tiles * 4;       // run index and finished-CTA count
+    L.counters = L.gen_idx + 2;
     return L;
 }
 
@@ -834,7 +788,7 @@ forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     if (tiles_n > sm_count / info->cluster) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_BF16_TCGEN05_LN;
     wl->partial_floats = 4 * 2 * (size_t)tiles_n * (size_t)d.M;          // one float4 per row and half tile
-    wl->counters = (size_t)tiles_m;
+    wl->counters = (size_t)tiles_m + 2;                                   // strips, then run index and finished-CTA count
     return FORGE_OK;
 }
 
@@ -903,35 +857,23 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     p.tiles_m = (int)((d.M + K2_BM - 1) / K2_BM);
     p.tiles_n = (int)((d.N + K2_BN - 1) / K2_BN);
     p.num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
-    p.ln_target = 0;
-    {
-        static int env = -1;        // FORGE_K2_GROUP_M overrides the rasterisation group (tuning aid)
-        if (env < 0) {
-            const char *e = std::getenv("FORGE_K2_GROUP_M");
-            env = e ? std::atoi(e) : 0;
-        }
-        p.group_m = env > 0 ? env : (pair ? K2_GROUP_M / 2 : K2_GROUP_M);      // 2048 rows either way
-    }
-    // The counters that CTAs wait on only ever grow: run r is complete at r times the arrivals of one run
-    // (mean chain: strips; K split: parts 1..S-1 of a tile; LayerNorm: half tiles of a strip).
-    h.run_gen += 1;
+    p.group_m = pair ? K2_GROUP_M / 2 : K2_GROUP_M;      // 2048 rows either way
     if (!ln) {
         const K2Layout L = k2_layout(d, h.sm_count);
         p.rowg = h.ws.partial + L.rowg_off;
         p.strips_done = h.ws.counters + L.strips_done_idx;
-        p.strips_target = h.run_gen * (unsigned)p.tiles_m;
         p.tail_parts = L.tail_parts;
         p.tail_kb = L.tail_kb;
         p.tail_scratch = reinterpret_cast<float4 *>(h.ws.partial + L.scratch_off);
         p.tail_flags = h.ws.counters + L.tail_flags_idx;
-        p.tail_target = h.run_gen * (unsigned)(L.tail_parts - 1);
+        p.gen = h.ws.counters + L.gen_idx;
         p.cooperative = d.red == FORGE_RED_MEAN_GELU_RESIDUAL || L.tail_parts > 1;
         return pair ? k2_launch_t<false, true>(h, p, a.stream) : k2_launch_t<false, false>(h, p, a.stream);
     }
     p.tail_parts = 1;
     p.tail_kb = p.num_kb;
     p.cooperative = 1;
-    p.ln_target = h.run_gen * 2u * (unsigned)p.tiles_n;      // half tiles of a strip
+    p.gen = h.ws.counters + p.tiles_m;
     return pair ? k2_launch_t<true, true>(h, p, a.stream) : k2_launch_t<true, false>(h, p, a.stream);
 }
 

@@ -53,8 +53,6 @@
 // (bounded) for the strip's other half tiles, combines the statistics in part order and normalises
 // out of TMEM.  The mean chain publishes gelu(mean) per row and the whole grid writes the residual
 // rows at the end.  In both, and with the K cut, CTAs wait on one another: the launch is cooperative.
-#include <cstdlib>
-
 #include "common.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
@@ -73,8 +71,18 @@ constexpr uint32_t K5_RAW_BYTES = K5_A_BYTES + K5_B_BYTES;         // what TMA w
 constexpr uint32_t K5_STAGE_BYTES = 2 * K5_RAW_BYTES;              // raw/hi, then lo
 constexpr uint32_t K5_RING_BYTES = K5_STAGES * K5_STAGE_BYTES;     // 192 KiB
 constexpr uint32_t K5_TMEM_COLS = 512;
-constexpr int K5_GROUP_M = 8;       // 256-row units per rasterisation group
-constexpr int K5_CHUNK_KB = 4;      // ring stages (32 k each) accumulated in TMEM before the epilogue drains them
+// Tuning builds may override these three (-DFORGE_K5_GROUP_M=.. and so on); the defaults are the measured best.
+#ifndef FORGE_K5_GROUP_M
+#define FORGE_K5_GROUP_M 8
+#endif
+#ifndef FORGE_K5_CHUNK_KB
+#define FORGE_K5_CHUNK_KB 4
+#endif
+#ifndef FORGE_K5_TAIL_SPLIT
+#define FORGE_K5_TAIL_SPLIT 1      // 0: never cut the last wave's tiles along K
+#endif
+constexpr int K5_GROUP_M = FORGE_K5_GROUP_M;       // 256-row units per rasterisation group
+constexpr int K5_CHUNK_KB = FORGE_K5_CHUNK_KB;     // ring stages (32 k each) accumulated in TMEM before the epilogue drains them
 // Register shares after setmaxnreg: the epilogue warpgroups hold a 128-value running sum per
 // thread; producer, issuer and splitters need little.  The sum of the shares must not exceed the
 // registers the CTA was launched with (checked on the host before the first launch).
@@ -110,15 +118,15 @@ struct K5Params {
     const float *X;             // mean chain only: the residual input
     const void *aux;            // mean chain: sub[N] (float); cross-entropy: target[M] (int32); LayerNorm: gamma[N]
     const float *beta;          // LayerNorm
-    unsigned ln_target;         // LayerNorm: value a strip's counter reaches when all its half tiles of this run are in
+    unsigned *gen;              // launches whose CTAs wait on one another: run index (see run_index_begin)
+    int cooperative;            // CTAs of this launch wait on one another
     void *out;
     int M, N, K;
     Epilogue e;
     float *partial;             // per half tile: [2*tiles_n][M] floats (float4 for the softmax statistics)
     unsigned *counters;         // [tiles_m]
     float *rowg;                // mean chain: gelu(mean) per row, [M]
-    unsigned *strips_done;      // mean chain: strips whose rowg values are published; only ever grows
-    unsigned strips_target;     // ... and the value it reaches when this run's strips are all done
+    unsigned *strips_done;      // mean chain: strips whose rowg values are published; only ever grows: tiles_m per run
     int *status;
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     int group_m;
@@ -127,8 +135,7 @@ struct K5Params {
     int tail_parts;             // S
     int tail_kb;                // k-blocks per part
     float4 *tail_scratch;       // [tail tile][part - 1][rank][column half][32][128] float4
-    unsigned *tail_flags;       // [tail tile][rank][column half]; only ever grow
-    unsigned tail_target;       // value a flag reaches when parts 1..S-1 of this run have arrived
+    unsigned *tail_flags;       // [tail tile][rank][column half]; only ever grow: tail_parts - 1 arrivals per run
 };
 
 // One unit of work of a cluster: a pair tile and a range of k-blocks.  Cluster c takes the whole
@@ -185,13 +192,6 @@ __device__ __forceinline__ void k5_tile_coords(int t, int units_m, int tiles_n, 
     tn = r / gm;
 }
 
-__device__ __forceinline__ unsigned ld_acquire_gpu_u32(const unsigned *p)
-{
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-
 __device__ __forceinline__ void k5_epi_bar_sync(int g) { asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(K5_EPI_THREADS) : "memory"); }
 
 __global__ void __launch_bounds__(K5_THREADS, 1)
@@ -206,6 +206,8 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     const int units_m = (p.tiles_m + 1) / 2;              // 256-row units
     const int cluster = (int)(blockIdx.x >> 1), clusters = (int)(gridDim.x >> 1);
     bool ok = true;
+    // counters that CTAs wait on only ever grow: this run is complete at `run` times the arrivals of one run
+    const unsigned run = p.cooperative ? run_index_begin(p.gen) : 0u;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < K5_STAGES; ++i) {
@@ -412,22 +414,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     if ((acc ^= 1) == 0) acc_phase ^= 1;
                     continue;
                 }
-                if (et == 0) {
-                    uint64_t t0 = 0;
-                    for (uint32_t it = 1; (int)(ld_acquire_gpu_u32(flag) - p.tail_target) < 0; ++it) {
-                        __nanosleep(100);
-                        if ((it & 0x3f) == 0) {
-                            if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
-                            const uint64_t now = ptx::globaltimer_ns();
-                            if (t0 == 0) t0 = now;
-                            else if (now - t0 > ptx::kWaitBudgetNs) {
-                                report_timeout(p.status, SITE_ARRIVAL, w.tail);
-                                s.abort_flag = 1;
-                                break;
-                            }
-                        }
-                    }
-                }
+                if (et == 0 && !wait_counter<100>(flag, run * (unsigned)(p.tail_parts - 1), p.status, SITE_ARRIVAL, w.tail)) s.abort_flag = 1;
                 k5_epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
                 __threadfence();
@@ -499,19 +486,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 k5_epi_bar_sync(h);
                 if (et == 0) {
                     atomicAdd(&p.counters[tm], 1u);
-                    uint64_t t0 = 0;
-                    for (uint32_t it = 1; (int)(ld_acquire_gpu_u32(&p.counters[tm]) - p.ln_target) < 0; ++it) {
-                        if ((it & 0xff) == 0) {
-                            if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
-                            const uint64_t now = ptx::globaltimer_ns();
-                            if (t0 == 0) t0 = now;
-                            else if (now - t0 > ptx::kWaitBudgetNs) {
-                                report_timeout(p.status, SITE_ARRIVAL, tm);
-                                s.abort_flag = 1;
-                                break;
-                            }
-                        }
-                    }
+                    if (!wait_counter<0>(&p.counters[tm], run * 2u * (unsigned)p.tiles_n, p.status, SITE_ARRIVAL, tm)) s.abort_flag = 1;
                 }
                 k5_epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
@@ -688,22 +663,8 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     // strip by whichever epilogue group finished a strip (which stalled that CTA's pipeline).
     // CTAs wait on one another here: the launch is cooperative (all CTAs resident) and the wait is bounded.
     if (p.e.red == FORGE_RED_MEAN_GELU_RESIDUAL) {
-        if (threadIdx.x == 0) {
-            uint64_t t0 = 0;
-            for (uint32_t it = 1; (int)(ld_acquire_gpu_u32(p.strips_done) - p.strips_target) < 0; ++it) {
-                __nanosleep(200);
-                if ((it & 0x3f) == 0) {
-                    if (*(volatile int *)p.status != 0) { s.abort_flag = 1; break; }
-                    const uint64_t now = ptx::globaltimer_ns();
-                    if (t0 == 0) t0 = now;
-                    else if (now - t0 > ptx::kWaitBudgetNs) {
-                        report_timeout(p.status, SITE_ARRIVAL, (int)blockIdx.x);
-                        s.abort_flag = 1;
-                        break;
-                    }
-                }
-            }
-        }
+        if (threadIdx.x == 0 && !wait_counter<200>(p.strips_done, run * (unsigned)p.tiles_m, p.status, SITE_ARRIVAL, (int)blockIdx.x))
+            s.abort_flag = 1;
         __syncthreads();
         if (!*(volatile int *)&s.abort_flag) {
             const size_t k4 = (size_t)(p.K >> 2), total = (size_t)p.M * k4;
@@ -729,6 +690,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         ptx::tc_fence_after();
         ptx::tmem_dealloc_pair(tmem_base, K5_TMEM_COLS);
     }
+    if (p.cooperative && threadIdx.x == 0) run_index_end(p.gen, run);
 }
 
 // ---- host side ---------------------------------------------------------------------------
@@ -744,7 +706,7 @@ struct K5Layout {
     size_t rowg_off;          // mean chain: gelu(mean) per row (float offset into the partial area)
     size_t scratch_off;       // K split: hand-over area (float offset, multiple of 4)
     size_t partial_floats;
-    size_t strips_done_idx, tail_flags_idx, counters;
+    size_t strips_done_idx, tail_flags_idx, gen_idx, counters;
 };
 
 static K5Layout k5_layout(const forge_fused_linear_desc_t &d, int sm_count)
@@ -756,10 +718,7 @@ static K5Layout k5_layout(const forge_fused_linear_desc_t &d, int sm_count)
     L.clusters = sm_count / 2;
     const int64_t full = L.units / L.clusters, rest = L.units % L.clusters;
     const int num_kb = (int)((d.K + K5_BK - 1) / K5_BK);
-    static const int env = [] {          // FORGE_K5_TAIL_SPLIT=0: never cut the last wave's tiles along K
-        const char *e = std::getenv("FORGE_K5_TAIL_SPLIT");
-        return e ? std::atoi(e) : 1;
-    }();
+    constexpr bool env = FORGE_K5_TAIL_SPLIT != 0;
     const bool ln = d.red == FORGE_RED_LAYERNORM;
     int parts = 1;
     if (env && rest > 0 && full < K5_TAIL_MAX_FULL_WAVES && !ln) {        // LayerNorm: a tile already waits for its strip; no second dependency
@@ -781,7 +740,8 @@ static K5Layout k5_layout(const forge_fused_linear_desc_t &d, int sm_count)
     L.partial_floats = L.scratch_off + (size_t)L.tail_tiles * (L.tail_parts - 1) * 2 * 2 * (4 * 32 * K5_EPI_THREADS);
     L.strips_done_idx = fold ? (size_t)L.tiles_m : 0;
     L.tail_flags_idx = L.strips_done_idx + (chain ? 1 : 0);
-    L.counters = L.tail_flags_idx + (size_t)L.tail_tiles * 4;
+    L.gen_idx = L.tail_flags_idx + (size_t)L.tail_tiles * 4;       // run index and finished-CTA count
+    L.counters = L.gen_idx + 2;
     return L;
 }
 
@@ -860,35 +820,19 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
     p.status = h.ws.status;
     p.tiles_m = (int)((d.M + K5_BM - 1) / K5_BM);
     const K5Layout L = k5_layout(d, h.sm_count);
-    h.run_gen += 1;                                          // the wait counters only ever grow: run r ends at r * arrivals per run
+    p.gen = h.ws.counters + L.gen_idx;
+    p.cooperative = k5_ctas_wait(h);
     p.rowg = h.ws.partial + L.rowg_off;
     p.strips_done = h.ws.counters + L.strips_done_idx;
-    p.strips_target = h.run_gen * (unsigned)p.tiles_m;
     p.tail_parts = L.tail_parts;
     p.tail_kb = L.tail_kb;
     p.tail_scratch = reinterpret_cast<float4 *>(h.ws.partial + L.scratch_off);
     p.tail_flags = h.ws.counters + L.tail_flags_idx;
-    p.tail_target = h.run_gen * (unsigned)(L.tail_parts - 1);
     p.beta = (const float *)a.beta;
-    p.ln_target = h.run_gen * 2u * (unsigned)L.tiles_n;      // strip counters only ever grow under LayerNorm
     p.tiles_n = (int)((d.N + K5_BN - 1) / K5_BN);
     p.num_kb = (int)((d.K + K5_BK - 1) / K5_BK);
-    {
-        static int env = -1;        // FORGE_K5_GROUP_M overrides the rasterisation group (tuning aid)
-        if (env < 0) {
-            const char *e = std::getenv("FORGE_K5_GROUP_M");
-            env = e ? std::atoi(e) : 0;
-        }
-        p.group_m = d.red == FORGE_RED_LAYERNORM ? 0 : (env > 0 ? env : K5_GROUP_M);
-    }
-    {
-        static int env = -1;        // FORGE_K5_CHUNK_KB overrides the accumulation chunk (32 k per unit; tuning aid)
-        if (env < 0) {
-            const char *e = std::getenv("FORGE_K5_CHUNK_KB");
-            env = e ? std::atoi(e) : 0;
-        }
-        p.chunk_kb = env > 0 ? env : K5_CHUNK_KB;
-    }
+    p.group_m = d.red == FORGE_RED_LAYERNORM ? 0 : K5_GROUP_M;
+    p.chunk_kb = K5_CHUNK_KB;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)h.info.grid);
     cfg.blockDim = dim3(K5_THREADS);
@@ -901,7 +845,7 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (k5_ctas_wait(h) && cooperative_launch_enabled()) {
+    if (p.cooperative && cooperative_launch_enabled()) {
         attr[1].id = cudaLaunchAttributeCooperative;
         attr[1].val.cooperative = 1;
         cfg.numAttrs = 2;

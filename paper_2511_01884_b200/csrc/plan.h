@@ -5,8 +5,6 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include <cstdlib>
-
 #include "../../include/forge.h"
 
 namespace forge {
@@ -41,7 +39,6 @@ struct Handle {
     forge_plan_info_t info;
     int sm_count = 0;
     int last_detail[4] = {0, 0, 0, 0};   // status area as read by the last last_status() call
-    unsigned run_gen = 0;            // runs launched since the workspace was last cleared
     Workspace ws;
     // staging buffers of run_host()
     void *hX = nullptr, *hW = nullptr, *hb = nullptr, *hg = nullptr, *hbe = nullptr, *hout = nullptr;
@@ -55,16 +52,17 @@ struct Handle {
 };
 
 // Kernels whose CTAs wait on one another are launched cooperatively (all CTAs resident at once).
-// FORGE_K4_COOPERATIVE=0 drops the attribute: profilers refuse cooperative cluster launches.  The
-// grids never exceed the SM count and every wait is bounded, so the worst case on a GPU that is
-// busy with other work is a reported time-out, not a hang.
-inline bool cooperative_launch_enabled()
+// A profiling build (-DFORGE_PROFILING_NO_COOPERATIVE) drops the attribute, because profilers
+// refuse cooperative launches of clusters; it is not for production use: the grids never exceed
+// the SM count and every wait is bounded, so the worst case on a GPU that is busy with other work
+// is a reported time-out, not a hang, but co-residency is no longer guaranteed.
+constexpr bool cooperative_launch_enabled()
 {
-    static const int v = [] {
-        const char *e = std::getenv("FORGE_K4_COOPERATIVE");
-        return e ? (std::atoi(e) != 0) : 1;
-    }();
-    return v != 0;
+#ifdef FORGE_PROFILING_NO_COOPERATIVE
+    return false;
+#else
+    return true;
+#endif
 }
 
 // Layout of the workspace (element counts) for a plan; filled by the planners.

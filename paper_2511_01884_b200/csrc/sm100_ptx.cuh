@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the bf16 kernels use: mbarrier with
-// bounded waits, TMA tensor loads/stores (never multicast), tcgen05 (TMEM allocation, MMA,
+// bounded waits, TMA tensor loads (never multicast), tcgen05 (TMEM allocation, MMA,
 // commit, loads, fences), ldmatrix / mma.sync for the skinny kernel.  Written from the
 // public PTX ISA description of these instructions.
 #pragma once
@@ -15,12 +15,7 @@ namespace ptx {
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ uint64_t globaltimer_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
+__device__ __forceinline__ uint64_t globaltimer_ns() { return wait_clock_ns(); }
 
 __device__ __forceinline__ bool elect_one()
 {
@@ -80,10 +75,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 
-// Wait budget of every device-side wait: about two seconds of wall clock, checked every few
-// thousand polls.  On expiry -- or as soon as another thread has reported a give-up -- the
-// wait returns false; callers then leave their loops and fall through to the teardown.
-constexpr uint64_t kWaitBudgetNs = 2000000000ull;
+// The wait budget (forge::kWaitBudgetNs) is checked every few thousand polls.  On expiry -- or as
+// soon as another thread has reported a give-up -- the wait returns false; callers then leave
+// their loops and fall through to the teardown.
+using forge::kWaitBudgetNs;
 
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *status, int site, int detail = 0,
                                           uint64_t budget_ns = kWaitBudgetNs)
@@ -118,18 +113,7 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *tm, ui
         ::"r"(smem_u32(dst)), "l"((uint64_t)tm), "r"(smem_u32(bar)), "r"(x), "r"(y)
         : "memory");
 }
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *tm, const void *src, int x, int y)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"((uint64_t)tm), "r"(smem_u32(src)), "r"(x), "r"(y)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-template <int N>
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
-// generic-proxy writes to shared memory -> visible to the async proxy (TMA store)
+// generic-proxy writes to shared memory -> visible to the async proxy (tensor-core operand reads)
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---- tcgen05 / TMEM ------------------------------------------------------------------------

@@ -29,6 +29,24 @@ def test_library_exports_every_declared_symbol():
     assert declared == set(B.EXPORTS)
 
 
+def test_header_compiles_and_links_as_c99(tmp_path):
+    """include/forge.h is a C interface: a strict C99 translation unit includes it, links the library and
+    calls the host-only entry points and every NULL-argument path."""
+    exe = str(tmp_path / "header_c99")
+    pkg = os.path.dirname(B.LIB_PATH)
+    cmd = ["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+           os.path.join(ROOT, "tests", "c", "header_c99.c"), "-o", exe, "-L", pkg, "-lforge", f"-Wl,-rpath,{pkg}"]
+    r = subprocess.run(cmd, capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    r = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0, r.stdout + r.stderr
+    assert "ok" in r.stdout
+
+
+def test_kernel_name_of_a_handle_needs_a_handle():
+    assert B.forge_fused_linear_kernel_name(None) == "no handle"
+
+
 def test_no_vendor_gemm_library_is_linked():
     out = subprocess.run(["ldd", B.LIB_PATH], capture_output=True, text=True).stdout
     for lib in ("cublas", "cudnn", "cutlass", "nccl"):

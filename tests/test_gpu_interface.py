@@ -251,3 +251,61 @@ def test_nothing_is_written_outside_the_output(case):
     op.close()
     assert bool((buf[:guard] == 12345.0).all()) and bool((buf[guard + n_out:] == 12345.0).all())
     pu.assert_parity(wl, out.float().cpu().numpy().astype(np.float64), pu.run_oracle(wl, inp))
+
+
+@pytest.mark.parametrize("name", ["ln_bf16", "chain_bf16", "tailsplit_bf16", "ln_tf32x3", "rowsum_f32"])
+def test_run_captured_in_a_graph_replays_correctly(name):
+    """run() keeps no per-call state on the host: the counters that the CTAs of the LayerNorm, chain
+    and K-cut launches wait on take their run index from device memory.  So a run captured into a
+    CUDA graph and replayed (with other direct runs on the same handle in between) gives the same
+    bits as a direct run."""
+    import torch
+    wl = {"ln_bf16": wk.custom_workload("g_ln", wk.BF16, 300, 1032, 128, wk.ACT_GELU_TANH, wk.RED_LAYERNORM, w_std=0.05),
+          "chain_bf16": wk.custom_workload("g_chain", wk.BF16, 300, 520, 128, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL, w_std=0.05),
+          "tailsplit_bf16": wk.custom_workload("g_tail", wk.BF16, 256, 512, 4096, wk.ACT_SILU, wk.RED_NONE, w_std=0.02),
+          "ln_tf32x3": wk.custom_workload("g_ln5", wk.F32_TF32X3, 300, 520, 256, wk.ACT_GELU_TANH, wk.RED_LAYERNORM),
+          "rowsum_f32": wk.custom_workload("g_sum", wk.F32, 300, 700, 96, wk.ACT_RELU, wk.RED_SUM)}[name]
+    inp = wk.make_inputs(wl)
+    dev = {k: pu.to_device(v, wl.dtype) for k, v in inp.items() if k != "target"}
+    aux = dev["sub"] if wl.red == wk.RED_MEAN_GELU_RESIDUAL else dev["gamma"]
+    dt = {wk.F32: torch.float32, wk.BF16: torch.bfloat16, wk.F32_TF32X3: torch.float32}[wl.dtype]
+    shape = (wl.M,) if wl.out_cols == 0 else (wl.M, wl.out_cols)
+    direct = torch.full(shape, float("nan"), dtype=torch.float32 if wl.out_cols == 0 else dt, device="cuda")
+    replay = torch.full_like(direct, float("nan"))
+    op = B.FusedLinear(pu.desc_of(wl))
+    op(dev["X"], dev["W"], dev["b"], aux, dev["beta"], direct)            # first use outside any capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            op(dev["X"], dev["W"], dev["b"], aux, dev["beta"], replay, stream=side.cuda_stream)
+    torch.cuda.synchronize()
+    for i in range(3):
+        replay.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(replay, direct), (name, i)
+        op(dev["X"], dev["W"], dev["b"], aux, dev["beta"], direct)        # a direct run between the replays
+        torch.cuda.synchronize()
+    op.check()
+    op.close()
+    g = replay.float().cpu().numpy().astype(np.float64)
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
+def test_kernel_name_of_a_handle():
+    wl = wk.custom_workload("kn", wk.BF16, 16, 1024, 256, wk.ACT_GELU_ERF, wk.RED_MAX, w_std=0.05)
+    op = B.FusedLinear(pu.desc_of(wl))
+    assert B.forge_fused_linear_kernel_name(op.h) == B.kernel_name(op.plan.kernel) == "bf16_skinny_splitk"
+    op.close()
+
+
+def test_measured_ffma_rate_is_plausible():
+    import torch
+    st, tflops, mhz = B.forge_selftest_ffma_rate(0, 50)
+    assert st == B.FORGE_OK
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    nominal = sms * 128 * 2 * 1.965e9 / 1e12
+    assert 0.5 * nominal < tflops < 1.05 * nominal, (tflops, nominal)
+    assert 900.0 < mhz < 2100.0

@@ -60,6 +60,32 @@ def test_c1_through_static_scratch():
         assert pu.rel_err(g, want) <= pu.TOL[wk.F32]
 
 
+def test_calls_allocate_no_device_memory_and_bias_is_optional():
+    """What the entry point is for: after the first call on the device (which looks the array's address
+    up) further calls leave the amount of free device memory exactly as it was.  Also: b = NULL means
+    no bias."""
+    import torch
+    wl = wk.custom_workload("noalloc_nobias", wk.F32, 300, 700, 96, wk.ACT_SILU, wk.RED_SUM, seed=12, has_bias=False)
+    inp = wk.make_inputs(wl)
+    assert inp["b"] is None
+    dev = {k: pu.to_device(v, wl.dtype) for k, v in inp.items()}
+    out = torch.full((wl.M,), float("nan"), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        st = B.forge_fused_linear_f32_reduce_static(wl.M, wl.N, wl.K, wl.act, wl.red, wl.scale, dev["X"], dev["W"], None, out, stream)
+        assert st == B.FORGE_OK, B.status_string(st)
+    call()                                                          # first call on this device: symbol lookup
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(5):
+        call()
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
+    pu.assert_parity(wl, out.cpu().numpy().astype(np.float64), pu.run_oracle(wl, inp))
+
+
 def test_sizes_beyond_the_array_are_refused():
     import torch
     x = torch.zeros(16, device="cuda")
