@@ -1,7 +1,18 @@
-"""Build the CUDA library in-tree: ``python -m paper_2511_01884_b200.build``.
+"""Build the CUDA library in-tree: ``python -m paper_2511_01884_b200.build [-v] [-f] [-DNAME[=VALUE] ...]``.
 
 One shared object, ``libforge.so``, next to this file, from every ``csrc/*.cu``; compiled
 for sm_100a only (the kernels use tcgen05 / TMEM / TMA and have no other target).
+
+``-D`` options make a special-purpose build in place of the normal one (they force a full
+rebuild, and so does the next build without them):
+  -DFORGE_PROFILING_NO_COOPERATIVE   launch the kernels whose CTAs wait on one another without the
+                                     cooperative attribute (profilers refuse cooperative launches of
+                                     clusters); not for production use
+  -DFORGE_DEBUG_BOUNDS               check shared-memory ring offsets, TMEM columns and workspace indices
+                                     against their allocations and report the first violation through the
+                                     handle's status word instead of making the access
+  -DFORGE_K2_GROUP_M=.. -DFORGE_K2_PAIR=0 -DFORGE_K2_TAIL_SPLIT=0 -DFORGE_K5_GROUP_M=.. -DFORGE_K5_CHUNK_KB=..
+  -DFORGE_K5_TAIL_SPLIT=0 -DFORGE_TMA_L2_PROMOTION=0|64|128|256 -DFORGE_SKINNY_MAX_M=0..32   tuning variants
 """
 from __future__ import annotations
 
@@ -27,7 +38,16 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(verbose: bool = False, force: bool = False) -> str:
+def build(verbose: bool = False, force: bool = False, defines=()) -> str:
+    # a build with -D options, and the first build after one, recompile everything
+    stamp = os.path.join(OBJ, "defines.txt")
+    os.makedirs(OBJ, exist_ok=True)
+    want = " ".join(sorted(defines))
+    have = open(stamp).read() if os.path.exists(stamp) else ""
+    if want != have:
+        force = True
+        with open(stamp, "w") as f:
+            f.write(want)
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     hdrs = sorted(glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h")) +
                   glob.glob(os.path.join(HERE, "..", "include", "*.h")))
@@ -37,7 +57,7 @@ def build(verbose: bool = False, force: bool = False) -> str:
         o = os.path.join(OBJ, os.path.basename(s)[:-3] + ".o")
         objs.append(o)
         if force or _stale(o, [s] + hdrs):
-            cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            cmd = [NVCC] + FLAGS + list(defines) + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
 
     def run(cmd):
@@ -62,4 +82,4 @@ def build(verbose: bool = False, force: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv))
+    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, defines=[a for a in sys.argv[1:] if a.startswith("-D")]))

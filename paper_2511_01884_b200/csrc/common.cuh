@@ -146,6 +146,17 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
     return v;
 }
 
+// Count an arrival.  Release: everything this thread has observed -- its own writes and, through a
+// CTA barrier it has passed, the writes of the CTA's other threads -- is visible to whoever acquires
+// the counter later.  Acquire: what earlier arrivals had released is visible to this thread and, after
+// another CTA barrier, to the rest of the CTA (which must read it past L1, e.g. with __ldcg).
+__device__ __forceinline__ unsigned arrive_acq_rel(unsigned *counter)
+{
+    unsigned old;
+    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
+    return old;
+}
+
 __device__ __forceinline__ uint64_t wait_clock_ns()
 {
     uint64_t t;
@@ -189,11 +200,9 @@ __device__ __forceinline__ bool wait_counter(const unsigned *counter, unsigned t
 __device__ __forceinline__ unsigned run_index_begin(const unsigned *gen) { return ld_acquire_u32(gen) + 1u; }
 __device__ __forceinline__ void run_index_end(unsigned *gen, unsigned run)
 {
-    __threadfence();
-    if (atomicAdd(gen + 1, 1u) == gridDim.x - 1) {
+    if (arrive_acq_rel(gen + 1) == gridDim.x - 1) {      // the next reader is a later launch: nothing else to order
         gen[1] = 0u;
-        __threadfence();
-        *(volatile unsigned *)gen = run;
+        gen[0] = run;
     }
 }
 

@@ -55,6 +55,14 @@ forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_
     return FORGE_OK;
 }
 
+// Status word and counters to zero, the partial area to the byte its kernel expects between runs.
+bool clear_workspace(const Workspace &ws)
+{
+    const size_t head = (size_t)((char *)ws.partial - (char *)ws.base);
+    if (cudaMemset(ws.base, 0, head) != cudaSuccess) return false;
+    return ws.bytes == head || cudaMemset(ws.partial, ws.partial_fill, ws.bytes - head) == cudaSuccess;
+}
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;
@@ -298,11 +306,12 @@ forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, 
     if (!g.ok) { delete h; return FORGE_ERR_CUDA; }
     h->ws.bytes = (size_t)h->info.workspace_bytes;
     if (cudaMalloc(&h->ws.base, h->ws.bytes) != cudaSuccess) { cudaGetLastError(); delete h; return FORGE_ERR_ALLOC; }
-    if (cudaMemset(h->ws.base, 0, h->ws.bytes) != cudaSuccess) { cudaFree(h->ws.base); delete h; return FORGE_ERR_CUDA; }
     char *base = (char *)h->ws.base;
     h->ws.status = (int *)base;
     h->ws.counters = (unsigned *)(base + kStatusBytes);
     h->ws.partial = (float *)(base + kStatusBytes + ((wl.counters * sizeof(unsigned) + 255) / 256) * 256);
+    h->ws.partial_fill = wl.partial_fill;
+    if (!clear_workspace(h->ws)) { cudaFree(h->ws.base); delete h; return FORGE_ERR_CUDA; }
 
     switch (h->info.kernel) {
     case FORGE_KERNEL_F32_FFMA: st = k1_setup(*h); break;
@@ -493,7 +502,7 @@ forge_status_t forge_fused_linear_last_status(forge_fused_linear_t hh)
     const int word = h.last_detail[0];
     if (word != 0) {
         // a give-up may have left arrival counters half way: clear the whole workspace
-        cudaMemset(h.ws.base, 0, h.ws.bytes);
+        clear_workspace(h.ws);
         return (forge_status_t)(word >> 16);
     }
     return FORGE_OK;

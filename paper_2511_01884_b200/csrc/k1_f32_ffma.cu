@@ -295,12 +295,12 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         for (int i = 0; i < R; ++i)
 #pragma unroll
             for (int j = 0; j < R / 4; ++j) mine[i * (R / 4) + j] = make_float4(acc[i][4 * j], acc[i][4 * j + 1], acc[i][4 * j + 2], acc[i][4 * j + 3]);
-        __threadfence();
+        // one arrival per CTA by one thread: its release covers what the barrier has ordered before it, its acquire
+        // (and the next barrier) what the other slices' CTAs had written (read below past L1)
         __syncthreads();
-        if (tid == 0) s_last = (atomicAdd(&slice_counters[tile], 1u) == (unsigned)(k_slices - 1));
+        if (tid == 0) s_last = (arrive_acq_rel(&slice_counters[tile]) == (unsigned)(k_slices - 1));
         __syncthreads();
         if (!s_last) return;
-        __threadfence();
 #pragma unroll
         for (int i = 0; i < R; ++i)
 #pragma unroll
@@ -381,12 +381,10 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         }
         if (p.tiles_n > 1) {
             // the last CTA to arrive at this row strip folds the partials in tile order
-            __threadfence();
             __syncthreads();
-            if (tid == 0) s_last = (atomicAdd(&p.counters[tile_m], 1u) == (unsigned)(p.tiles_n - 1));
+            if (tid == 0) s_last = (arrive_acq_rel(&p.counters[tile_m]) == (unsigned)(p.tiles_n - 1));
             __syncthreads();
             if (!s_last) return;
-            __threadfence();
             if (tid < BM && m0 + tid < M) {
                 const int row = m0 + tid;
                 float v = __ldcg(&p.partial[row]);
@@ -464,12 +462,10 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
             }
         }
         if (p.tiles_n == 1) return;
-        __threadfence();
         __syncthreads();
-        if (tid == 0) s_last = (atomicAdd(&p.counters[tile_m], 1u) == (unsigned)(p.tiles_n - 1));
+        if (tid == 0) s_last = (arrive_acq_rel(&p.counters[tile_m]) == (unsigned)(p.tiles_n - 1));
         __syncthreads();
         if (!s_last) return;
-        __threadfence();
         if (tid < BM && m0 + tid < M) {
             const int row = m0 + tid;
             float4 f = __ldcg(&part4[row]);

@@ -330,9 +330,8 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                             dst[(c * 8 + i) * K2_EPI_THREADS + et] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
                                                                                  __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
                     }
-                    __threadfence();
                     epi_bar_sync(h);
-                    if (et == 0) atomicAdd(flag, 1u);
+                    if (et == 0) arrive_acq_rel(flag);      // its release covers the group's stores, ordered before it by the barrier
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
@@ -342,7 +341,6 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 if (et == 0 && !wait_counter<100>(flag, run * (unsigned)(p.tail_parts - 1), p.status, SITE_ARRIVAL, w.tail)) s.abort_flag = 1;
                 epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
-                __threadfence();
 #pragma unroll 1
                 for (int c = 0; c < CHUNKS; ++c) {
                     uint32_t r[32];
@@ -409,16 +407,16 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 ptx::tmem_st_wait();
                 float4 *stats = reinterpret_cast<float4 *>(p.partial);
                 if (row < p.M) stats[(size_t)part * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
-                // ---- publish, then wait (bounded) for the other parts of this strip ----
-                __threadfence();
+                // ---- publish, then wait (bounded) for the other parts of this strip: one arrival per group by one
+                //      thread (release: the group's triples, which the barrier orders before it; the acquiring polls
+                //      and the next barrier make the other groups' triples readable past L1) ----
                 epi_bar_sync(h);
                 if (et == 0) {
-                    atomicAdd(&p.counters[tm], 1u);
+                    arrive_acq_rel(&p.counters[tm]);
                     if (!wait_counter<0>(&p.counters[tm], run * (unsigned)parts, p.status, SITE_ARRIVAL, tm)) s.abort_flag = 1;
                 }
                 epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
-                __threadfence();
                 // Combine the strip's parts in part order, all at once (same result on every CTA):
                 // mean = sum n_i mean_i / sum n_i,  M2 = sum (M2_i + n_i (mean_i - mean)^2).
                 float rstd = 0.f, shift = 0.f;
@@ -513,13 +511,11 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 
                 float4 *part4 = reinterpret_cast<float4 *>(p.partial);
                 if (row < p.M) part4[(size_t)part * p.M + row] = make_float4(mx, se, tl, 0.f);
-                __threadfence();
                 epi_bar_sync(h);
-                if (et == 0) s.last_flag[h] = (atomicAdd(&p.counters[tm], 1u) == (unsigned)(parts - 1));
+                if (et == 0) s.last_flag[h] = (arrive_acq_rel(&p.counters[tm]) == (unsigned)(parts - 1));
                 epi_bar_sync(h);
                 if (s.last_flag[h]) {
                     // the group that arrives last at the strip merges the parts in order
-                    __threadfence();
                     if (row < p.M) {
                         float4 f = __ldcg(&part4[row]);
                         mx = f.x; se = f.y; tl = f.z;
@@ -591,12 +587,10 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 // per-part row partials; the group that arrives last at the strip folds them in order
                 float *out = reinterpret_cast<float *>(p.out);
                 if (row < p.M) p.partial[(size_t)part * p.M + row] = red;
-                __threadfence();
                 epi_bar_sync(h);
-                if (et == 0) s.last_flag[h] = (atomicAdd(&p.counters[tm], 1u) == (unsigned)(parts - 1));
+                if (et == 0) s.last_flag[h] = (arrive_acq_rel(&p.counters[tm]) == (unsigned)(parts - 1));
                 epi_bar_sync(h);
                 if (s.last_flag[h]) {
-                    __threadfence();
                     if (row < p.M) {
                         float v = __ldcg(&p.partial[row]);
                         int i = 1;
@@ -617,9 +611,8 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                     if (et == 0) p.counters[tm] = 0u;
                     if (chain) {
                         // the strip's gelu(mean) values are published; the rows are written at the end, by the whole grid
-                        __threadfence();
                         epi_bar_sync(h);
-                        if (et == 0) atomicAdd(p.strips_done, 1u);
+                        if (et == 0) arrive_acq_rel(p.strips_done);
                     }
                 }
             }

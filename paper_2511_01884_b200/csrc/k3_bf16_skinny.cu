@@ -339,12 +339,13 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                         else p.partial[slot_i] = running[mt];
                     }
                 }
-                __threadfence();
+                // one arrival per CTA, by one thread: its release covers the partials the barrier has ordered before
+                // it, its acquire (and the next barrier) the other CTAs' partials read below.  No fence per thread: a
+                // sequentially consistent fence on an SM with copies in flight costs microseconds.
                 k3_consumer_sync();
-                if (t == 0) s.last_flag = (atomicAdd(&p.counters[0], 1u) == gridDim.x - 1);
+                if (t == 0) s.last_flag = (arrive_acq_rel(&p.counters[0]) == gridDim.x - 1);
                 k3_consumer_sync();
                 if (s.last_flag) {
-                    __threadfence();
                     constexpr int CHUNKS = K3_CONSUMERS / ROWS;            // 16 or 8 chunks of CTAs per row
                     const int row = t % ROWS, chunk = t / ROWS;
                     float mx = p.e.red == FORGE_RED_SUM ? 0.f : -INFINITY, se = 0.f, tl = 0.f;

@@ -405,9 +405,8 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 #pragma unroll
                     for (int i = 0; i < HALF / 4; ++i)
                         dst[i * K5_EPI_THREADS + et] = make_float4(sum[4 * i], sum[4 * i + 1], sum[4 * i + 2], sum[4 * i + 3]);
-                    __threadfence();
                     k5_epi_bar_sync(h);
-                    if (et == 0) atomicAdd(flag, 1u);
+                    if (et == 0) arrive_acq_rel(flag);      // its release covers the group's stores, ordered before it by the barrier
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
@@ -417,7 +416,6 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 if (et == 0 && !wait_counter<100>(flag, run * (unsigned)(p.tail_parts - 1), p.status, SITE_ARRIVAL, w.tail)) s.abort_flag = 1;
                 k5_epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
-                __threadfence();
                 for (int pp = 1; pp < p.tail_parts; ++pp) {
                     const float4 *src = p.tail_scratch + ((((size_t)w.tail * (p.tail_parts - 1) + (pp - 1)) * 2 + rank) * 2 + h) * (32 * K5_EPI_THREADS);
 #pragma unroll
@@ -481,16 +479,16 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 ptx::tmem_st_wait();
                 float4 *stats = reinterpret_cast<float4 *>(p.partial);
                 if (row < p.M) stats[(size_t)part * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
-                // publish, then wait (bounded) for the other half tiles of the strip
-                __threadfence();
+                // publish, then wait (bounded) for the other half tiles of the strip: one arrival per group by one thread
+                // (release: the group's triples, ordered before it by the barrier; the acquiring polls and the next
+                // barrier make the other groups' triples readable past L1)
                 k5_epi_bar_sync(h);
                 if (et == 0) {
-                    atomicAdd(&p.counters[tm], 1u);
+                    arrive_acq_rel(&p.counters[tm]);
                     if (!wait_counter<0>(&p.counters[tm], run * 2u * (unsigned)p.tiles_n, p.status, SITE_ARRIVAL, tm)) s.abort_flag = 1;
                 }
                 k5_epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
-                __threadfence();
                 // the strip's parts combined in part order: mean = sum n_i mean_i / sum n_i, M2 = sum (M2_i + n_i (mean_i - mean)^2)
                 float rstd = 0.f, shift = 0.f;
                 if (row < p.M) {
@@ -598,12 +596,10 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     if (lse) part4[(size_t)part * p.M + row] = make_float4(mx, se, tl, 0.f);
                     else p.partial[(size_t)part * p.M + row] = acc_red;
                 }
-                __threadfence();
                 k5_epi_bar_sync(h);
-                if (et == 0) s.last_flag[h] = (atomicAdd(&p.counters[tm], 1u) == (unsigned)(parts - 1));
+                if (et == 0) s.last_flag[h] = (arrive_acq_rel(&p.counters[tm]) == (unsigned)(parts - 1));
                 k5_epi_bar_sync(h);
                 if (s.last_flag[h]) {
-                    __threadfence();
                     float *out = reinterpret_cast<float *>(p.out);
                     if (row < p.M) {
                         if (lse) {
@@ -647,9 +643,8 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     if (et == 0) p.counters[tm] = 0u;
                     if (chain) {
                         // the strip's gelu(mean) values are published; the rows are written at the end, by the whole grid
-                        __threadfence();
                         k5_epi_bar_sync(h);
-                        if (et == 0) atomicAdd(p.strips_done, 1u);
+                        if (et == 0) arrive_acq_rel(p.strips_done);
                     }
                 }
             }
