@@ -55,13 +55,8 @@ forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_
     return FORGE_OK;
 }
 
-// Status word and counters to zero, the partial area to the byte its kernel expects between runs.
-bool clear_workspace(const Workspace &ws)
-{
-    const size_t head = (size_t)((char *)ws.partial - (char *)ws.base);
-    if (cudaMemset(ws.base, 0, head) != cudaSuccess) return false;
-    return ws.bytes == head || cudaMemset(ws.partial, ws.partial_fill, ws.bytes - head) == cudaSuccess;
-}
+// Status word, counters and partials all start from zero.
+bool clear_workspace(const Workspace &ws) { return cudaMemset(ws.base, 0, ws.bytes) == cudaSuccess; }
 
 struct DeviceGuard {
     int prev = -1;
@@ -310,7 +305,6 @@ forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, 
     h->ws.status = (int *)base;
     h->ws.counters = (unsigned *)(base + kStatusBytes);
     h->ws.partial = (float *)(base + kStatusBytes + ((wl.counters * sizeof(unsigned) + 255) / 256) * 256);
-    h->ws.partial_fill = wl.partial_fill;
     if (!clear_workspace(h->ws)) { cudaFree(h->ws.base); delete h; return FORGE_ERR_CUDA; }
 
     switch (h->info.kernel) {

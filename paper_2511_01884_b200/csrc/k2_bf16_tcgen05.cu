@@ -13,14 +13,17 @@
 //
 // K4 (LayerNorm over N) is the same kernel with a different tile order and epilogue: the
 // N-tiles of one 128-row strip are consecutive tiles, hence run on different SMs at about
-// the same time.  Each epilogue makes one sweep over its accumulator (bias, activation,
-// scale, per-row (n, mean, M2) of its 256 columns, activated values written back to TMEM),
-// publishes the row triples to a small workspace, waits -- bounded -- until the strip's
-// other tiles have published theirs, merges the triples in tile order (Chan et al.), and
-// makes a second sweep over TMEM to normalise and store.  Only the 16-byte triples travel
-// through global memory; the un-normalised tile never leaves the SM.  The wait is hidden
-// behind the MMAs of the next tile (other TMEM buffer).  CTAs wait on one another, so the
-// launch is cooperative and a strip may not have more tiles than there are CTAs.
+// the same time.  Each epilogue group makes one sweep over its half of the accumulator (bias,
+// activation, scale, per-row (n, mean, M2) of its 128 columns), keeps the activated values in
+// registers (128 per thread; the epilogue warpgroups take a larger register share with
+// setmaxnreg, which is why this form runs 384 threads: warpgroup 0 = producer, issuer and two idle
+// warps) and hands the TMEM buffer back at once.  It then publishes the row triples to a small
+// workspace, waits -- bounded -- until the strip's other tiles have published theirs, merges the
+// triples in tile order (Chan et al.), normalises the registers and stores.  Only the 16-byte
+// triples travel through global memory; the un-normalised tile never leaves the SM.  The wait
+// costs the tensor cores nothing as long as it is shorter than two tiles: the MMAs of the next
+// two tiles have both TMEM buffers to go to.  CTAs wait on one another, so the launch is
+// cooperative and a strip may not have more tiles than there are CTAs.
 #include "common.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
@@ -29,8 +32,18 @@ namespace forge {
 
 constexpr int K2_BM = 128, K2_BN = 256, K2_BK = 64;
 constexpr int K2_MAX_STAGES = 6;
-constexpr int K2_THREADS = 320;              // TMA warp, MMA warp, 2 x 4 epilogue warps
 constexpr int K2_EPI_THREADS = 128;
+// Threads per CTA and first epilogue warp.  Plain form: TMA warp, MMA warp, 2 x 4 epilogue warps.  LayerNorm:
+// warpgroup 0 = TMA warp, MMA warp and two idle warps, warpgroups 1 and 2 = the two epilogue groups, so that
+// setmaxnreg (a warpgroup-wide instruction) can move registers from the former to the latter.
+template <bool LN> struct K2Shape {
+    static constexpr int THREADS = LN ? 384 : 320;
+    static constexpr int EPI_WARP0 = LN ? 4 : 2;
+};
+// LayerNorm register shares: 128 x 40 + 256 x 232 = 64512 = 384 x 168, what the CTA is launched with
+// (checked on the host before the first launch: setmaxnreg.inc waits for ever for registers that are not there).
+constexpr int K4_REGS_EPI = 232, K4_REGS_OTHER = 40;
+constexpr int K4_REGS_NEEDED = 128 * K4_REGS_OTHER + 256 * K4_REGS_EPI;
 constexpr uint32_t K2_A_BYTES = K2_BM * K2_BK * 2;
 constexpr uint32_t K2_TMEM_COLS = 512;
 // Shared-memory ring.  One CTA per tile: a stage holds the 128-row X tile and the 256-row W tile
@@ -162,7 +175,7 @@ __device__ __forceinline__ void epi_bar_sync(int g) { asm volatile("bar.sync %0,
 // full" barriers of both CTAs, the epilogues of both CTAs arrive on the leader's "accumulator
 // empty" barrier.
 template <bool LN, bool PAIR>
-__global__ void __launch_bounds__(K2_THREADS, 1)
+__global__ void __launch_bounds__(K2Shape<LN>::THREADS, 1)
 k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const K2Params p)
 {
     using Ring = K2Ring<PAIR>;
@@ -205,6 +218,10 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
     ptx::tc_fence_after();
     const uint32_t tmem_base = s.tmem_base;
 
+    constexpr int EPI_WARP0 = K2Shape<LN>::EPI_WARP0, THREADS = K2Shape<LN>::THREADS;
+    // LayerNorm: warpgroup 0 hands registers to the epilogue warpgroups (each warp of a warpgroup executes its own
+    // setmaxnreg; the compiler sizes the code that follows each one accordingly)
+    if (LN && warp < EPI_WARP0) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(K4_REGS_OTHER));
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (ptx::elect_one()) {
@@ -264,13 +281,14 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 if ((acc ^= 1) == 0) acc_phase ^= 1;
             }
         }
-    } else {
+    } else if (warp >= EPI_WARP0) {
         // ---------------- epilogue ----------------
+        if (LN) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(K4_REGS_EPI));
         // Two independent groups of four warps; group h owns columns [128h, 128h+128) of every
         // tile ("part" 2*tn + h of the row strip) and has its own named barrier.
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
-        const int h = (warp - 2) >> 2;                // column half
-        const int et = (threadIdx.x - 64) & (K2_EPI_THREADS - 1);     // 0..127 inside the group
+        const int h = (warp - EPI_WARP0) >> 2;        // column half
+        const int et = (threadIdx.x - 32 * EPI_WARP0) & (K2_EPI_THREADS - 1);     // 0..127 inside the group
         constexpr int HALF = K2_BN / 2, CHUNKS = HALF / 32;
         const int parts = 2 * p.tiles_n;
         int acc = 0;
@@ -363,48 +381,50 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             }
 
             if (LN) {
-                // ---- sweep 1: activated values back to TMEM, row statistics of this half tile ----
+                // ---- sweep 1: activated values into registers, row statistics of this half tile ----
+                float v[HALF];
                 RowStat rs{0.f, 0.f, 0.f};
-#pragma unroll 1
+#pragma unroll
                 for (int c = 0; c < CHUNKS; ++c) {
                     const int col0 = n0 + c * 32;
-                    if (col0 >= p.N) break;
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(taddr + c * 32, r);
-                    ptx::tmem_ld_wait();
-                    float v[32];
+                    if (col0 < p.N) {
+                        uint32_t r[32];
+                        ptx::tmem_ld_32x32(taddr + c * 32, r);
+                        ptx::tmem_ld_wait();
+                        float (&x)[32] = reinterpret_cast<float (&)[32]>(v[c * 32]);      // this chunk's slice of the registers
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
-                    apply_act_array<false>(p.e.act, v, p.e.scale);
+                        for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
+                        apply_act_array<false>(p.e.act, x, p.e.scale);
+                        const int nv = min(32, p.N - col0);
+                        RowStat cs;
+                        cs.n = (float)nv;
+                        if (nv == 32) {
+                            float sum = 0.f;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(v[j]);
-                    ptx::tmem_st_32x32(taddr + c * 32, r);
-                    const int nv = min(32, p.N - col0);
-                    RowStat cs;
-                    cs.n = (float)nv;
-                    if (nv == 32) {
-                        float sum = 0.f;
+                            for (int j = 0; j < 32; ++j) sum += x[j];
+                            cs.mean = sum * (1.0f / 32.0f);
+                            cs.m2 = 0.f;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) sum += v[j];
-                        cs.mean = sum * (1.0f / 32.0f);
-                        cs.m2 = 0.f;
+                            for (int j = 0; j < 32; ++j) { const float dlt = x[j] - cs.mean; cs.m2 = fmaf(dlt, dlt, cs.m2); }
+                        } else {
+                            float sum = 0.f;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) { const float dlt = v[j] - cs.mean; cs.m2 = fmaf(dlt, dlt, cs.m2); }
-                    } else {
-                        float sum = 0.f;
+                            for (int j = 0; j < 32; ++j) sum += j < nv ? x[j] : 0.f;
+                            cs.mean = sum / cs.n;
+                            cs.m2 = 0.f;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) sum += j < nv ? v[j] : 0.f;
-                        cs.mean = sum / cs.n;
-                        cs.m2 = 0.f;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const float dlt = j < nv ? v[j] - cs.mean : 0.f;
-                            cs.m2 = fmaf(dlt, dlt, cs.m2);
+                            for (int j = 0; j < 32; ++j) {
+                                const float dlt = j < nv ? x[j] - cs.mean : 0.f;
+                                cs.m2 = fmaf(dlt, dlt, cs.m2);
+                            }
                         }
+                        rs = merge_stat(rs, cs);
                     }
-                    rs = merge_stat(rs, cs);
                 }
-                ptx::tmem_st_wait();
+                // the accumulator is in registers: the TMEM buffer goes back to the MMA warp before the wait
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
                 float4 *stats = reinterpret_cast<float4 *>(p.partial);
                 if (row < p.M) stats[(size_t)part * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
                 // ---- publish, then wait (bounded) for the other parts of this strip: one arrival per group by one
@@ -437,38 +457,27 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                     rstd = rsqrtf(m2 / cnt + p.e.eps);
                     shift = -mean * rstd;
                 }
-                // ---- sweep 2: normalise out of TMEM and store ----
-#pragma unroll 1
-                for (int c = 0; c < CHUNKS; ++c) {
-                    const int col0 = n0 + c * 32;
-                    if (col0 >= p.N) break;
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(taddr + c * 32, r);
-                    ptx::tmem_ld_wait();
-                    if (row < p.M) {
-                        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)row * p.N + col0;
+                // ---- sweep 2: normalise the registers and store ----
+                if (row < p.M) {
+                    __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)row * p.N + n0;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            if (col0 + i * 8 < p.N) {
-                                float y[8];
+                    for (int i = 0; i < HALF / 8; ++i) {
+                        if (n0 + i * 8 < p.N) {
+                            float y[8];
 #pragma unroll
-                                for (int j = 0; j < 8; ++j) {
-                                    const int cc = c * 32 + i * 8 + j;
-                                    y[j] = fmaf(fmaf(__uint_as_float(r[i * 8 + j]), rstd, shift), sg[cc], sbe[cc]);
-                                }
-                                uint4 w;
-                                w.x = ptx::pack16x2(y[0], y[1], p.f16);
-                                w.y = ptx::pack16x2(y[2], y[3], p.f16);
-                                w.z = ptx::pack16x2(y[4], y[5], p.f16);
-                                w.w = ptx::pack16x2(y[6], y[7], p.f16);
-                                *reinterpret_cast<uint4 *>(dst + i * 8) = w;
+                            for (int j = 0; j < 8; ++j) {
+                                const int cc = i * 8 + j;
+                                y[j] = fmaf(fmaf(v[cc], rstd, shift), sg[cc], sbe[cc]);
                             }
+                            uint4 w4;
+                            w4.x = ptx::pack16x2(y[0], y[1], p.f16);
+                            w4.y = ptx::pack16x2(y[2], y[3], p.f16);
+                            w4.z = ptx::pack16x2(y[4], y[5], p.f16);
+                            w4.w = ptx::pack16x2(y[6], y[7], p.f16);
+                            *reinterpret_cast<uint4 *>(dst + i * 8) = w4;
                         }
                     }
                 }
-                ptx::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
                 if ((acc ^= 1) == 0) acc_phase ^= 1;
                 continue;
             }
@@ -633,7 +642,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             const size_t k8 = (size_t)(p.K >> 3), total = (size_t)p.M * k8;
             const uint4 *X8 = reinterpret_cast<const uint4 *>(p.X);
             uint4 *Y8 = reinterpret_cast<uint4 *>(p.out);
-            for (size_t e = (size_t)blockIdx.x * K2_THREADS + threadIdx.x; e < total; e += (size_t)gridDim.x * K2_THREADS) {
+            for (size_t e = (size_t)blockIdx.x * THREADS + threadIdx.x; e < total; e += (size_t)gridDim.x * THREADS) {
                 const float g = __ldcg(p.rowg + e / k8);
                 uint4 x = __ldg(X8 + e);
                 uint32_t *w = reinterpret_cast<uint32_t *>(&x);
@@ -733,7 +742,7 @@ forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     info->tile_k = K2_BK;
     info->stages = L.pair ? K2Ring<true>::STAGES : K2Ring<false>::STAGES;
     info->cluster = L.pair ? 2 : 1;
-    info->threads = K2_THREADS;
+    info->threads = K2Shape<false>::THREADS;
     info->grid = L.grid;
     info->smem_bytes = (int64_t)K2_SMEM_BYTES;
     wl->partial_floats = L.partial_floats;
@@ -758,7 +767,7 @@ static forge_status_t k2_check_residency(const Handle &h)
 {
     int coop = 0, per_sm = 0;
     if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h.d.device) != cudaSuccess || !coop) return FORGE_ERR_CUDA;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2_bf16_tcgen05_kernel<LN, PAIR>, K2_THREADS, K2_SMEM_BYTES) != cudaSuccess ||
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2_bf16_tcgen05_kernel<LN, PAIR>, K2Shape<LN>::THREADS, K2_SMEM_BYTES) != cudaSuccess ||
         (int64_t)per_sm * h.sm_count < h.info.grid)
         return FORGE_ERR_CUDA;
     return FORGE_OK;
@@ -780,14 +789,26 @@ forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     // the tiles of a strip wait for one another: they must all be resident at once
     if (tiles_n > sm_count / info->cluster) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_BF16_TCGEN05_LN;
+    info->threads = K2Shape<true>::THREADS;
     wl->partial_floats = 4 * 2 * (size_t)tiles_n * (size_t)d.M;          // one float4 per row and half tile
     wl->counters = (size_t)tiles_m + 2;                                   // strips, then run index and finished-CTA count
     return FORGE_OK;
 }
 
+// setmaxnreg.inc waits until the registers it asks for are free: the shares must fit into what a CTA is
+// launched with, or the kernel is never launched.
+template <bool PAIR>
+static bool k4_register_shares_fit()
+{
+    cudaFuncAttributes fa;
+    return cudaFuncGetAttributes(&fa, k2_bf16_tcgen05_kernel<true, PAIR>) == cudaSuccess &&
+           fa.numRegs * K2Shape<true>::THREADS >= K4_REGS_NEEDED;
+}
+
 forge_status_t k4_setup(Handle &h)
 {
     const bool pair = h.info.cluster == 2;
+    if (!(pair ? k4_register_shares_fit<true>() : k4_register_shares_fit<false>())) return FORGE_ERR_CUDA;
     if ((pair ? k2_prepare<true, true>() : k2_prepare<true, false>()) != FORGE_OK) return FORGE_ERR_CUDA;
     return pair ? k2_check_residency<true, true>(h) : k2_check_residency<true, false>(h);
 }
@@ -797,7 +818,7 @@ static forge_status_t k2_launch_t(const Handle &h, const K2Params &p, cudaStream
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)h.info.grid);
-    cfg.blockDim = dim3(K2_THREADS);
+    cfg.blockDim = dim3(K2Shape<LN>::THREADS);
     cfg.dynamicSmemBytes = K2_SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];

@@ -22,7 +22,6 @@ struct Workspace {
     int *status = nullptr;           // status word
     void *base = nullptr;            // the single allocation the three point into
     size_t bytes = 0;
-    int partial_fill = 0;            // byte the partial area holds between runs (0, or 0xff: "not written yet")
 };
 
 struct Handle;
@@ -70,7 +69,6 @@ constexpr bool cooperative_launch_enabled()
 struct WorkspaceLayout {
     size_t partial_floats = 0;
     size_t counters = 0;
-    int partial_fill = 0;            // byte value the partial area starts from (status and counters start from zero)
 };
 
 // Each kernel family: a host-only planner (no device access), a one-time setup on the
