@@ -56,7 +56,8 @@ typedef enum {
      * each operand is split into a TF32 head and a TF32 tail and X W^T is accumulated in fp32
      * from the three products head*head, head*tail, tail*head (relative error of a product
      * about 2^-21), so the result stays within the 1e-4 of Section 2.2 with two orders of
-     * magnitude to spare.  Needs K % 4 == 0, N % 4 == 0 and 16-byte aligned pointers.          */
+     * magnitude to spare.  Needs K % 4 == 0, N % 4 == 0 and 16-byte aligned pointers; LayerNorm
+     * needs ceil(N / 256) to be at most the number of CTA pairs of the grid (74 on a B200).  */
 } forge_dtype_t;
 
 typedef enum {
@@ -71,7 +72,14 @@ typedef enum {
     FORGE_RED_NONE = 0,
     FORGE_RED_SUM = 1,
     FORGE_RED_MAX = 2,
-    FORGE_RED_LAYERNORM = 3,     /* population variance, eps inside the square root      */
+    FORGE_RED_LAYERNORM = 3,
+    /* Population variance, eps inside the square root, gamma and beta applied after the
+     * normalisation.  The N-tiles of a row strip exchange per-row (count, mean, M2) triples (the
+     * "cross-tile aggregation" of Appendix B.1); the un-normalised values never leave the SM.
+     * Row width: 16-bit storage, any N (rows of more than 256 x [CTA pairs in the grid] columns --
+     * 18944 on a B200 -- are served by computing every tile twice, once for the statistics and
+     * once to normalise: twice the arithmetic); FORGE_F32, N up to 128 x [2 x SM count] (37888);
+     * FORGE_F32_TF32X3, N up to 256 x [SM count / 2] (18944).  Beyond: FORGE_ERR_UNSUPPORTED.     */
     FORGE_RED_MEAN_GELU_RESIDUAL = 4,
     /* The chain of the paper's Appendix B.1 case study (Linear, subtract, row mean, GELU,
      * residual add of the layer's input, all in one kernel):
@@ -130,9 +138,8 @@ typedef struct {
  * is compute- or memory-bound): fp32 -> F32_FFMA; fp32 with TF32x3 arithmetic -> F32_TF32X3; 16-bit with M <= 32 and neither LayerNorm nor
  * the mean-GELU-residual chain -> BF16_SKINNY; 16-bit LayerNorm -> BF16_TCGEN05_LN; other 16-bit
  * -> BF16_TCGEN05.
- * Unsupported: bf16 with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); fp32 LayerNorm with
- * N > 1024 (one 8-CTA cluster); bf16 LayerNorm with more 256-column tiles per row than
- * clusters in the grid.
+ * Unsupported: 16-bit storage with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); LayerNorm
+ * rows wider than forge_red_t states for fp32 storage; TF32x3 with K % 4 != 0 or N % 4 != 0.
  */
 forge_status_t forge_fused_linear_query_plan(const forge_fused_linear_desc_t *desc, int sm_count,
                                              forge_plan_info_t *info);
@@ -154,7 +161,10 @@ forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, 
  *   (mean-gelu-residual, whose subtract vector travels in `gamma`).
  * Allocates nothing and does not synchronise.  Returns only argument / launch errors;
  * device-side give-ups are reported by forge_fused_linear_last_status().  At most one run
- * per handle may be in flight (the workspace belongs to the handle).
+ * per handle may be in flight (the workspace belongs to the handle).  A call leaves nothing
+ * on the host that a later call depends on (counters that CTAs wait on take their run index
+ * from device memory), so a run captured into a CUDA graph can be replayed, also interleaved
+ * with direct runs of the same handle.
  * Steps: operand fetch, contraction with fp32 accumulation, bias, activation, scale, row
  * reduction and store all happen inside the single kernel launched here (the fused form of
  * Appendix A.1 / B.1; nothing but the final result reaches global memory).

@@ -5,22 +5,20 @@
 // Row reductions across the N-tiles of one row strip:
 //   sum/max   per-tile partials in a small workspace, folded in tile order by the CTA that
 //             arrives last at the strip's counter (deterministic, no float atomics);
-//   layernorm the N-tiles of a strip form one thread-block cluster; per-row (n, mean, M2)
-//             triples are exchanged through distributed shared memory and merged, then
-//             each CTA normalises the tile it still holds in registers.
-#include <cooperative_groups.h>
-
+//   layernorm persistent CTAs walk the tiles strip by strip, so the N-tiles of a strip are worked on
+//             at about the same time; each tile publishes its per-row (n, mean, M2) triples, waits
+//             (bounded) until the strip's counter shows all of them, combines them in tile order and
+//             normalises the tile it still holds in registers.  CTAs wait on one another: cooperative
+//             launch, and a strip may not have more tiles than there are CTAs.
 #include <mutex>
 
 #include "common.cuh"
 #include "plan.h"
 
-namespace cg = cooperative_groups;
-
 namespace forge {
 
 constexpr int K1_BM = 128, K1_BN = 128, K1_BK = 16, K1_THREADS = 256, K1_PAD = 4;
-constexpr int K1_LN_MAX_CLUSTER = 8;
+constexpr int K1_CTAS_PER_SM = 2;            // the kernels are built for two resident CTAs per SM
 
 struct K1Params {
     const float *X, *W, *b, *gamma, *beta;
@@ -34,8 +32,9 @@ struct K1Params {
     int res_vec4;          // mean chain: X and Y rows ([M,K]) can be moved with 128-bit accesses
     int warm_l2;           // small grids: request the CTA's operand panels into L2 before the k loop
     // (Small grids: K is cut into gridDim.z slices, one CTA each; the slice length and the hand-over
-    // area follow from the fields above -- see k1_slice_len() -- so that this structure, whose size
-    // the code generated for the large tile turned out to be sensitive to, stays as it is.)
+    // area follow from the fields above -- see k1_slice_len().)
+    int *status;           // LayerNorm: status word of the bounded strip wait
+    unsigned *gen;         // LayerNorm: run index of the strip counters (see run_index_begin)
 };
 
 // Length of a K slice when K is cut into `slices`: a multiple of the small tile's 32-wide k-tile.
@@ -137,20 +136,20 @@ __device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &
 // T = 2: 128x128 CTA tile, 8x8 accumulators per thread.  T = 1: 64x64 tile, 4x4 per thread, for
 // problems with too few 128x128 tiles to occupy the SMs (a grid of a handful of CTAs is bound by
 // the FMA rate of the few SMs it runs on, not by the GPU's).
+// One output tile (for small grids: one K slice of it).  `run` is the run index of the LayerNorm strip counters.
+// Returns false only when a bounded wait gave up.
 template <bool VEC, int RED, int T>
-__global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Params p)
+__device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, const int tile_n, const unsigned run)
 {
     constexpr int BM = 64 * T, BN = 64 * T, R = 4 * T;       // tile and per-thread extent
     constexpr int BK = T == 1 ? 32 : K1_BK;                  // the small tile takes longer k steps (fewer round trips)
     __shared__ __align__(16) float As[2][BK][BM + K1_PAD];
     __shared__ __align__(16) float Bs[2][BK][BN + K1_PAD];
-    __shared__ RowStat s_stat[BM];
     __shared__ float s_mean[BM], s_rstd[BM];
     __shared__ int s_last;
 
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
-    const int tile_n = blockIdx.x, tile_m = blockIdx.y;
     const int m0 = tile_m * BM, n0 = tile_n * BN;
     const int M = p.M, N = p.N, K = p.K;
 
@@ -300,7 +299,7 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
         __syncthreads();
         if (tid == 0) s_last = (arrive_acq_rel(&slice_counters[tile]) == (unsigned)(k_slices - 1));
         __syncthreads();
-        if (!s_last) return;
+        if (!s_last) return true;
 #pragma unroll
         for (int i = 0; i < R; ++i)
 #pragma unroll
@@ -350,7 +349,7 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
                     if (cok[j]) dst[col[j]] = acc[i][j];
             }
         }
-        return;
+        return true;
     }
 
     if (RED == FORGE_RED_SUM || RED == FORGE_RED_MAX || RED == FORGE_RED_MEAN_GELU_RESIDUAL) {
@@ -384,7 +383,7 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
             __syncthreads();
             if (tid == 0) s_last = (arrive_acq_rel(&p.counters[tile_m]) == (unsigned)(p.tiles_n - 1));
             __syncthreads();
-            if (!s_last) return;
+            if (!s_last) return true;
             if (tid < BM && m0 + tid < M) {
                 const int row = m0 + tid;
                 float v = __ldcg(&p.partial[row]);
@@ -425,7 +424,7 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
                 }
             }
         }
-        return;
+        return true;
     }
 
     if (RED == FORGE_RED_LOGSUMEXP || RED == FORGE_RED_CROSS_ENTROPY) {
@@ -461,11 +460,11 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
                 else part4[(size_t)tile_n * M + row] = make_float4(mx, se, tl, 0.f);
             }
         }
-        if (p.tiles_n == 1) return;
+        if (p.tiles_n == 1) return true;
         __syncthreads();
         if (tid == 0) s_last = (arrive_acq_rel(&p.counters[tile_m]) == (unsigned)(p.tiles_n - 1));
         __syncthreads();
-        if (!s_last) return;
+        if (!s_last) return true;
         if (tid < BM && m0 + tid < M) {
             const int row = m0 + tid;
             float4 f = __ldcg(&part4[row]);
@@ -489,38 +488,62 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
             p.out[row] = mx + logf(se) - tl;
         }
         if (tid == 0) p.counters[tile_m] = 0u;
-        return;
+        return true;
     }
 
     if (RED == FORGE_RED_LAYERNORM) {
-        cg::cluster_group cluster = cg::this_cluster();
-        // per-thread statistics of its <= 8 columns of each row, two sweeps over registers
+        float4 *stats = reinterpret_cast<float4 *>(p.partial);      // [tiles_n][M] (n, mean, M2, -)
+        // per-thread statistics of its <= 8 columns of each row, two sweeps over registers, then the 16 lanes
+        // that share the row
 #pragma unroll
         for (int i = 0; i < R; ++i) {
-            RowStat s;
+            RowStat st;
             float sum = 0.f;
-            s.n = 0.f;
+            st.n = 0.f;
 #pragma unroll
             for (int j = 0; j < R; ++j)
-                if (cok[j]) { sum += acc[i][j]; s.n += 1.f; }
-            s.mean = s.n > 0.f ? sum / s.n : 0.f;
-            s.m2 = 0.f;
+                if (cok[j]) { sum += acc[i][j]; st.n += 1.f; }
+            st.mean = st.n > 0.f ? sum / st.n : 0.f;
+            st.m2 = 0.f;
 #pragma unroll
             for (int j = 0; j < R; ++j)
-                if (cok[j]) { const float d = acc[i][j] - s.mean; s.m2 = fmaf(d, d, s.m2); }
+                if (cok[j]) { const float d = acc[i][j] - st.mean; st.m2 = fmaf(d, d, st.m2); }
 #pragma unroll
-            for (int sft = 1; sft <= 8; sft <<= 1) s = merge_stat(s, shfl_xor_stat(s, sft));
-            if (tx == 0) s_stat[ty * 4 + (i & 3) + (i >> 2) * 64] = s;
+            for (int sft = 1; sft <= 8; sft <<= 1) st = merge_stat(st, shfl_xor_stat(st, sft));
+            const int row = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
+            if (tx == 0 && row < M) stats[(size_t)tile_n * M + row] = make_float4(st.n, st.mean, st.m2, 0.f);
         }
-        cluster.sync();
-        if (tid < BM) {
-            const unsigned nranks = cluster.num_blocks();
-            RowStat s = *cluster.map_shared_rank(&s_stat[tid], 0);
-            for (unsigned r = 1; r < nranks; ++r) s = merge_stat(s, *cluster.map_shared_rank(&s_stat[tid], r));
-            s_mean[tid] = s.mean;
-            s_rstd[tid] = rsqrtf(s.m2 / s.n + p.e.eps);
+        // publish, then wait (bounded) for the strip's other tiles: one arrival per CTA by one thread (release: the
+        // CTA's triples, ordered before it by the barrier; the acquiring polls and the next barrier make the other
+        // tiles' triples readable past L1)
+        __syncthreads();
+        if (tid == 0) {
+            arrive_acq_rel(&p.counters[tile_m]);
+            s_last = wait_counter<0>(&p.counters[tile_m], run * (unsigned)p.tiles_n, p.status, SITE_ARRIVAL, tile_m) ? 1 : 0;
         }
-        cluster.sync();      // also keeps every CTA's s_stat alive until all have read it
+        __syncthreads();
+        if (!s_last) return false;
+        // the strip's tiles combined in tile order, all at once (same result in every CTA):
+        // mean = sum n_i mean_i / sum n_i,  M2 = sum (M2_i + n_i (mean_i - mean)^2)
+        if (tid < BM && m0 + tid < M) {
+            const int row = m0 + tid;
+            float cnt = 0.f, wsum = 0.f;
+            for (int t = 0; t < p.tiles_n; ++t) {
+                const float4 o = __ldcg(&stats[(size_t)t * M + row]);
+                cnt += o.x;
+                wsum = fmaf(o.x, o.y, wsum);
+            }
+            const float mean = wsum / cnt;
+            float m2 = 0.f;
+            for (int t = 0; t < p.tiles_n; ++t) {
+                const float4 o = __ldcg(&stats[(size_t)t * M + row]);
+                const float dm = o.y - mean;
+                m2 += fmaf(o.x * dm, dm, o.z);
+            }
+            s_mean[tid] = mean;
+            s_rstd[tid] = rsqrtf(m2 / cnt + p.e.eps);
+        }
+        __syncthreads();
         float g[R], be[R];
 #pragma unroll
         for (int j = 0; j < R; ++j) {
@@ -547,6 +570,25 @@ __global__ void __launch_bounds__(K1_THREADS, 2) k1_f32_ffma_kernel(const K1Para
                     if (cok[j]) dst[col[j]] = y[j];
             }
         }
+    }
+    return true;
+}
+
+// Grid: one CTA per tile (and K slice), blockIdx = (N-tile, M-tile, slice).  LayerNorm: a one-dimensional grid of
+// persistent CTAs that take the tiles strip by strip.
+template <bool VEC, int RED, int T>
+__global__ void __launch_bounds__(K1_THREADS, K1_CTAS_PER_SM) k1_f32_ffma_kernel(const K1Params p)
+{
+    if (RED == FORGE_RED_LAYERNORM) {
+        const unsigned run = run_index_begin(p.gen);
+        const int tiles = (int)((p.M + 64 * T - 1) / (64 * T)) * p.tiles_n;
+        for (int t = (int)blockIdx.x; t < tiles; t += (int)gridDim.x) {
+            if (!k1_tile<VEC, RED, T>(p, t / p.tiles_n, t % p.tiles_n, run)) break;
+            __syncthreads();          // the tile's shared memory is free for the next one
+        }
+        if (threadIdx.x == 0) run_index_end(p.gen, run);
+    } else {
+        k1_tile<VEC, RED, T>(p, (int)blockIdx.y, (int)blockIdx.x, 0u);
     }
 }
 
@@ -579,21 +621,27 @@ forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     const int64_t tiles_m = (d.M + bm - 1) / bm, tiles_n = (d.N + bn - 1) / bn;
     if (tiles_m > 65535 || tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
     if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
-    if (d.red == FORGE_RED_LAYERNORM && tiles_n > K1_LN_MAX_CLUSTER) return FORGE_ERR_UNSUPPORTED;
+    // LayerNorm: persistent CTAs, and the tiles of a strip wait for one another, so all of them must be resident
+    const int64_t ln_grid = tiles_m * tiles_n < (int64_t)K1_CTAS_PER_SM * sm_count ? tiles_m * tiles_n : (int64_t)K1_CTAS_PER_SM * sm_count;
+    if (d.red == FORGE_RED_LAYERNORM && tiles_n > ln_grid) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_F32_FFMA;
     info->tile_m = bm;
     info->tile_n = bn;
     info->tile_k = small ? 32 : K1_BK;
     info->stages = 2;
-    info->cluster = d.red == FORGE_RED_LAYERNORM ? (int)tiles_n : 1;
+    info->cluster = 1;
     info->threads = K1_THREADS;
     const int slices = small ? k1_slices(d, sm_count, tiles_m * tiles_n) : 1;
-    info->grid = tiles_m * tiles_n * slices;
+    info->grid = d.red == FORGE_RED_LAYERNORM ? ln_grid : tiles_m * tiles_n * slices;
     info->smem_bytes = 0;
     const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;      // float4 partials
     const bool partials = (d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || d.red == FORGE_RED_MEAN_GELU_RESIDUAL || lse) && tiles_n > 1;
     wl->partial_floats = partials ? (lse ? 4 : 1) * (size_t)tiles_n * (size_t)d.M : 0;
     wl->counters = partials ? (size_t)tiles_m : 0;
+    if (d.red == FORGE_RED_LAYERNORM) {       // one (n, mean, M2, -) per row and tile; strip counters, then run index and finished-CTA count
+        wl->partial_floats = 4 * (size_t)tiles_n * (size_t)d.M;
+        wl->counters = (size_t)tiles_m + 2;
+    }
     if (slices > 1) {         // hand-over area of the K slices (64x64 floats per tile and slice) after the row partials
         wl->partial_floats = (wl->partial_floats + 3) / 4 * 4 + (size_t)(tiles_m * tiles_n) * slices * 64 * 64;
         wl->counters += (size_t)(tiles_m * tiles_n);
@@ -601,10 +649,20 @@ forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     return FORGE_OK;
 }
 
-forge_status_t k1_setup(Handle &) { return FORGE_OK; }
+// LayerNorm: CTAs wait on one another, so the whole grid must be resident at once.
+forge_status_t k1_setup(Handle &h)
+{
+    if (h.d.red != FORGE_RED_LAYERNORM) return FORGE_OK;
+    int coop = 0, a = 0, b = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, h.d.device) != cudaSuccess || !coop) return FORGE_ERR_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, k1_f32_ffma_kernel<true, FORGE_RED_LAYERNORM, 2>, K1_THREADS, 0) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, k1_f32_ffma_kernel<false, FORGE_RED_LAYERNORM, 2>, K1_THREADS, 0) != cudaSuccess)
+        return FORGE_ERR_CUDA;
+    return (int64_t)(a < b ? a : b) * h.sm_count >= h.info.grid ? FORGE_OK : FORGE_ERR_CUDA;
+}
 
 template <bool VEC, int RED, int T = 2>
-static forge_status_t k1_launch_t(const K1Params &p, dim3 grid, int cluster, cudaStream_t stream)
+static forge_status_t k1_launch_t(const K1Params &p, dim3 grid, cudaStream_t stream)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
@@ -612,11 +670,9 @@ static forge_status_t k1_launch_t(const K1Params &p, dim3 grid, int cluster, cud
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
-    if (RED == FORGE_RED_LAYERNORM) {
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = cluster;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
+    if (RED == FORGE_RED_LAYERNORM && cooperative_launch_enabled()) {
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
     }
@@ -639,6 +695,7 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
     p.e = Epilogue{(int)d.act, (int)d.red, d.scale, d.ln_eps, d.has_bias};
     p.partial = h.ws.partial;
     p.counters = h.ws.counters;
+    p.status = h.ws.status;
     const int bm = h.info.tile_m, bn = h.info.tile_n;          // 128 or 64
     p.warm_l2 = (h.info.grid < h.sm_count) && (d.K <= 4096);   // latency-bound grids with modest panels
     p.tiles_n = (int)((d.N + bn - 1) / bn);
@@ -646,14 +703,15 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
     p.res_vec4 = (d.K % 4 == 0) && ((uintptr_t)a.out % 16 == 0) && ((uintptr_t)a.X % 16 == 0);
     const int64_t tiles_m = (d.M + bm - 1) / bm;
     const int k_slices = bm != K1_BM ? k1_slices(d, h.sm_count, tiles_m * p.tiles_n) : 1;
-    const dim3 grid((unsigned)p.tiles_n, (unsigned)tiles_m, (unsigned)k_slices);
+    p.gen = h.ws.counters + tiles_m;          // LayerNorm: behind the strip counters
+    const dim3 grid = d.red == FORGE_RED_LAYERNORM ? dim3((unsigned)h.info.grid)
+                                                   : dim3((unsigned)p.tiles_n, (unsigned)tiles_m, (unsigned)k_slices);
     const bool vec = (d.K % 4 == 0) && ((uintptr_t)a.X % 16 == 0) && ((uintptr_t)a.W % 16 == 0);
 #define K1_CASE(R)                                                                                   \
     case R:                                                                                          \
         if (bm == K1_BM)                                                                             \
-            return vec ? k1_launch_t<true, R, 2>(p, grid, h.info.cluster, a.stream)                  \
-                       : k1_launch_t<false, R, 2>(p, grid, h.info.cluster, a.stream);                \
-        return vec ? k1_launch_t<true, R, 1>(p, grid, 1, a.stream) : k1_launch_t<false, R, 1>(p, grid, 1, a.stream);
+            return vec ? k1_launch_t<true, R, 2>(p, grid, a.stream) : k1_launch_t<false, R, 2>(p, grid, a.stream); \
+        return vec ? k1_launch_t<true, R, 1>(p, grid, a.stream) : k1_launch_t<false, R, 1>(p, grid, a.stream);
     switch (d.red) {
         K1_CASE(FORGE_RED_NONE)
         K1_CASE(FORGE_RED_SUM)
@@ -743,9 +801,11 @@ extern "C" forge_status_t forge_fused_linear_f32_reduce_static(int64_t M, int64_
     p.out_vec4 = 0;
     p.res_vec4 = 0;
     p.warm_l2 = 0;
+    p.status = nullptr;
+    p.gen = nullptr;
     const dim3 grid((unsigned)tiles_n, (unsigned)tiles_m);
     const bool vec = (K % 4 == 0) && ((uintptr_t)X % 16 == 0) && ((uintptr_t)W % 16 == 0);
     if (red == FORGE_RED_SUM)
-        return vec ? k1_launch_t<true, FORGE_RED_SUM>(p, grid, 1, stream) : k1_launch_t<false, FORGE_RED_SUM>(p, grid, 1, stream);
-    return vec ? k1_launch_t<true, FORGE_RED_MAX>(p, grid, 1, stream) : k1_launch_t<false, FORGE_RED_MAX>(p, grid, 1, stream);
+        return vec ? k1_launch_t<true, FORGE_RED_SUM>(p, grid, stream) : k1_launch_t<false, FORGE_RED_SUM>(p, grid, stream);
+    return vec ? k1_launch_t<true, FORGE_RED_MAX>(p, grid, stream) : k1_launch_t<false, FORGE_RED_MAX>(p, grid, stream);
 }

@@ -97,6 +97,7 @@ struct K2Params {
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     int group_m;          // row units per rasterisation group
     unsigned *gen;        // launches whose CTAs wait on one another: run index (see run_index_begin)
+    int two_pass;         // LayerNorm of rows with more tiles than CTAs (pairs): see K2Item::pass
     // K split of the last wave's tiles (tail_parts = 1: none)
     int tail_parts;           // S
     int tail_kb;              // k-blocks per part
@@ -134,6 +135,7 @@ struct K2Item {
     int tm, tn;                 // row unit, 256-column tile
     int kb_lo, kb_hi;           // k-blocks [kb_lo, kb_hi)
     int part, tail;             // part of the K split (0 leads), index of the tile among the split ones (-1: whole tile)
+    int pass;                   // LayerNorm of rows wider than the grid: 0 = statistics only, 1 = normalise and store
 };
 
 template <bool LN>
@@ -145,6 +147,12 @@ __device__ __forceinline__ bool k2_item(const K2Params &p, int j, int unit, int 
     w.kb_hi = p.num_kb;
     w.part = 0;
     w.tail = -1;
+    w.pass = 0;
+    if (LN && p.two_pass) {
+        // every tile twice: this unit's whole list once for the statistics, then once more to normalise
+        const int mine = full + (unit < rest ? 1 : 0);
+        if (j >= mine) { j -= mine; w.pass = 1; }
+    }
     if (j < full) {
         t = j * units + unit;
     } else if (j == full && p.tail_parts <= 1) {
@@ -426,17 +434,27 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 __syncwarp();
                 if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
                 float4 *stats = reinterpret_cast<float4 *>(p.partial);
-                if (row < p.M) stats[(size_t)part * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
+                // Rows with more tiles than the grid has CTAs (pairs) cannot all be held on chip at once: every tile is
+                // then computed twice.  Pass 0 publishes its triples and moves on (it never waits, so the grid always
+                // gets through it); pass 1, which starts only when this unit has finished pass 0, recomputes the tile,
+                // waits for the strip's triples (normally long there) and normalises.  Twice the arithmetic, and the
+                // un-normalised tile still never leaves the SM.
+                const bool publish = !p.two_pass || w.pass == 0, finish = !p.two_pass || w.pass == 1;
+                if (publish && row < p.M) stats[(size_t)part * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
                 // ---- publish, then wait (bounded) for the other parts of this strip: one arrival per group by one
                 //      thread (release: the group's triples, which the barrier orders before it; the acquiring polls
                 //      and the next barrier make the other groups' triples readable past L1) ----
                 epi_bar_sync(h);
                 if (et == 0) {
-                    arrive_acq_rel(&p.counters[tm]);
-                    if (!wait_counter<0>(&p.counters[tm], run * (unsigned)parts, p.status, SITE_ARRIVAL, tm)) s.abort_flag = 1;
+                    if (publish) arrive_acq_rel(&p.counters[tm]);
+                    if (finish && !wait_counter<0>(&p.counters[tm], run * (unsigned)parts, p.status, SITE_ARRIVAL, tm)) s.abort_flag = 1;
                 }
                 epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
+                if (!finish) {
+                    if ((acc ^= 1) == 0) acc_phase ^= 1;
+                    continue;
+                }
                 // Combine the strip's parts in part order, all at once (same result on every CTA):
                 // mean = sum n_i mean_i / sum n_i,  M2 = sum (M2_i + n_i (mean_i - mean)^2).
                 float rstd = 0.f, shift = 0.f;
@@ -786,8 +804,8 @@ forge_status_t k4_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     const forge_status_t st = k2_plan(d, sm_count, info, wl);
     if (st != FORGE_OK) return st;
     const int64_t tiles_m = (d.M + K2_BM - 1) / K2_BM, tiles_n = (d.N + K2_BN - 1) / K2_BN;
-    // the tiles of a strip wait for one another: they must all be resident at once
-    if (tiles_n > sm_count / info->cluster) return FORGE_ERR_UNSUPPORTED;
+    // the tiles of a strip wait for one another: they must all be resident at once, or every tile is computed
+    // twice (see K2Item::pass)
     info->kernel = FORGE_KERNEL_BF16_TCGEN05_LN;
     info->threads = K2Shape<true>::THREADS;
     wl->partial_floats = 4 * 2 * (size_t)tiles_n * (size_t)d.M;          // one float4 per row and half tile
@@ -888,6 +906,7 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     p.tail_kb = p.num_kb;
     p.cooperative = 1;
     p.gen = h.ws.counters + p.tiles_m;
+    p.two_pass = p.tiles_n > h.info.grid / h.info.cluster;
     return pair ? k2_launch_t<true, true>(h, p, a.stream) : k2_launch_t<true, false>(h, p, a.stream);
 }
 

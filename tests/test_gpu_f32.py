@@ -54,14 +54,25 @@ def test_every_activation(act):
     pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
 
 
-def test_no_bias_and_layernorm_edge_of_cluster():
-    wl = wk.custom_workload("f32_ln_1024", wk.F32, 130, 1024, 40, wk.ACT_GELU_ERF, wk.RED_LAYERNORM,
-                            has_bias=False, seed=4)
+# one tile per strip, 8 and 9 tiles (past the width a thread-block cluster would span), 32 tiles with many strips
+# per CTA (several waves of persistent CTAs), a row as wide as a language-model head with few rows
+@pytest.mark.parametrize("M,N,K,bias", [(130, 1024, 40, False), (70, 1032, 36, True), (1500, 4096, 64, True),
+                                        (40, 32768, 24, True), (128 * 5 + 3, 128 * 59 + 8, 20, True)])
+def test_layernorm_of_wide_rows(M, N, K, bias):
+    wl = wk.custom_workload(f"f32_ln_{N}", wk.F32, M, N, K, wk.ACT_GELU_ERF, wk.RED_LAYERNORM, has_bias=bias, seed=4)
     inp = wk.make_inputs(wl)
-    g, plan = pu.run_gpu(wl, inp)
-    assert plan["cluster"] == 8
+    op = B.FusedLinear(pu.desc_of(wl))
+    g, plan = pu.run_gpu(wl, inp, op=op, repeats=3)           # the strip counters are never reset between runs
+    op.close()
+    assert plan["kernel"] == B.FORGE_KERNEL_F32_FFMA and plan["cluster"] == 1 and plan["grid"] <= 2 * 148
     pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
-    st, _ = B.forge_fused_linear_query_plan(B.make_desc(8, 1025, 8, wk.F32, 0, wk.RED_LAYERNORM))
+
+
+def test_layernorm_rows_wider_than_the_grid_are_refused():
+    # the tiles of a strip wait for one another: more 128-column tiles than resident CTAs cannot be served
+    st, _ = B.forge_fused_linear_query_plan(B.make_desc(8, 128 * 296, 8, wk.F32, 0, wk.RED_LAYERNORM))
+    assert st == B.FORGE_OK
+    st, _ = B.forge_fused_linear_query_plan(B.make_desc(8, 128 * 296 + 1, 8, wk.F32, 0, wk.RED_LAYERNORM))
     assert st == B.FORGE_ERR_UNSUPPORTED
 
 

@@ -24,8 +24,6 @@ def _cases(dtype, n, seed, step, m_hi, n_hi, k_hi):
         if rng.random() < 0.3:                      # long K with few tiles: slices / K cuts
             K = int(rng.integers(k_hi // step, 4 * k_hi // step + 1)) * step
         act, red = ACTS[int(rng.integers(5))], REDS[int(rng.integers(7))]
-        if dtype == wk.F32 and red == wk.RED_LAYERNORM and N > 1024:
-            continue                                 # the FFMA kernel's LayerNorm spans one 8-CTA cluster (refused beyond)
         out.append((M, N, K, act, red, bool(rng.integers(2)), len(out)))
     return out
 

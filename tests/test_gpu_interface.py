@@ -253,7 +253,7 @@ def test_nothing_is_written_outside_the_output(case):
     pu.assert_parity(wl, out.float().cpu().numpy().astype(np.float64), pu.run_oracle(wl, inp))
 
 
-@pytest.mark.parametrize("name", ["ln_bf16", "chain_bf16", "tailsplit_bf16", "ln_tf32x3", "rowsum_f32"])
+@pytest.mark.parametrize("name", ["ln_bf16", "chain_bf16", "tailsplit_bf16", "ln_tf32x3", "rowsum_f32", "ln_f32", "ln_bf16_two_pass"])
 def test_run_captured_in_a_graph_replays_correctly(name):
     """run() keeps no per-call state on the host: the counters that the CTAs of the LayerNorm, chain
     and K-cut launches wait on take their run index from device memory.  So a run captured into a
@@ -264,7 +264,9 @@ def test_run_captured_in_a_graph_replays_correctly(name):
           "chain_bf16": wk.custom_workload("g_chain", wk.BF16, 300, 520, 128, wk.ACT_IDENTITY, wk.RED_MEAN_GELU_RESIDUAL, w_std=0.05),
           "tailsplit_bf16": wk.custom_workload("g_tail", wk.BF16, 256, 512, 4096, wk.ACT_SILU, wk.RED_NONE, w_std=0.02),
           "ln_tf32x3": wk.custom_workload("g_ln5", wk.F32_TF32X3, 300, 520, 256, wk.ACT_GELU_TANH, wk.RED_LAYERNORM),
-          "rowsum_f32": wk.custom_workload("g_sum", wk.F32, 300, 700, 96, wk.ACT_RELU, wk.RED_SUM)}[name]
+          "rowsum_f32": wk.custom_workload("g_sum", wk.F32, 300, 700, 96, wk.ACT_RELU, wk.RED_SUM),
+          "ln_f32": wk.custom_workload("g_ln1", wk.F32, 300, 1300, 96, wk.ACT_GELU_TANH, wk.RED_LAYERNORM),
+          "ln_bf16_two_pass": wk.custom_workload("g_ln2", wk.BF16, 130, 256 * 80, 64, wk.ACT_SILU, wk.RED_LAYERNORM, w_std=0.05)}[name]
     inp = wk.make_inputs(wl)
     dev = {k: pu.to_device(v, wl.dtype) for k, v in inp.items() if k != "target"}
     aux = dev["sub"] if wl.red == wk.RED_MEAN_GELU_RESIDUAL else dev["gamma"]

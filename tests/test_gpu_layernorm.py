@@ -33,6 +33,20 @@ def test_shapes(M, N, K):
     pu.assert_parity(wl, g, pu.run_oracle(wl, inp), f"act={act}")
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 32768, 64), (130, 256 * 75, 72), (16, 256 * 200 + 8, 16)])
+def test_rows_with_more_tiles_than_the_grid_are_computed_twice(M, N, K):
+    """A row strip of more 256-column tiles than there are CTA pairs cannot be held on chip at once: the kernel
+    then makes a statistics pass and a normalising pass over every tile.  Same results, same tolerance; the
+    strip counters carry over from run to run."""
+    wl = _case(M, N, K, wk.ACT_GELU_TANH, seed=N % 97)
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    g, plan = pu.run_gpu(wl, inp, op=op, repeats=3)
+    op.close()
+    assert plan["kernel"] == B.FORGE_KERNEL_BF16_TCGEN05_LN
+    pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+
+
 def test_unit_affine_rows_have_zero_mean_and_unit_variance():
     wl = _case(256, 2048, 256, wk.ACT_GELU_ERF, seed=1, eps=1e-12)
     inp = wk.make_inputs(wl)
