@@ -206,6 +206,107 @@ __device__ __forceinline__ void run_index_end(unsigned *gen, unsigned run)
     }
 }
 
+// ---- folds of what the tiles of a row strip leave in the workspace -------------------------------
+// All of them walk the parts in part order whichever CTA does the walking, so the result does not depend
+// on arrival order; loads are issued eight at a time (a dependent round trip per part made the fold of a
+// wide row the longest thing in the kernel) and read past L1 (the values come from other SMs).
+
+// Row sums or maxima: partial[part * M + row], part = 0 .. parts-1.
+template <bool ADD>
+__device__ __forceinline__ float fold_row_partials(const float *partial, int parts, int M, int row)
+{
+    float v = __ldcg(&partial[row]);
+    int i = 1;
+    for (; i + 8 <= parts; i += 8) {
+        float o[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) o[u] = __ldcg(&partial[(size_t)(i + u) * M + row]);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v = ADD ? v + o[u] : fmaxf(v, o[u]);
+    }
+    for (; i < parts; ++i) {
+        const float o = __ldcg(&partial[(size_t)i * M + row]);
+        v = ADD ? v + o : fmaxf(v, o);
+    }
+    return v;
+}
+
+// Softmax statistics (max, sum exp, target logit, -) per part: returns logsumexp - target logit.
+template <bool ACCURATE>
+__device__ __forceinline__ float fold_row_lse(const float4 *part4, int parts, int M, int row)
+{
+    float4 f = __ldcg(&part4[row]);
+    float mx = f.x, se = f.y, tl = f.z;
+    int i = 1;
+    for (; i + 8 <= parts; i += 8) {
+        float4 g[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) g[u] = __ldcg(&part4[(size_t)(i + u) * M + row]);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            lse_merge<ACCURATE>(mx, se, g[u].x, g[u].y);
+            tl += g[u].z;
+        }
+    }
+    for (; i < parts; ++i) {
+        f = __ldcg(&part4[(size_t)i * M + row]);
+        lse_merge<ACCURATE>(mx, se, f.x, f.y);
+        tl += f.z;
+    }
+    return mx + (ACCURATE ? logf(se) : __logf(se)) - tl;
+}
+
+// LayerNorm: the strip's (n, mean, M2, -) triples combined all at once, with one division for the mean
+// and one for the variance (the pairwise merge costs a division per part):
+//     mean = sum n_i mean_i / sum n_i,   M2 = sum (M2_i + n_i (mean_i - mean)^2).
+// Returns the mean and writes 1 / sqrt(M2 / n + eps).
+template <bool ACCURATE>
+__device__ __forceinline__ float combine_row_moments(const float4 *stats, int parts, int M, int row, float eps, float &rstd)
+{
+    float cnt = 0.f, wsum = 0.f;
+    for (int i = 0; i < parts; ++i) {
+        const float4 o = __ldcg(&stats[(size_t)i * M + row]);
+        cnt += o.x;
+        wsum = fmaf(o.x, o.y, wsum);
+    }
+    const float mean = wsum / cnt;
+    float m2 = 0.f;
+    for (int i = 0; i < parts; ++i) {
+        const float4 o = __ldcg(&stats[(size_t)i * M + row]);
+        const float dm = o.y - mean;
+        m2 += fmaf(o.x * dm, dm, o.z);
+    }
+    rstd = ACCURATE ? 1.0f / sqrtf(m2 / cnt + eps) : rsqrtf(m2 / cnt + eps);
+    return mean;
+}
+
+// (n, mean, M2) of the first nv of 32 values held in registers: two sweeps, no division per element.
+__device__ __forceinline__ RowStat chunk_moments(const float (&v)[32], int nv)
+{
+    RowStat cs;
+    cs.n = (float)nv;
+    cs.m2 = 0.f;
+    if (nv == 32) {
+        float sum = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sum += v[j];
+        cs.mean = sum * (1.0f / 32.0f);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) { const float dlt = v[j] - cs.mean; cs.m2 = fmaf(dlt, dlt, cs.m2); }
+    } else {
+        float sum = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sum += j < nv ? v[j] : 0.f;
+        cs.mean = sum / cs.n;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const float dlt = j < nv ? v[j] - cs.mean : 0.f;
+            cs.m2 = fmaf(dlt, dlt, cs.m2);
+        }
+    }
+    return cs;
+}
+
 constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 }  // namespace forge

@@ -40,39 +40,10 @@ struct K1Params {
 // Length of a K slice when K is cut into `slices`: a multiple of the small tile's 32-wide k-tile.
 __host__ __device__ inline int k1_slice_len(int K, int slices) { return ((K + slices - 1) / slices + 31) / 32 * 32; }
 
-// One CTA-tile slab (128 rows x 16 k, or 64 rows x 32 k) from a K-major matrix into registers:
-// two float4 per thread either way.
+// One CTA-tile slab (128 rows x 16 k, or 64 rows x 32 k) from a K-major matrix into registers: two float4 per
+// thread either way.  k_end is the end of this CTA's range of k (K itself unless K is cut into slices).
 template <bool VEC, int T>
 __device__ __forceinline__ void k1_fetch(const float *__restrict__ base, int rows_total, int K,
-                                         int row0, int kt, int tid, float4 (&r)[2])
-{
-    constexpr int KQ = (T == 1 ? 32 : 16) / 4;          // float4 per row of the slab
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int idx = tid + i * K1_THREADS;
-        const int row = row0 + idx / KQ;
-        const int k = kt + (idx % KQ) * 4;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (row < rows_total) {
-            const float *src = base + (size_t)row * K + k;
-            if (VEC) {
-                if (k < K) v = __ldg(reinterpret_cast<const float4 *>(src));
-            } else {
-                if (k + 0 < K) v.x = __ldg(src + 0);
-                if (k + 1 < K) v.y = __ldg(src + 1);
-                if (k + 2 < K) v.z = __ldg(src + 2);
-                if (k + 3 < K) v.w = __ldg(src + 3);
-            }
-        }
-        r[i] = v;
-    }
-}
-
-// The same with an explicit end of the k range (K slices of the small tile).
-// One CTA-tile slab (128 rows x 16 k, or 64 rows x 32 k) from a K-major matrix into registers:
-// two float4 per thread either way.
-template <bool VEC, int T>
-__device__ __forceinline__ void k1_fetch_range(const float *__restrict__ base, int rows_total, int K,
                                          int row0, int kt, int tid, float4 (&r)[2], int k_end)
 {
     constexpr int KQ = (T == 1 ? 32 : 16) / 4;          // float4 per row of the slab
@@ -159,26 +130,26 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
 #pragma unroll
         for (int j = 0; j < R / 2; ++j) acc2[i][j] = 0ull;
 
-    if (T == 1) {
-        // small tile: this CTA may own only a slice of K (blockIdx.z of gridDim.z slices)
+    {
+        // this CTA's range of k: the whole of K unless a small grid (T == 1) is cut into gridDim.z slices
+        const int k_per = T == 1 ? k1_slice_len(K, (int)gridDim.z) : K, k_lo = T == 1 ? (int)blockIdx.z * k_per : 0;
+        const int k_hi = min(K, k_lo + k_per);
         if (p.warm_l2) {
             // A small grid walks K with one tile of look-ahead, i.e. it pays the memory latency once
             // per k-tile.  Asking L2 for both operand panels up front puts all of those requests in
             // flight at once; the k loop then runs at L2 latency.
-            const int w_per = k1_slice_len(K, (int)gridDim.z), w_lo = (int)blockIdx.z * w_per, w_len = min(K, w_lo + w_per) - w_lo;
+            const int w_len = k_hi - k_lo;
             const int lines_per_row = (w_len * 4 + 127) / 128;
             const int rows_a = min(BM, M - m0), rows_b = min(BN, N - n0);
             for (int i = tid; i < (rows_a + rows_b) * lines_per_row; i += K1_THREADS) {
                 const int r = i / lines_per_row, c = i - r * lines_per_row;
                 const float *ptr = r < rows_a ? p.X + (size_t)(m0 + r) * K : p.W + (size_t)(n0 + r - rows_a) * K;
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr + w_lo + min(c * 32, w_len - 1)));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr + k_lo + min(c * 32, w_len - 1)));
             }
         }
-        // this CTA's range of k (the whole of K unless a small grid is cut into slices)
-        const int k_per = k1_slice_len(K, (int)gridDim.z), k_lo = (int)blockIdx.z * k_per, k_hi = min(K, k_lo + k_per);
         float4 ra[2], rb[2];
-        k1_fetch_range<VEC, T>(p.X, M, K, m0, k_lo, tid, ra, k_hi);
-        k1_fetch_range<VEC, T>(p.W, N, K, n0, k_lo, tid, rb, k_hi);
+        k1_fetch<VEC, T>(p.X, M, K, m0, k_lo, tid, ra, k_hi);
+        k1_fetch<VEC, T>(p.W, N, K, n0, k_lo, tid, rb, k_hi);
         k1_stash<T>(As[0], tid, ra);
         k1_stash<T>(Bs[0], tid, rb);
         __syncthreads();
@@ -187,8 +158,8 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
         for (int kt = k_lo; kt < k_hi; kt += BK) {
             const bool more = kt + BK < k_hi;
             if (more) {
-                k1_fetch_range<VEC, T>(p.X, M, K, m0, kt + BK, tid, ra, k_hi);
-                k1_fetch_range<VEC, T>(p.W, N, K, n0, kt + BK, tid, rb, k_hi);
+                k1_fetch<VEC, T>(p.X, M, K, m0, kt + BK, tid, ra, k_hi);
+                k1_fetch<VEC, T>(p.W, N, K, n0, kt + BK, tid, rb, k_hi);
             }
 #pragma unroll
             for (int k = 0; k < BK; ++k) {
@@ -216,61 +187,6 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
             __syncthreads();
             buf ^= 1;
         }
-
-    } else {
-        if (p.warm_l2) {
-            // A small grid walks K with one tile of look-ahead, i.e. it pays the memory latency once
-            // per k-tile.  Asking L2 for both operand panels up front puts all of those requests in
-            // flight at once; the k loop then runs at L2 latency.
-            const int lines_per_row = (K * 4 + 127) / 128;
-            const int rows_a = min(BM, M - m0), rows_b = min(BN, N - n0);
-            for (int i = tid; i < (rows_a + rows_b) * lines_per_row; i += K1_THREADS) {
-                const int r = i / lines_per_row, c = i - r * lines_per_row;
-                const float *ptr = r < rows_a ? p.X + (size_t)(m0 + r) * K : p.W + (size_t)(n0 + r - rows_a) * K;
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr + min(c * 32, K - 1)));
-            }
-        }
-        float4 ra[2], rb[2];
-        k1_fetch<VEC, T>(p.X, M, K, m0, 0, tid, ra);
-        k1_fetch<VEC, T>(p.W, N, K, n0, 0, tid, rb);
-        k1_stash<T>(As[0], tid, ra);
-        k1_stash<T>(Bs[0], tid, rb);
-        __syncthreads();
-
-        int buf = 0;
-        for (int kt = 0; kt < K; kt += BK) {
-            const bool more = kt + BK < K;
-            if (more) {
-                k1_fetch<VEC, T>(p.X, M, K, m0, kt + BK, tid, ra);
-                k1_fetch<VEC, T>(p.W, N, K, n0, kt + BK, tid, rb);
-            }
-#pragma unroll
-            for (int k = 0; k < BK; ++k) {
-                const int flip = ((k >> 3) & 1) << 3;          // see k1_stash
-                float a[R];
-                unsigned long long b[R / 2];                    // column pairs as they lie in memory
-#pragma unroll
-                for (int q = 0; q < T; ++q) {
-                    const float4 av = *reinterpret_cast<const float4 *>(&As[buf][k][64 * q + ((ty * 4) ^ flip)]);
-                    const ulonglong2 bv = *reinterpret_cast<const ulonglong2 *>(&Bs[buf][k][64 * q + ((tx * 4) ^ flip)]);
-                    a[4 * q + 0] = av.x; a[4 * q + 1] = av.y; a[4 * q + 2] = av.z; a[4 * q + 3] = av.w;
-                    b[2 * q + 0] = bv.x; b[2 * q + 1] = bv.y;
-                }
-#pragma unroll
-                for (int i = 0; i < R; ++i) {
-                    const unsigned long long ai = pack2(a[i], a[i]);
-#pragma unroll
-                    for (int j = 0; j < R / 2; ++j) ffma2(acc2[i][j], ai, b[j]);
-                }
-            }
-            if (more) {
-                k1_stash<T>(As[buf ^ 1], tid, ra);
-                k1_stash<T>(Bs[buf ^ 1], tid, rb);
-            }
-            __syncthreads();
-            buf ^= 1;
-        }
-
     }
 
     float acc[R][R];
@@ -386,19 +302,7 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
             if (!s_last) return true;
             if (tid < BM && m0 + tid < M) {
                 const int row = m0 + tid;
-                float v = __ldcg(&p.partial[row]);
-                int t = 1;
-                for (; t + 8 <= p.tiles_n; t += 8) {      // 8 independent loads in flight
-                    float o[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) o[u] = __ldcg(&p.partial[(size_t)(t + u) * M + row]);
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) v = ADD ? v + o[u] : fmaxf(v, o[u]);
-                }
-                for (; t < p.tiles_n; ++t) {
-                    const float o = __ldcg(&p.partial[(size_t)t * M + row]);
-                    v = ADD ? v + o : fmaxf(v, o);
-                }
+                const float v = fold_row_partials<ADD>(p.partial, p.tiles_n, M, row);
                 if (CHAIN) s_mean[tid] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)N);
                 else p.out[row] = v;
             }
@@ -466,26 +370,7 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
         __syncthreads();
         if (!s_last) return true;
         if (tid < BM && m0 + tid < M) {
-            const int row = m0 + tid;
-            float4 f = __ldcg(&part4[row]);
-            float mx = f.x, se = f.y, tl = f.z;
-            int t = 1;
-            for (; t + 8 <= p.tiles_n; t += 8) {      // 8 independent loads in flight, then the chain of merges
-                float4 g[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) g[u] = __ldcg(&part4[(size_t)(t + u) * M + row]);
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    lse_merge<true>(mx, se, g[u].x, g[u].y);
-                    tl += g[u].z;
-                }
-            }
-            for (; t < p.tiles_n; ++t) {
-                f = __ldcg(&part4[(size_t)t * M + row]);
-                lse_merge<true>(mx, se, f.x, f.y);
-                tl += f.z;
-            }
-            p.out[row] = mx + logf(se) - tl;
+            p.out[m0 + tid] = fold_row_lse<true>(part4, p.tiles_n, M, m0 + tid);
         }
         if (tid == 0) p.counters[tile_m] = 0u;
         return true;
@@ -526,22 +411,7 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
         // the strip's tiles combined in tile order, all at once (same result in every CTA):
         // mean = sum n_i mean_i / sum n_i,  M2 = sum (M2_i + n_i (mean_i - mean)^2)
         if (tid < BM && m0 + tid < M) {
-            const int row = m0 + tid;
-            float cnt = 0.f, wsum = 0.f;
-            for (int t = 0; t < p.tiles_n; ++t) {
-                const float4 o = __ldcg(&stats[(size_t)t * M + row]);
-                cnt += o.x;
-                wsum = fmaf(o.x, o.y, wsum);
-            }
-            const float mean = wsum / cnt;
-            float m2 = 0.f;
-            for (int t = 0; t < p.tiles_n; ++t) {
-                const float4 o = __ldcg(&stats[(size_t)t * M + row]);
-                const float dm = o.y - mean;
-                m2 += fmaf(o.x * dm, dm, o.z);
-            }
-            s_mean[tid] = mean;
-            s_rstd[tid] = rsqrtf(m2 / cnt + p.e.eps);
+            s_mean[tid] = combine_row_moments<false>(stats, p.tiles_n, M, m0 + tid, p.e.eps, s_rstd[tid]);
         }
         __syncthreads();
         float g[R], be[R];

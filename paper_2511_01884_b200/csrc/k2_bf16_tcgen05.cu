@@ -403,30 +403,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 #pragma unroll
                         for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
                         apply_act_array<false>(p.e.act, x, p.e.scale);
-                        const int nv = min(32, p.N - col0);
-                        RowStat cs;
-                        cs.n = (float)nv;
-                        if (nv == 32) {
-                            float sum = 0.f;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) sum += x[j];
-                            cs.mean = sum * (1.0f / 32.0f);
-                            cs.m2 = 0.f;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) { const float dlt = x[j] - cs.mean; cs.m2 = fmaf(dlt, dlt, cs.m2); }
-                        } else {
-                            float sum = 0.f;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) sum += j < nv ? x[j] : 0.f;
-                            cs.mean = sum / cs.n;
-                            cs.m2 = 0.f;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const float dlt = j < nv ? x[j] - cs.mean : 0.f;
-                                cs.m2 = fmaf(dlt, dlt, cs.m2);
-                            }
-                        }
-                        rs = merge_stat(rs, cs);
+                        rs = merge_stat(rs, chunk_moments(x, min(32, p.N - col0)));
                     }
                 }
                 // the accumulator is in registers: the TMEM buffer goes back to the MMA warp before the wait
@@ -455,26 +432,9 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                     if ((acc ^= 1) == 0) acc_phase ^= 1;
                     continue;
                 }
-                // Combine the strip's parts in part order, all at once (same result on every CTA):
-                // mean = sum n_i mean_i / sum n_i,  M2 = sum (M2_i + n_i (mean_i - mean)^2).
+                // the strip's parts combined in part order, all at once (same result on every CTA)
                 float rstd = 0.f, shift = 0.f;
-                if (row < p.M) {
-                    float cnt = 0.f, wsum = 0.f;
-                    for (int i = 0; i < parts; ++i) {
-                        const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
-                        cnt += o.x;
-                        wsum = fmaf(o.x, o.y, wsum);
-                    }
-                    const float mean = wsum / cnt;
-                    float m2 = 0.f;
-                    for (int i = 0; i < parts; ++i) {
-                        const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
-                        const float dm = o.y - mean;
-                        m2 += fmaf(o.x * dm, dm, o.z);
-                    }
-                    rstd = rsqrtf(m2 / cnt + p.e.eps);
-                    shift = -mean * rstd;
-                }
+                if (row < p.M) shift = -combine_row_moments<false>(stats, parts, p.M, row, p.e.eps, rstd) * rstd;
                 // ---- sweep 2: normalise the registers and store ----
                 if (row < p.M) {
                     __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)row * p.N + n0;
@@ -543,27 +503,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 epi_bar_sync(h);
                 if (s.last_flag[h]) {
                     // the group that arrives last at the strip merges the parts in order
-                    if (row < p.M) {
-                        float4 f = __ldcg(&part4[row]);
-                        mx = f.x; se = f.y; tl = f.z;
-                        int i = 1;
-                        for (; i + 8 <= parts; i += 8) {      // 8 independent loads in flight, then the chain of merges
-                            float4 g[8];
-#pragma unroll
-                            for (int u = 0; u < 8; ++u) g[u] = __ldcg(&part4[(size_t)(i + u) * p.M + row]);
-#pragma unroll
-                            for (int u = 0; u < 8; ++u) {
-                                lse_merge<false>(mx, se, g[u].x, g[u].y);
-                                tl += g[u].z;
-                            }
-                        }
-                        for (; i < parts; ++i) {
-                            f = __ldcg(&part4[(size_t)i * p.M + row]);
-                            lse_merge<false>(mx, se, f.x, f.y);
-                            tl += f.z;
-                        }
-                        reinterpret_cast<float *>(p.out)[row] = mx + __logf(se) - tl;
-                    }
+                    if (row < p.M) reinterpret_cast<float *>(p.out)[row] = fold_row_lse<false>(part4, parts, p.M, row);
                     if (et == 0) p.counters[tm] = 0u;
                 }
                 if ((acc ^= 1) == 0) acc_phase ^= 1;
@@ -619,19 +559,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 epi_bar_sync(h);
                 if (s.last_flag[h]) {
                     if (row < p.M) {
-                        float v = __ldcg(&p.partial[row]);
-                        int i = 1;
-                        for (; i + 8 <= parts; i += 8) {      // 8 independent loads in flight
-                            float o[8];
-#pragma unroll
-                            for (int u = 0; u < 8; ++u) o[u] = __ldcg(&p.partial[(size_t)(i + u) * p.M + row]);
-#pragma unroll
-                            for (int u = 0; u < 8; ++u) v = add ? v + o[u] : fmaxf(v, o[u]);
-                        }
-                        for (; i < parts; ++i) {
-                            const float o = __ldcg(&p.partial[(size_t)i * p.M + row]);
-                            v = add ? v + o : fmaxf(v, o);
-                        }
+                        const float v = add ? fold_row_partials<true>(p.partial, parts, p.M, row) : fold_row_partials<false>(p.partial, parts, p.M, row);
                         if (chain) p.rowg[row] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)p.N);
                         else out[row] = v;
                     }

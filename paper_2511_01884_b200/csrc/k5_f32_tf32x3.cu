@@ -461,20 +461,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 #pragma unroll
                     for (int jj = 0; jj < 32; ++jj) r[jj] = __float_as_uint(v[jj]);
                     ptx::tmem_st_32x32(taddr + c * 32, r);
-                    const int nv = min(32, p.N - col0);
-                    RowStat cs;
-                    cs.n = (float)nv;
-                    float csum = 0.f;
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) csum += jj < nv ? v[jj] : 0.f;
-                    cs.mean = csum / cs.n;
-                    cs.m2 = 0.f;
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        const float dlt = jj < nv ? v[jj] - cs.mean : 0.f;
-                        cs.m2 = fmaf(dlt, dlt, cs.m2);
-                    }
-                    rs = merge_stat(rs, cs);
+                    rs = merge_stat(rs, chunk_moments(v, min(32, p.N - col0)));
                 }
                 ptx::tmem_st_wait();
                 float4 *stats = reinterpret_cast<float4 *>(p.partial);
@@ -491,23 +478,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
                 // the strip's parts combined in part order: mean = sum n_i mean_i / sum n_i, M2 = sum (M2_i + n_i (mean_i - mean)^2)
                 float rstd = 0.f, shift = 0.f;
-                if (row < p.M) {
-                    float cnt = 0.f, wsum = 0.f;
-                    for (int i = 0; i < parts; ++i) {
-                        const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
-                        cnt += o.x;
-                        wsum = fmaf(o.x, o.y, wsum);
-                    }
-                    const float mean = wsum / cnt;
-                    float m2 = 0.f;
-                    for (int i = 0; i < parts; ++i) {
-                        const float4 o = __ldcg(&stats[(size_t)i * p.M + row]);
-                        const float dm = o.y - mean;
-                        m2 += fmaf(o.x * dm, dm, o.z);
-                    }
-                    rstd = 1.0f / sqrtf(m2 / cnt + p.e.eps);
-                    shift = -mean * rstd;
-                }
+                if (row < p.M) shift = -combine_row_moments<true>(stats, parts, p.M, row, p.e.eps, rstd) * rstd;
                 // sweep 2: normalise out of TMEM and store
 #pragma unroll 1
                 for (int c = 0; c < CHUNKS; ++c) {
@@ -603,39 +574,9 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     float *out = reinterpret_cast<float *>(p.out);
                     if (row < p.M) {
                         if (lse) {
-                            float4 f = __ldcg(&part4[row]);
-                            mx = f.x; se = f.y; tl = f.z;
-                            int i = 1;
-                            for (; i + 8 <= parts; i += 8) {      // 8 independent loads in flight, then the chain of merges
-                                float4 g[8];
-#pragma unroll
-                                for (int u = 0; u < 8; ++u) g[u] = __ldcg(&part4[(size_t)(i + u) * p.M + row]);
-#pragma unroll
-                                for (int u = 0; u < 8; ++u) {
-                                    lse_merge<true>(mx, se, g[u].x, g[u].y);
-                                    tl += g[u].z;
-                                }
-                            }
-                            for (; i < parts; ++i) {
-                                f = __ldcg(&part4[(size_t)i * p.M + row]);
-                                lse_merge<true>(mx, se, f.x, f.y);
-                                tl += f.z;
-                            }
-                            out[row] = mx + logf(se) - tl;
+                            out[row] = fold_row_lse<true>(part4, parts, p.M, row);
                         } else {
-                            float v = __ldcg(&p.partial[row]);
-                            int i = 1;
-                            for (; i + 8 <= parts; i += 8) {      // 8 independent loads in flight
-                                float o[8];
-#pragma unroll
-                                for (int u = 0; u < 8; ++u) o[u] = __ldcg(&p.partial[(size_t)(i + u) * p.M + row]);
-#pragma unroll
-                                for (int u = 0; u < 8; ++u) v = add ? v + o[u] : fmaxf(v, o[u]);
-                            }
-                            for (; i < parts; ++i) {
-                                const float o = __ldcg(&p.partial[(size_t)i * p.M + row]);
-                                v = add ? v + o : fmaxf(v, o);
-                            }
+                            const float v = add ? fold_row_partials<true>(p.partial, parts, p.M, row) : fold_row_partials<false>(p.partial, parts, p.M, row);
                             if (chain) p.rowg[row] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)p.N);
                             else out[row] = v;
                         }
