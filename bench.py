@@ -214,7 +214,7 @@ class Rotation:
 
 def w_copies(wl):
     """Distinct copies of W the timed loop rotates through (only the HBM-bound workload needs more than one)."""
-    return 3 if wl.name == "c4" else 1
+    return 3 if wl.hbm_bound else 1
 
 
 def time_steps(rot, steps, warmup, torch, flush_buf=None, barrier=None):
@@ -289,7 +289,7 @@ def sustained_block(rot, wl, peaks, local, torch, seconds=2.5):
     rot.check()
     ms = e0.elapsed_time(e1) / n
     v, u = unit_value(wl, ms)
-    key = "hbm_gbs" if wl.name == "c4" else "bf16_tflops_sustained"
+    key = "hbm_gbs" if wl.hbm_bound else "bf16_tflops_sustained"
     blk = {"steps": n, "seconds": round(ms * n / 1e3, 3), "ms_per_step": round(ms, 5), "value": round(v, 2), "unit": u,
            "clocks": cs.summary()}
     if wl.dtype == wk.BF16 and peaks.get(key):
@@ -360,7 +360,7 @@ def eager_context_us(wl, d, torch, steps=10):
 def roofline_of(wl, ms, peaks, kernel, sm_max_mhz, sm_count, alu_peak=None):
     """Roofline of the (single) kernel of a step: achieved = algorithmic work / measured time."""
     src = peaks["_source"]
-    if wl.name == "c4":
+    if wl.hbm_bound:
         ach = wl.algorithmic_bytes / ms / 1e6
         peak, unit, bound = peaks["hbm_gbs"], "GB/s", "hbm"
         note = f"{wl.algorithmic_bytes} algorithmic bytes per launch; peak = copy bandwidth, of {src}"
@@ -392,7 +392,7 @@ def roofline_of(wl, ms, peaks, kernel, sm_max_mhz, sm_count, alu_peak=None):
 
 def unit_value(wl, ms, n_units=1):
     """Whole-job rate: the units (bytes or flops of one workload) all ranks processed / the slowest rank's time."""
-    if wl.name == "c4":
+    if wl.hbm_bound:
         return multigpu.aggregate_rate(wl.algorithmic_bytes, n_units, ms) / 1e9, "GB/s"
     return multigpu.aggregate_rate(wl.flops, n_units, ms) / 1e12, "TFLOP/s"
 
@@ -420,7 +420,7 @@ def oracle_sample(wl, inp, target_s=12.0, max_rows=None):
                         red=wl.red, eps=wl.ln_eps, rows=rows, **extra)
     dt = time.perf_counter() - t
     flops = 2.0 * len(rows) * wl.N * wl.K
-    if wl.name == "c4":
+    if wl.hbm_bound:
         value, unit = (len(rows) / M) * wl.algorithmic_bytes / dt / 1e9, "GB/s"
     else:
         value, unit = flops / dt / 1e12, "TFLOP/s"
@@ -449,7 +449,7 @@ def run_reference(args):
         if i >= args.warmup:
             times.append(time.perf_counter() - t)
     ms = 1e3 * sum(times) / len(times)
-    if wl.name == "c4":
+    if wl.hbm_bound:
         value, unit = (rows / wl.M) * wl.algorithmic_bytes / ms / 1e6, "GB/s"
     else:
         value, unit = 2.0 * rows * wl.N * wl.K / ms / 1e9, "TFLOP/s"
@@ -557,7 +557,7 @@ def config_of(wl, n_gpus, extra=None):
     return c
 
 
-EXTRA_STEPS = {"c1": 200, "c2": 20, "c4": 300, "c5": 50, "c3": 50, "n1": 20, "n2": 10, "c2t": 50, "n1t": 50, "n1b": 50}
+EXTRA_STEPS = {"c1": 200, "c2": 20, "c4": 300, "c5": 50, "c3": 50, "n1": 20, "n2": 10, "c2t": 50, "n1t": 50, "n1b": 50, "m64": 150}
 
 
 def measure_extra(w2, local, torch, peaks, props, alu_peak):
@@ -578,7 +578,7 @@ def measure_extra(w2, local, torch, peaks, props, alu_peak):
     if fl is not None:            # latency-bound workload: also the figure without the flush
         entry["us_per_call_back_to_back_warm_l2"] = round(back_to_back_us(rot, torch), 2)
         launches += 1020
-    if w2.name == "c4":           # HBM-bound: one call alone on the device, beside the back-to-back figure
+    if w2.hbm_bound:           # HBM-bound: one call alone on the device, beside the back-to-back figure
         med, best = isolated_us(rot, torch)
         entry["us_per_call_isolated"] = {"median": round(med, 2), "min": round(best, 2), "calls": 30,
                                          "how": "a synchronise after every call; W copies rotated as in the timed loop"}
@@ -616,8 +616,9 @@ def run_kernel_only(args, wl, torch, local):
 
 
 def l2_policy(wl):
-    if wl.name == "c4":
-        return "HBM-bound: three distinct copies of W (768 MiB) rotated, no byte of a W is in L2 when it is read again"
+    if wl.hbm_bound:
+        return (f"HBM-bound: three distinct copies of W ({3 * wl.N * wl.K * wl.elem_bytes >> 20} MiB) rotated, "
+                "no byte of a W is in L2 when it is read again")
     if wl.algorithmic_bytes > 130e6:
         return "operands larger than L2 (126 MB), compute-bound: no flush"
     return "L2 flushed (256 MiB write) before every call"
@@ -728,7 +729,7 @@ def main():
                     "matches_device_run": same, "how": "forge_fused_linear_run_host, pinned host buffers, wall clock"},
             "gpu_launches": launches,
             "roofline": roofline_of(wl, ms * wl.M / rows, peaks, op.plan.kernel, clocks.get("sm_max_mhz"), props.multi_processor_count, alu_peak),
-            "nominal_frac": round((value / world) / (NOMINAL["hbm_gbs"] if wl.name == "c4" else NOMINAL["bf16_tflops"]), 4)
+            "nominal_frac": round((value / world) / (NOMINAL["hbm_gbs"] if wl.hbm_bound else NOMINAL["bf16_tflops"]), 4)
             if wl.dtype == wk.BF16 else None}
     if alu_peak:
         line["alu_peak_measured"] = {"value": round(alu_peak, 2), "unit": "TFLOP/s", "effective_sm_mhz": round(mhz, 1),

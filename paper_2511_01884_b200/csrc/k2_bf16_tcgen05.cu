@@ -80,8 +80,16 @@ struct K2Smem {
     float gamma[2][K2_BN];
     float beta[2][K2_BN];
 };
-constexpr size_t K2_SMEM_BYTES = 1024 + (size_t)K2Ring<false>::BYTES + sizeof(K2Smem);
-static_assert(K2Ring<false>::BYTES == K2Ring<true>::BYTES, "both ring layouts use the same shared memory");
+// One CTA per tile with at most 64 rows of X: the X box is 64 rows (8 KiB), which makes room for a fifth stage
+// (5 x 40 KiB): these problems are bound by the stream of W, and what counts is the bytes in flight.  The MMA
+// still spans 128 rows; rows 64..127 of its A operand are the first rows of the stage's W tile (finite values),
+// and the accumulator rows they produce are never read.
+constexpr uint32_t K2_A_BYTES_SHORT = K2_A_BYTES / 2;
+constexpr int K2_STAGES_SHORT = 5;
+constexpr size_t K2_RING_BYTES = (size_t)K2_STAGES_SHORT * (K2_A_BYTES_SHORT + K2Ring<false>::B_BYTES);     // 200 KiB, the largest
+static_assert(K2Ring<false>::BYTES <= K2_RING_BYTES && K2Ring<true>::BYTES <= K2_RING_BYTES && K2_STAGES_SHORT <= K2_MAX_STAGES, "ring");
+constexpr size_t K2_SMEM_BYTES = 1024 + K2_RING_BYTES + sizeof(K2Smem);
+static_assert(K2_SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
 
 struct K2Params {
     int f16;                    // storage format of X, W, b, gamma, beta, Y: IEEE half (1) or bfloat16 (0)
@@ -98,6 +106,7 @@ struct K2Params {
     int group_m;          // row units per rasterisation group
     unsigned *gen;        // launches whose CTAs wait on one another: run index (see run_index_begin)
     int two_pass;         // LayerNorm of rows with more tiles than CTAs (pairs): see K2Item::pass
+    int short_x;          // one CTA per tile and M <= 64: 64-row X box, five stages
     // K split of the last wave's tiles (tail_parts = 1: none)
     int tail_parts;           // S
     int tail_kb;              // k-blocks per part
@@ -187,11 +196,12 @@ __global__ void __launch_bounds__(K2Shape<LN>::THREADS, 1)
 k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const K2Params p)
 {
     using Ring = K2Ring<PAIR>;
-    constexpr int STAGES = Ring::STAGES;
-    constexpr uint32_t STAGE_BYTES = Ring::STAGE_BYTES;
+    const bool short_x = !PAIR && p.short_x;
+    const int STAGES = short_x ? K2_STAGES_SHORT : Ring::STAGES;
+    const uint32_t A_BYTES = short_x ? K2_A_BYTES_SHORT : K2_A_BYTES, STAGE_BYTES = A_BYTES + Ring::B_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    K2Smem &s = *reinterpret_cast<K2Smem *>(tiles + (size_t)Ring::BYTES);
+    K2Smem &s = *reinterpret_cast<K2Smem *>(tiles + K2_RING_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;        // position in the pair; 0 leads
@@ -204,7 +214,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
     const unsigned run = p.cooperative ? run_index_begin(p.gen) : 0u;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < STAGES; ++i) { ptx::mbar_init(&s.full[i], 1); ptx::mbar_init(&s.empty[i], 1); }
+        for (int i = 0; i < K2_MAX_STAGES; ++i) { ptx::mbar_init(&s.full[i], 1); ptx::mbar_init(&s.empty[i], 1); }
         for (int i = 0; i < 2; ++i) { ptx::mbar_init(&s.acc_full[i], 1); ptx::mbar_init(&s.acc_empty[i], PAIR ? 16 : 8); }
         s.abort_flag = 0;
         ptx::fence_mbar_init();
@@ -247,11 +257,11 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                         if (rank == 0) ptx::mbar_expect_tx(&s.full[stage], 2 * STAGE_BYTES);
                         const uint32_t bar = ptx::mapa_u32(ptx::smem_u32(&s.full[stage]), 0);
                         ptx::tma_load_2d_pair(a, &tmX, bar, kb * K2_BK, tm * K2_BM);
-                        ptx::tma_load_2d_pair(a + K2_A_BYTES, &tmW, bar, kb * K2_BK, tn * K2_BN + (int)rank * (K2_BN / 2));
+                        ptx::tma_load_2d_pair(a + A_BYTES, &tmW, bar, kb * K2_BK, tn * K2_BN + (int)rank * (K2_BN / 2));
                     } else {
                         ptx::mbar_expect_tx(&s.full[stage], STAGE_BYTES);
                         ptx::tma_load_2d(a, &tmX, &s.full[stage], kb * K2_BK, tm * K2_BM);
-                        ptx::tma_load_2d(a + K2_A_BYTES, &tmW, &s.full[stage], kb * K2_BK, tn * K2_BN);
+                        ptx::tma_load_2d(a + A_BYTES, &tmW, &s.full[stage], kb * K2_BK, tn * K2_BN);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -273,7 +283,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                     ptx::tc_fence_after();
                     const uint8_t *a = tiles + (size_t)stage * STAGE_BYTES;
                     const uint64_t adesc = ptx::smem_desc_k_sw128(a);
-                    const uint64_t bdesc = ptx::smem_desc_k_sw128(a + K2_A_BYTES);
+                    const uint64_t bdesc = ptx::smem_desc_k_sw128(a + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < K2_BK / 16; ++k) {     // 16 bf16 = 32 bytes = 2 descriptor units
                         if (PAIR) ptx::umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb != w.kb_lo) | (k != 0));
@@ -686,7 +696,7 @@ forge_status_t k2_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     info->tile_m = L.pair ? 2 * K2_BM : K2_BM;
     info->tile_n = K2_BN;
     info->tile_k = K2_BK;
-    info->stages = L.pair ? K2Ring<true>::STAGES : K2Ring<false>::STAGES;
+    info->stages = L.pair ? K2Ring<true>::STAGES : (d.M <= K2_BM / 2 ? K2_STAGES_SHORT : K2Ring<false>::STAGES);
     info->cluster = L.pair ? 2 : 1;
     info->threads = K2Shape<false>::THREADS;
     info->grid = L.grid;
@@ -793,7 +803,8 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     const bool pair = h.info.cluster == 2;
     forge_status_t st;
     if (h.tmX_ptr != a.X) {
-        if ((st = encode_tmap_16(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, K2_BM, K2_BK, d.dtype == FORGE_F16)) != FORGE_OK) return st;
+        const bool short_x = !pair && d.M <= K2_BM / 2;          // the box is what TMA writes: 64 rows, 8 KiB
+        if ((st = encode_tmap_16(&h.tmX, a.X, (uint64_t)d.M, (uint64_t)d.K, short_x ? K2_BM / 2 : K2_BM, K2_BK, d.dtype == FORGE_F16)) != FORGE_OK) return st;
         h.tmX_ptr = a.X;
     }
     if (h.tmW_ptr != a.W) {
@@ -817,6 +828,7 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     p.tiles_m = (int)((d.M + K2_BM - 1) / K2_BM);
     p.tiles_n = (int)((d.N + K2_BN - 1) / K2_BN);
     p.num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
+    p.short_x = !pair && d.M <= K2_BM / 2;
     p.group_m = pair ? K2_GROUP_M / 2 : K2_GROUP_M;      // 2048 rows either way
     if (!ln) {
         const K2Layout L = k2_layout(d, h.sm_count);

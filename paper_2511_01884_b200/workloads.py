@@ -148,6 +148,12 @@ class Workload:
         return 2 * self.M * self.N * self.K
 
     @property
+    def hbm_bound(self) -> bool:
+        """Few rows of X on 16-bit storage: streaming W once is the whole cost (below 128 flop per byte the
+        tensor cores wait for the memory), so the rate that means something is bytes per second."""
+        return self.dtype in (BF16, F16) and self.M < 128
+
+    @property
     def elem_bytes(self) -> int:
         return 4 if self.dtype in (F32, F32_TF32X3) else 2
 
@@ -213,6 +219,10 @@ EXTRA_WORKLOADS: Dict[str, Workload] = {
     "n1b": Workload("n1b", BF16, 8192, 8192, 8192, ACT_IDENTITY, RED_MEAN_GELU_RESIDUAL, 1.0, 0.0,
                     Dist("normal", 1.0), Dist("normal", 0.02), Dist("normal", 0.02),
                     note="bf16, subtract, row mean, GELU-erf, residual add", sub=Dist("uniform", -0.5, 0.5)),
+    # between the skinny kernel's 32 rows and a full 128-row tile: still bound by the stream of W
+    "m64": Workload("m64", BF16, 64, 32768, 8192, ACT_GELU_TANH, RED_NONE, 1.0, 0.0,
+                    Dist("normal", 1.0), Dist("normal", 0.02), Dist("normal", 0.02),
+                    note="bf16, 64 rows against a 32768 x 8192 weight, GELU-tanh"),
     "c2t": dataclasses.replace(WORKLOADS["c2"], name="c2t", dtype=F32_TF32X3,
                                note="C2's tensors, contraction as three TF32 tensor-core products"),
 }

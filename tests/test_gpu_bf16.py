@@ -1,5 +1,7 @@
 """GPU parity of the bf16 tcgen05 path (TMA -> shared-memory ring -> tcgen05.mma -> TMEM ->
 fused epilogue) against the CPU oracle."""
+import dataclasses
+
 import numpy as np
 import pytest
 
@@ -115,3 +117,18 @@ def test_tiles_of_the_last_wave_cut_along_k(M, N, K, grid, red):
     assert np.array_equal(a, b)
     rows = np.unique(np.concatenate([np.arange(0, M, 7), [M - 1]]))
     pu.assert_parity(wl, a[rows], pu.run_oracle(wl, inp, rows))
+
+
+def test_row_counts_between_the_skinny_kernel_and_a_full_tile():
+    """M = 48, 64, 96 against a 32768 x 8192 weight: more rows than the skinny kernel carries, fewer than a 128-row
+    tile -- the problem is still bound by the stream of W.  Served by this kernel (one CTA per tile, the last wave cut
+    along K); every output element against the oracle."""
+    base = wk.EXTRA_WORKLOADS["m64"]
+    full = wk.make_inputs(dataclasses.replace(base, M=96))
+    for M in (48, 64, 96):
+        wl = dataclasses.replace(base, name=f"m{M}", M=M)
+        inp = dict(full)
+        inp["X"] = np.ascontiguousarray(full["X"][:M])
+        g, plan = pu.run_gpu(wl, inp)
+        assert plan["kernel"] == B.FORGE_KERNEL_BF16_TCGEN05 and plan["cluster"] == 1
+        pu.assert_parity(wl, g, pu.run_oracle(wl, inp), f"M={M}")
