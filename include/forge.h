@@ -43,8 +43,11 @@ typedef enum {
     FORGE_ERR_CUDA = 3,          /* a CUDA runtime/driver call failed (or no sm_100 GPU)  */
     FORGE_ERR_ALLOC = 4,         /* host or device allocation failed                      */
     FORGE_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up                    */
-    FORGE_ERR_SCRATCH_LIMIT = 6  /* problem needs more scratch than the fixed buffer of   */
+    FORGE_ERR_SCRATCH_LIMIT = 6, /* problem needs more scratch than the fixed buffer of   */
                                  /* forge_fused_linear_f32_reduce_static() holds          */
+    FORGE_ERR_BOUNDS = 7         /* bounds-checked build only (-DFORGE_DEBUG_BOUNDS): a    */
+                                 /* kernel computed an index outside its allocation; the  */
+                                 /* access was skipped (last_status / last_wait_detail)   */
 } forge_status_t;
 
 typedef enum {
@@ -190,8 +193,11 @@ forge_status_t forge_fused_linear_last_status(forge_fused_linear_t h);
 /*
  * Diagnostics of the give-up that the most recent last_status() call reported (host pointer
  * to 4 ints): [0] which wait (1 operand tile arrival, 2 ring stage release, 3 accumulator
- * ready, 4 accumulator release, 5 arrival of the other tiles of a row strip), [1] a
- * kernel-specific detail word, [2] CTA index, [3] thread index.  All zero if none.
+ * ready, 4 accumulator release, 5 arrival of the other tiles of a row strip) or, for
+ * FORGE_ERR_BOUNDS, which allocation (16 shared-memory ring, 17 tensor-memory columns,
+ * 18 workspace partials, 19 workspace counters, 20 other shared memory), [1] a kernel-specific
+ * detail word (FORGE_ERR_BOUNDS: the offending index), [2] CTA index, [3] thread index.  All
+ * zero if none.
  */
 forge_status_t forge_fused_linear_last_wait_detail(forge_fused_linear_t h, int detail[4]);
 

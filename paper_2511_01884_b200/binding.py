@@ -7,11 +7,12 @@ import os
 from typing import Optional
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libforge.so")
+# FORGE_LIBRARY names another build of the same library to load instead (the bounds-checked one, say)
+LIB_PATH = os.environ.get("FORGE_LIBRARY") or os.path.join(_HERE, "libforge.so")
 
 # enums of forge.h
 (FORGE_OK, FORGE_ERR_INVALID_ARG, FORGE_ERR_UNSUPPORTED, FORGE_ERR_CUDA, FORGE_ERR_ALLOC, FORGE_ERR_TIMEOUT,
- FORGE_ERR_SCRATCH_LIMIT) = range(7)
+ FORGE_ERR_SCRATCH_LIMIT, FORGE_ERR_BOUNDS) = range(8)
 FORGE_STATIC_SCRATCH_BYTES = 1 << 20
 FORGE_F32, FORGE_BF16, FORGE_F16, FORGE_F32_TF32X3 = 0, 1, 2, 3
 FORGE_ACT_IDENTITY, FORGE_ACT_RELU, FORGE_ACT_GELU_ERF, FORGE_ACT_GELU_TANH, FORGE_ACT_SILU = range(5)

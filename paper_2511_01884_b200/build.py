@@ -1,4 +1,5 @@
-"""Build the CUDA library in-tree: ``python -m paper_2511_01884_b200.build [-v] [-f] [-DNAME[=VALUE] ...]``.
+"""Build the CUDA library in-tree: ``python -m paper_2511_01884_b200.build [-v] [-f] [-DNAME[=VALUE] ...]``
+(``--debug-bounds``: the bounds-checked build as a second library, ``libforge_debug_bounds.so``).
 
 One shared object, ``libforge.so``, next to this file, from every ``csrc/*.cu``; compiled
 for sm_100a only (the kernels use tcgen05 / TMEM / TMA and have no other target).
@@ -38,7 +39,18 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(verbose: bool = False, force: bool = False, defines=()) -> str:
+DEBUG_LIB = os.path.join(HERE, "libforge_debug_bounds.so")
+
+
+def build_debug_bounds(verbose: bool = False) -> str:
+    """The bounds-checked build, beside the normal one (load it with FORGE_LIBRARY=<path>)."""
+    return build(verbose=verbose, defines=["-DFORGE_DEBUG_BOUNDS"], out=DEBUG_LIB)
+
+
+def build(verbose: bool = False, force: bool = False, defines=(), out: str = LIB) -> str:
+    global OBJ
+    LIB_OUT = out
+    OBJ = os.path.join(HERE, "_build" if out == LIB else "_build_" + os.path.splitext(os.path.basename(out))[0])
     # a build with -D options, and the first build after one, recompile everything
     stamp = os.path.join(OBJ, "defines.txt")
     os.makedirs(OBJ, exist_ok=True)
@@ -74,12 +86,15 @@ def build(verbose: bool = False, force: bool = False, defines=()) -> str:
     for o in glob.glob(os.path.join(OBJ, "*.o")):
         if o not in objs:
             os.remove(o)
-    if force or jobs or _stale(LIB, objs):
-        tmp = LIB + f".tmp{os.getpid()}"
+    if force or jobs or _stale(LIB_OUT, objs):
+        tmp = LIB_OUT + f".tmp{os.getpid()}"
         subprocess.check_call([NVCC, "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, LIB_OUT)
+    return LIB_OUT
 
 
 if __name__ == "__main__":
-    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, defines=[a for a in sys.argv[1:] if a.startswith("-D")]))
+    if "--debug-bounds" in sys.argv:
+        print(build_debug_bounds(verbose="-v" in sys.argv))
+    else:
+        print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, defines=[a for a in sys.argv[1:] if a.startswith("-D")]))

@@ -25,15 +25,35 @@ enum WaitSite : int {
     SITE_ARRIVAL = 5, SITE_SPLIT = 8
 };
 
-// Words 1..3 of the status area describe the first give-up: a caller-chosen detail word, the
+// Words 1..3 of the status area describe the first report: a caller-chosen detail word, the
 // CTA index and the thread index.
-__device__ __forceinline__ void report_timeout(int *status, int site, int detail = 0)
+__device__ __forceinline__ void report_status(int *status, int code, int site, int detail)
 {
-    if (atomicCAS(status, 0, (int(FORGE_ERR_TIMEOUT) << 16) | site) == 0) {
+    if (atomicCAS(status, 0, (code << 16) | site) == 0) {
         status[1] = detail;
         status[2] = (int)blockIdx.x;
         status[3] = (int)threadIdx.x;
     }
+}
+__device__ __forceinline__ void report_timeout(int *status, int site, int detail = 0) { report_status(status, FORGE_ERR_TIMEOUT, site, detail); }
+
+// ---- bounds-checked build ------------------------------------------------------------------------
+// With -DFORGE_DEBUG_BOUNDS every offset into the shared-memory ring, every tensor-memory column range and
+// every workspace index a kernel computes is compared with the extent of its allocation before it is used;
+// the first one outside is recorded in the status word (FORGE_ERR_BOUNDS, which allocation, the index) and the
+// access is skipped -- never a trap.  In a normal build in_bounds() is the constant true.
+enum BoundsSite : int { BOUNDS_RING = 16, BOUNDS_TMEM = 17, BOUNDS_PARTIAL = 18, BOUNDS_COUNTER = 19, BOUNDS_SMEM = 20 };
+#ifdef FORGE_DEBUG_BOUNDS
+constexpr bool kDebugBounds = true;
+#else
+constexpr bool kDebugBounds = false;
+#endif
+__device__ __forceinline__ bool in_bounds(int *status, int site, long long first, long long count, long long extent)
+{
+    if (!kDebugBounds) return true;
+    if (first >= 0 && count >= 0 && first + count <= extent) return true;
+    if (status) report_status(status, FORGE_ERR_BOUNDS, site, (int)first);
+    return false;
 }
 
 // ---- activations -------------------------------------------------------------------

@@ -305,6 +305,8 @@ forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, 
     h->ws.status = (int *)base;
     h->ws.counters = (unsigned *)(base + kStatusBytes);
     h->ws.partial = (float *)(base + kStatusBytes + ((wl.counters * sizeof(unsigned) + 255) / 256) * 256);
+    h->ws.partial_floats = (long long)wl.partial_floats;
+    h->ws.counter_words = (long long)wl.counters;
     if (!clear_workspace(h->ws)) { cudaFree(h->ws.base); delete h; return FORGE_ERR_CUDA; }
 
     switch (h->info.kernel) {
@@ -551,6 +553,7 @@ const char *forge_status_string(forge_status_t s)
     case FORGE_ERR_ALLOC: return "allocation failed";
     case FORGE_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case FORGE_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the fixed no-allocation buffer holds";
+    case FORGE_ERR_BOUNDS: return "bounds-checked build: an index outside its allocation (the access was skipped)";
     }
     return "unknown status";
 }

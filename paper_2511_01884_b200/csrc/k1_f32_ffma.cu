@@ -35,6 +35,7 @@ struct K1Params {
     // area follow from the fields above -- see k1_slice_len().)
     int *status;           // LayerNorm: status word of the bounded strip wait
     unsigned *gen;         // LayerNorm: run index of the strip counters (see run_index_begin)
+    long long ws_floats, ws_counters;      // extents of `partial` and `counters` (bounds-checked build)
 };
 
 // Length of a K slice when K is cut into `slices`: a multiple of the small tile's 32-wide k-tile.
@@ -206,6 +207,11 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
         const int k_slices = (int)gridDim.z;
         const int tile = tile_m * (int)gridDim.x + tile_n;
         float4 *mine = slice_partial + (((size_t)tile * k_slices + blockIdx.z) * K1_THREADS + tid) * (R * R / 4);
+        // (the same verdict in every thread: the check is on the tile's whole hand-over area and its counter)
+        if (!in_bounds(p.status, BOUNDS_PARTIAL, (long long)(reinterpret_cast<float *>(slice_partial) - p.partial) + (long long)tile * k_slices * K1_THREADS * (R * R),
+                       (long long)k_slices * K1_THREADS * (R * R), p.ws_floats) ||
+            !in_bounds(p.status, BOUNDS_COUNTER, (long long)(slice_counters - p.counters) + tile, 1, p.ws_counters))
+            return true;
 #pragma unroll
         for (int i = 0; i < R; ++i)
 #pragma unroll
@@ -235,6 +241,15 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
     }
 
     // ---- epilogue: bias, activation, scale, in registers --------------------------------
+    if (kDebugBounds && RED != FORGE_RED_NONE && (p.tiles_n > 1 || RED == FORGE_RED_LAYERNORM)) {
+        // the rows of this tile's partials in the workspace (one float, or one float4, per row) and the strip's
+        // counter, checked before either is touched (the same verdict in every thread)
+        constexpr bool WIDE = RED == FORGE_RED_LAYERNORM || RED == FORGE_RED_LOGSUMEXP || RED == FORGE_RED_CROSS_ENTROPY;
+        const long long first = (long long)tile_n * M + m0, rows = min(BM, M - m0);
+        if (!in_bounds(p.status, BOUNDS_PARTIAL, WIDE ? 4 * first : first, WIDE ? 4 * rows : rows, p.ws_floats) ||
+            !in_bounds(p.status, BOUNDS_COUNTER, tile_m, 1, p.ws_counters))
+            return true;
+    }
     int col[R];
     bool cok[R];
     float bias[R];
@@ -566,6 +581,8 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
     p.partial = h.ws.partial;
     p.counters = h.ws.counters;
     p.status = h.ws.status;
+    p.ws_floats = h.ws.partial_floats;
+    p.ws_counters = h.ws.counter_words;
     const int bm = h.info.tile_m, bn = h.info.tile_n;          // 128 or 64
     p.warm_l2 = (h.info.grid < h.sm_count) && (d.K <= 4096);   // latency-bound grids with modest panels
     p.tiles_n = (int)((d.N + bn - 1) / bn);
@@ -673,6 +690,8 @@ extern "C" forge_status_t forge_fused_linear_f32_reduce_static(int64_t M, int64_
     p.warm_l2 = 0;
     p.status = nullptr;
     p.gen = nullptr;
+    p.ws_floats = (long long)((K1_STATIC_SCRATCH_BYTES - counter_bytes) / sizeof(float));
+    p.ws_counters = (long long)(counter_bytes / sizeof(unsigned));
     const dim3 grid((unsigned)tiles_n, (unsigned)tiles_m);
     const bool vec = (K % 4 == 0) && ((uintptr_t)X % 16 == 0) && ((uintptr_t)W % 16 == 0);
     if (red == FORGE_RED_SUM)

@@ -107,6 +107,7 @@ struct K2Params {
     unsigned *gen;        // launches whose CTAs wait on one another: run index (see run_index_begin)
     int two_pass;         // LayerNorm of rows with more tiles than CTAs (pairs): see K2Item::pass
     int short_x;          // one CTA per tile and M <= 64: 64-row X box, five stages
+    long long ws_floats, ws_counters;      // extents of `partial` and `counters` (bounds-checked build)
     // K split of the last wave's tiles (tail_parts = 1: none)
     int tail_parts;           // S
     int tail_kb;              // k-blocks per part
@@ -250,6 +251,7 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 const int tm = PAIR ? 2 * w.tm + (int)rank : w.tm, tn = w.tn;
                 for (int kb = w.kb_lo; kb < w.kb_hi; ++kb) {
                     if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
+                    if (!in_bounds(p.status, BOUNDS_RING, (long long)stage * STAGE_BYTES, STAGE_BYTES, (long long)K2_RING_BYTES)) { ok = false; break; }
                     uint8_t *a = tiles + (size_t)stage * STAGE_BYTES;
                     if (PAIR) {
                         // the leader's barrier counts the bytes of both CTAs (rows past M or N are zero fill
@@ -278,8 +280,10 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 if (!ptx::mbar_wait(&s.acc_empty[acc], acc_phase ^ 1, p.status, SITE_ACC_EMPTY)) { ok = false; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * K2_BN;
+                if (!in_bounds(p.status, BOUNDS_TMEM, acc * K2_BN, K2_BN, K2_TMEM_COLS)) { ok = false; break; }
                 for (int kb = w.kb_lo; kb < w.kb_hi; ++kb) {
                     if (!ptx::mbar_wait(&s.full[stage], phase, p.status, SITE_TMA_FULL)) { ok = false; break; }
+                    if (!in_bounds(p.status, BOUNDS_RING, (long long)stage * STAGE_BYTES, STAGE_BYTES, (long long)K2_RING_BYTES)) { ok = false; break; }
                     ptx::tc_fence_after();
                     const uint8_t *a = tiles + (size_t)stage * STAGE_BYTES;
                     const uint64_t adesc = ptx::smem_desc_k_sw128(a);
@@ -341,6 +345,23 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
 
             const int row = m0 + q * 32 + lane;
             const uint32_t taddr = tmem_base + (uint32_t)(acc * K2_BN + h * HALF) + ((uint32_t)(q * 32) << 16);
+            if (kDebugBounds && m0 < p.M) {
+                // what this group will touch for this tile, checked before any of it is touched (the same verdict in
+                // every thread of the group): its tensor-memory columns, the strip's counter, the rows of its part
+                // in the workspace (one float or one float4 per row), the hand-over area of a K cut
+                const bool wide = LN || p.e.red == FORGE_RED_LOGSUMEXP || p.e.red == FORGE_RED_CROSS_ENTROPY;
+                const bool uses_ws = LN || reduce || wide;
+                const long long rows = min(K2_BM, p.M - m0), first = (long long)part * p.M + m0;
+                bool fine = in_bounds(p.status, BOUNDS_TMEM, acc * K2_BN + h * HALF, HALF, K2_TMEM_COLS);
+                if (uses_ws) fine = fine && in_bounds(p.status, BOUNDS_COUNTER, tm, 1, p.ws_counters) &&
+                                    in_bounds(p.status, BOUNDS_PARTIAL, wide ? 4 * first : first, wide ? 4 * rows : rows, p.ws_floats);
+                if (!LN && w.tail >= 0)
+                    fine = fine && in_bounds(p.status, BOUNDS_PARTIAL, (long long)(reinterpret_cast<float *>(p.tail_scratch) - p.partial) +
+                                             ((((long long)w.tail * (p.tail_parts - 1) + (p.tail_parts - 2)) * 2 + rank) * 2 + h) * (4ll * 32 * K2_EPI_THREADS),
+                                             4ll * 32 * K2_EPI_THREADS, p.ws_floats) &&
+                           in_bounds(p.status, BOUNDS_COUNTER, (long long)(p.tail_flags - p.counters) + ((long long)w.tail * 2 + rank) * 2 + h, 1, p.ws_counters);
+                if (!fine) { ok = false; break; }
+            }
             if (PAIR && m0 >= p.M) {
                 // second half of the last pair tile lies past M: nothing to publish, free the accumulator
                 ptx::tc_fence_before();
@@ -829,6 +850,8 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     p.tiles_n = (int)((d.N + K2_BN - 1) / K2_BN);
     p.num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
     p.short_x = !pair && d.M <= K2_BM / 2;
+    p.ws_floats = h.ws.partial_floats;
+    p.ws_counters = h.ws.counter_words;
     p.group_m = pair ? K2_GROUP_M / 2 : K2_GROUP_M;      // 2048 rows either way
     if (!ln) {
         const K2Layout L = k2_layout(d, h.sm_count);

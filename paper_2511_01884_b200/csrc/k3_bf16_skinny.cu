@@ -77,6 +77,7 @@ struct K3Params {
     int num_kb;
     int groups;           // N / 8
     int box_groups;       // groups per strip = rows of the W box / 8
+    long long ws_floats;  // extent of `partial` (bounds-checked build)
 };
 
 __device__ __forceinline__ void k3_consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(K3_CONSUMERS) : "memory"); }
@@ -131,6 +132,7 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                     int kb = i + kb_rot;
                     if (kb >= p.num_kb) kb -= p.num_kb;
                     if (!ptx::mbar_wait(&s.empty[slot], phase ^ 1, p.status, SITE_STAGE_EMPTY, (slot << 16) | (kb & 0xffff))) { ok = false; break; }
+                    if (!in_bounds(p.status, BOUNDS_RING, (long long)slot * STAGE_BYTES, STAGE_BYTES, (long long)K3_RING_BYTES)) { ok = false; break; }
                     uint8_t *dst = ring + (size_t)slot * STAGE_BYTES;
                     ptx::mbar_expect_tx(&s.full[slot], stage_tx);
                     // a box that starts at or past K (ragged last stage) is all zero fill
@@ -183,6 +185,7 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
 
             for (; seq < seq_end; seq += K3_KSPLIT) {
                 if (ok && !ptx::mbar_wait(&s.full[slot], phase, p.status, SITE_TMA_FULL, (slot << 16) | (seq & 0xffff))) ok = false;
+                if (ok && !in_bounds(p.status, BOUNDS_RING, (long long)slot * STAGE_BYTES, STAGE_BYTES, (long long)K3_RING_BYTES)) ok = false;
                 if (ok) {
                     const uint32_t wbase = ptx::smem_u32(ring + (size_t)slot * STAGE_BYTES);
                     const uint32_t xbase = wbase + K3_W_BYTES;
@@ -335,6 +338,7 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
                         const size_t slot_i = (size_t)blockIdx.x * ROWS + mt * 16 + t;
+                        if (!in_bounds(p.status, BOUNDS_PARTIAL, (long long)slot_i * (softmax ? 4 : 1), softmax ? 4 : 1, p.ws_floats)) continue;
                         if (softmax) part4[slot_i] = make_float4(running[mt], running_s[mt], running_t[mt], 0.f);
                         else p.partial[slot_i] = running[mt];
                     }
@@ -464,6 +468,7 @@ forge_status_t k3_launch(Handle &h, const RunArgs &a)
     p.num_kb = (int)((d.K + K3_KB * K3_BK - 1) / (K3_KB * K3_BK));
     p.groups = (int)(d.N / 8);
     p.box_groups = h.info.tile_n / 8;
+    p.ws_floats = h.ws.partial_floats;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)h.info.grid);
     cfg.blockDim = dim3(K3_THREADS);

@@ -130,6 +130,7 @@ struct K5Params {
     int *status;
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     int group_m;
+    long long ws_floats, ws_counters;   // extents of `partial` and `counters` (bounds-checked build)
     int chunk_kb;               // stages per TMEM accumulation chunk
     // K split of the last wave's tiles (tail_parts = 1: none)
     int tail_parts;             // S
@@ -243,6 +244,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     const int tm = 2 * w.um + (int)rank, tn = w.tn;
                     for (int kb = w.kb_lo; kb < w.kb_hi; ++kb) {
                         if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
+                        if (!in_bounds(p.status, BOUNDS_RING, (long long)stage * K5_STAGE_BYTES, K5_RAW_BYTES, K5_RING_BYTES)) { ok = false; break; }
                         uint8_t *a = tiles + (size_t)stage * K5_STAGE_BYTES;
                         ptx::mbar_expect_tx(&s.full[stage], K5_RAW_BYTES);      // rows past M or N are zero fill and count in full
                         ptx::tma_load_2d(a, &tmX, &s.full[stage], kb * K5_BK, tm * K5_BM);
@@ -264,9 +266,11 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                         if (!ptx::mbar_wait(&s.acc_empty[acc], acc_phase ^ 1, p.status, SITE_ACC_EMPTY)) { ok = false; break; }
                         ptx::tc_fence_after();
                         const uint32_t d_tmem = tmem_base + (uint32_t)acc * K5_BN;
+                        if (!in_bounds(p.status, BOUNDS_TMEM, acc * K5_BN, K5_BN, K5_TMEM_COLS)) { ok = false; break; }
                         const int kb1 = min(kb0 + p.chunk_kb, w.kb_hi);
                         for (int kb = kb0; kb < kb1; ++kb) {
                             if (!ptx::mbar_wait(&s.split[stage], phase, p.status, SITE_SPLIT)) { ok = false; break; }
+                            if (!in_bounds(p.status, BOUNDS_RING, (long long)stage * K5_STAGE_BYTES, K5_STAGE_BYTES, K5_RING_BYTES)) { ok = false; break; }
                             ptx::tc_fence_after();
                             const uint8_t *a = tiles + (size_t)stage * K5_STAGE_BYTES;
                             const uint64_t a_hi = ptx::smem_desc_k_sw128(a), b_hi = ptx::smem_desc_k_sw128(a + K5_A_BYTES);
@@ -358,6 +362,22 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             }
             const int row = m0 + q * 32 + lane;
             const uint32_t lane_addr = tmem_base + (uint32_t)(h * HALF) + ((uint32_t)(q * 32) << 16);
+            if (kDebugBounds && m0 < p.M) {
+                // what this group will touch for this tile, checked before any of it is touched (the same verdict in
+                // every thread of the group): its tensor-memory columns in both buffers, the strip's counter, the rows
+                // of its part in the workspace (one float or one float4 per row), the hand-over area of a K cut
+                const bool wide = ln || lse, uses_ws = wide || fold;
+                const long long rows = min(K5_BM, p.M - m0), first = (long long)part * p.M + m0;
+                bool fine = in_bounds(p.status, BOUNDS_TMEM, K5_BN + h * HALF, HALF, K5_TMEM_COLS);
+                if (uses_ws) fine = fine && in_bounds(p.status, BOUNDS_COUNTER, tm, 1, p.ws_counters) &&
+                                    in_bounds(p.status, BOUNDS_PARTIAL, wide ? 4 * first : first, wide ? 4 * rows : rows, p.ws_floats);
+                if (w.tail >= 0)
+                    fine = fine && in_bounds(p.status, BOUNDS_PARTIAL, (long long)(reinterpret_cast<float *>(p.tail_scratch) - p.partial) +
+                                             ((((long long)w.tail * (p.tail_parts - 1) + (p.tail_parts - 2)) * 2 + rank) * 2 + h) * (4ll * 32 * K5_EPI_THREADS),
+                                             4ll * 32 * K5_EPI_THREADS, p.ws_floats) &&
+                           in_bounds(p.status, BOUNDS_COUNTER, (long long)(p.tail_flags - p.counters) + ((long long)w.tail * 2 + rank) * 2 + h, 1, p.ws_counters);
+                if (!fine) { ok = false; break; }
+            }
             // ---- chunks of K: drain every finished accumulator into the running sum (round to nearest) ----
             float sum[HALF];
 #pragma unroll
@@ -757,6 +777,8 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
     p.tiles_m = (int)((d.M + K5_BM - 1) / K5_BM);
     const K5Layout L = k5_layout(d, h.sm_count);
     p.gen = h.ws.counters + L.gen_idx;
+    p.ws_floats = h.ws.partial_floats;
+    p.ws_counters = h.ws.counter_words;
     p.cooperative = k5_ctas_wait(h);
     p.rowg = h.ws.partial + L.rowg_off;
     p.strips_done = h.ws.counters + L.strips_done_idx;

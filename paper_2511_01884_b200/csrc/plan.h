@@ -22,6 +22,7 @@ struct Workspace {
     int *status = nullptr;           // status word
     void *base = nullptr;            // the single allocation the three point into
     size_t bytes = 0;
+    long long partial_floats = 0, counter_words = 0;     // extents of the two areas (for the bounds-checked build)
 };
 
 struct Handle;

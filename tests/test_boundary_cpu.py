@@ -114,8 +114,8 @@ def test_tf32x3_plan():
 
 
 def test_status_and_kernel_strings():
-    seen = {B.status_string(s) for s in range(7)}
-    assert len(seen) == 7 and "unknown status" not in seen
+    seen = {B.status_string(s) for s in range(8)}
+    assert len(seen) == 8 and "unknown status" not in seen
     assert B.status_string(99) == "unknown status"
     assert "f32" in B.kernel_name(B.FORGE_KERNEL_F32_FFMA)
 
