@@ -53,6 +53,11 @@
 // (bounded) for the strip's other half tiles, combines the statistics in part order and normalises
 // out of TMEM.  The mean chain publishes gelu(mean) per row and the whole grid writes the residual
 // rows at the end.  In both, and with the K cut, CTAs wait on one another: the launch is cooperative.
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+
 #include "common.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
@@ -91,9 +96,12 @@ constexpr int K5_REGS_NEEDED = 256 * K5_REGS_EPI + 256 * K5_REGS_OTHER;
 // A kind::tf32 MMA reading a full fp32 word uses its upper 19 bits and ignores the 13 low
 // fraction bits (measured on B200: with an identity weight and inputs that run through all 8192
 // tail patterns the result is exact, which it would not be if the word were rounded), so the raw
-// tile serves as hi.  K5_WRITE_HI = 1 instead stores hi explicitly (words that are TF32 numbers
-// whatever the hardware does with low bits) at the price of a third more shared-memory traffic
-// in the splitters: 717 us instead of 615 us on a 4096^3 problem.
+// tile serves as hi.  That is a property of the hardware, not of the instruction set's definition, so it
+// is not taken on trust: the first handle created on a device runs a small problem with an identity weight
+// whose exact result depends on it (k5_probe_heads); where it does not hold -- or in a build with
+// -DK5_WRITE_HI=1 -- the splitters store hi explicitly (words that are TF32 numbers whatever the hardware
+// does with low bits) at the price of a third more shared-memory traffic: 717 us instead of 615 us on a
+// 4096^3 problem.
 #ifndef K5_WRITE_HI
 #define K5_WRITE_HI 0
 #endif
@@ -131,6 +139,7 @@ struct K5Params {
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     int group_m;
     long long ws_floats, ws_counters;   // extents of `partial` and `counters` (bounds-checked build)
+    int write_hi;               // the splitters also store the TF32 heads (the raw words do not serve as such here)
     int chunk_kb;               // stages per TMEM accumulation chunk
     // K split of the last wave's tiles (tail_parts = 1: none)
     int tail_parts;             // S
@@ -318,7 +327,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                     hi.z = __uint_as_float(__float_as_uint(v.z) & 0xffffe000u);
                     hi.w = __uint_as_float(__float_as_uint(v.w) & 0xffffe000u);
                     lo[idx] = make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);
-                    if (K5_WRITE_HI) raw[idx] = hi;
+                    if (p.write_hi) raw[idx] = hi;
                 }
                 ptx::fence_proxy_async_smem();      // these writes are read by the tensor core (async proxy)
                 __syncwarp();
@@ -730,8 +739,71 @@ static bool k5_ctas_wait(const Handle &h)
     return h.d.red == FORGE_RED_MEAN_GELU_RESIDUAL || h.d.red == FORGE_RED_LAYERNORM || k5_layout(h.d, h.sm_count).tail_parts > 1;
 }
 
+// Do the raw fp32 words serve as TF32 heads on this device, i.e. does a kind::tf32 MMA ignore the 13 low
+// fraction bits rather than round them away?  Per device: 0 not known yet, 1 yes, 2 no (heads are written),
+// 3 being found out right now (by the nested handle of the probe itself).
+static int k5_heads_mode[64];
+static std::mutex k5_heads_mutex;
+
+// X = 128 x 32 values whose low 13 fraction bits run through many patterns, W = the first 32 rows of an
+// identity (256 x 32), no bias, no activation: Y[:, :32] must reproduce X to 2^-20 if the scheme holds
+// (1 * x = hi + lo, of which the tensor core drops at most the two lowest bits of lo); a tensor core that
+// rounded the raw word to the nearest TF32 number instead would be off by up to 2^-11 |x| on about half of them.
+static forge_status_t k5_probe_heads(int device, int *mode)
+{
+    constexpr int M = 128, N = 256, K = 32;
+    float *hx = new (std::nothrow) float[M * K + N * K + M * N];
+    if (!hx) return FORGE_ERR_ALLOC;
+    float *hw = hx + M * K, *hy = hw + N * K;
+    for (int i = 0; i < M * K; ++i) {
+        const uint32_t tail = ((uint32_t)i * 2654435761u) & 0x1fffu, head = ((uint32_t)i * 40503u) & 0x3ffu;
+        const uint32_t bits = ((uint32_t)(120 + i % 16) << 23) | (head << 13) | tail | (((uint32_t)i & 1u) << 31);
+        std::memcpy(&hx[i], &bits, 4);
+    }
+    for (int i = 0; i < N * K; ++i) hw[i] = (i / K == i % K) ? 1.0f : 0.0f;
+    forge_fused_linear_desc_t d = {};
+    d.M = M; d.N = N; d.K = K;
+    d.dtype = FORGE_F32_TF32X3; d.act = FORGE_ACT_IDENTITY; d.red = FORGE_RED_NONE;
+    d.scale = 1.0f; d.ln_eps = 0.f; d.has_bias = 0; d.device = device;
+    float *dx = nullptr;
+    forge_fused_linear_t probe = nullptr;
+    forge_status_t st = cudaMalloc(&dx, sizeof(float) * (M * K + N * K + M * N)) == cudaSuccess ? FORGE_OK : FORGE_ERR_ALLOC;
+    if (st == FORGE_OK) st = forge_fused_linear_create(&d, &probe);
+    if (st == FORGE_OK && cudaMemcpy(dx, hx, sizeof(float) * (M * K + N * K), cudaMemcpyHostToDevice) != cudaSuccess) st = FORGE_ERR_CUDA;
+    if (st == FORGE_OK) st = forge_fused_linear_run(probe, dx, dx + M * K, nullptr, nullptr, nullptr, dx + M * K + N * K, nullptr);
+    if (st == FORGE_OK) st = forge_fused_linear_last_status(probe);
+    if (st == FORGE_OK && cudaMemcpy(hy, dx + M * K + N * K, sizeof(float) * M * N, cudaMemcpyDeviceToHost) != cudaSuccess) st = FORGE_ERR_CUDA;
+    if (st == FORGE_OK) {
+        bool holds = true;
+        for (int m = 0; m < M && holds; ++m)
+            for (int k = 0; k < K; ++k) {
+                const float x = hx[m * K + k], y = hy[m * N + k];
+                if (!(std::fabs(y - x) <= std::fabs(x) * (1.0f / 262144.0f))) { holds = false; break; }      // 2^-18
+            }
+        *mode = holds ? 1 : 2;
+    }
+    if (probe) forge_fused_linear_destroy(probe);
+    if (dx) cudaFree(dx); else cudaGetLastError();
+    delete[] hx;
+    return st;
+}
+
 forge_status_t k5_setup(Handle &h)
 {
+    if (h.d.device >= 64) return FORGE_ERR_UNSUPPORTED;
+    {
+        std::unique_lock<std::mutex> lock(k5_heads_mutex);
+        if (K5_WRITE_HI) k5_heads_mode[h.d.device] = 2;
+        if (k5_heads_mode[h.d.device] == 0) {
+            k5_heads_mode[h.d.device] = 3;
+            lock.unlock();                       // the probe creates a handle of its own, which comes through here
+            int mode = 0;
+            const forge_status_t st = k5_probe_heads(h.d.device, &mode);
+            lock.lock();
+            k5_heads_mode[h.d.device] = st == FORGE_OK ? mode : 0;
+            if (st != FORGE_OK) return st;
+        }
+    }
     // setmaxnreg.inc waits until the registers it asks for are free: the shares must fit into what
     // a CTA is launched with, or the kernel is never launched
     cudaFuncAttributes fa;
@@ -779,6 +851,7 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
     p.gen = h.ws.counters + L.gen_idx;
     p.ws_floats = h.ws.partial_floats;
     p.ws_counters = h.ws.counter_words;
+    p.write_hi = k5_heads_mode[d.device] == 2;
     p.cooperative = k5_ctas_wait(h);
     p.rowg = h.ws.partial + L.rowg_off;
     p.strips_done = h.ws.counters + L.strips_done_idx;
