@@ -719,6 +719,11 @@ def main():
         st, tf, mhz = B.forge_selftest_ffma_rate(local, 200)
         if st == B.FORGE_OK:
             alu_peak = tf
+        time.sleep(0.5)
+        st, rs_b2b, rs_single = B.forge_selftest_read_stream(local)
+        read_stream = {"back_to_back_gbs": round(rs_b2b, 1), "single_launch_gbs": round(rs_single, 1),
+                       "how": "forge_selftest_read_stream: load-only kernel (four 32-KiB bulk copies in flight per SM) over three "
+                              "rotating 256-MiB buffers, CUDA events"} if st == B.FORGE_OK else None
     line = {"metric": f"fused-op {unit} ({wl.name})", "value": round(value, 2), "unit": unit, "n_gpus": n_gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_max, 5), "higher_is_better": True,
             "scaling": args.scaling, "vs_baseline": None, "dtype": "bf16" if wl.dtype == wk.BF16 else "f32",
@@ -731,6 +736,8 @@ def main():
             "roofline": roofline_of(wl, ms * wl.M / rows, peaks, op.plan.kernel, clocks.get("sm_max_mhz"), props.multi_processor_count, alu_peak),
             "nominal_frac": round((value / world) / (NOMINAL["hbm_gbs"] if wl.hbm_bound else NOMINAL["bf16_tflops"]), 4)
             if wl.dtype == wk.BF16 else None}
+    if rank == 0 and world == 1 and read_stream:
+        line["hbm_read_measured"] = read_stream          # what a kernel that only reads gets: the ceiling of the HBM-bound workloads
     if alu_peak:
         line["alu_peak_measured"] = {"value": round(alu_peak, 2), "unit": "TFLOP/s", "effective_sm_mhz": round(mhz, 1),
                                      "how": "forge_selftest_ffma_rate: 200 ms of independent register-to-register fma.rn.f32x2 on every SM, CUDA events"}

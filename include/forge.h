@@ -233,6 +233,18 @@ const char *forge_fused_linear_kernel_name(forge_fused_linear_t h);
 forge_status_t forge_selftest_ffma_rate(int device, int milliseconds, double *tflops, double *sm_mhz_effective);
 
 /*
+ * Measure what the memory system of this device delivers to a kernel that only reads: one thread per
+ * SM keeps four 32-KiB bulk copies (global -> shared memory) in flight over a contiguous share of a
+ * 256-MiB buffer, nothing is computed.  Three such buffers (768 MiB, allocated and freed here) are read in
+ * turn, so nothing is served from L2.  Writes GB/s (1e9 bytes) of 30 launches issued back to back to
+ * *gbs_back_to_back and, if the pointer is not NULL, of the median of 11 launches with a synchronise
+ * after each to *gbs_single (host pointers).  This is the measured ceiling the HBM-bound skinny-M
+ * kernel is compared with -- the paper's Judge reads `dram__throughput` for the same question
+ * (Appendix C).  Synchronous.
+ */
+forge_status_t forge_selftest_read_stream(int device, double *gbs_back_to_back, double *gbs_single);
+
+/*
  * Row sum / row max of the fp32 fused linear without a handle and without any allocation.
  * (The paper has no counterpart to this entry point: it exists for the benefit of callers,
  * not of the method.)

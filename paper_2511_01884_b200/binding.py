@@ -26,7 +26,7 @@ EXPORTS = [
     "forge_fused_linear_run_host", "forge_fused_linear_last_status", "forge_fused_linear_get_plan",
     "forge_fused_linear_launches_per_run", "forge_fused_linear_destroy", "forge_fused_linear_last_wait_detail",
     "forge_fused_linear_f32_reduce_static", "forge_selftest_bounded_wait", "forge_selftest_ffma_rate",
-    "forge_status_string", "forge_kernel_name", "forge_fused_linear_kernel_name",
+    "forge_selftest_read_stream", "forge_status_string", "forge_kernel_name", "forge_fused_linear_kernel_name",
 ]
 
 
@@ -84,7 +84,8 @@ def lib() -> ctypes.CDLL:
         L.forge_selftest_ffma_rate.argtypes = [i, i, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
         L.forge_fused_linear_kernel_name.argtypes = [vp]
         L.forge_fused_linear_kernel_name.restype = ctypes.c_char_p
-        for n in EXPORTS[:12]:
+        L.forge_selftest_read_stream.argtypes = [i, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+        for n in EXPORTS[:13]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -161,6 +162,13 @@ def forge_selftest_ffma_rate(device: int = 0, milliseconds: int = 200):
     t, f = ctypes.c_double(0.0), ctypes.c_double(0.0)
     st = lib().forge_selftest_ffma_rate(int(device), int(milliseconds), ctypes.byref(t), ctypes.byref(f))
     return st, t.value, f.value
+
+
+def forge_selftest_read_stream(device: int = 0):
+    """(status, GB/s back to back, GB/s of a single launch) of the load-only stream: the measured HBM read ceiling."""
+    a, b = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    st = lib().forge_selftest_read_stream(int(device), ctypes.byref(a), ctypes.byref(b))
+    return st, a.value, b.value
 
 
 def forge_fused_linear_kernel_name(h) -> str:

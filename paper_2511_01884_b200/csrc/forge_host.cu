@@ -199,7 +199,100 @@ __global__ void __launch_bounds__(512, 2) forge_ffma_rate_kernel(float *sink, fl
     if (x == 0x7ff0dead7ff0beefull) sink[0] = 1.f;      // keeps the chains alive; practically never true
 }
 
+// Load-only stream: one thread per CTA keeps `stages` contiguous bulk copies of `piece` bytes in flight into a ring
+// of shared memory (global -> shared, completion counted in bytes on an mbarrier per slot); nothing is computed.
+// What it sustains is what the memory system delivers to a kernel that only reads.
+__global__ void __launch_bounds__(32, 1) forge_read_stream_kernel(const uint8_t *src, size_t bytes, uint32_t piece, int stages, int *status)
+{
+    extern __shared__ uint8_t stream_raw[];
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(stream_raw) + 127) & ~uintptr_t(127));
+    __shared__ uint64_t full[8];
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < stages; ++i) ptx::mbar_init(&full[i], 1);
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    const size_t pieces = bytes / piece;
+    const size_t lo = pieces * blockIdx.x / gridDim.x, hi = pieces * (blockIdx.x + 1) / gridDim.x;
+    long long issued = 0;
+    bool ok = true;
+    for (size_t i = lo; i < hi && ok; ++i, ++issued) {
+        const int slot = (int)(issued % stages);
+        // the slot's previous copy must have landed before it is overwritten
+        if (issued >= stages && !ptx::mbar_wait(&full[slot], (uint32_t)((issued / stages - 1) & 1), status, SITE_TMA_FULL, slot)) { ok = false; break; }
+        ptx::mbar_expect_tx(&full[slot], piece);
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(ptx::smem_u32(ring + (size_t)slot * piece)), "l"(src + i * piece), "r"(piece), "r"(ptx::smem_u32(&full[slot])) : "memory");
+    }
+    // every copy still in flight lands before the CTA leaves
+    for (long long j = issued > stages ? issued - stages : 0; j < issued && ok; ++j)
+        ok = ptx::mbar_wait(&full[(int)(j % stages)], (uint32_t)((j / stages) & 1), status, SITE_TMA_FULL, (int)(j % stages));
+    if (!ok) __nanosleep(500000);
+}
+
 extern "C" {
+
+forge_status_t forge_selftest_read_stream(int device, double *gbs_back_to_back, double *gbs_single)
+{
+    if (!gbs_back_to_back || device < 0) return FORGE_ERR_INVALID_ARG;
+    DeviceGuard g(device);
+    if (!g.ok) return FORGE_ERR_CUDA;
+    int sms = 0, major = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms <= 0 ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess || major != 10)
+        return FORGE_ERR_CUDA;
+    constexpr size_t kPart = (size_t)256 << 20;          // one "weight": twice the L2
+    constexpr int kParts = 3, kStages = 4;
+    constexpr uint32_t kPiece = 32768;
+    constexpr size_t kSmem = (size_t)kStages * kPiece + 128;
+    uint8_t *buf = nullptr;
+    int *status = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaMalloc(&buf, kParts * kPart) != cudaSuccess || cudaMalloc(&status, 256) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(buf);
+        return FORGE_ERR_ALLOC;
+    }
+    forge_status_t st = FORGE_ERR_CUDA;
+    bool ok = cudaMemset(buf, 1, kParts * kPart) == cudaSuccess && cudaMemset(status, 0, 256) == cudaSuccess &&
+              cudaFuncSetAttribute(forge_read_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem) == cudaSuccess &&
+              cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess;
+    auto launch = [&](int i) { forge_read_stream_kernel<<<sms, 32, kSmem>>>(buf + (size_t)(i % kParts) * kPart, kPart, kPiece, kStages, status); };
+    float ms = 0.f;
+    if (ok) {
+        constexpr int kRuns = 30;
+        for (int i = 0; i < kParts; ++i) launch(i);
+        ok = cudaDeviceSynchronize() == cudaSuccess && cudaEventRecord(e0) == cudaSuccess;
+        for (int i = 0; i < kRuns; ++i) launch(i);
+        ok = ok && cudaEventRecord(e1) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess &&
+             cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess && ms > 0.f;
+        if (ok) *gbs_back_to_back = (double)kPart * kRuns / (ms * 1e-3) / 1e9;
+    }
+    if (ok && gbs_single) {
+        float best[11];
+        for (int i = 0; i < 11 && ok; ++i) {
+            ok = cudaEventRecord(e0) == cudaSuccess;
+            launch(i);
+            ok = ok && cudaEventRecord(e1) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess &&
+                 cudaEventElapsedTime(&best[i], e0, e1) == cudaSuccess;
+        }
+        if (ok) {
+            for (int i = 0; i < 11; ++i)
+                for (int j = i + 1; j < 11; ++j)
+                    if (best[j] < best[i]) { const float t = best[i]; best[i] = best[j]; best[j] = t; }
+            *gbs_single = (double)kPart / (best[5] * 1e-3) / 1e9;          // the median launch
+        }
+    }
+    int word = 0;
+    if (ok && cudaMemcpy(&word, status, sizeof(word), cudaMemcpyDeviceToHost) == cudaSuccess) st = word == 0 ? FORGE_OK : (forge_status_t)(word >> 16);
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(buf);
+    cudaFree(status);
+    if (!ok) cudaGetLastError();
+    return st;
+}
 
 forge_status_t forge_selftest_ffma_rate(int device, int milliseconds, double *tflops, double *sm_mhz_effective)
 {

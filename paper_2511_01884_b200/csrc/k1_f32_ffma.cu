@@ -35,8 +35,21 @@ struct K1Params {
     // area follow from the fields above -- see k1_slice_len().)
     int *status;           // LayerNorm: status word of the bounded strip wait
     unsigned *gen;         // LayerNorm: run index of the strip counters (see run_index_begin)
-    long long ws_floats, ws_counters;      // extents of `partial` and `counters` (bounds-checked build)
+#ifdef FORGE_DEBUG_BOUNDS
+    // extents of `partial` and `counters`.  Only in the bounds-checked build: the code generated for the large tile
+    // is sensitive to the size of this structure (two more words cost 5 % on a 4096^3 problem).
+    long long ws_floats, ws_counters;
+#endif
 };
+#ifdef FORGE_DEBUG_BOUNDS
+#define K1_WS_FLOATS(p) ((p).ws_floats)
+#define K1_WS_COUNTERS(p) ((p).ws_counters)
+#define K1_SET_EXTENTS(p, f, c) ((p).ws_floats = (f), (p).ws_counters = (c))
+#else
+#define K1_WS_FLOATS(p) 0ll
+#define K1_WS_COUNTERS(p) 0ll
+#define K1_SET_EXTENTS(p, f, c) ((void)0)
+#endif
 
 // Length of a K slice when K is cut into `slices`: a multiple of the small tile's 32-wide k-tile.
 __host__ __device__ inline int k1_slice_len(int K, int slices) { return ((K + slices - 1) / slices + 31) / 32 * 32; }
@@ -209,8 +222,8 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
         float4 *mine = slice_partial + (((size_t)tile * k_slices + blockIdx.z) * K1_THREADS + tid) * (R * R / 4);
         // (the same verdict in every thread: the check is on the tile's whole hand-over area and its counter)
         if (!in_bounds(p.status, BOUNDS_PARTIAL, (long long)(reinterpret_cast<float *>(slice_partial) - p.partial) + (long long)tile * k_slices * K1_THREADS * (R * R),
-                       (long long)k_slices * K1_THREADS * (R * R), p.ws_floats) ||
-            !in_bounds(p.status, BOUNDS_COUNTER, (long long)(slice_counters - p.counters) + tile, 1, p.ws_counters))
+                       (long long)k_slices * K1_THREADS * (R * R), K1_WS_FLOATS(p)) ||
+            !in_bounds(p.status, BOUNDS_COUNTER, (long long)(slice_counters - p.counters) + tile, 1, K1_WS_COUNTERS(p)))
             return true;
 #pragma unroll
         for (int i = 0; i < R; ++i)
@@ -246,8 +259,8 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
         // counter, checked before either is touched (the same verdict in every thread)
         constexpr bool WIDE = RED == FORGE_RED_LAYERNORM || RED == FORGE_RED_LOGSUMEXP || RED == FORGE_RED_CROSS_ENTROPY;
         const long long first = (long long)tile_n * M + m0, rows = min(BM, M - m0);
-        if (!in_bounds(p.status, BOUNDS_PARTIAL, WIDE ? 4 * first : first, WIDE ? 4 * rows : rows, p.ws_floats) ||
-            !in_bounds(p.status, BOUNDS_COUNTER, tile_m, 1, p.ws_counters))
+        if (!in_bounds(p.status, BOUNDS_PARTIAL, WIDE ? 4 * first : first, WIDE ? 4 * rows : rows, K1_WS_FLOATS(p)) ||
+            !in_bounds(p.status, BOUNDS_COUNTER, tile_m, 1, K1_WS_COUNTERS(p)))
             return true;
     }
     int col[R];
@@ -581,8 +594,7 @@ forge_status_t k1_launch(Handle &h, const RunArgs &a)
     p.partial = h.ws.partial;
     p.counters = h.ws.counters;
     p.status = h.ws.status;
-    p.ws_floats = h.ws.partial_floats;
-    p.ws_counters = h.ws.counter_words;
+    K1_SET_EXTENTS(p, h.ws.partial_floats, h.ws.counter_words);
     const int bm = h.info.tile_m, bn = h.info.tile_n;          // 128 or 64
     p.warm_l2 = (h.info.grid < h.sm_count) && (d.K <= 4096);   // latency-bound grids with modest panels
     p.tiles_n = (int)((d.N + bn - 1) / bn);
@@ -690,8 +702,7 @@ extern "C" forge_status_t forge_fused_linear_f32_reduce_static(int64_t M, int64_
     p.warm_l2 = 0;
     p.status = nullptr;
     p.gen = nullptr;
-    p.ws_floats = (long long)((K1_STATIC_SCRATCH_BYTES - counter_bytes) / sizeof(float));
-    p.ws_counters = (long long)(counter_bytes / sizeof(unsigned));
+    K1_SET_EXTENTS(p, (long long)((K1_STATIC_SCRATCH_BYTES - counter_bytes) / sizeof(float)), (long long)(counter_bytes / sizeof(unsigned)));
     const dim3 grid((unsigned)tiles_n, (unsigned)tiles_m);
     const bool vec = (K % 4 == 0) && ((uintptr_t)X % 16 == 0) && ((uintptr_t)W % 16 == 0);
     if (red == FORGE_RED_SUM)

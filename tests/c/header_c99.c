@@ -57,6 +57,7 @@ int main(void)
     CHECK(forge_selftest_bounded_wait(0, 0, detail) == FORGE_ERR_INVALID_ARG);
     CHECK(forge_selftest_ffma_rate(0, 0, &rate, NULL) == FORGE_ERR_INVALID_ARG);
     CHECK(forge_selftest_ffma_rate(0, 10, NULL, NULL) == FORGE_ERR_INVALID_ARG);
+    CHECK(forge_selftest_read_stream(0, NULL, NULL) == FORGE_ERR_INVALID_ARG);
     CHECK(forge_fused_linear_f32_reduce_static(0, 1, 1, FORGE_ACT_RELU, FORGE_RED_SUM, 1.0f, NULL, NULL, NULL, NULL,
                                                NULL) == FORGE_ERR_INVALID_ARG);
 

@@ -303,6 +303,12 @@ def test_kernel_name_of_a_handle():
     op.close()
 
 
+def test_measured_read_stream_is_plausible():
+    st, b2b, single = B.forge_selftest_read_stream(0)
+    assert st == B.FORGE_OK
+    assert 4000.0 < b2b < 8000.0 and 3500.0 < single <= 1.02 * b2b, (b2b, single)      # GB/s; nominal HBM3e: 8000
+
+
 def test_measured_ffma_rate_is_plausible():
     import torch
     st, tflops, mhz = B.forge_selftest_ffma_rate(0, 50)
