@@ -53,11 +53,14 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # from the ncu captures summarised under profiles/, keyed by workload, with the sha256 of the
 # kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
 NCU_TRAFFIC = {
-    "c2": {"bytes": 539106048, "sha": "83c493efb815777f"},
-    "c3": {"bytes": 1150823328, "sha": "b0fa426747d03e58"},
-    "c4": {"bytes": 273_142_272, "sha": "d1f4e9fb22aed839"},
-    "c5": {"bytes": 304678656, "sha": "b0fa426747d03e58"},
-    "c2t": {"bytes": 353031168, "sha": "cb0f91a3d90a1e4c"},
+    "c2": {"bytes": 550_270_976, "sha": "feb632b4df2f6da9"},
+    "c3": {"bytes": 1_163_608_832, "sha": "638fa5d97469a021"},
+    "c4": {"bytes": 272_563_200, "sha": "6a936c6f5c8bc382"},
+    "c5": {"bytes": 300_992_768, "sha": "638fa5d97469a021"},
+    "c2t": {"bytes": 350_918_656, "sha": "5ec8bbf3c13bfe6a"},
+    "n2": {"bytes": 1_134_139_944, "sha": "638fa5d97469a021"},
+    "m64": {"bytes": 542_402_816, "sha": "638fa5d97469a021"},
+    "n1b": {"bytes": 1_220_658_896, "sha": "638fa5d97469a021"},
 }
 
 
