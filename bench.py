@@ -56,7 +56,7 @@ NCU_TRAFFIC = {
     "c2": {"bytes": 550_270_976, "sha": "feb632b4df2f6da9"},
     "c3": {"bytes": 1_163_608_832, "sha": "638fa5d97469a021"},
     "c4": {"bytes": 272_563_200, "sha": "6a936c6f5c8bc382"},
-    "c5": {"bytes": 300_992_768, "sha": "638fa5d97469a021"},
+    "c5": {"bytes": 300_095_232, "sha": "638fa5d97469a021"},
     "c2t": {"bytes": 350_918_656, "sha": "5ec8bbf3c13bfe6a"},
     "n2": {"bytes": 1_134_139_944, "sha": "638fa5d97469a021"},
     "m64": {"bytes": 542_402_816, "sha": "638fa5d97469a021"},

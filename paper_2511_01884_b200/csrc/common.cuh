@@ -276,28 +276,42 @@ __device__ __forceinline__ float fold_row_lse(const float4 *part4, int parts, in
     return mx + (ACCURATE ? logf(se) : __logf(se)) - tl;
 }
 
-// LayerNorm: the strip's (n, mean, M2, -) triples combined all at once, with one division for the mean
-// and one for the variance (the pairwise merge costs a division per part):
-//     mean = sum n_i mean_i / sum n_i,   M2 = sum (M2_i + n_i (mean_i - mean)^2).
-// Returns the mean and writes 1 / sqrt(M2 / n + eps).
+// LayerNorm: the strip's (n, mean, M2, -) triples combined in one walk, with one division for the mean and
+// one for the variance (the pairwise merge costs a division per part).  With d_i = mean_i - mean_0:
+//     mean = mean_0 + sum n_i d_i / n,   M2 = sum M2_i + sum n_i d_i^2 - (sum n_i d_i)^2 / n,   n = sum n_i.
+// Shifting by the first part's mean keeps the subtraction in M2 harmless: what cancels is of the size of the
+// spread of the parts' means, not of the mean itself.  Returns the mean and writes 1 / sqrt(M2 / n + eps).
 template <bool ACCURATE>
 __device__ __forceinline__ float combine_row_moments(const float4 *stats, int parts, int M, int row, float eps, float &rstd)
 {
-    float cnt = 0.f, wsum = 0.f;
-    for (int i = 0; i < parts; ++i) {
+    const float4 first = __ldcg(&stats[row]);
+    float cnt = first.x, s1 = 0.f, s2 = 0.f, m2 = first.z;
+    int i = 1;
+    for (; i + 8 <= parts; i += 8) {
+        float4 o[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) o[u] = __ldcg(&stats[(size_t)(i + u) * M + row]);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float d = o[u].y - first.y, nd = o[u].x * d;
+            cnt += o[u].x;
+            s1 += nd;
+            s2 = fmaf(nd, d, s2);
+            m2 += o[u].z;
+        }
+    }
+    for (; i < parts; ++i) {
         const float4 o = __ldcg(&stats[(size_t)i * M + row]);
+        const float d = o.y - first.y, nd = o.x * d;
         cnt += o.x;
-        wsum = fmaf(o.x, o.y, wsum);
+        s1 += nd;
+        s2 = fmaf(nd, d, s2);
+        m2 += o.z;
     }
-    const float mean = wsum / cnt;
-    float m2 = 0.f;
-    for (int i = 0; i < parts; ++i) {
-        const float4 o = __ldcg(&stats[(size_t)i * M + row]);
-        const float dm = o.y - mean;
-        m2 += fmaf(o.x * dm, dm, o.z);
-    }
-    rstd = ACCURATE ? 1.0f / sqrtf(m2 / cnt + eps) : rsqrtf(m2 / cnt + eps);
-    return mean;
+    const float inv = 1.0f / cnt, shift = s1 * inv;
+    const float var = fmaxf((m2 + s2 - s1 * shift) * inv, 0.f);
+    rstd = ACCURATE ? 1.0f / sqrtf(var + eps) : rsqrtf(var + eps);
+    return first.y + shift;
 }
 
 // (n, mean, M2) of the first nv of 32 values held in registers: two sweeps, no division per element.
