@@ -59,8 +59,7 @@ typedef enum {
      * each operand is split into a TF32 head and a TF32 tail and X W^T is accumulated in fp32
      * from the three products head*head, head*tail, tail*head (relative error of a product
      * about 2^-21), so the result stays within the 1e-4 of Section 2.2 with two orders of
-     * magnitude to spare.  Needs K % 4 == 0, N % 4 == 0 and 16-byte aligned pointers; LayerNorm
-     * needs ceil(N / 256) to be at most the number of CTA pairs of the grid (74 on a B200).  */
+     * magnitude to spare.  Needs K % 4 == 0, N % 4 == 0 and 16-byte aligned pointers.          */
 } forge_dtype_t;
 
 typedef enum {
@@ -79,10 +78,10 @@ typedef enum {
     /* Population variance, eps inside the square root, gamma and beta applied after the
      * normalisation.  The N-tiles of a row strip exchange per-row (count, mean, M2) triples (the
      * "cross-tile aggregation" of Appendix B.1); the un-normalised values never leave the SM.
-     * Row width: 16-bit storage, any N (rows of more than 256 x [CTA pairs in the grid] columns --
-     * 18944 on a B200 -- are served by computing every tile twice, once for the statistics and
-     * once to normalise: twice the arithmetic); FORGE_F32, N up to 128 x [2 x SM count] (37888);
-     * FORGE_F32_TF32X3, N up to 256 x [SM count / 2] (18944).  Beyond: FORGE_ERR_UNSUPPORTED.     */
+     * Any N: the tiles of a strip wait for one another, so when a strip has more tiles than the
+     * grid has CTAs (pairs) -- N > 18944 on the tensor-core kernels, N > 37888 on the fp32 FFMA
+     * kernel, on a B200 -- every tile is computed twice, once for the statistics and once to
+     * normalise: twice the arithmetic, and still nothing un-normalised in global memory.         */
     FORGE_RED_MEAN_GELU_RESIDUAL = 4,
     /* The chain of the paper's Appendix B.1 case study (Linear, subtract, row mean, GELU,
      * residual add of the layer's input, all in one kernel):
@@ -141,8 +140,8 @@ typedef struct {
  * is compute- or memory-bound): fp32 -> F32_FFMA; fp32 with TF32x3 arithmetic -> F32_TF32X3; 16-bit with M <= 32 and neither LayerNorm nor
  * the mean-GELU-residual chain -> BF16_SKINNY; 16-bit LayerNorm -> BF16_TCGEN05_LN; other 16-bit
  * -> BF16_TCGEN05.
- * Unsupported: 16-bit storage with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); LayerNorm
- * rows wider than forge_red_t states for fp32 storage; TF32x3 with K % 4 != 0 or N % 4 != 0.
+ * Unsupported: 16-bit storage with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); TF32x3 with
+ * K % 4 != 0 or N % 4 != 0.
  */
 forge_status_t forge_fused_linear_query_plan(const forge_fused_linear_desc_t *desc, int sm_count,
                                              forge_plan_info_t *info);

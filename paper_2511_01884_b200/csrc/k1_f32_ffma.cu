@@ -122,9 +122,11 @@ __device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &
 // problems with too few 128x128 tiles to occupy the SMs (a grid of a handful of CTAs is bound by
 // the FMA rate of the few SMs it runs on, not by the GPU's).
 // One output tile (for small grids: one K slice of it).  `run` is the run index of the LayerNorm strip counters.
-// Returns false only when a bounded wait gave up.
+// LayerNorm of rows with more tiles than CTAs computes every tile twice: ln_pass 1 = statistics only (publish, never
+// wait), 2 = recompute, wait for the strip, normalise and store; 0 = both in one visit.  Returns false only when a
+// bounded wait gave up.
 template <bool VEC, int RED, int T>
-__device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, const int tile_n, const unsigned run)
+__device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, const int tile_n, const unsigned run, const int ln_pass = 0)
 {
     constexpr int BM = 64 * T, BN = 64 * T, R = 4 * T;       // tile and per-thread extent
     constexpr int BK = T == 1 ? 32 : K1_BK;                  // the small tile takes longer k steps (fewer round trips)
@@ -424,18 +426,19 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
 #pragma unroll
             for (int sft = 1; sft <= 8; sft <<= 1) st = merge_stat(st, shfl_xor_stat(st, sft));
             const int row = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
-            if (tx == 0 && row < M) stats[(size_t)tile_n * M + row] = make_float4(st.n, st.mean, st.m2, 0.f);
+            if (ln_pass != 2 && tx == 0 && row < M) stats[(size_t)tile_n * M + row] = make_float4(st.n, st.mean, st.m2, 0.f);
         }
         // publish, then wait (bounded) for the strip's other tiles: one arrival per CTA by one thread (release: the
         // CTA's triples, ordered before it by the barrier; the acquiring polls and the next barrier make the other
         // tiles' triples readable past L1)
         __syncthreads();
         if (tid == 0) {
-            arrive_acq_rel(&p.counters[tile_m]);
-            s_last = wait_counter<0>(&p.counters[tile_m], run * (unsigned)p.tiles_n, p.status, SITE_ARRIVAL, tile_m) ? 1 : 0;
+            if (ln_pass != 2) arrive_acq_rel(&p.counters[tile_m]);
+            s_last = (ln_pass == 1 || wait_counter<0>(&p.counters[tile_m], run * (unsigned)p.tiles_n, p.status, SITE_ARRIVAL, tile_m)) ? 1 : 0;
         }
         __syncthreads();
         if (!s_last) return false;
+        if (ln_pass == 1) return true;
         // the strip's tiles combined in tile order, all at once (same result in every CTA):
         // mean = sum n_i mean_i / sum n_i,  M2 = sum (M2_i + n_i (mean_i - mean)^2)
         if (tid < BM && m0 + tid < M) {
@@ -480,10 +483,15 @@ __global__ void __launch_bounds__(K1_THREADS, K1_CTAS_PER_SM) k1_f32_ffma_kernel
     if (RED == FORGE_RED_LAYERNORM) {
         const unsigned run = run_index_begin(p.gen);
         const int tiles = (int)((p.M + 64 * T - 1) / (64 * T)) * p.tiles_n;
-        for (int t = (int)blockIdx.x; t < tiles; t += (int)gridDim.x) {
-            if (!k1_tile<VEC, RED, T>(p, t / p.tiles_n, t % p.tiles_n, run)) break;
-            __syncthreads();          // the tile's shared memory is free for the next one
-        }
+        // a strip with more tiles than the grid has CTAs cannot wait for itself: statistics first (no CTA waits in that
+        // pass, so the grid always gets through it), then every tile once more
+        const bool two_pass = p.tiles_n > (int)gridDim.x;
+        bool fine = true;
+        for (int pass = two_pass ? 1 : 0; fine && pass <= (two_pass ? 2 : 0); ++pass)
+            for (int t = (int)blockIdx.x; t < tiles; t += (int)gridDim.x) {
+                if (!k1_tile<VEC, RED, T>(p, t / p.tiles_n, t % p.tiles_n, run, pass)) { fine = false; break; }
+                __syncthreads();          // the tile's shared memory is free for the next one
+            }
         if (threadIdx.x == 0) run_index_end(p.gen, run);
     } else {
         k1_tile<VEC, RED, T>(p, (int)blockIdx.y, (int)blockIdx.x, 0u);
@@ -519,9 +527,9 @@ forge_status_t k1_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     const int64_t tiles_m = (d.M + bm - 1) / bm, tiles_n = (d.N + bn - 1) / bn;
     if (tiles_m > 65535 || tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
     if (d.M > 0x7fffffff || d.N > 0x7fffffff || d.K > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
-    // LayerNorm: persistent CTAs, and the tiles of a strip wait for one another, so all of them must be resident
+    // LayerNorm: persistent CTAs; the tiles of a strip wait for one another (a strip with more tiles than CTAs is
+    // served by computing every tile twice)
     const int64_t ln_grid = tiles_m * tiles_n < (int64_t)K1_CTAS_PER_SM * sm_count ? tiles_m * tiles_n : (int64_t)K1_CTAS_PER_SM * sm_count;
-    if (d.red == FORGE_RED_LAYERNORM && tiles_n > ln_grid) return FORGE_ERR_UNSUPPORTED;
     info->kernel = FORGE_KERNEL_F32_FFMA;
     info->tile_m = bm;
     info->tile_n = bn;

@@ -140,6 +140,7 @@ struct K5Params {
     int group_m;
     long long ws_floats, ws_counters;   // extents of `partial` and `counters` (bounds-checked build)
     int write_hi;               // the splitters also store the TF32 heads (the raw words do not serve as such here)
+    int two_pass;               // LayerNorm of rows with more tiles than CTA pairs: see K5Item::pass
     int chunk_kb;               // stages per TMEM accumulation chunk
     // K split of the last wave's tiles (tail_parts = 1: none)
     int tail_parts;             // S
@@ -154,6 +155,7 @@ struct K5Item {
     int um, tn;                 // 256-row unit, 256-column tile
     int kb_lo, kb_hi;           // k-blocks [kb_lo, kb_hi)
     int part, tail;             // part of the K split (0 leads), index of the tile among the split ones (-1: whole tile)
+    int pass;                   // LayerNorm of rows wider than the grid: 0 = statistics only, 1 = normalise and store
 };
 
 __device__ __forceinline__ void k5_tile_coords(int t, int units_m, int tiles_n, int group_m, int &um, int &tn);
@@ -166,6 +168,12 @@ __device__ __forceinline__ bool k5_item(const K5Params &p, int j, int cluster, i
     w.kb_hi = p.num_kb;
     w.part = 0;
     w.tail = -1;
+    w.pass = 0;
+    if (p.two_pass) {
+        // every tile twice: this cluster's whole list once for the statistics, then once more to normalise
+        const int mine = full + (cluster < rest ? 1 : 0);
+        if (j >= mine) { j -= mine; w.pass = 1; }
+    }
     if (j < full) {
         t = j * clusters + cluster;
     } else if (j == full && p.tail_parts <= 1) {
@@ -494,17 +502,30 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 }
                 ptx::tmem_st_wait();
                 float4 *stats = reinterpret_cast<float4 *>(p.partial);
-                if (row < p.M) stats[(size_t)part * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
+                // Rows with more tiles than the grid has CTA pairs cannot all be held on chip at once: every tile is then
+                // computed twice.  Pass 0 publishes its triples and moves on (it never waits, so the grid always gets
+                // through it); pass 1, which a cluster starts only when it has finished pass 0, recomputes the tile, waits
+                // for the strip's triples and normalises.  Twice the arithmetic; the un-normalised tile still never
+                // leaves the SM.
+                const bool publish = !p.two_pass || w.pass == 0, finish = !p.two_pass || w.pass == 1;
+                if (publish && row < p.M) stats[(size_t)part * p.M + row] = make_float4(rs.n, rs.mean, rs.m2, 0.f);
                 // publish, then wait (bounded) for the other half tiles of the strip: one arrival per group by one thread
                 // (release: the group's triples, ordered before it by the barrier; the acquiring polls and the next
                 // barrier make the other groups' triples readable past L1)
                 k5_epi_bar_sync(h);
                 if (et == 0) {
-                    arrive_acq_rel(&p.counters[tm]);
-                    if (!wait_counter<0>(&p.counters[tm], run * 2u * (unsigned)p.tiles_n, p.status, SITE_ARRIVAL, tm)) s.abort_flag = 1;
+                    if (publish) arrive_acq_rel(&p.counters[tm]);
+                    if (finish && !wait_counter<0>(&p.counters[tm], run * 2u * (unsigned)p.tiles_n, p.status, SITE_ARRIVAL, tm)) s.abort_flag = 1;
                 }
                 k5_epi_bar_sync(h);
                 if (*(volatile int *)&s.abort_flag) { ok = false; break; }
+                if (!finish) {
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
+                    if ((acc ^= 1) == 0) acc_phase ^= 1;
+                    continue;
+                }
                 // the strip's parts combined in part order: mean = sum n_i mean_i / sum n_i, M2 = sum (M2_i + n_i (mean_i - mean)^2)
                 float rstd = 0.f, shift = 0.f;
                 if (row < p.M) shift = -combine_row_moments<true>(stats, parts, p.M, row, p.e.eps, rstd) * rstd;
@@ -717,8 +738,8 @@ forge_status_t k5_plan(const forge_fused_linear_desc_t &d, int sm_count, forge_p
     if (d.K % 4 != 0 || d.N % 4 != 0 || sm_count < 2) return FORGE_ERR_UNSUPPORTED;
     const K5Layout L = k5_layout(d, sm_count);
     if (L.tiles_m * L.tiles_n > 0x7fffffff) return FORGE_ERR_UNSUPPORTED;
-    // LayerNorm: the tiles of a strip wait for one another, so they must all be resident at once
-    if (d.red == FORGE_RED_LAYERNORM && L.tiles_n > L.clusters) return FORGE_ERR_UNSUPPORTED;
+    // (LayerNorm: the tiles of a strip wait for one another; with more of them than CTA pairs every tile is
+    // computed twice, see K5Item::pass)
     info->kernel = FORGE_KERNEL_F32_TF32X3;
     info->tile_m = 2 * K5_BM;
     info->tile_n = K5_BN;
@@ -852,6 +873,7 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
     p.ws_floats = h.ws.partial_floats;
     p.ws_counters = h.ws.counter_words;
     p.write_hi = k5_heads_mode[d.device] == 2;
+    p.two_pass = d.red == FORGE_RED_LAYERNORM && L.tiles_n > L.grid / 2;
     p.cooperative = k5_ctas_wait(h);
     p.rowg = h.ws.partial + L.rowg_off;
     p.strips_done = h.ws.counters + L.strips_done_idx;

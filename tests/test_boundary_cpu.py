@@ -87,12 +87,14 @@ def test_unsupported_is_reported_not_rerouted():
     # LayerNorm: the tiles of a row strip wait for one another, so a row may not have more tiles than resident CTAs
     st, p = B.forge_fused_linear_query_plan(B.make_desc(64, 4096, 8, wk.F32, 0, wk.RED_LAYERNORM))
     assert st == B.FORGE_OK and p.kernel == B.FORGE_KERNEL_F32_FFMA and p.cluster == 1 and p.grid == 32
-    st, _ = B.forge_fused_linear_query_plan(B.make_desc(64, 128 * 296 + 1, 8, wk.F32, 0, wk.RED_LAYERNORM))
-    assert st == B.FORGE_ERR_UNSUPPORTED
+    st, p = B.forge_fused_linear_query_plan(B.make_desc(64, 128 * 296 + 1, 8, wk.F32, 0, wk.RED_LAYERNORM))
+    assert st == B.FORGE_OK and p.grid == 296          # more tiles per strip than CTAs: every tile is computed twice
     # fp32 on the tensor cores: 16-byte pitch of X, W and Y rows; LayerNorm rows of at most 74 tiles
-    for M, N, K, red in ((64, 64, 66, wk.RED_NONE), (64, 66, 64, wk.RED_NONE), (64, 256 * 74 + 4, 64, wk.RED_LAYERNORM)):
+    for M, N, K, red in ((64, 64, 66, wk.RED_NONE), (64, 66, 64, wk.RED_NONE)):
         st, _ = B.forge_fused_linear_query_plan(B.make_desc(M, N, K, wk.F32_TF32X3, 0, red))
         assert st == B.FORGE_ERR_UNSUPPORTED
+    st, _ = B.forge_fused_linear_query_plan(B.make_desc(64, 256 * 74 + 4, 64, wk.F32_TF32X3, 0, wk.RED_LAYERNORM))
+    assert st == B.FORGE_OK
 
 
 def test_tf32x3_plan():

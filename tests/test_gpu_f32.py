@@ -57,7 +57,8 @@ def test_every_activation(act):
 # one tile per strip, 8 and 9 tiles (past the width a thread-block cluster would span), 32 tiles with many strips
 # per CTA (several waves of persistent CTAs), a row as wide as a language-model head with few rows
 @pytest.mark.parametrize("M,N,K,bias", [(130, 1024, 40, False), (70, 1032, 36, True), (1500, 4096, 64, True),
-                                        (40, 32768, 24, True), (128 * 5 + 3, 128 * 59 + 8, 20, True)])
+                                        (40, 32768, 24, True), (128 * 5 + 3, 128 * 59 + 8, 20, True),
+                                        (130, 128 * 300 + 5, 12, True)])      # more tiles per strip than CTAs: two passes
 def test_layernorm_of_wide_rows(M, N, K, bias):
     wl = wk.custom_workload(f"f32_ln_{N}", wk.F32, M, N, K, wk.ACT_GELU_ERF, wk.RED_LAYERNORM, has_bias=bias, seed=4)
     inp = wk.make_inputs(wl)
@@ -68,12 +69,11 @@ def test_layernorm_of_wide_rows(M, N, K, bias):
     pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
 
 
-def test_layernorm_rows_wider_than_the_grid_are_refused():
-    # the tiles of a strip wait for one another: more 128-column tiles than resident CTAs cannot be served
-    st, _ = B.forge_fused_linear_query_plan(B.make_desc(8, 128 * 296, 8, wk.F32, 0, wk.RED_LAYERNORM))
-    assert st == B.FORGE_OK
-    st, _ = B.forge_fused_linear_query_plan(B.make_desc(8, 128 * 296 + 1, 8, wk.F32, 0, wk.RED_LAYERNORM))
-    assert st == B.FORGE_ERR_UNSUPPORTED
+def test_layernorm_rows_wider_than_the_grid_are_planned():
+    # the tiles of a strip wait for one another; with more 128-column tiles than resident CTAs every tile is computed twice
+    for N in (128 * 296, 128 * 296 + 1, 1 << 20):
+        st, p = B.forge_fused_linear_query_plan(B.make_desc(8, N, 8, wk.F32, 0, wk.RED_LAYERNORM))
+        assert st == B.FORGE_OK and p.grid <= 296
 
 
 def test_layernorm_constant_rows_give_beta():

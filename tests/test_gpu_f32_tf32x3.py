@@ -155,6 +155,19 @@ def test_layernorm_constant_rows_give_beta():
 
 
 def test_what_the_kernel_does_not_serve_is_refused():
-    for M, N, K, red in [(64, 64, 66, wk.RED_NONE), (64, 66, 64, wk.RED_NONE), (64, 256 * 74 + 4, 64, wk.RED_LAYERNORM)]:
+    for M, N, K, red in [(64, 64, 66, wk.RED_NONE), (64, 66, 64, wk.RED_NONE)]:
         st, _ = B.forge_fused_linear_query_plan(B.make_desc(M, N, K, T, 0, red))
         assert st == B.FORGE_ERR_UNSUPPORTED
+
+
+def test_layernorm_rows_with_more_tiles_than_cta_pairs():
+    """More 256-column tiles per row strip than the grid has CTA pairs: every tile is computed twice (statistics,
+    then normalisation); the strip counters carry over from run to run."""
+    wl = wk.custom_workload("t_ln_2pass", T, 140, 256 * 80 + 8, 64, wk.ACT_GELU_TANH, wk.RED_LAYERNORM, seed=9)
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    g, plan = pu.run_gpu(wl, inp, op=op, repeats=3)
+    op.close()
+    assert plan["kernel"] == B.FORGE_KERNEL_F32_TF32X3
+    e = pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
+    assert e <= 2e-5, e
