@@ -25,6 +25,7 @@
 // two tiles have both TMEM buffers to go to.  CTAs wait on one another, so the launch is
 // cooperative and a strip may not have more tiles than there are CTAs.
 #include "common.cuh"
+#include "epilogue_tmem.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
 
@@ -317,7 +318,6 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
         uint32_t acc_phase = 0;
         const bool chain = p.e.red == FORGE_RED_MEAN_GELU_RESIDUAL;       // subtract, row mean, GELU, residual add
         const bool reduce = p.e.red == FORGE_RED_SUM || p.e.red == FORGE_RED_MAX || chain;
-        const bool add = p.e.red != FORGE_RED_MAX;
         const uint32_t acc_empty_addr[2] = {ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[0]), 0),
                                             ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[1]), 0)};   // the leader's (PAIR)
         K2Item w;
@@ -491,117 +491,32 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 continue;
             }
 
-            if (p.e.red == FORGE_RED_LOGSUMEXP || p.e.red == FORGE_RED_CROSS_ENTROPY) {
-                // online (max, sum exp) over this thread's row of the half tile; the target's logit
-                // is picked up on the way (cross-entropy); Y is never written
-                const int tgt = (p.e.red == FORGE_RED_CROSS_ENTROPY && row < p.M)
-                                    ? __ldg(reinterpret_cast<const int *>(p.gamma) + row) : -1;
-                float mx = -INFINITY, se = 0.f, tl = 0.f;
-#pragma unroll 1
-                for (int c = 0; c < CHUNKS; ++c) {
-                    const int col0 = n0 + c * 32;
-                    if (col0 >= p.N) break;
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(taddr + c * 32, r);
-                    ptx::tmem_ld_wait();
-                    float v[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
-                    apply_act_array<false>(p.e.act, v, p.e.scale);
-                    const int nv = min(32, p.N - col0);
-                    float cm = -INFINITY;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) cm = j < nv ? fmaxf(cm, v[j]) : cm;
-                    const float nm = fmaxf(mx, cm);
-                    float cs = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) cs += j < nv ? __expf(v[j] - nm) : 0.f;
-                    se = (mx == -INFINITY ? 0.f : se * __expf(mx - nm)) + cs;
-                    mx = nm;
-                    if (tgt >= col0 && tgt < col0 + 32) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) tl = (col0 + j == tgt) ? v[j] : tl;
-                    }
-                }
-                ptx::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
-
-                float4 *part4 = reinterpret_cast<float4 *>(p.partial);
-                if (row < p.M) part4[(size_t)part * p.M + row] = make_float4(mx, se, tl, 0.f);
-                epi_bar_sync(h);
-                if (et == 0) s.last_flag[h] = (arrive_acq_rel(&p.counters[tm]) == (unsigned)(parts - 1));
-                epi_bar_sync(h);
-                if (s.last_flag[h]) {
-                    // the group that arrives last at the strip merges the parts in order
-                    if (row < p.M) reinterpret_cast<float *>(p.out)[row] = fold_row_lse<false>(part4, parts, p.M, row);
-                    if (et == 0) p.counters[tm] = 0u;
-                }
-                if ((acc ^= 1) == 0) acc_phase ^= 1;
-                continue;
-            }
-
-            float red = add ? 0.f : -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < CHUNKS; ++c) {
-                const int col0 = n0 + c * 32;
-                if (col0 >= p.N) break;
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(taddr + c * 32, r);
-                ptx::tmem_ld_wait();
-                float v[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
-                apply_act_array<false>(p.e.act, v, p.e.scale);
-                if (reduce) {
-                    if (chain) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] -= sg[c * 32 + j];
-                    }
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (col0 + j < p.N) red = add ? red + v[j] : fmaxf(red, v[j]);
-                } else if (row < p.M) {
+            // ---- plain epilogue and the row reductions: one sweep over the half tile (epilogue_tmem.cuh) ----
+            const int tgt = (p.e.red == FORGE_RED_CROSS_ENTROPY && row < p.M) ? __ldg(reinterpret_cast<const int *>(p.gamma) + row) : -1;
+            HalfTileRow mine;
+            half_tile_sweep<false, CHUNKS>(taddr, n0, p.N, p.e, sb, sg, tgt,
+                [&](int col0, const float (&v)[32], int) {
+                    if (row >= p.M) return;
                     __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)row * p.N + col0;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        if (col0 + i * 8 < p.N) {
-                            uint4 w;
-                            w.x = ptx::pack16x2(v[i * 8 + 0], v[i * 8 + 1], p.f16);
-                            w.y = ptx::pack16x2(v[i * 8 + 2], v[i * 8 + 3], p.f16);
-                            w.z = ptx::pack16x2(v[i * 8 + 4], v[i * 8 + 5], p.f16);
-                            w.w = ptx::pack16x2(v[i * 8 + 6], v[i * 8 + 7], p.f16);
-                            *reinterpret_cast<uint4 *>(dst + i * 8) = w;
+                        if (col0 + i * 8 < p.N) {          // N % 8 == 0: whole 16-byte pieces
+                            uint4 w4;
+                            w4.x = ptx::pack16x2(v[i * 8 + 0], v[i * 8 + 1], p.f16);
+                            w4.y = ptx::pack16x2(v[i * 8 + 2], v[i * 8 + 3], p.f16);
+                            w4.z = ptx::pack16x2(v[i * 8 + 4], v[i * 8 + 5], p.f16);
+                            w4.w = ptx::pack16x2(v[i * 8 + 6], v[i * 8 + 7], p.f16);
+                            *reinterpret_cast<uint4 *>(dst + i * 8) = w4;
                         }
                     }
-                }
-            }
+                }, mine);
             // accumulator drained: hand the TMEM buffer back to the MMA warp
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) { if (PAIR) ptx::mbar_arrive_cluster(acc_empty_addr[acc]); else ptx::mbar_arrive(&s.acc_empty[acc]); }
-
-            if (reduce) {
-                // per-part row partials; the group that arrives last at the strip folds them in order
-                float *out = reinterpret_cast<float *>(p.out);
-                if (row < p.M) p.partial[(size_t)part * p.M + row] = red;
-                epi_bar_sync(h);
-                if (et == 0) s.last_flag[h] = (arrive_acq_rel(&p.counters[tm]) == (unsigned)(parts - 1));
-                epi_bar_sync(h);
-                if (s.last_flag[h]) {
-                    if (row < p.M) {
-                        const float v = add ? fold_row_partials<true>(p.partial, parts, p.M, row) : fold_row_partials<false>(p.partial, parts, p.M, row);
-                        if (chain) p.rowg[row] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)p.N);
-                        else out[row] = v;
-                    }
-                    if (et == 0) p.counters[tm] = 0u;
-                    if (chain) {
-                        // the strip's gelu(mean) values are published; the rows are written at the end, by the whole grid
-                        epi_bar_sync(h);
-                        if (et == 0) arrive_acq_rel(p.strips_done);
-                    }
-                }
-            }
+            if (reduce || p.e.red == FORGE_RED_LOGSUMEXP || p.e.red == FORGE_RED_CROSS_ENTROPY)
+                strip_fold<false>(p.e, mine, p.partial, part, parts, p.M, p.N, row, et == 0, &p.counters[tm], &s.last_flag[h],
+                                  [h] { epi_bar_sync(h); }, reinterpret_cast<float *>(p.out), p.rowg, p.strips_done);
             if ((acc ^= 1) == 0) acc_phase ^= 1;
         }
     }

@@ -59,6 +59,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "epilogue_tmem.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
 
@@ -358,7 +359,6 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         const bool ln = red == FORGE_RED_LAYERNORM;
         const bool lse = red == FORGE_RED_LOGSUMEXP || red == FORGE_RED_CROSS_ENTROPY;
         const bool fold = red == FORGE_RED_SUM || red == FORGE_RED_MAX || chain;
-        const bool add = red != FORGE_RED_MAX;
         const uint32_t acc_empty_addr[2] = {ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[0]), 0),
                                             ptx::mapa_u32(ptx::smem_u32(&s.acc_empty[1]), 0)};     // the leader's
         int tile_parity = 0;            // bias / sub staging alternates per tile (a slow thread may still read the last one)
@@ -561,84 +561,24 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 continue;
             }
 
+            // ---- plain epilogue and the row reductions: one sweep over the half tile (epilogue_tmem.cuh) ----
             const int tgt = (red == FORGE_RED_CROSS_ENTROPY && row < p.M) ? __ldg(reinterpret_cast<const int *>(p.aux) + row) : -1;
-            float acc_red = add ? 0.f : -INFINITY;        // row sum / max of this half tile
-            float mx = -INFINITY, se = 0.f, tl = 0.f;     // (max, sum exp) and the target's logit
-#pragma unroll 1
-            for (int c = 0; c < CHUNKS; ++c) {
-                const int col0 = n0 + c * 32;
-                if (col0 >= p.N) break;
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(taddr + c * 32, r);
-                ptx::tmem_ld_wait();
-                float v[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) + sb[c * 32 + j];
-                apply_act_array<true>(p.e.act, v, p.e.scale);
-                const int nv = min(32, p.N - col0);
-                if (lse) {
-                    float cm = -INFINITY;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) cm = j < nv ? fmaxf(cm, v[j]) : cm;
-                    const float nm = fmaxf(mx, cm);
-                    float cs = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) cs += j < nv ? expf(v[j] - nm) : 0.f;
-                    se = (mx == -INFINITY ? 0.f : se * expf(mx - nm)) + cs;
-                    mx = nm;
-                    if (tgt >= col0 && tgt < col0 + 32) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) tl = (col0 + j == tgt) ? v[j] : tl;
-                    }
-                } else if (fold) {
-                    if (chain) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] -= ss[c * 32 + j];
-                    }
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (j < nv) acc_red = add ? acc_red + v[j] : fmaxf(acc_red, v[j]);
-                } else if (row < p.M) {
+            HalfTileRow mine;
+            half_tile_sweep<true, CHUNKS>(taddr, n0, p.N, p.e, sb, ss, tgt,
+                [&](int col0, const float (&v)[32], int nv) {
+                    if (row >= p.M) return;
                     float *dst = reinterpret_cast<float *>(p.out) + (size_t)row * p.N + col0;      // N % 4 == 0: 16-byte aligned
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                         if (i * 4 < nv) *reinterpret_cast<float4 *>(dst + i * 4) = make_float4(v[i * 4], v[i * 4 + 1], v[i * 4 + 2], v[i * 4 + 3]);
-                }
-            }
+                }, mine);
             // accumulator drained: hand the TMEM buffer back to the MMA warp
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_addr[acc]);
-
-            if (lse || fold) {
-                // per-part row partials; the group that arrives last at the strip folds them in part order
-                float4 *part4 = reinterpret_cast<float4 *>(p.partial);
-                if (row < p.M) {
-                    if (lse) part4[(size_t)part * p.M + row] = make_float4(mx, se, tl, 0.f);
-                    else p.partial[(size_t)part * p.M + row] = acc_red;
-                }
-                k5_epi_bar_sync(h);
-                if (et == 0) s.last_flag[h] = (arrive_acq_rel(&p.counters[tm]) == (unsigned)(parts - 1));
-                k5_epi_bar_sync(h);
-                if (s.last_flag[h]) {
-                    float *out = reinterpret_cast<float *>(p.out);
-                    if (row < p.M) {
-                        if (lse) {
-                            out[row] = fold_row_lse<true>(part4, parts, p.M, row);
-                        } else {
-                            const float v = add ? fold_row_partials<true>(p.partial, parts, p.M, row) : fold_row_partials<false>(p.partial, parts, p.M, row);
-                            if (chain) p.rowg[row] = apply_act<true>(FORGE_ACT_GELU_ERF, v / (float)p.N);
-                            else out[row] = v;
-                        }
-                    }
-                    if (et == 0) p.counters[tm] = 0u;
-                    if (chain) {
-                        // the strip's gelu(mean) values are published; the rows are written at the end, by the whole grid
-                        k5_epi_bar_sync(h);
-                        if (et == 0) arrive_acq_rel(p.strips_done);
-                    }
-                }
-            }
+            if (lse || fold)
+                strip_fold<true>(p.e, mine, p.partial, part, parts, p.M, p.N, row, et == 0, &p.counters[tm], &s.last_flag[h],
+                                 [h] { k5_epi_bar_sync(h); }, reinterpret_cast<float *>(p.out), p.rowg, p.strips_done);
             if ((acc ^= 1) == 0) acc_phase ^= 1;
         }
     }
