@@ -377,9 +377,10 @@ forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, 
 
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || desc->device >= ndev) { cudaGetLastError(); return FORGE_ERR_CUDA; }
-    int major = 0, sms = 0;
+    int major = 0, sms = 0, l2 = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, desc->device) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, desc->device) != cudaSuccess)
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, desc->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, desc->device) != cudaSuccess)
         return FORGE_ERR_CUDA;
     if (major != 10) return FORGE_ERR_CUDA;     // the kernels are sm_100a only
 
@@ -387,6 +388,7 @@ forge_status_t forge_fused_linear_create(const forge_fused_linear_desc_t *desc, 
     if (!h) return FORGE_ERR_ALLOC;
     h->d = *desc;
     h->sm_count = sms;
+    h->l2_bytes = l2;
     st = plan_for(*desc, sms, &h->info, &wl);
     if (st != FORGE_OK) { delete h; return st; }
 

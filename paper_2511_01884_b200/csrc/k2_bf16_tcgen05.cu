@@ -61,6 +61,9 @@ template <bool PAIR> struct K2Ring {
 #ifndef FORGE_K2_GROUP_M
 #define FORGE_K2_GROUP_M 16
 #endif
+#ifndef FORGE_K2_K_SERPENTINE
+#define FORGE_K2_K_SERPENTINE 1    // 0: every tile walks K upwards
+#endif
 #ifndef FORGE_K2_PAIR
 #define FORGE_K2_PAIR 1            // 0: one CTA per tile, never CTA pairs
 #endif
@@ -108,6 +111,7 @@ struct K2Params {
     unsigned *gen;        // launches whose CTAs wait on one another: run index (see run_index_begin)
     int two_pass;         // LayerNorm of rows with more tiles than CTAs (pairs): see K2Item::pass
     int short_x;          // one CTA per tile and M <= 64: 64-row X box, five stages
+    int k_serpentine;     // every other tile of a unit walks K downwards (a wave's operands exceed half of L2)
     long long ws_floats, ws_counters;      // extents of `partial` and `counters` (bounds-checked build)
     // K split of the last wave's tiles (tail_parts = 1: none)
     int tail_parts;           // S
@@ -250,7 +254,9 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             K2Item w;
             for (int j = 0; ok && k2_item<LN>(p, j, unit, units, unit_rows, w); ++j) {
                 const int tm = PAIR ? 2 * w.tm + (int)rank : w.tm, tn = w.tn;
-                for (int kb = w.kb_lo; kb < w.kb_hi; ++kb) {
+                for (int it = w.kb_lo; it < w.kb_hi; ++it) {
+                    // K serpentine (see k2_k_serpentine)
+                    const int kb = (p.k_serpentine && (j & 1)) ? w.kb_lo + w.kb_hi - 1 - it : it;
                     if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
                     if (!in_bounds(p.status, BOUNDS_RING, (long long)stage * STAGE_BYTES, STAGE_BYTES, (long long)K2_RING_BYTES)) { ok = false; break; }
                     uint8_t *a = tiles + (size_t)stage * STAGE_BYTES;
@@ -768,6 +774,7 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     p.ws_floats = h.ws.partial_floats;
     p.ws_counters = h.ws.counter_words;
     p.group_m = pair ? K2_GROUP_M / 2 : K2_GROUP_M;      // 2048 rows either way
+    p.k_serpentine = FORGE_K2_K_SERPENTINE && k_serpentine_pays(d, h.info.grid / h.info.cluster, pair ? 2 * K2_BM : K2_BM, K2_BN, ln ? 0 : K2_GROUP_M * K2_BM, 2, h.l2_bytes);
     if (!ln) {
         const K2Layout L = k2_layout(d, h.sm_count);
         p.rowg = h.ws.partial + L.rowg_off;

@@ -78,6 +78,9 @@ constexpr uint32_t K5_STAGE_BYTES = 2 * K5_RAW_BYTES;              // raw/hi, th
 constexpr uint32_t K5_RING_BYTES = K5_STAGES * K5_STAGE_BYTES;     // 192 KiB
 constexpr uint32_t K5_TMEM_COLS = 512;
 // Tuning builds may override these three (-DFORGE_K5_GROUP_M=.. and so on); the defaults are the measured best.
+#ifndef FORGE_K5_K_SERPENTINE
+#define FORGE_K5_K_SERPENTINE 1    // 0: every tile walks K upwards
+#endif
 #ifndef FORGE_K5_GROUP_M
 #define FORGE_K5_GROUP_M 8
 #endif
@@ -139,6 +142,7 @@ struct K5Params {
     int *status;
     int tiles_m, tiles_n, num_kb;      // tiles_m counts 128-row strips
     int group_m;
+    int k_serpentine;           // every other tile of a cluster walks K downwards (see k_serpentine_pays)
     long long ws_floats, ws_counters;   // extents of `partial` and `counters` (bounds-checked build)
     int write_hi;               // the splitters also store the TF32 heads (the raw words do not serve as such here)
     int two_pass;               // LayerNorm of rows with more tiles than CTA pairs: see K5Item::pass
@@ -260,7 +264,8 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 K5Item w;
                 for (int j = 0; ok && k5_item(p, j, cluster, clusters, units_m, w); ++j) {
                     const int tm = 2 * w.um + (int)rank, tn = w.tn;
-                    for (int kb = w.kb_lo; kb < w.kb_hi; ++kb) {
+                    for (int it = w.kb_lo; it < w.kb_hi; ++it) {
+                        const int kb = (p.k_serpentine && (j & 1)) ? w.kb_lo + w.kb_hi - 1 - it : it;
                         if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
                         if (!in_bounds(p.status, BOUNDS_RING, (long long)stage * K5_STAGE_BYTES, K5_RAW_BYTES, K5_RING_BYTES)) { ok = false; break; }
                         uint8_t *a = tiles + (size_t)stage * K5_STAGE_BYTES;
@@ -826,6 +831,7 @@ forge_status_t k5_launch(Handle &h, const RunArgs &a)
     p.num_kb = (int)((d.K + K5_BK - 1) / K5_BK);
     p.group_m = d.red == FORGE_RED_LAYERNORM ? 0 : K5_GROUP_M;
     p.chunk_kb = K5_CHUNK_KB;
+    p.k_serpentine = FORGE_K5_K_SERPENTINE && k_serpentine_pays(d, h.info.grid / 2, 2 * K5_BM, K5_BN, p.group_m * 2 * K5_BM, 4, h.l2_bytes);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)h.info.grid);
     cfg.blockDim = dim3(K5_THREADS);
