@@ -343,4 +343,35 @@ __device__ __forceinline__ RowStat chunk_moments(const float (&v)[32], int nv)
 
 constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// ---- residual rows of the mean chain --------------------------------------------------------------------
+// Y[r, :] = X[r, :] + g(r) over `total` 16-byte pieces (`per_row` of them to a row), this thread taking the pieces
+// first, first + step, ...  BATCH loads are issued before the first is used: with one load in flight per thread the
+// grid keeps well under a megabyte in flight, a fraction of what the memory system needs to stream.  g(row) yields
+// the row's addend, add(piece, addend) applies it to the values packed in the piece.  Y is written once and not read
+// again here: streaming stores.
+template <int BATCH, class Vec, class RowValue, class Add>
+__device__ __forceinline__ void residual_rows(const Vec *__restrict__ X, Vec *__restrict__ Y, size_t per_row, size_t total,
+                                              size_t first, size_t step, RowValue g, Add add)
+{
+    static_assert(sizeof(Vec) == 16, "16-byte pieces");
+    const bool narrow = total <= 0xffffffffull;              // 32-bit division where the indices allow it
+    for (size_t e0 = first; e0 < total; e0 += BATCH * step) {
+        Vec x[BATCH];
+#pragma unroll
+        for (int u = 0; u < BATCH; ++u) {
+            const size_t e = e0 + (size_t)u * step;
+            if (e < total) x[u] = __ldg(X + e);
+        }
+#pragma unroll
+        for (int u = 0; u < BATCH; ++u) {
+            const size_t e = e0 + (size_t)u * step;
+            if (e < total) {
+                const size_t row = narrow ? (size_t)((uint32_t)e / (uint32_t)per_row) : e / per_row;
+                add(x[u], g(row));
+                __stcs(Y + e, x[u]);
+            }
+        }
+    }
+}
+
 }  // namespace forge

@@ -537,21 +537,20 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             s.abort_flag = 1;
         __syncthreads();
         if (!*(volatile int *)&s.abort_flag) {
-            const size_t k8 = (size_t)(p.K >> 3), total = (size_t)p.M * k8;
-            const uint4 *X8 = reinterpret_cast<const uint4 *>(p.X);
-            uint4 *Y8 = reinterpret_cast<uint4 *>(p.out);
-            for (size_t e = (size_t)blockIdx.x * THREADS + threadIdx.x; e < total; e += (size_t)gridDim.x * THREADS) {
-                const float g = __ldcg(p.rowg + e / k8);
-                uint4 x = __ldg(X8 + e);
-                uint32_t *w = reinterpret_cast<uint32_t *>(&x);
+            const size_t k8 = (size_t)(p.K >> 3);
+            const bool f16 = p.f16;
+            residual_rows<8>(reinterpret_cast<const uint4 *>(p.X), reinterpret_cast<uint4 *>(p.out), k8, (size_t)p.M * k8,
+                          (size_t)blockIdx.x * THREADS + threadIdx.x, (size_t)gridDim.x * THREADS,
+                          [&](size_t row) { return __ldcg(p.rowg + row); },
+                          [f16](uint4 &x, float g) {
+                              uint32_t *w = reinterpret_cast<uint32_t *>(&x);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float lo, hi;
-                    ptx::unpack16x2(w[i], p.f16, lo, hi);
-                    w[i] = ptx::pack16x2(lo + g, hi + g, p.f16);
-                }
-                Y8[e] = x;
-            }
+                              for (int i = 0; i < 4; ++i) {
+                                  float lo, hi;
+                                  ptx::unpack16x2(w[i], f16, lo, hi);
+                                  w[i] = ptx::pack16x2(lo + g, hi + g, f16);
+                              }
+                          });
         } else {
             ok = false;
         }

@@ -598,15 +598,11 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             s.abort_flag = 1;
         __syncthreads();
         if (!*(volatile int *)&s.abort_flag) {
-            const size_t k4 = (size_t)(p.K >> 2), total = (size_t)p.M * k4;
-            const float4 *X4 = reinterpret_cast<const float4 *>(p.X);
-            float4 *Y4 = reinterpret_cast<float4 *>(p.out);
-            for (size_t e = (size_t)blockIdx.x * K5_THREADS + threadIdx.x; e < total; e += (size_t)gridDim.x * K5_THREADS) {
-                const float g = __ldcg(p.rowg + e / k4);
-                float4 x = __ldg(X4 + e);
-                x.x += g; x.y += g; x.z += g; x.w += g;
-                Y4[e] = x;
-            }
+            const size_t k4 = (size_t)(p.K >> 2);
+            residual_rows<4>(reinterpret_cast<const float4 *>(p.X), reinterpret_cast<float4 *>(p.out), k4, (size_t)p.M * k4,
+                          (size_t)blockIdx.x * K5_THREADS + threadIdx.x, (size_t)gridDim.x * K5_THREADS,
+                          [&](size_t row) { return __ldcg(p.rowg + row); },
+                          [](float4 &x, float g) { x.x += g; x.y += g; x.z += g; x.w += g; });
         } else {
             ok = false;
         }
