@@ -118,9 +118,6 @@ __device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &
     asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
 
-// Lane distance of two threads whose column groups differ by s (a power of two below 16): see the lane layout in k1_tile.
-__device__ __forceinline__ constexpr int k1_tx_lanes(int s) { return s == 8 ? 16 : s; }
-
 // T = 2: 128x128 CTA tile, 8x8 accumulators per thread.  T = 1: 64x64 tile, 4x4 per thread, for
 // problems with too few 128x128 tiles to occupy the SMs (a grid of a handful of CTAs is bound by
 // the FMA rate of the few SMs it runs on, not by the GPU's).
@@ -139,11 +136,7 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
     __shared__ int s_last;
 
     const int tid = threadIdx.x;
-    // A warp owns 2 row groups x 16 column groups.  Its lanes are laid out so that each half-warp holds 2 row groups
-    // x 8 column groups: a 128-bit shared-memory load is served per half-warp, one wavefront per 128 distinct
-    // bytes, and this footprint (32 B of the X slab, 128 B of the W slab) needs one each where 1 x 16 needs 1 + 2.
-    const int lane = tid & 31;
-    const int tx = (lane & 7) | ((lane >> 4) << 3), ty = 2 * (tid >> 5) + ((lane >> 3) & 1);
+    const int tx = tid & 15, ty = tid >> 4;
     const int m0 = tile_m * BM, n0 = tile_n * BN;
     const int M = p.M, N = p.N, K = p.K;
 
@@ -320,7 +313,7 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
                 if (cok[j]) v = ADD ? v + (acc[i][j] - sub[j]) : fmaxf(v, acc[i][j]);
 #pragma unroll
             for (int s = 8; s >= 1; s >>= 1) {
-                const float o = __shfl_xor_sync(0xffffffffu, v, k1_tx_lanes(s));
+                const float o = __shfl_xor_sync(0xffffffffu, v, s);
                 v = ADD ? v + o : fmaxf(v, o);
             }
             const int rl = ty * 4 + (i & 3) + (i >> 2) * 64;
@@ -391,9 +384,9 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
             // the 16 lanes that share the row: shuffles, no block-wide barrier
 #pragma unroll
             for (int s = 8; s >= 1; s >>= 1) {
-                const float om = __shfl_xor_sync(0xffffffffu, mx, k1_tx_lanes(s));
-                const float os = __shfl_xor_sync(0xffffffffu, se, k1_tx_lanes(s));
-                tl += __shfl_xor_sync(0xffffffffu, tl, k1_tx_lanes(s));                    // exactly one lane holds it
+                const float om = __shfl_xor_sync(0xffffffffu, mx, s);
+                const float os = __shfl_xor_sync(0xffffffffu, se, s);
+                tl += __shfl_xor_sync(0xffffffffu, tl, s);                    // exactly one lane holds it
                 lse_merge<true>(mx, se, om, os);
             }
             if (tx == 0 && row < M) {
@@ -431,7 +424,7 @@ __device__ __forceinline__ bool k1_tile(const K1Params &p, const int tile_m, con
             for (int j = 0; j < R; ++j)
                 if (cok[j]) { const float d = acc[i][j] - st.mean; st.m2 = fmaf(d, d, st.m2); }
 #pragma unroll
-            for (int sft = 1; sft <= 8; sft <<= 1) st = merge_stat(st, shfl_xor_stat(st, k1_tx_lanes(sft)));
+            for (int sft = 1; sft <= 8; sft <<= 1) st = merge_stat(st, shfl_xor_stat(st, sft));
             const int row = m0 + ty * 4 + (i & 3) + (i >> 2) * 64;
             if (ln_pass != 2 && tx == 0 && row < M) stats[(size_t)tile_n * M + row] = make_float4(st.n, st.mean, st.m2, 0.f);
         }
