@@ -59,7 +59,7 @@ template <bool PAIR> struct K2Ring {
 };
 // Tuning builds may override these three (-DFORGE_K2_GROUP_M=.. and so on); the defaults are the measured best.
 #ifndef FORGE_K2_GROUP_M
-#define FORGE_K2_GROUP_M 16
+#define FORGE_K2_GROUP_M 32
 #endif
 #ifndef FORGE_K2_K_SERPENTINE
 #define FORGE_K2_K_SERPENTINE 1    // 0: every tile walks K upwards
@@ -772,7 +772,7 @@ static forge_status_t k24_launch(Handle &h, const RunArgs &a, bool ln)
     p.short_x = !pair && d.M <= K2_BM / 2;
     p.ws_floats = h.ws.partial_floats;
     p.ws_counters = h.ws.counter_words;
-    p.group_m = pair ? K2_GROUP_M / 2 : K2_GROUP_M;      // 2048 rows either way
+    p.group_m = pair ? K2_GROUP_M / 2 : K2_GROUP_M;      // 4096 rows either way
     p.k_serpentine = FORGE_K2_K_SERPENTINE && k_serpentine_pays(d, h.info.grid / h.info.cluster, pair ? 2 * K2_BM : K2_BM, K2_BN, ln ? 0 : K2_GROUP_M * K2_BM, 2, h.l2_bytes);
     if (!ln) {
         const K2Layout L = k2_layout(d, h.sm_count);

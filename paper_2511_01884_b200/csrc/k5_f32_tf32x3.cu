@@ -82,7 +82,7 @@ constexpr uint32_t K5_TMEM_COLS = 512;
 #define FORGE_K5_K_SERPENTINE 1    // 0: every tile walks K upwards
 #endif
 #ifndef FORGE_K5_GROUP_M
-#define FORGE_K5_GROUP_M 8
+#define FORGE_K5_GROUP_M 16
 #endif
 #ifndef FORGE_K5_CHUNK_KB
 #define FORGE_K5_CHUNK_KB 4
