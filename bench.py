@@ -711,7 +711,13 @@ def main():
     e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
     e2e_ms = multigpu.max_over_ranks(e2e_ms, dist if world > 1 else None, device="cuda")
     e2e_val, _ = unit_value(wl, e2e_ms, n_units=n_units)
-    same = bool(torch.equal(host_out.cuda(), d["out"]))
+    # run_host() plans its blocks of rows for their own row count, so a block may walk K in another order than the
+    # whole problem does: the two results agree to the last place of the storage type, not always bit for bit
+    e2e_out, dev_out = host_out.cuda().float(), d["out"].float()
+    ulp = 2.0 ** -7 if wl.dtype != wk.F32 else 2.0 ** -22
+    same = bool(((e2e_out - dev_out).abs() <= ulp * torch.maximum(e2e_out.abs(), dev_out.abs())).all())
+    differing = int((e2e_out != dev_out).sum())
+    del e2e_out, dev_out
     op.check()
 
     # the measured fp32 ceiling: a register-only FMA loop on every SM
@@ -734,7 +740,7 @@ def main():
             "clocks": clocks,
             "e2e": {"value": round(e2e_val, 3), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": round(e2e_ms, 3),
-                    "matches_device_run": same, "how": "forge_fused_linear_run_host, pinned host buffers, wall clock"},
+                    "matches_device_run": same, "elements_differing_in_the_last_place": differing, "how": "forge_fused_linear_run_host, pinned host buffers, wall clock"},
             "gpu_launches": launches,
             "roofline": roofline_of(wl, ms * wl.M / rows, peaks, op.plan.kernel, clocks.get("sm_max_mhz"), props.multi_processor_count, alu_peak),
             "nominal_frac": round((value / world) / (NOMINAL["hbm_gbs"] if wl.hbm_bound else NOMINAL["bf16_tflops"]), 4)

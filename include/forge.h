@@ -178,6 +178,9 @@ forge_status_t forge_fused_linear_run(forge_fused_linear_t h, const void *X, con
  * Same operation with HOST buffers (pageable or pinned): copies the inputs to device
  * staging buffers owned by the handle (allocated on first use), runs, copies the result
  * back and synchronises.  Layouts and dtypes as for run(); bf16 data are raw 16-bit words.
+ * A large X is walked in blocks of rows, each planned for its own row count, so a block's tiles may
+ * accumulate over k in another order than run() on the whole problem: the results agree within
+ * fp32 accumulation rounding (for 16-bit outputs: the last place), not necessarily bit for bit.
  */
 forge_status_t forge_fused_linear_run_host(forge_fused_linear_t h, const void *X, const void *W, const void *b,
                                            const void *gamma, const void *beta, void *out);
