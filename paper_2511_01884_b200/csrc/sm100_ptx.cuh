@@ -75,22 +75,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 
-// Non-blocking look at a phase (no suspension): for a thread that has other things to poll.
-__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
 // The wait budget (forge::kWaitBudgetNs) is checked every few thousand polls.  On expiry -- or as
 // soon as another thread has reported a give-up -- the wait returns false; callers then leave
 // their loops and fall through to the teardown.

@@ -165,10 +165,6 @@ class Workload:
         return self.K if self.red == RED_MEAN_GELU_RESIDUAL else self.N
 
     @property
-    def out_elems(self) -> int:
-        return self.M * max(self.out_cols, 1)
-
-    @property
     def out_bytes(self) -> int:
         return self.M * 4 if self.out_cols == 0 else self.M * self.out_cols * self.elem_bytes
 
