@@ -712,11 +712,13 @@ def main():
     e2e_ms = multigpu.max_over_ranks(e2e_ms, dist if world > 1 else None, device="cuda")
     e2e_val, _ = unit_value(wl, e2e_ms, n_units=n_units)
     # run_host() plans its blocks of rows for their own row count, so a block may walk K in another order than the
-    # whole problem does: the two results agree to the last place of the storage type, not always bit for bit
+    # whole problem does: the two results agree to the last place of the storage type (where the pre-activation is
+    # near zero: to the rounding of the fp32 accumulation over K, bounded here by 1e-4), not always bit for bit
     e2e_out, dev_out = host_out.cuda().float(), d["out"].float()
     ulp = 2.0 ** -7 if wl.dtype != wk.F32 else 2.0 ** -22
-    same = bool(((e2e_out - dev_out).abs() <= ulp * torch.maximum(e2e_out.abs(), dev_out.abs())).all())
+    same = bool(((e2e_out - dev_out).abs() <= ulp * torch.maximum(e2e_out.abs(), dev_out.abs()) + 1e-4).all())
     differing = int((e2e_out != dev_out).sum())
+    max_abs_diff = float((e2e_out - dev_out).abs().max())
     del e2e_out, dev_out
     op.check()
 
@@ -740,7 +742,7 @@ def main():
             "clocks": clocks,
             "e2e": {"value": round(e2e_val, 3), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": round(e2e_ms, 3),
-                    "matches_device_run": same, "elements_differing_in_the_last_place": differing, "how": "forge_fused_linear_run_host, pinned host buffers, wall clock"},
+                    "matches_device_run": same, "elements_differing_in_the_last_place": differing, "max_abs_difference": max_abs_diff, "how": "forge_fused_linear_run_host, pinned host buffers, wall clock"},
             "gpu_launches": launches,
             "roofline": roofline_of(wl, ms * wl.M / rows, peaks, op.plan.kernel, clocks.get("sm_max_mhz"), props.multi_processor_count, alu_peak),
             "nominal_frac": round((value / world) / (NOMINAL["hbm_gbs"] if wl.hbm_bound else NOMINAL["bf16_tflops"]), 4)

@@ -119,6 +119,25 @@ def test_tiles_of_the_last_wave_cut_along_k(M, N, K, grid, red):
     pu.assert_parity(wl, a[rows], pu.run_oracle(wl, inp, rows))
 
 
+@pytest.mark.parametrize("red", [wk.RED_NONE, wk.RED_SUM])
+def test_one_wave_then_a_k_cut_tail_walked_downwards(red):
+    """90 pair tiles on 74 CTA pairs with operands past half of L2: every pair computes one whole tile (K upwards),
+    then 16 tiles are left, each cut into 4 parts along K, and these second items walk their k-blocks downwards
+    (the K serpentine).  The ring, the part ranges and the hand-over must not care about the direction."""
+    M, N, K = 512, 256 * 45, 4096
+    wl = wk.custom_workload("bf16_wave_tail_serpentine", wk.BF16, M, N, K, wk.ACT_SILU, red, seed=77 + red, w_std=0.02)
+    st, plan = B.forge_fused_linear_query_plan(pu.desc_of(wl))
+    assert st == B.FORGE_OK and plan.kernel == B.FORGE_KERNEL_BF16_TCGEN05 and plan.cluster == 2 and plan.grid == 148
+    inp = wk.make_inputs(wl)
+    op = B.FusedLinear(pu.desc_of(wl))
+    a, _ = pu.run_gpu(wl, inp, op=op, repeats=2)
+    b, _ = pu.run_gpu(wl, inp, op=op)
+    op.close()
+    assert np.array_equal(a, b)
+    rows = np.unique(np.concatenate([np.arange(0, M, 5), [M - 1]]))
+    pu.assert_parity(wl, a[rows], pu.run_oracle(wl, inp, rows))
+
+
 def test_row_counts_between_the_skinny_kernel_and_a_full_tile():
     """M = 48, 64, 96 against a 32768 x 8192 weight: more rows than the skinny kernel carries, fewer than a 128-row
     tile -- the problem is still bound by the stream of W.  Served by this kernel (one CTA per tile, the last wave cut
