@@ -80,6 +80,7 @@ struct K2Smem {
     uint32_t tmem_base;
     int last_flag[2];
     int abort_flag;
+    uint4 store_patch[8][128];  // 2 KiB per epilogue warp: see k2_store_row_pieces
     float bias[2][K2_BN];
     float gamma[2][K2_BN];
     float beta[2][K2_BN];
@@ -185,6 +186,26 @@ __device__ __forceinline__ bool k2_item(const K2Params &p, int j, int unit, int 
     }
     k2_tile_coords<LN>(t, unit_rows, p.tiles_n, p.group_m, w.tm, w.tn);
     return true;
+}
+
+// 32 columns of Y for the 32 rows of a warp (thread <-> row, four 16-byte pieces each) -> global memory through a
+// 2-KiB patch of shared memory, so that one store instruction writes 8 rows x 64 contiguous bytes (whole sectors)
+// instead of 32 rows x 16 bytes.  Piece i of row r lies at slot i ^ ((r >> 1) & 3) of the row's 64 bytes: both the
+// row-wise writes and the transposed reads are free of bank conflicts.  row0 = the warp's first row.
+__device__ __forceinline__ void k2_store_row_pieces(uint4 *patch, int lane, const uint4 (&w4)[4], __nv_bfloat16 *out,
+                                                    int row0, int M, int N, int col0)
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) patch[lane * 4 + (i ^ ((lane >> 1) & 3))] = w4[i];
+    __syncwarp();
+    const int piece = lane & 3, col = col0 + piece * 8;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = 8 * i + (lane >> 2), row = row0 + r;
+        const uint4 x = patch[r * 4 + (piece ^ ((r >> 1) & 3))];
+        if (row < M && col < N) *reinterpret_cast<uint4 *>(out + (size_t)row * N + col) = x;      // N % 8 == 0: whole pieces
+    }
+    __syncwarp();          // the patch is free for the next 32 columns
 }
 
 // named barrier of epilogue group g (ids 1 and 2; 0 is __syncthreads)
@@ -473,24 +494,26 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
                 float rstd = 0.f, shift = 0.f;
                 if (row < p.M) shift = -combine_row_moments<false>(stats, parts, p.M, row, p.e.eps, rstd) * rstd;
                 // ---- sweep 2: normalise the registers and store ----
-                if (row < p.M) {
-                    __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)row * p.N + n0;
+                {
+                    uint4 *patch = s.store_patch[warp - EPI_WARP0];
 #pragma unroll
-                    for (int i = 0; i < HALF / 8; ++i) {
-                        if (n0 + i * 8 < p.N) {
+                    for (int c = 0; c < HALF / 32; ++c) {
+                        uint4 w4[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
                             float y[8];
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
-                                const int cc = i * 8 + j;
+                                const int cc = c * 32 + i * 8 + j;
                                 y[j] = fmaf(fmaf(v[cc], rstd, shift), sg[cc], sbe[cc]);
                             }
-                            uint4 w4;
-                            w4.x = ptx::pack16x2(y[0], y[1], p.f16);
-                            w4.y = ptx::pack16x2(y[2], y[3], p.f16);
-                            w4.z = ptx::pack16x2(y[4], y[5], p.f16);
-                            w4.w = ptx::pack16x2(y[6], y[7], p.f16);
-                            *reinterpret_cast<uint4 *>(dst + i * 8) = w4;
+                            w4[i].x = ptx::pack16x2(y[0], y[1], p.f16);
+                            w4[i].y = ptx::pack16x2(y[2], y[3], p.f16);
+                            w4[i].z = ptx::pack16x2(y[4], y[5], p.f16);
+                            w4[i].w = ptx::pack16x2(y[6], y[7], p.f16);
                         }
+                        if (n0 + c * 32 < p.N)
+                            k2_store_row_pieces(patch, lane, w4, reinterpret_cast<__nv_bfloat16 *>(p.out), m0 + 32 * q, p.M, p.N, n0 + c * 32);
                     }
                 }
                 if ((acc ^= 1) == 0) acc_phase ^= 1;
@@ -502,19 +525,16 @@ k2_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_con
             HalfTileRow mine;
             half_tile_sweep<false, CHUNKS>(taddr, n0, p.N, p.e, sb, sg, tgt,
                 [&](int col0, const float (&v)[32], int) {
-                    if (row >= p.M) return;
-                    __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)row * p.N + col0;
+                    uint4 w4[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        if (col0 + i * 8 < p.N) {          // N % 8 == 0: whole 16-byte pieces
-                            uint4 w4;
-                            w4.x = ptx::pack16x2(v[i * 8 + 0], v[i * 8 + 1], p.f16);
-                            w4.y = ptx::pack16x2(v[i * 8 + 2], v[i * 8 + 3], p.f16);
-                            w4.z = ptx::pack16x2(v[i * 8 + 4], v[i * 8 + 5], p.f16);
-                            w4.w = ptx::pack16x2(v[i * 8 + 6], v[i * 8 + 7], p.f16);
-                            *reinterpret_cast<uint4 *>(dst + i * 8) = w4;
-                        }
+                        w4[i].x = ptx::pack16x2(v[i * 8 + 0], v[i * 8 + 1], p.f16);
+                        w4[i].y = ptx::pack16x2(v[i * 8 + 2], v[i * 8 + 3], p.f16);
+                        w4[i].z = ptx::pack16x2(v[i * 8 + 4], v[i * 8 + 5], p.f16);
+                        w4[i].w = ptx::pack16x2(v[i * 8 + 6], v[i * 8 + 7], p.f16);
                     }
+                    k2_store_row_pieces(s.store_patch[warp - EPI_WARP0], lane, w4, reinterpret_cast<__nv_bfloat16 *>(p.out),
+                                        m0 + 32 * q, p.M, p.N, col0);
                 }, mine);
             // accumulator drained: hand the TMEM buffer back to the MMA warp
             ptx::tc_fence_before();
