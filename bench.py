@@ -53,14 +53,14 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # from the ncu captures summarised under profiles/, keyed by workload, with the sha256 of the
 # kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
 NCU_TRAFFIC = {
-    "c2": {"bytes": 539_586_560, "sha": "a8edcb07ff7a7bdb"},
-    "c3": {"bytes": 988_228_352, "sha": "4749161a9c0e9ad6"},
-    "c4": {"bytes": 272_427_264, "sha": "6a936c6f5c8bc382"},
-    "c5": {"bytes": 305_583_616, "sha": "4749161a9c0e9ad6"},
-    "c2t": {"bytes": 304_035_328, "sha": "15258430dc7d2dc8"},
-    "n2": {"bytes": 866_688_256, "sha": "4749161a9c0e9ad6"},
-    "m64": {"bytes": 542_019_328, "sha": "4749161a9c0e9ad6"},
-    "n1b": {"bytes": 1_041_674_752, "sha": "4749161a9c0e9ad6"},
+    "c2": {"bytes": 546_686_976, "sha": "a8edcb07ff7a7bdb"},
+    "c3": {"bytes": 1_095_412_480, "sha": "4459306c224e7c19"},
+    "c4": {"bytes": 273_465_344, "sha": "6a936c6f5c8bc382"},
+    "c5": {"bytes": 326_996_992, "sha": "4459306c224e7c19"},
+    "c2t": {"bytes": 305_881_088, "sha": "15258430dc7d2dc8"},
+    "n2": {"bytes": 992_057_344, "sha": "4459306c224e7c19"},
+    "m64": {"bytes": 542_097_408, "sha": "4459306c224e7c19"},
+    "n1b": {"bytes": 1_102_634_976, "sha": "4459306c224e7c19"},
 }
 
 
