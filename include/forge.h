@@ -114,7 +114,8 @@ typedef enum {
     FORGE_KERNEL_F32_FFMA = 1,        /* fp32 register-tiled FFMA GEMM, fused epilogue        */
     FORGE_KERNEL_BF16_TCGEN05 = 2,    /* bf16 TMA -> smem ring -> tcgen05.mma -> TMEM; CTA     */
                                       /* pairs (cta_group::2, 256x256 tiles) when M > 128      */
-    FORGE_KERNEL_BF16_SKINNY = 3,     /* 16-bit, M <= 32: split-K over warps, HBM-bound        */
+    FORGE_KERNEL_BF16_SKINNY = 3,     /* 16-bit, M <= 96: HBM-bound; rows of W are the M       */
+                                      /* dimension of tcgen05.mma, X the N dimension (swap)    */
     FORGE_KERNEL_BF16_TCGEN05_LN = 4, /* bf16 tcgen05 whose epilogue merges row statistics    */
                                       /* across the N-tiles of a row strip (LayerNorm)         */
     FORGE_KERNEL_F32_TF32X3 = 5       /* fp32 operands split in shared memory into TF32 head   */
@@ -137,7 +138,7 @@ typedef struct {
  * `sm_count` multiprocessors.  Touches no device.  Returns FORGE_ERR_INVALID_ARG /
  * FORGE_ERR_UNSUPPORTED exactly as create() would for the same descriptor.
  * Kernel selection (Appendix B.1's point that the right fusion depends on whether the chain
- * is compute- or memory-bound): fp32 -> F32_FFMA; fp32 with TF32x3 arithmetic -> F32_TF32X3; 16-bit with M <= 32 and neither LayerNorm nor
+ * is compute- or memory-bound): fp32 -> F32_FFMA; fp32 with TF32x3 arithmetic -> F32_TF32X3; 16-bit with M <= 96 and neither LayerNorm nor
  * the mean-GELU-residual chain -> BF16_SKINNY; 16-bit LayerNorm -> BF16_TCGEN05_LN; other 16-bit
  * -> BF16_TCGEN05.
  * Unsupported: 16-bit storage with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); TF32x3 with

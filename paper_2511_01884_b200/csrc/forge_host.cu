@@ -20,14 +20,16 @@ bool desc_enums_ok(const forge_fused_linear_desc_t &d)
            d.act <= FORGE_ACT_SILU && d.red >= FORGE_RED_NONE && d.red <= FORGE_RED_CROSS_ENTROPY;
 }
 
-// Largest M served by the skinny kernel.  Up to 32 rows it streams W a few percent faster than
-// the tensor-core tile kernel (148 CTAs against N/256 tiles); from there on its mma.sync rate,
-// not the stream, sets the time and the tile kernel wins.  A tuning build may lower the limit
-// (-DFORGE_SKINNY_MAX_M=0..32) to compare the two kernels on the same problem.
+// Largest M served by the skinny kernel.  These problems are bound by the stream of W, and the skinny kernel
+// spreads W over all SMs in equal shares, whatever N; the tile kernel has N/256 tiles to hand out.  As M grows the
+// skinny kernel re-reads X from L2 once per 112-128 rows of W (the tile kernel once per 256), and past about 96 rows
+// the tile kernel is level or ahead (measured on 16384 x 8192 and 32768 x 8192 weights, rotating copies:
+// M = 96: 58 / 97 us against 66 / 104; M = 128: 63 / 113 against 67 / 105).  A tuning build may move the limit
+// (-DFORGE_SKINNY_MAX_M=0..128) to compare the two kernels on the same problem.
 #ifndef FORGE_SKINNY_MAX_M
-#define FORGE_SKINNY_MAX_M 32
+#define FORGE_SKINNY_MAX_M 96
 #endif
-static_assert(FORGE_SKINNY_MAX_M >= 0 && FORGE_SKINNY_MAX_M <= 32, "the skinny kernel carries at most 32 rows");
+static_assert(FORGE_SKINNY_MAX_M >= 0 && FORGE_SKINNY_MAX_M <= 128, "the skinny kernel carries at most 128 rows");
 constexpr int64_t skinny_max_m() { return FORGE_SKINNY_MAX_M; }
 
 forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
@@ -658,7 +660,7 @@ const char *forge_kernel_name(forge_kernel_t k)
     switch (k) {
     case FORGE_KERNEL_F32_FFMA: return "f32_ffma_128x128x16";
     case FORGE_KERNEL_BF16_TCGEN05: return "bf16_tcgen05_tma";
-    case FORGE_KERNEL_BF16_SKINNY: return "bf16_skinny_splitk";
+    case FORGE_KERNEL_BF16_SKINNY: return "bf16_skinny_swapab_tcgen05";
     case FORGE_KERNEL_BF16_TCGEN05_LN: return "bf16_tcgen05_tma_layernorm";
     case FORGE_KERNEL_F32_TF32X3: return "f32_tf32x3_tcgen05_tma";
     }

@@ -101,14 +101,18 @@ def test_c3_sampled_rows_full_size():
     pu.assert_parity(wl, g[rows], pu.run_oracle(wl, inp, rows))
 
 
-@pytest.mark.parametrize("M,N,K,grid", [(64, 2048, 4096, 8 * 4), (300, 520, 4096, 2 * 6 * 4), (128, 16384, 2048, 64 * 2)])
+@pytest.mark.parametrize("M,N,K,grid", [(64, 2048, 4096, 8 * 4), (112, 2048, 4096, 8 * 4), (300, 520, 4096, 2 * 6 * 4), (128, 16384, 2048, 64 * 2)])
 @pytest.mark.parametrize("red", [wk.RED_NONE, wk.RED_SUM, wk.RED_MEAN_GELU_RESIDUAL, wk.RED_CROSS_ENTROPY])
 def test_tiles_of_the_last_wave_cut_along_k(M, N, K, grid, red):
     """Fewer tiles than CTAs (or CTA pairs): every tile is computed by several of them, a slice of K
-    each, and put together by the first.  Same bits on every run (the arrival flags only ever grow)."""
+    each, and put together by the first.  Same bits on every run (the arrival flags only ever grow).  (With at most
+    96 rows only the chain takes this kernel; the other reductions go to the skinny kernel and are checked all the same.)"""
     wl = wk.custom_workload(f"bf16_ksplit_{M}", wk.BF16, M, N, K, wk.ACT_GELU_TANH, red, seed=M + red, w_std=0.02)
     st, plan = B.forge_fused_linear_query_plan(pu.desc_of(wl))
-    assert st == B.FORGE_OK and plan.kernel == B.FORGE_KERNEL_BF16_TCGEN05 and plan.grid == grid
+    if M <= 96 and red != wk.RED_MEAN_GELU_RESIDUAL:
+        assert st == B.FORGE_OK and plan.kernel == B.FORGE_KERNEL_BF16_SKINNY
+    else:
+        assert st == B.FORGE_OK and plan.kernel == B.FORGE_KERNEL_BF16_TCGEN05 and plan.grid == grid
     inp = wk.make_inputs(wl)
     op = B.FusedLinear(pu.desc_of(wl))
     a, _ = pu.run_gpu(wl, inp, op=op, repeats=3)
@@ -139,15 +143,15 @@ def test_one_wave_then_a_k_cut_tail_walked_downwards(red):
 
 
 def test_row_counts_between_the_skinny_kernel_and_a_full_tile():
-    """M = 48, 64, 96 against a 32768 x 8192 weight: more rows than the skinny kernel carries, fewer than a 128-row
-    tile -- the problem is still bound by the stream of W.  Served by this kernel (one CTA per tile, the last wave cut
-    along K); every output element against the oracle."""
+    """M = 48, 64, 96, 112 against a 32768 x 8192 weight: fewer rows than a 128-row tile -- the problem is bound by
+    the stream of W.  Up to 96 rows the skinny kernel serves it, beyond that this kernel (one CTA per tile, the last
+    wave cut along K); every output element against the oracle."""
     base = wk.EXTRA_WORKLOADS["m64"]
-    full = wk.make_inputs(dataclasses.replace(base, M=96))
-    for M in (48, 64, 96):
+    full = wk.make_inputs(dataclasses.replace(base, M=112))
+    for M in (48, 64, 96, 112):
         wl = dataclasses.replace(base, name=f"m{M}", M=M)
         inp = dict(full)
         inp["X"] = np.ascontiguousarray(full["X"][:M])
         g, plan = pu.run_gpu(wl, inp)
-        assert plan["kernel"] == B.FORGE_KERNEL_BF16_TCGEN05 and plan["cluster"] == 1
+        assert plan["kernel"] == (B.FORGE_KERNEL_BF16_SKINNY if M <= 96 else B.FORGE_KERNEL_BF16_TCGEN05) and plan["cluster"] == 1
         pu.assert_parity(wl, g, pu.run_oracle(wl, inp), f"M={M}")

@@ -299,7 +299,7 @@ def test_run_captured_in_a_graph_replays_correctly(name):
 def test_kernel_name_of_a_handle():
     wl = wk.custom_workload("kn", wk.BF16, 16, 1024, 256, wk.ACT_GELU_ERF, wk.RED_MAX, w_std=0.05)
     op = B.FusedLinear(pu.desc_of(wl))
-    assert B.forge_fused_linear_kernel_name(op.h) == B.kernel_name(op.plan.kernel) == "bf16_skinny_splitk"
+    assert B.forge_fused_linear_kernel_name(op.h) == B.kernel_name(op.plan.kernel) == "bf16_skinny_swapab_tcgen05"
     op.close()
 
 

@@ -1,5 +1,5 @@
-"""GPU parity of the skinny-M bf16 path (M <= 32: split-K over warps, mma.sync from a TMA
-ring, warp-shuffle row reductions) against the CPU oracle."""
+"""GPU parity of the skinny-M bf16 path (M <= 96: rows of W as the M dimension of tcgen05.mma, X as its
+N dimension, a TMA ring, warp-shuffle row reductions) against the CPU oracle."""
 import numpy as np
 import pytest
 
@@ -30,11 +30,14 @@ def test_identity_weight_reproduces_x():
 # N/8 below, at and far above the SM count (1, several and many strips per CTA); K with a
 # ragged last block and fewer blocks than K-slices; M below 16
 # ... and K long enough for many passes over the shared-memory ring
-# ... and two 16-row tiles of X per CTA (M up to 32), full and ragged
+# ... and more than 16 rows of X (padded to a multiple of 16: the MMA's N dimension), full and ragged, up to
+# the largest row count this kernel serves, with one or two TMA boxes per ring stage
 SHAPES = [(16, 8, 8), (1, 64, 16), (5, 1184, 72), (16, 1192, 200), (16, 4096, 1024), (7, 20000, 264),
           (16, 148 * 8 * 17, 128), (16, 148 * 8 * 40 + 8, 64), (16, 2368, 4096), (3, 1184 * 13, 2048),
           (17, 8, 8), (32, 1192, 200), (27, 20000, 264), (24, 4096, 1024), (32, 148 * 8 * 17, 128),
-          (19, 1184 * 13, 2048), (32, 2368, 4096)]
+          (19, 1184 * 13, 2048), (32, 2368, 4096),
+          (33, 8, 8), (48, 1192, 200), (64, 4096, 1024), (80, 148 * 8 * 17, 128), (96, 20000, 264), (85, 2368, 4096),
+          (96, 148 * 8 * 40 + 8, 64)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -69,10 +72,10 @@ def test_repeatable_bits_and_back_to_back_runs():
 
 
 def test_row_tiles_follow_m():
-    for M, rows in ((1, 16), (16, 16), (17, 32), (32, 32)):
+    for M, rows in ((1, 16), (16, 16), (17, 32), (32, 32), (33, 48), (96, 96)):
         st, plan = B.forge_fused_linear_query_plan(pu.desc_of(_case(M, 4096, 256, wk.ACT_RELU, wk.RED_SUM)))
         assert st == B.FORGE_OK and plan.kernel == B.FORGE_KERNEL_BF16_SKINNY and plan.tile_m == rows
-    st, plan = B.forge_fused_linear_query_plan(pu.desc_of(_case(33, 4096, 256, wk.ACT_RELU, wk.RED_SUM)))
+    st, plan = B.forge_fused_linear_query_plan(pu.desc_of(_case(97, 4096, 256, wk.ACT_RELU, wk.RED_SUM)))
     assert st == B.FORGE_OK and plan.kernel == B.FORGE_KERNEL_BF16_TCGEN05
 
 

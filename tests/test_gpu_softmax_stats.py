@@ -13,9 +13,9 @@ pytestmark = pytest.mark.gpu
 REDS = [wk.RED_LOGSUMEXP, wk.RED_CROSS_ENTROPY]
 F32_SHAPES = [(1, 1, 1), (5, 100, 7), (128, 128, 16), (130, 300, 36), (257, 1000, 64), (64, 2500, 19)]
 BF16_SHAPES = [(128, 256, 64), (300, 520, 200), (1000, 776, 328), (260, 4104, 64),
-               # M <= 32: skinny kernel, one and two 16-row tiles
+               # M <= 96: skinny kernel, rows of X padded to a multiple of 16
                (17, 8, 8), (16, 1024, 128), (1, 64, 16), (7, 20000, 264), (16, 148 * 8 * 17, 128), (3, 1184 * 13, 2048),
-               (30, 20000, 264), (32, 148 * 8 * 17, 128), (21, 1184 * 13, 2048)]
+               (30, 20000, 264), (32, 148 * 8 * 17, 128), (21, 1184 * 13, 2048), (70, 20000, 264), (96, 1184 * 13, 512)]
 
 
 @pytest.mark.parametrize("M,N,K", F32_SHAPES)
@@ -34,7 +34,7 @@ def test_bf16(M, N, K, red):
     wl = wk.custom_workload(f"lse_bf16_{M}x{N}x{K}", wk.BF16, M, N, K, wk.ACT_IDENTITY, red, scale=2.0, seed=M + N)
     inp = wk.make_inputs(wl)
     g, plan = pu.run_gpu(wl, inp)
-    assert plan["kernel"] == (B.FORGE_KERNEL_BF16_SKINNY if M <= 32 else B.FORGE_KERNEL_BF16_TCGEN05)
+    assert plan["kernel"] == (B.FORGE_KERNEL_BF16_SKINNY if M <= 96 else B.FORGE_KERNEL_BF16_TCGEN05)
     pu.assert_parity(wl, g, pu.run_oracle(wl, inp))
 
 
