@@ -44,7 +44,7 @@ struct K3Smem {
     float red[K3_EPI_WARPS][K3_MAX_M];        // per warp and row of X: sum or max over the warp's 32 columns ...
     float red_s[K3_EPI_WARPS][K3_MAX_M];      // ... softmax: sum of exponentials ...
     float red_t[K3_EPI_WARPS][K3_MAX_M];      // ... and the target's logit
-    float fold[3][K3_EPI_THREADS];             // the last CTA's fold: (row, chunk of CTAs)
+    float fold[4][K3_EPI_THREADS];             // the last CTA's fold: (row, chunk of CTAs) results
     uint32_t tmem_base;
     int last_flag;
     int abort_flag;
@@ -327,34 +327,57 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                 k3_epi_sync();
                 if (et == 0) s.last_flag = (arrive_acq_rel(&p.counters[0]) == gridDim.x - 1);
                 k3_epi_sync();
-                if (s.last_flag) {
+                if (s.last_flag && !softmax) {
+                    // sum / max: a thread takes four rows (one 16-byte load per CTA) of every chunks-th CTA, eight
+                    // loads in flight, merged in CTA order (an absent CTA is the neutral element); the chunks'
+                    // results meet in shared memory and are merged in chunk order
+                    const int quads = p.xr / 4, chunks = K3_EPI_THREADS / quads;       // 32 .. 4 chunks of CTAs
+                    const int quad = et % quads, chunk = et / quads;
+                    float *ff = &s.fold[0][0];                                          // [chunk][row], at most 512 floats
+                    if (chunk < chunks) {
+                        float a[4] = {neutral, neutral, neutral, neutral};
+                        for (unsigned c0 = chunk; c0 < gridDim.x; c0 += 8 * chunks) {
+                            float4 f[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                const unsigned c = c0 + u * chunks;
+                                f[u] = c < gridDim.x ? __ldcg(&part4[(size_t)c * quads + quad]) : make_float4(neutral, neutral, neutral, neutral);
+                            }
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                a[0] = sum ? a[0] + f[u].x : fmaxf(a[0], f[u].x);
+                                a[1] = sum ? a[1] + f[u].y : fmaxf(a[1], f[u].y);
+                                a[2] = sum ? a[2] + f[u].z : fmaxf(a[2], f[u].z);
+                                a[3] = sum ? a[3] + f[u].w : fmaxf(a[3], f[u].w);
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) ff[chunk * p.xr + quad * 4 + j] = a[j];
+                    }
+                    k3_epi_sync();
+                    if (et < p.M) {
+                        float r = ff[et];
+                        for (int j = 1; j < chunks; ++j) r = sum ? r + ff[j * p.xr + et] : fmaxf(r, ff[j * p.xr + et]);
+                        out[et] = r;
+                    }
+                    if (et == 0) p.counters[0] = 0u;
+                } else if (s.last_flag) {
+                    // softmax statistics: one 16-byte triple per row and CTA
                     const int chunks = K3_EPI_THREADS / p.xr;              // 8 .. 1 chunks of CTAs per row
                     const int row = et % p.xr, chunk = et / p.xr;
-                    float mx = neutral, se = 0.f, tl = 0.f;
+                    float mx = -INFINITY, se = 0.f, tl = 0.f;
                     if (chunk < chunks) {
-                        // eight loads in flight, then the merges in CTA order (an absent CTA is the neutral element)
                         for (unsigned c0 = chunk; c0 < gridDim.x; c0 += 8 * chunks) {
-                            if (softmax) {
-                                float4 f[8];
+                            float4 f[8];
 #pragma unroll
-                                for (int u = 0; u < 8; ++u) {
-                                    const unsigned c = c0 + u * chunks;
-                                    f[u] = c < gridDim.x ? __ldcg(&part4[(size_t)c * p.xr + row]) : make_float4(-INFINITY, 0.f, 0.f, 0.f);
-                                }
+                            for (int u = 0; u < 8; ++u) {
+                                const unsigned c = c0 + u * chunks;
+                                f[u] = c < gridDim.x ? __ldcg(&part4[(size_t)c * p.xr + row]) : make_float4(-INFINITY, 0.f, 0.f, 0.f);
+                            }
 #pragma unroll
-                                for (int u = 0; u < 8; ++u) {
-                                    lse_merge<false>(mx, se, f[u].x, f[u].y);
-                                    tl += f[u].z;
-                                }
-                            } else {
-                                float o[8];
-#pragma unroll
-                                for (int u = 0; u < 8; ++u) {
-                                    const unsigned c = c0 + u * chunks;
-                                    o[u] = c < gridDim.x ? __ldcg(&p.partial[(size_t)c * p.xr + row]) : neutral;
-                                }
-#pragma unroll
-                                for (int u = 0; u < 8; ++u) mx = sum ? mx + o[u] : fmaxf(mx, o[u]);
+                            for (int u = 0; u < 8; ++u) {
+                                lse_merge<false>(mx, se, f[u].x, f[u].y);
+                                tl += f[u].z;
                             }
                         }
                     }
@@ -363,15 +386,10 @@ k3_bf16_skinny_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                     if (et < p.M) {
                         mx = s.fold[0][et]; se = s.fold[1][et]; tl = s.fold[2][et];
                         for (int j = 1; j < chunks; ++j) {
-                            if (softmax) {
-                                lse_merge<false>(mx, se, s.fold[0][j * p.xr + et], s.fold[1][j * p.xr + et]);
-                                tl += s.fold[2][j * p.xr + et];
-                            } else {
-                                const float o = s.fold[0][j * p.xr + et];
-                                mx = sum ? mx + o : fmaxf(mx, o);
-                            }
+                            lse_merge<false>(mx, se, s.fold[0][j * p.xr + et], s.fold[1][j * p.xr + et]);
+                            tl += s.fold[2][j * p.xr + et];
                         }
-                        out[et] = softmax ? mx + __logf(se) - tl : mx;
+                        out[et] = mx + __logf(se) - tl;
                     }
                     if (et == 0) p.counters[0] = 0u;
                 }
