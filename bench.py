@@ -55,11 +55,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC = {
     "c2": {"bytes": 546_686_976, "sha": "a8edcb07ff7a7bdb"},
     "c3": {"bytes": 1_095_412_480, "sha": "4459306c224e7c19"},
-    "c4": {"bytes": 273_465_344, "sha": "6a936c6f5c8bc382"},
+    "c4": {"bytes": 273_227_520, "sha": "31f38eb6ee54b347"},
     "c5": {"bytes": 326_996_992, "sha": "4459306c224e7c19"},
     "c2t": {"bytes": 305_881_088, "sha": "15258430dc7d2dc8"},
     "n2": {"bytes": 992_057_344, "sha": "4459306c224e7c19"},
-    "m64": {"bytes": 542_097_408, "sha": "4459306c224e7c19"},
+    "m64": {"bytes": 551_581_952, "sha": "31f38eb6ee54b347"},
     "n1b": {"bytes": 1_102_634_976, "sha": "4459306c224e7c19"},
 }
 
