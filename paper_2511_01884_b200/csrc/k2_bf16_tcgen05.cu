@@ -28,6 +28,7 @@
 #include "epilogue_tmem.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
+#include "tile_schedule.cuh"
 
 namespace forge {
 
@@ -124,68 +125,14 @@ struct K2Params {
     unsigned *strips_done;    // mean chain: strips whose rowg values are published; only ever grows: tiles_m per run
 };
 
-template <bool LN>
-__device__ __forceinline__ void k2_tile_coords(int t, int tiles_m, int tiles_n, int group_m, int &tm, int &tn)
-{
-    if (LN) {            // a strip's N-tiles are neighbours in the schedule
-        tm = t / tiles_n;
-        tn = t - tm * tiles_n;
-        return;
-    }
-    const int group_size = group_m * tiles_n;
-    const int g = t / group_size, r = t - g * group_size;
-    const int gm = min(group_m, tiles_m - g * group_m);
-    tm = g * group_m + r % gm;
-    tn = r / gm;
-    if (g & 1) tn = tiles_n - 1 - tn;      // every other group walks the N-tiles backwards: the W panels last used are still in L2
-}
-
-// One unit of work of a CTA (or CTA pair): a tile and a range of k-blocks.  Unit c of C takes the whole
-// tiles c, c + C, ... of the full waves and then at most one item of the last wave.  When the tiles
-// left for the last wave are at most half the units, each is cut along K into S parts that run on S
-// units at once: parts 1..S-1 leave their raw accumulators in a scratch area and count themselves
-// in; part 0 waits for them (bounded), adds them into its accumulator in part order and runs the
-// epilogue.  The same cut lets a problem with fewer tiles than SMs (M <= 128 with a few thousand
-// columns, say) stream its weights with most of the GPU.
-struct K2Item {
-    int tm, tn;                 // row unit, 256-column tile
-    int kb_lo, kb_hi;           // k-blocks [kb_lo, kb_hi)
-    int part, tail;             // part of the K split (0 leads), index of the tile among the split ones (-1: whole tile)
-    int pass;                   // LayerNorm of rows wider than the grid: 0 = statistics only, 1 = normalise and store
-};
-
+// Item j of this unit's work list (tile_schedule.cuh).  LayerNorm: the N-tiles of a strip are neighbours in the
+// schedule (group_m = 0) and rows wider than the grid take every tile twice.
+using K2Item = TileItem;
 template <bool LN>
 __device__ __forceinline__ bool k2_item(const K2Params &p, int j, int unit, int units, int unit_rows, K2Item &w)
 {
-    const int total = unit_rows * p.tiles_n, full = total / units, rest = total - full * units;
-    int t;
-    w.kb_lo = 0;
-    w.kb_hi = p.num_kb;
-    w.part = 0;
-    w.tail = -1;
-    w.pass = 0;
-    if (LN && p.two_pass) {
-        // every tile twice: this unit's whole list once for the statistics, then once more to normalise
-        const int mine = full + (unit < rest ? 1 : 0);
-        if (j >= mine) { j -= mine; w.pass = 1; }
-    }
-    if (j < full) {
-        t = j * units + unit;
-    } else if (j == full && p.tail_parts <= 1) {
-        if (unit >= rest) return false;
-        t = full * units + unit;
-    } else if (j == full) {
-        if (unit >= rest * p.tail_parts) return false;
-        w.tail = unit / p.tail_parts;
-        w.part = unit - w.tail * p.tail_parts;
-        t = full * units + w.tail;
-        w.kb_lo = w.part * p.tail_kb;
-        w.kb_hi = min(w.kb_lo + p.tail_kb, p.num_kb);
-    } else {
-        return false;
-    }
-    k2_tile_coords<LN>(t, unit_rows, p.tiles_n, p.group_m, w.tm, w.tn);
-    return true;
+    return schedule_item<true>(j, unit, units, unit_rows, p.tiles_n, p.num_kb, p.tail_parts, p.tail_kb, LN && p.two_pass,
+                               LN ? 0 : p.group_m, w);
 }
 
 // 32 columns of Y for the 32 rows of a warp (thread <-> row, four 16-byte pieces each) -> global memory through a
@@ -597,54 +544,27 @@ static bool k2_use_pair(const forge_fused_linear_desc_t &d, int sm_count)
     return FORGE_K2_PAIR != 0 && d.M > K2_BM && sm_count >= 2;
 }
 
-// Grid, K split of the last wave and workspace layout of the non-LayerNorm kernel: a pure function of
-// the problem and the SM count, used by the planner and by the launcher.
-constexpr int K2_TAIL_MAX_PARTS = 8;      // bounds the scratch area and the serial adds of part 0
+// Grid, K split of the last wave and workspace layout of the non-LayerNorm kernel (tile_schedule.cuh).
 constexpr int K2_TAIL_MIN_KB = 16;        // a part is worth its hand-over only with 1024 k or more
-constexpr int K2_TAIL_MAX_FULL_WAVES = 8; // after that many full waves the last one is too small a share to matter
-                                          // (55 waves: measured 3 % slower with the cut than without)
-struct K2Layout {
+struct K2Layout : ScheduleLayout {
     bool pair;
-    int64_t tiles_m, tiles_n, units, slots, grid;      // slots: CTAs (or CTA pairs) the GPU offers
-    int tail_parts, tail_kb, tail_tiles;
-    size_t rowg_off, scratch_off, partial_floats;      // float offsets into the partial area
-    size_t strips_done_idx, tail_flags_idx, gen_idx, counters;
+    int64_t grid;
 };
 
 static K2Layout k2_layout(const forge_fused_linear_desc_t &d, int sm_count)
 {
-    K2Layout L = {};
-    L.pair = k2_use_pair(d, sm_count);
-    L.tiles_m = (d.M + K2_BM - 1) / K2_BM;
-    L.tiles_n = (d.N + K2_BN - 1) / K2_BN;
-    L.units = (L.pair ? (L.tiles_m + 1) / 2 : L.tiles_m) * L.tiles_n;
-    L.slots = L.pair ? sm_count / 2 : sm_count;
-    const int64_t full = L.units / L.slots, rest = L.units % L.slots;
-    const int num_kb = (int)((d.K + K2_BK - 1) / K2_BK);
-    constexpr bool env = FORGE_K2_TAIL_SPLIT != 0;
-    int parts = 1;
-    if (env && rest > 0 && full < K2_TAIL_MAX_FULL_WAVES && d.red != FORGE_RED_LAYERNORM) {
-        int64_t s = L.slots / rest;
-        if (s > K2_TAIL_MAX_PARTS) s = K2_TAIL_MAX_PARTS;
-        if (s > num_kb / K2_TAIL_MIN_KB) s = num_kb / K2_TAIL_MIN_KB;
-        parts = s < 1 ? 1 : (int)s;
-    }
-    L.tail_kb = (num_kb + parts - 1) / parts;
-    L.tail_parts = (num_kb + L.tail_kb - 1) / L.tail_kb;       // no empty part
-    L.tail_tiles = L.tail_parts > 1 ? (int)rest : 0;
-    const int64_t ctas = full > 0 ? L.slots : rest * L.tail_parts;
-    L.grid = L.pair ? 2 * ctas : ctas;
+    const bool pair = k2_use_pair(d, sm_count);
+    const int64_t tiles_m = (d.M + K2_BM - 1) / K2_BM, tiles_n = (d.N + K2_BN - 1) / K2_BN;
     const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;      // float4 partials
     const bool chain = d.red == FORGE_RED_MEAN_GELU_RESIDUAL;
     const bool fold = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || chain || lse;      // one partial per row and half tile
-    const size_t fold_floats = fold ? (lse ? 4 : 1) * 2 * (size_t)L.tiles_n * (size_t)d.M : 0;
-    L.rowg_off = fold_floats;                                  // mean chain: gelu(mean) per row after the partials
-    L.scratch_off = (L.rowg_off + (chain ? (size_t)d.M : 0) + 3) / 4 * 4;
-    L.partial_floats = L.scratch_off + (size_t)L.tail_tiles * (L.tail_parts - 1) * 2 * 2 * (4 * 32 * K2_EPI_THREADS);
-    L.strips_done_idx = fold ? (size_t)L.tiles_m : 0;
-    L.tail_flags_idx = L.strips_done_idx + (chain ? 1 : 0);
-    L.gen_idx = L.tail_flags_idx + (size_t)L.tail_tiles * 4;       // run index and finished-CTA count
-    L.counters = L.gen_idx + 2;
+    K2Layout L = {};
+    static_cast<ScheduleLayout &>(L) = schedule_layout(
+        tiles_m, tiles_n, (pair ? (tiles_m + 1) / 2 : tiles_m) * tiles_n, pair ? sm_count / 2 : sm_count,
+        (int)((d.K + K2_BK - 1) / K2_BK), FORGE_K2_TAIL_SPLIT != 0 && d.red != FORGE_RED_LAYERNORM, K2_TAIL_MIN_KB,
+        fold ? (lse ? 4 : 1) * 2 * (size_t)tiles_n * (size_t)d.M : 0, chain, d.M);
+    L.pair = pair;
+    L.grid = pair ? 2 * L.ctas : L.ctas;
     return L;
 }
 

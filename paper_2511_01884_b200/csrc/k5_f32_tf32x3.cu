@@ -62,6 +62,7 @@
 #include "epilogue_tmem.cuh"
 #include "plan.h"
 #include "sm100_ptx.cuh"
+#include "tile_schedule.cuh"
 
 namespace forge {
 
@@ -154,66 +155,15 @@ struct K5Params {
     unsigned *tail_flags;       // [tail tile][rank][column half]; only ever grow: tail_parts - 1 arrivals per run
 };
 
-// One unit of work of a cluster: a pair tile and a range of k-blocks.  Cluster c takes the whole
-// tiles c, c + C, ... of the full waves and then at most one item of the last wave.
-struct K5Item {
-    int um, tn;                 // 256-row unit, 256-column tile
-    int kb_lo, kb_hi;           // k-blocks [kb_lo, kb_hi)
-    int part, tail;             // part of the K split (0 leads), index of the tile among the split ones (-1: whole tile)
-    int pass;                   // LayerNorm of rows wider than the grid: 0 = statistics only, 1 = normalise and store
-};
-
-__device__ __forceinline__ void k5_tile_coords(int t, int units_m, int tiles_n, int group_m, int &um, int &tn);
-
+// Item j of this cluster's work list (tile_schedule.cuh): a pair tile (tm = 256-row unit) and a range of k-blocks.
+using K5Item = TileItem;
 __device__ __forceinline__ bool k5_item(const K5Params &p, int j, int cluster, int clusters, int units_m, K5Item &w)
 {
-    const int total = units_m * p.tiles_n, full = total / clusters, rest = total - full * clusters;
-    int t;
-    w.kb_lo = 0;
-    w.kb_hi = p.num_kb;
-    w.part = 0;
-    w.tail = -1;
-    w.pass = 0;
-    if (p.two_pass) {
-        // every tile twice: this cluster's whole list once for the statistics, then once more to normalise
-        const int mine = full + (cluster < rest ? 1 : 0);
-        if (j >= mine) { j -= mine; w.pass = 1; }
-    }
-    if (j < full) {
-        t = j * clusters + cluster;
-    } else if (j == full && p.tail_parts <= 1) {
-        if (cluster >= rest) return false;
-        t = full * clusters + cluster;
-    } else if (j == full) {
-        if (cluster >= rest * p.tail_parts) return false;
-        w.tail = cluster / p.tail_parts;
-        w.part = cluster - w.tail * p.tail_parts;
-        t = full * clusters + w.tail;
-        w.kb_lo = w.part * p.tail_kb;
-        w.kb_hi = min(w.kb_lo + p.tail_kb, p.num_kb);
-    } else {
-        return false;
-    }
-    k5_tile_coords(t, units_m, p.tiles_n, p.group_m, w.um, w.tn);
-    return true;
+    return schedule_item<false>(j, cluster, clusters, units_m, p.tiles_n, p.num_kb, p.tail_parts, p.tail_kb, p.two_pass != 0, p.group_m, w);
 }
 
 template <int N> __device__ __forceinline__ void k5_reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void k5_reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-
-__device__ __forceinline__ void k5_tile_coords(int t, int units_m, int tiles_n, int group_m, int &um, int &tn)
-{
-    if (group_m <= 0) {          // LayerNorm: the N-tiles of a row strip are neighbours in the schedule
-        um = t / tiles_n;
-        tn = t - um * tiles_n;
-        return;
-    }
-    const int group_size = group_m * tiles_n;
-    const int g = t / group_size, r = t - g * group_size;
-    const int gm = min(group_m, units_m - g * group_m);
-    um = g * group_m + r % gm;
-    tn = r / gm;
-}
 
 __device__ __forceinline__ void k5_epi_bar_sync(int g) { asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(K5_EPI_THREADS) : "memory"); }
 
@@ -263,7 +213,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
                 uint32_t phase = 0;
                 K5Item w;
                 for (int j = 0; ok && k5_item(p, j, cluster, clusters, units_m, w); ++j) {
-                    const int tm = 2 * w.um + (int)rank, tn = w.tn;
+                    const int tm = 2 * w.tm + (int)rank, tn = w.tn;
                     for (int it = w.kb_lo; it < w.kb_hi; ++it) {
                         const int kb = (p.k_serpentine && (j & 1)) ? w.kb_lo + w.kb_hi - 1 - it : it;
                         if (!ptx::mbar_wait(&s.empty[stage], phase ^ 1, p.status, SITE_STAGE_EMPTY)) { ok = false; break; }
@@ -369,7 +319,7 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         int tile_parity = 0;            // bias / sub staging alternates per tile (a slow thread may still read the last one)
         K5Item w;
         for (int j = 0; k5_item(p, j, cluster, clusters, units_m, w); ++j, tile_parity ^= 1) {
-            const int tn = w.tn, tm = 2 * w.um + (int)rank;
+            const int tn = w.tn, tm = 2 * w.tm + (int)rank;
             const int m0 = tm * K5_BM, n0 = tn * K5_BN + h * HALF;
             const int part = 2 * tn + h;
             float *sb = s.bias[tile_parity] + h * HALF, *ss = s.sub[tile_parity] + h * HALF;
@@ -621,54 +571,26 @@ k5_f32_tf32x3_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 }
 
 // ---- host side ---------------------------------------------------------------------------
-// Grid, K split of the last wave and workspace layout: a pure function of the problem and the SM count,
-// used by the planner and by the launcher.
-constexpr int K5_TAIL_MAX_PARTS = 8;      // bounds the scratch area and the serial adds of part 0
+// Grid, K split of the last wave and workspace layout (tile_schedule.cuh).
 constexpr int K5_TAIL_MIN_KB = 16;        // a part is worth its hand-over only with 512 k or more
-constexpr int K5_TAIL_MAX_FULL_WAVES = 8; // after that many full waves the last one is too small a share to matter
-struct K5Layout {
-    int64_t tiles_m, tiles_n, units, clusters, grid;
-    int tail_parts, tail_kb, tail_tiles;
-    size_t fold_floats;       // per half tile row partials of the row reductions
-    size_t rowg_off;          // mean chain: gelu(mean) per row (float offset into the partial area)
-    size_t scratch_off;       // K split: hand-over area (float offset, multiple of 4)
-    size_t partial_floats;
-    size_t strips_done_idx, tail_flags_idx, gen_idx, counters;
+struct K5Layout : ScheduleLayout {
+    int64_t grid;
 };
 
 static K5Layout k5_layout(const forge_fused_linear_desc_t &d, int sm_count)
 {
-    K5Layout L = {};
-    L.tiles_m = (d.M + K5_BM - 1) / K5_BM;
-    L.tiles_n = (d.N + K5_BN - 1) / K5_BN;
-    L.units = ((L.tiles_m + 1) / 2) * L.tiles_n;
-    L.clusters = sm_count / 2;
-    const int64_t full = L.units / L.clusters, rest = L.units % L.clusters;
-    const int num_kb = (int)((d.K + K5_BK - 1) / K5_BK);
-    constexpr bool env = FORGE_K5_TAIL_SPLIT != 0;
+    const int64_t tiles_m = (d.M + K5_BM - 1) / K5_BM, tiles_n = (d.N + K5_BN - 1) / K5_BN;
     const bool ln = d.red == FORGE_RED_LAYERNORM;
-    int parts = 1;
-    if (env && rest > 0 && full < K5_TAIL_MAX_FULL_WAVES && !ln) {        // LayerNorm: a tile already waits for its strip; no second dependency
-        int64_t s = L.clusters / rest;
-        if (s > K5_TAIL_MAX_PARTS) s = K5_TAIL_MAX_PARTS;
-        if (s > num_kb / K5_TAIL_MIN_KB) s = num_kb / K5_TAIL_MIN_KB;
-        parts = s < 1 ? 1 : (int)s;
-    }
-    L.tail_kb = (num_kb + parts - 1) / parts;
-    L.tail_parts = (num_kb + L.tail_kb - 1) / L.tail_kb;       // no empty part
-    L.tail_tiles = L.tail_parts > 1 ? (int)rest : 0;
-    L.grid = 2 * (full > 0 ? L.clusters : rest * L.tail_parts);
     const bool lse = d.red == FORGE_RED_LOGSUMEXP || d.red == FORGE_RED_CROSS_ENTROPY;
     const bool chain = d.red == FORGE_RED_MEAN_GELU_RESIDUAL;
     const bool fold = d.red == FORGE_RED_SUM || d.red == FORGE_RED_MAX || chain || lse || ln;
-    L.fold_floats = fold ? ((lse || ln) ? 4 : 1) * 2 * (size_t)L.tiles_n * (size_t)d.M : 0;
-    L.rowg_off = L.fold_floats;
-    L.scratch_off = (L.rowg_off + (chain ? (size_t)d.M : 0) + 3) / 4 * 4;
-    L.partial_floats = L.scratch_off + (size_t)L.tail_tiles * (L.tail_parts - 1) * 2 * 2 * (4 * 32 * K5_EPI_THREADS);
-    L.strips_done_idx = fold ? (size_t)L.tiles_m : 0;
-    L.tail_flags_idx = L.strips_done_idx + (chain ? 1 : 0);
-    L.gen_idx = L.tail_flags_idx + (size_t)L.tail_tiles * 4;       // run index and finished-CTA count
-    L.counters = L.gen_idx + 2;
+    K5Layout L = {};
+    // LayerNorm: a tile already waits for its strip; no second dependency, so no K split
+    static_cast<ScheduleLayout &>(L) = schedule_layout(
+        tiles_m, tiles_n, ((tiles_m + 1) / 2) * tiles_n, sm_count / 2, (int)((d.K + K5_BK - 1) / K5_BK),
+        FORGE_K5_TAIL_SPLIT != 0 && !ln, K5_TAIL_MIN_KB,
+        fold ? ((lse || ln) ? 4 : 1) * 2 * (size_t)tiles_n * (size_t)d.M : 0, chain, d.M);
+    L.grid = 2 * L.ctas;
     return L;
 }
 
