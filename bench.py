@@ -53,14 +53,14 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # from the ncu captures summarised under profiles/, keyed by workload, with the sha256 of the
 # kernel source the capture was taken from.  A changed source invalidates the figure (-> null).
 NCU_TRAFFIC = {
-    "c2": {"bytes": 546_686_976, "sha": "a8edcb07ff7a7bdb"},
-    "c3": {"bytes": 1_095_412_480, "sha": "4459306c224e7c19"},
-    "c4": {"bytes": 273_227_520, "sha": "31f38eb6ee54b347"},
-    "c5": {"bytes": 326_996_992, "sha": "4459306c224e7c19"},
-    "c2t": {"bytes": 305_881_088, "sha": "15258430dc7d2dc8"},
-    "n2": {"bytes": 992_057_344, "sha": "4459306c224e7c19"},
-    "m64": {"bytes": 551_581_952, "sha": "31f38eb6ee54b347"},
-    "n1b": {"bytes": 1_102_634_976, "sha": "4459306c224e7c19"},
+    "c2": {"bytes": 556_733_184, "sha": "a8edcb07ff7a7bdb"},
+    "c3": {"bytes": 1_001_968_384, "sha": "ab482763f83be5c8"},
+    "c4": {"bytes": 273_177_344, "sha": "8c72391c87c56a84"},
+    "c5": {"bytes": 326_729_728, "sha": "ab482763f83be5c8"},
+    "c2t": {"bytes": 304_342_528, "sha": "29bae20a963fe65f"},
+    "n2": {"bytes": 876_474_368, "sha": "ab482763f83be5c8"},
+    "m64": {"bytes": 551_515_136, "sha": "8c72391c87c56a84"},
+    "n1b": {"bytes": 1_025_926_656, "sha": "ab482763f83be5c8"},
 }
 
 

@@ -28,7 +28,7 @@ constexpr int K3_BK = 64;                      // k per TMA box: one 128-byte sw
 #ifndef FORGE_K3_KB
 #define FORGE_K3_KB 0
 #endif
-constexpr int K3_MAX_KB = 2;
+static_assert(FORGE_K3_KB >= 0 && FORGE_K3_KB <= 2, "one or two 64-k blocks per stage");
 constexpr int K3_MAX_ROWS_W = 128;             // rows of W per strip (the MMA's M)
 constexpr int K3_MAX_M = 128;                  // rows of X (the MMA's N, padded to a multiple of 16)
 constexpr int K3_MAX_STAGES = 16;
