@@ -55,11 +55,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC = {
     "c2": {"bytes": 556_733_184, "sha": "a8edcb07ff7a7bdb"},
     "c3": {"bytes": 1_001_968_384, "sha": "ab482763f83be5c8"},
-    "c4": {"bytes": 273_177_344, "sha": "8c72391c87c56a84"},
+    "c4": {"bytes": 273_245_696, "sha": "7f82c84d18aa5daf"},
     "c5": {"bytes": 326_729_728, "sha": "ab482763f83be5c8"},
     "c2t": {"bytes": 304_342_528, "sha": "29bae20a963fe65f"},
     "n2": {"bytes": 876_474_368, "sha": "ab482763f83be5c8"},
-    "m64": {"bytes": 551_515_136, "sha": "8c72391c87c56a84"},
+    "m64": {"bytes": 554_519_552, "sha": "7f82c84d18aa5daf"},
     "n1b": {"bytes": 1_025_926_656, "sha": "ab482763f83be5c8"},
 }
 

@@ -138,9 +138,10 @@ typedef struct {
  * `sm_count` multiprocessors.  Touches no device.  Returns FORGE_ERR_INVALID_ARG /
  * FORGE_ERR_UNSUPPORTED exactly as create() would for the same descriptor.
  * Kernel selection (Appendix B.1's point that the right fusion depends on whether the chain
- * is compute- or memory-bound): fp32 -> F32_FFMA; fp32 with TF32x3 arithmetic -> F32_TF32X3; 16-bit with M <= 96 and neither LayerNorm nor
- * the mean-GELU-residual chain -> BF16_SKINNY; 16-bit LayerNorm -> BF16_TCGEN05_LN; other 16-bit
- * -> BF16_TCGEN05.
+ * is compute- or memory-bound): fp32 -> F32_FFMA; fp32 with TF32x3 arithmetic -> F32_TF32X3;
+ * 16-bit with M <= 96 and neither LayerNorm nor the mean-GELU-residual chain -> BF16_SKINNY
+ * (except a long K against few rows of W: K >= 24576 with N <= 16 x sm_count); 16-bit LayerNorm
+ * -> BF16_TCGEN05_LN; other 16-bit -> BF16_TCGEN05.
  * Unsupported: 16-bit storage with K % 8 != 0 or N % 8 != 0 (16-byte row pitch); TF32x3 with
  * K % 4 != 0 or N % 4 != 0.
  */

@@ -14,7 +14,7 @@ rebuild, and so does the next build without them):
                                      handle's status word instead of making the access
   -DFORGE_K2_GROUP_M=.. -DFORGE_K2_PAIR=0 -DFORGE_K2_TAIL_SPLIT=0 -DFORGE_K2_K_SERPENTINE=0 -DFORGE_K5_K_SERPENTINE=0
   -DFORGE_K5_GROUP_M=.. -DFORGE_K5_CHUNK_KB=..
-  -DFORGE_K5_TAIL_SPLIT=0 -DFORGE_TMA_L2_PROMOTION=0|64|128|256 -DFORGE_SKINNY_MAX_M=0..128 -DFORGE_K3_KB=1|2   tuning variants
+  -DFORGE_K5_TAIL_SPLIT=0 -DFORGE_TMA_L2_PROMOTION=0|64|128|256 -DFORGE_SKINNY_MAX_M=0..128 -DFORGE_K3_KB=1..8   tuning variants
 """
 from __future__ import annotations
 

@@ -31,6 +31,17 @@ bool desc_enums_ok(const forge_fused_linear_desc_t &d)
 #endif
 static_assert(FORGE_SKINNY_MAX_M >= 0 && FORGE_SKINNY_MAX_M <= 128, "the skinny kernel carries at most 128 rows");
 constexpr int64_t skinny_max_m() { return FORGE_SKINNY_MAX_M; }
+// One more case goes to the tile kernel: a long K against so few rows of W that an SM's share is 16 rows or fewer
+// (N <= 16 x SMs).  The skinny kernel gives every CTA all of K for its rows, and 16 rows are too few bytes in flight
+// per SM however the ring is cut; the tile kernel cuts K over the CTAs instead (measured, M = 16: 1024 x 65536
+// 114 against 67 us, 2048 x 32768 61 against 52; but 2368 x 8192 21 against 35, 4096 x 16384 35 against 48).
+bool skinny_serves(const forge_fused_linear_desc_t &d, int sm_count)
+{
+    if (d.M > skinny_max_m() || d.red == FORGE_RED_MEAN_GELU_RESIDUAL) return false;
+    const int64_t groups = d.N / 8, ctas = groups < sm_count ? groups : sm_count;
+    const int64_t rows_per_cta = ctas > 0 ? (groups + ctas - 1) / ctas * 8 : 0;
+    return !(rows_per_cta <= 16 && d.K >= 24576);
+}
 
 forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_plan_info_t *info, WorkspaceLayout *wl)
 {
@@ -47,7 +58,7 @@ forge_status_t plan_for(const forge_fused_linear_desc_t &d, int sm_count, forge_
     } else {
         if (d.K % 8 != 0 || d.N % 8 != 0) return FORGE_ERR_UNSUPPORTED;     // 16-byte row pitch for TMA
         if (d.red == FORGE_RED_LAYERNORM) st = k4_plan(d, sm_count, info, wl);
-        else if (d.M <= skinny_max_m() && d.red != FORGE_RED_MEAN_GELU_RESIDUAL) st = k3_plan(d, sm_count, info, wl);
+        else if (skinny_serves(d, sm_count)) st = k3_plan(d, sm_count, info, wl);
         else st = k2_plan(d, sm_count, info, wl);
     }
     if (st != FORGE_OK) return st;

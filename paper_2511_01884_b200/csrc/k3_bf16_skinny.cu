@@ -5,8 +5,8 @@
 // and the (padded) rows of X its N dimension, so a TMA box of W is an operand as it lands -- no
 // warp touches the stream.  Each CTA owns a contiguous range of 8-row groups of W sized so that all
 // CTAs stream the same number of bytes, and walks it in strips of at most 128 rows.  Warp 0 streams W
-// and the matching slice of X (which stays L2-resident) through a deep ring of 64-k stages; one
-// thread of warp 1 issues four MMAs per stage (M = 128, N = padded rows of X, K = 16) into one of two
+// and the matching slice of X (which stays L2-resident) through a ring whose stages hold one to eight
+// 64-k boxes; one thread of warp 1 issues four MMAs per box (M = 128, N = padded rows of X, K = 16) into one of two
 // tensor-memory accumulators; warps 2..5 read a finished accumulator (thread <-> row of W = output
 // column), add the bias, apply the activation and either store Y or reduce over the strip's columns
 // with shuffles, then across strips and -- by the CTA that arrives last, in CTA order -- across CTAs.
@@ -24,11 +24,12 @@
 namespace forge {
 
 constexpr int K3_BK = 64;                      // k per TMA box: one 128-byte swizzle row
-// Boxes per stage (1 or 2; planned per problem, or forced by a tuning build with -DFORGE_K3_KB=1|2).
+// Boxes per stage (planned per problem, or forced by a tuning build with -DFORGE_K3_KB=1..8).
 #ifndef FORGE_K3_KB
 #define FORGE_K3_KB 0
 #endif
-static_assert(FORGE_K3_KB >= 0 && FORGE_K3_KB <= 2, "one or two 64-k blocks per stage");
+constexpr int K3_MAX_KB = 8;
+static_assert(FORGE_K3_KB >= 0 && FORGE_K3_KB <= K3_MAX_KB, "boxes per stage");
 constexpr int K3_MAX_ROWS_W = 128;             // rows of W per strip (the MMA's M)
 constexpr int K3_MAX_M = 128;                  // rows of X (the MMA's N, padded to a multiple of 16)
 constexpr int K3_MAX_STAGES = 16;
@@ -422,12 +423,24 @@ int k3_stage_count(uint32_t stage)
     const int n = (int)(K3_RING_BUDGET / stage);
     return n > K3_MAX_STAGES ? K3_MAX_STAGES : n;
 }
-// Two boxes per stage request 256 contiguous bytes of every row of W together, which the memory system serves
-// better than two requests of 128 bytes at different times -- as long as the ring then still has enough stages.
+// Boxes per stage: what counts is the bytes of W in flight (stages x boxes x box size) and, with two or more boxes,
+// that 256 contiguous bytes or more of every row are requested together (measured: at equal bytes in flight two boxes
+// beat one by 2-6 %).  A strip of few rows (small N, or N / 8 just above the SM count) has small boxes, and since an MMA
+// reads 16 KiB from the start of each -- boxes of one stage may overlap in that span -- only many boxes per stage fill
+// the ring: 8 rows of W, one box per stage: 12 KiB in flight; eight boxes: 72 KiB.
 int k3_boxes_per_stage(int box_groups, int xr)
 {
     if (FORGE_K3_KB != 0) return FORGE_K3_KB;
-    return k3_stage_count(k3_stage_bytes(box_groups, xr, 2)) >= 4 ? 2 : 1;
+    const uint32_t wbox = (uint32_t)box_groups * 8 * K3_BK * 2;
+    int best = 1;
+    double best_score = 0;
+    for (int kb = 1; kb <= K3_MAX_KB; ++kb) {
+        const int stages = k3_stage_count(k3_stage_bytes(box_groups, xr, kb));
+        if (stages < 4 && kb > 1) break;
+        const double score = (double)stages * kb * wbox * (kb >= 2 ? 1.0 : 0.9);
+        if (score > best_score) { best_score = score; best = kb; }
+    }
+    return best;
 }
 uint32_t k3_tmem_cols(int xr)
 {

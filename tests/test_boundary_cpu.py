@@ -131,6 +131,24 @@ def test_fp32_plan():
     assert st == B.FORGE_OK and p.grid == 32 * 32 and p.cluster == 1 and p.tile_m == 128
 
 
+def test_skinny_plan():
+    """The skinny kernel's plan: C4 on 148 SMs streams 104 or 112 rows of W per CTA in stages of two 64-k boxes; a strip of
+    few rows takes more boxes per stage; M beyond 96, and a long K against 16 rows of W per SM or fewer, go to the tile
+    kernel."""
+    st, p = B.forge_fused_linear_query_plan(pu_desc("c4"))
+    assert st == B.FORGE_OK and p.kernel == B.FORGE_KERNEL_BF16_SKINNY
+    assert (p.tile_m, p.tile_n, p.tile_k, p.stages, p.grid, p.threads, p.cluster) == (16, 112, 128, 6, 148, 192, 1)
+    assert p.smem_bytes <= 227 * 1024 and p.workspace_bytes >= 148 * 16 * 4
+    st, p = B.forge_fused_linear_query_plan(B.make_desc(16, 1184, 8192, wk.BF16, wk.ACT_RELU, wk.RED_SUM))
+    assert st == B.FORGE_OK and p.kernel == B.FORGE_KERNEL_BF16_SKINNY and (p.tile_n, p.tile_k) == (8, 512)
+    for M, N, K, kernel in ((96, 16384, 8192, B.FORGE_KERNEL_BF16_SKINNY), (97, 16384, 8192, B.FORGE_KERNEL_BF16_TCGEN05),
+                            (16, 1024, 65536, B.FORGE_KERNEL_BF16_TCGEN05), (16, 2368, 24576, B.FORGE_KERNEL_BF16_TCGEN05),
+                            (16, 2368, 16384, B.FORGE_KERNEL_BF16_SKINNY), (16, 4096, 65536, B.FORGE_KERNEL_BF16_SKINNY)):
+        st, p = B.forge_fused_linear_query_plan(B.make_desc(M, N, K, wk.BF16, wk.ACT_RELU, wk.RED_MAX))
+        assert st == B.FORGE_OK and p.kernel == kernel, (M, N, K)
+        assert p.smem_bytes <= 227 * 1024
+
+
 def pu_desc(name):
     wl = wk.WORKLOADS[name]
     return B.make_desc(wl.M, wl.N, wl.K, wl.dtype, wl.act, wl.red, wl.scale, wl.ln_eps, wl.bias.kind != "none")

@@ -37,7 +37,9 @@ SHAPES = [(16, 8, 8), (1, 64, 16), (5, 1184, 72), (16, 1192, 200), (16, 4096, 10
           (17, 8, 8), (32, 1192, 200), (27, 20000, 264), (24, 4096, 1024), (32, 148 * 8 * 17, 128),
           (19, 1184 * 13, 2048), (32, 2368, 4096),
           (33, 8, 8), (48, 1192, 200), (64, 4096, 1024), (80, 148 * 8 * 17, 128), (96, 20000, 264), (85, 2368, 4096),
-          (96, 148 * 8 * 40 + 8, 64)]
+          (96, 148 * 8 * 40 + 8, 64),
+          # few rows of W per CTA: up to eight 64-k boxes per ring stage, full and ragged in K
+          (16, 1184, 2048), (7, 2368, 1000), (40, 1184, 776), (16, 4096, 1536)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
