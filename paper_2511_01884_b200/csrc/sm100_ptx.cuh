@@ -1,7 +1,6 @@
 // Thin inline-PTX wrappers for the sm_100a features the bf16 kernels use: mbarrier with
 // bounded waits, TMA tensor loads (never multicast), tcgen05 (TMEM allocation, MMA,
-// commit, loads, fences), ldmatrix / mma.sync for the skinny kernel.  Written from the
-// public PTX ISA description of these instructions.
+// commit, loads, fences).  Written from the public PTX ISA description of these instructions.
 #pragma once
 
 #include <cuda.h>
@@ -300,28 +299,7 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint16_t cta_mas
                  ::"r"(smem_u32(bar)), "h"(cta_mask) : "memory");
 }
 
-// ---- legacy warp-level tensor path (skinny-M kernel) ---------------------------------------
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(saddr));
-}
-__device__ __forceinline__ void mma_m16n8k16_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void mma_m16n8k16_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
+// ---- 16-bit packing ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     uint32_t r;
